@@ -1,0 +1,479 @@
+"""Pins for the CPU oracle: it is checked against what the paper prints and what the
+mathematics fixes, never against itself and never against the CUDA path."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from mcsd_inputs import fork_parent_array, parent_array
+from oracle import mcsd_oracle as orc
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "paper_counts.txt")
+
+
+def _golden():
+    out = {}
+    with open(GOLDEN) as f:
+        for line in f:
+            line = line.split("#", 1)[0].strip()
+            if not line:
+                continue
+            k, v = line.split("=")
+            out[k.strip()] = [int(t) for t in v.split()]
+    return out
+
+
+# ----------------------------------------------------------------------------
+# trees and masks
+# ----------------------------------------------------------------------------
+
+def test_mask_sides_printed_for_fig1():
+    g = _golden()
+    # width 3, depth 2: the draft-initialised tree holds only the 6 draft tokens,
+    # the target-initialised one adds the 3 target tokens in front (Section 3.1)
+    draft = fork_parent_array(3, 2)
+    target = fork_parent_array(3, 3)
+    assert orc.dense_mask(draft).shape[0] == g["fig1_draft_init_mask_side"][0]
+    assert orc.dense_mask(target).shape[0] == g["fig1_target_init_mask_side"][0]
+
+
+def test_sliced_mask_sides_printed_for_fig2():
+    g = _golden()
+    parent = fork_parent_array(3, 3)
+    # stopping after draft iteration i keeps i levels: gamma = i - 1 levels below the first one
+    sides = [orc.sliced_mask(parent, gamma).shape[0] for gamma in (0, 1, 2)]
+    assert sides == g["fig2_slice_sides"]
+
+
+def test_counts_printed_for_static_configurations():
+    g = _golden()
+    parent = parent_array(2, (4, 3, 1, 1))
+    depth, level_start = orc.tree_levels(parent)
+    n_leaves = sum(1 for n in range(len(parent)) if not np.any(parent == n))
+    assert (len(parent) - 2) // 2 == g["cfg_2_4_3_1_1_draft_tokens_per_root"][0]
+    assert n_leaves == g["cfg_2_4_3_1_1_candidate_sequences"][0]
+    assert int(depth.max()) == g["cfg_2_4_3_1_1_gamma"][0]
+    parent = parent_array(1, (4, 2, 2, 1))
+    depth, level_start = orc.tree_levels(parent)
+    assert list(np.diff(level_start)[1:]) == g["cfg_4_2_2_1_level_sizes"]
+    assert len(parent) - 1 == 44
+
+
+def test_fork_mask_grows_linearly_expansion_tree_exponentially():
+    # Section 3.2: fork-shaped trees add `width` tokens per level, expansion trees multiply
+    fork = [len(fork_parent_array(3, d)) for d in (1, 2, 3, 4)]
+    assert list(np.diff(fork)) == [3, 3, 3]
+    exp = [len(parent_array(1, (3,) * d)) for d in (1, 2, 3, 4)]
+    assert list(np.diff(exp)) == [9, 27, 81]
+
+
+def _random_bfs_parent(rng, N, n_roots):
+    """Random level-ordered tree: parents non-decreasing, every level non-empty."""
+    parent = [-1] * n_roots
+    lo, hi = 0, n_roots          # current parent level [lo, hi)
+    while len(parent) < N:
+        start = len(parent)
+        n_new = int(rng.integers(1, max(2, min(N - start, 3 * (hi - lo)) + 1)))
+        n_new = min(n_new, N - start)
+        ps = np.sort(rng.integers(lo, hi, size=n_new))
+        parent.extend(int(x) for x in ps)
+        lo, hi = start, len(parent)
+    return np.asarray(parent[:N], dtype=np.int32)
+
+
+@pytest.mark.parametrize("N", [1, 2, 15, 63, 64, 65, 128, 129, 192])
+def test_mask_invariants_on_random_trees(N):
+    rng = np.random.default_rng(N)
+    parent = _random_bfs_parent(rng, N, n_roots=int(rng.integers(1, min(N, 8) + 1)))
+    depth, level_start = orc.tree_levels(parent)
+    m = orc.dense_mask(parent)
+    assert np.all(np.diag(m))
+    assert not np.any(np.triu(m, 1))                      # nothing attends to a later node
+    assert np.array_equal(m.sum(1), depth + 1)            # one bit per level of the root path
+    for n in range(N):
+        expect = np.zeros(N, dtype=bool)
+        expect[n] = True
+        if parent[n] >= 0:
+            expect |= m[parent[n]]
+        assert np.array_equal(m[n], expect)               # row = parent's row plus itself
+    bits = orc.pack_bitsets(m)
+    assert bits.shape == (N, (N + 63) // 64)
+    for n in range(N):
+        unpacked = [(int(bits[n, j // 64]) >> (j % 64)) & 1 for j in range(N)]
+        assert unpacked == [int(x) for x in m[n]]
+    # level_start brackets each depth
+    for l in range(len(level_start) - 1):
+        assert np.all(depth[level_start[l]:level_start[l + 1]] == l)
+
+
+def test_sliced_mask_equals_mask_rebuilt_for_truncated_tree():
+    for n_roots, br in [(1, (4, 2, 2, 1)), (8, (1, 2, 2, 1, 1, 1)), (1, (4, 2, 2, 1, 1, 1, 1, 1)), (3, (1, 1))]:
+        parent = parent_array(n_roots, br)
+        for gamma in range(len(br) + 1):
+            truncated = parent_array(n_roots, br[:gamma])
+            assert np.array_equal(orc.sliced_mask(parent, gamma), orc.dense_mask(truncated))
+            assert orc.n_active_for_gamma(parent, gamma) == len(truncated)
+
+
+def test_tree_levels_rejects_bad_orders():
+    with pytest.raises(ValueError):
+        orc.tree_levels([-1, 1])            # parent not earlier
+    with pytest.raises(ValueError):
+        orc.tree_levels([-1, 0, 1, 0])      # depth goes back down
+    with pytest.raises(ValueError):
+        orc.tree_levels([-1, -1, 1, 0])     # children out of parent order
+    with pytest.raises(ValueError):
+        orc.tree_levels([0, -1])            # node 0 is not a root
+
+
+# ----------------------------------------------------------------------------
+# attention
+# ----------------------------------------------------------------------------
+
+def _rand_attn(rng, B, H, N, D, L):
+    f = lambda *s: rng.standard_normal(s)
+    return f(B, H, N, D), f(B, H, L, D), f(B, H, L, D), f(B, H, N, D), f(B, H, N, D)
+
+
+def _sdpa_causal_last(q_seq, k_seq, v_seq, scale):
+    """Library causal attention over an explicit sequence [T][D]; returns all rows."""
+    t = lambda a: torch.from_numpy(np.ascontiguousarray(a))[None, None]
+    o = torch.nn.functional.scaled_dot_product_attention(t(q_seq), t(k_seq), t(v_seq), is_causal=True, scale=scale)
+    return o[0, 0].numpy()
+
+
+def test_single_chain_tree_is_ordinary_causal_attention():
+    rng = np.random.default_rng(1)
+    B, H, N, D, L = 2, 3, 6, 16, 11
+    q, kc, vc, kt, vt = _rand_attn(rng, B, H, N, D, L)
+    parent = parent_array(1, (1,) * (N - 1))
+    scale = 0.37
+    out = orc.tree_attention(q, kc, vc, kt, vt, [L] * B, None, parent, scale)
+    for b in range(B):
+        for h in range(H):
+            k_seq = np.concatenate([kc[b, h], kt[b, h]])
+            v_seq = np.concatenate([vc[b, h], vt[b, h]])
+            q_seq = np.concatenate([np.zeros((L, D)), q[b, h]])
+            ref = _sdpa_causal_last(q_seq, k_seq, v_seq, scale)[L:]
+            np.testing.assert_allclose(out[b, h], ref, rtol=0, atol=1e-12)
+
+
+def test_each_node_equals_causal_attention_over_its_own_root_path():
+    rng = np.random.default_rng(2)
+    parent = parent_array(2, (2, 3, 1))
+    N = len(parent)
+    B, H, D, L = 2, 2, 8, 9
+    q, kc, vc, kt, vt = _rand_attn(rng, B, H, N, D, L)
+    lens = [L, 5]
+    scale = 1.0 / np.sqrt(D)
+    out = orc.tree_attention(q, kc, vc, kt, vt, lens, None, parent, scale)
+    for b in range(B):
+        for h in range(H):
+            for n in range(N):
+                path = []
+                a = n
+                while a >= 0:
+                    path.append(a)
+                    a = parent[a]
+                path = path[::-1]
+                k_seq = np.concatenate([kc[b, h, :lens[b]], kt[b, h, path]])
+                v_seq = np.concatenate([vc[b, h, :lens[b]], vt[b, h, path]])
+                q_seq = np.zeros_like(k_seq)
+                q_seq[-1] = q[b, h, n]
+                ref = _sdpa_causal_last(q_seq, k_seq, v_seq, scale)[-1]
+                np.testing.assert_allclose(out[b, h, n], ref, rtol=0, atol=1e-12)
+
+
+def test_attention_invariants():
+    rng = np.random.default_rng(3)
+    parent = parent_array(1, (3, 2))
+    N = len(parent)
+    B, H, D, L = 1, 2, 8, 7
+    q, kc, vc, kt, vt = _rand_attn(rng, B, H, N, D, L)
+    scale = 0.5
+    base = orc.tree_attention(q, kc, vc, kt, vt, [L], None, parent, scale)
+    mask = orc.dense_mask(parent)
+    # changing K/V of nodes that are not on a node's root path leaves that node's output alone
+    for n in range(N):
+        kt2, vt2 = kt.copy(), vt.copy()
+        others = ~mask[n]
+        kt2[0, :, others] = rng.standard_normal((others.sum(), H, D)) * 5
+        vt2[0, :, others] = rng.standard_normal((others.sum(), H, D)) * 5
+        out = orc.tree_attention(q, kc, vc, kt2, vt2, [L], None, parent, scale)
+        np.testing.assert_allclose(out[0, :, n], base[0, :, n], rtol=0, atol=1e-13)
+    # each output is a convex combination of the values it may see
+    for n in range(N):
+        for h in range(H):
+            vals = np.concatenate([vc[0, h], vt[0, h, mask[n]]])
+            assert np.all(base[0, h, n] <= vals.max(0) + 1e-12)
+            assert np.all(base[0, h, n] >= vals.min(0) - 1e-12)
+    # no prefix at all: a root sees only itself, so its output is its own value row
+    out0 = orc.tree_attention(q, kc, vc, kt, vt, [0], None, parent, scale)
+    np.testing.assert_allclose(out0[0, :, 0], vt[0, :, 0], rtol=0, atol=1e-13)
+    # sliced tree: rows beyond n_active are not produced, the others do not change
+    outs = orc.tree_attention(q, kc, vc, kt, vt, [L], [4], parent, scale)
+    np.testing.assert_allclose(outs[0, :, :4], base[0, :, :4], rtol=0, atol=1e-13)
+    assert np.all(np.isnan(outs[0, :, 4:]))
+
+
+# ----------------------------------------------------------------------------
+# accept / reject
+# ----------------------------------------------------------------------------
+
+def _rand_dist(rng, *shape):
+    x = rng.random(shape) ** 2 + 1e-3
+    return x / x.sum(-1, keepdims=True)
+
+
+def _forced_run(p, q, tokens, parent, forced, u_bonus=0.5):
+    """Run the oracle with accept uniforms forced to 0 (accept if possible) or 1 (reject)."""
+    N = len(parent)
+    ua = np.ones((1, N))
+    for c, v in forced.items():
+        ua[0, c] = v
+    ub = np.full((1, N), u_bonus)
+    trace = []
+    res = orc.verify_tree(p, q, tokens, parent, None, ua, ub, trace=trace)
+    return res, trace
+
+
+def _inverse_cdf_measure(dist, n_grid=200001):
+    """Lebesgue measure of {u : inverse_cdf(dist, u) = t} estimated on a uniform grid."""
+    us = (np.arange(n_grid) + 0.5) / n_grid
+    counts = np.zeros(len(dist))
+    for u in us:
+        counts[orc.inverse_cdf(dist, u)] += 1
+    return counts / n_grid
+
+
+def test_inverse_cdf_samples_each_token_with_its_mass():
+    rng = np.random.default_rng(4)
+    dist = _rand_dist(rng, 7)
+    dist[2] = 0.0
+    dist = dist / dist.sum() * 3.0          # unnormalised input is allowed
+    meas = _inverse_cdf_measure(dist, 20001)
+    np.testing.assert_allclose(meas, dist / dist.sum(), atol=1e-4)
+    assert orc.inverse_cdf(dist, 0.0) == 0
+    assert orc.inverse_cdf(np.array([0.0, 0.0, 1.0, 0.0]), 0.3) == 2      # zero-mass ids are never drawn
+    assert orc.inverse_cdf(np.array([0.5, 0.5]), 0.5) == 1                # strict comparison at an edge
+
+
+@pytest.mark.parametrize("V,k", [(3, 1), (3, 2), (3, 3), (4, 1), (4, 2), (4, 3), (5, 1), (5, 2), (5, 3)])
+def test_exact_enumeration_output_distribution_is_target(V, k):
+    """One node with k sibling candidates drawn i.i.d. from q: the emitted token is distributed as p.
+
+    k = 1 is plain speculative decoding (Section 2.1: the output distribution stays the target's)."""
+    rng = np.random.default_rng(100 * V + k)
+    p = _rand_dist(rng, 1, 1 + k, V)
+    q = _rand_dist(rng, 1, 1 + k, V)
+    if V == 4:
+        q[0, 0, 1] = 0.0
+        q[0, 0] /= q[0, 0].sum()          # a token the draft never proposes
+        p[0, 0, 2] = 0.0
+        p[0, 0] /= p[0, 0].sum()          # a token the target never emits
+    parent = parent_array(1, (k,))
+    emitted = np.zeros(V)
+    for xs in itertools.product(range(V), repeat=k):
+        w = np.prod([q[0, 0, x] for x in xs])
+        if w == 0.0:
+            continue
+        tokens = np.array([[0] + list(xs)])
+        # all-rejected run gives every stage's acceptance probability and the final residual
+        res, trace = _forced_run(p, q, tokens, parent, {})
+        a = [t["a"] for t in trace if "child" in t]
+        stop = [t for t in trace if "stop" in t][0]
+        assert len(a) == k and stop["stop"] == 0
+        reach = 1.0
+        for i in range(k):
+            if a[i] > 0:
+                forced = {1 + j: 1.0 for j in range(i)}
+                forced[1 + i] = 0.0
+                r2, _ = _forced_run(p, q, tokens, parent, forced)
+                assert r2["accept_len"][0] == 1 and r2["out_tokens"][0, 0] == xs[i]
+                assert r2["out_nodes"][0, 0] == 1 + i
+            emitted[xs[i]] += w * reach * a[i]
+            reach *= 1.0 - a[i]
+        assert res["accept_len"][0] == 0
+        emitted += w * reach * stop["dist"] / stop["dist"].sum()
+    np.testing.assert_allclose(emitted, p[0, 0], rtol=0, atol=1e-12)
+
+
+def test_two_level_tree_joint_distribution():
+    """Tree (1; 2, 2): first emitted token ~ p(.), and given that it was an accepted
+    candidate x1, the second emitted token ~ p(. | x1)."""
+    V = 3
+    rng = np.random.default_rng(7)
+    p_root, q_root = _rand_dist(rng, V), _rand_dist(rng, V)
+    P2, Q2 = _rand_dist(rng, V, V), _rand_dist(rng, V, V)      # conditional rows given the first token
+    parent = parent_array(1, (2, 2))                            # nodes: 0 | 1 2 | 3 4 5 6
+    first = np.zeros(V)
+    joint = np.zeros((V, V))
+    moved = np.zeros(V)
+    for x1 in itertools.product(range(V), repeat=2):
+        w1 = q_root[x1[0]] * q_root[x1[1]]
+        for x2 in itertools.product(range(V), repeat=4):
+            w = w1 * np.prod([Q2[x1[i // 2], x2[i]] for i in range(4)])
+            tokens = np.array([[0, x1[0], x1[1], *x2]])
+            p = np.zeros((1, 7, V))
+            q = np.zeros((1, 7, V))
+            p[0, 0], q[0, 0] = p_root, q_root
+            for i in (0, 1):
+                p[0, 1 + i], q[0, 1 + i] = P2[x1[i]], Q2[x1[i]]
+            p[0, 3:] = 1.0 / V
+            q[0, 3:] = 1.0 / V
+            _, tr = _forced_run(p, q, tokens, parent, {})
+            a1 = [t["a"] for t in tr if t.get("node") == 0]
+            d1 = [t for t in tr if "stop" in t][0]["dist"]
+            reach = 1.0
+            for i in (0, 1):
+                pr = reach * a1[i]
+                reach *= 1.0 - a1[i]
+                if pr == 0.0:
+                    continue
+                first[x1[i]] += w * pr
+                moved[x1[i]] += w * pr
+                c = 1 + i
+                forced = {1 + j: 1.0 for j in range(i)}
+                forced[c] = 0.0
+                r2, tr2 = _forced_run(p, q, tokens, parent, forced)
+                assert r2["out_nodes"][0, 0] == c
+                a2 = [t["a"] for t in tr2 if t.get("node") == c]
+                d2 = [t for t in tr2 if "stop" in t][0]
+                assert d2["stop"] == c
+                kids = [3 + 2 * i, 4 + 2 * i]
+                reach2 = 1.0
+                for j in (0, 1):
+                    joint[x1[i], tokens[0, kids[j]]] += w * pr * reach2 * a2[j]
+                    reach2 *= 1.0 - a2[j]
+                joint[x1[i]] += w * pr * reach2 * d2["dist"] / d2["dist"].sum()
+            first += w * reach * d1 / d1.sum()
+    np.testing.assert_allclose(first, p_root, atol=1e-12)
+    np.testing.assert_allclose(joint, moved[:, None] * P2, atol=1e-12)
+
+
+def test_residual_matches_closed_form():
+    """After m rejections the target-side distribution is max(p - s_m q, 0) / Z_m with
+    s_0 = 0, Z_m = sum max(p - s_m q, 0), s_{m+1} = s_m + Z_m."""
+    rng = np.random.default_rng(8)
+    V, k = 50, 4
+    p = _rand_dist(rng, 1, 1 + k, V)
+    q = _rand_dist(rng, 1, 1 + k, V)
+    parent = parent_array(1, (k,))
+    tokens = np.array([[0] + [int(t) for t in rng.integers(0, V, k)]])
+    s = 0.0
+    for m in range(1, k + 1):
+        par_m = parent_array(1, (m,))
+        _, tr = _forced_run(p[:, :1 + m], q[:, :1 + m], tokens[:, :1 + m], par_m, {})
+        dist = [t for t in tr if "stop" in t][0]["dist"]
+        z = np.maximum(p[0, 0] - s * q[0, 0], 0).sum()
+        s = s + z
+        closed = np.maximum(p[0, 0] - s * q[0, 0], 0)
+        np.testing.assert_allclose(dist, closed / closed.sum(), rtol=0, atol=1e-12)
+        # acceptance probability of the next sibling against the closed form
+        a = [t["a"] for t in tr if "child" in t]
+        assert len(a) == m
+
+
+def test_verify_special_cases():
+    rng = np.random.default_rng(9)
+    parent = parent_array(1, (2, 2, 1))
+    N = len(parent)
+    V = 11
+    p = _rand_dist(rng, 2, N, V)
+    tokens = rng.integers(0, V, (2, N)).astype(np.int32)
+    ua = rng.random((2, N)) * 0.999
+    ub = rng.random((2, N))
+    # q = p: every first candidate is accepted, to full depth
+    r = orc.verify_tree(p, p.copy(), tokens, parent, None, ua, ub)
+    assert list(r["accept_len"]) == [3, 3]
+    assert np.array_equal(r["out_nodes"][0, :3], [1, 3, 7])
+    assert np.array_equal(r["out_tokens"][0, :3], tokens[0, [1, 3, 7]])
+    # gamma slices the walk: with gamma = 1 only one level is tested, bonus from the raw row of the stop node
+    r = orc.verify_tree(p, p.copy(), tokens, parent, [1, 0], ua, ub)
+    assert list(r["accept_len"]) == [1, 0]
+    assert r["out_tokens"][0, 1] == orc.inverse_cdf(p[0, 1], ub[0, 1])
+    assert r["out_tokens"][1, 0] == orc.inverse_cdf(p[1, 0], ub[1, 0])
+    assert np.all(r["out_tokens"][1, 1:] == -1) and np.all(r["out_nodes"][1] == -1)
+    # draft puts all its mass on a token the target never emits: everything rejected,
+    # the residual is the target row itself
+    p2 = p.copy()
+    p2[:, :, 0] = 0.0
+    p2 /= p2.sum(-1, keepdims=True)
+    q2 = np.zeros_like(p2)
+    q2[:, :, 0] = 1.0
+    tok0 = np.zeros_like(tokens)
+    r = orc.verify_tree(p2, q2, tok0, parent, None, ua, ub)
+    assert list(r["accept_len"]) == [0, 0]
+    assert r["out_tokens"][0, 0] == orc.inverse_cdf(p2[0, 0], ub[0, 0])
+
+
+def test_multi_root_selection_is_argmax_of_single_root_walks():
+    rng = np.random.default_rng(10)
+    n_roots, br = 4, (1, 2, 1)
+    parent = parent_array(n_roots, br)
+    N = len(parent)
+    B, V = 6, 9
+    p = _rand_dist(rng, B, N, V)
+    q = _rand_dist(rng, B, N, V)
+    tokens = rng.integers(0, V, (B, N)).astype(np.int32)
+    ua, ub = rng.random((B, N)), rng.random((B, N))
+    gam = rng.integers(0, 4, B)
+    res = orc.verify_tree(p, q, tokens, parent, gam, ua, ub, R=3)
+    mask = orc.dense_mask(parent)
+    for b in range(B):
+        lens = []
+        for r in range(n_roots):
+            # subtree of root r as a tree of its own
+            nodes = [n for n in range(N) if mask[n, r]]
+            remap = {n: i for i, n in enumerate(nodes)}
+            sub_parent = np.array([-1 if parent[n] < 0 else remap[parent[n]] for n in nodes])
+            rr = orc.verify_tree(p[b:b + 1, nodes], q[b:b + 1, nodes], tokens[b:b + 1, nodes], sub_parent,
+                                 gam[b:b + 1], ua[b:b + 1, nodes], ub[b:b + 1, nodes], R=3)
+            lens.append((int(rr["accept_len"][0]), rr, nodes))
+        best = int(np.argmax([l[0] for l in lens]))        # first maximum = lowest root index
+        assert res["best_root"][b] == best
+        ln, rr, nodes = lens[best]
+        assert res["accept_len"][b] == ln
+        assert np.array_equal(res["out_nodes"][b, :ln], [nodes[i] for i in rr["out_nodes"][0, :ln]])
+        # several roots: the selected root's own token is emitted first
+        assert res["out_tokens"][b, 0] == tokens[b, best]
+        assert np.array_equal(res["out_tokens"][b, 1:ln + 2], rr["out_tokens"][0, :ln + 1])
+        assert np.array_equal(res["next_roots"][b], rr["next_roots"][0])
+
+
+def test_next_roots_are_top_ids_with_ties_to_smaller_id():
+    parent = parent_array(1, ())
+    p = np.array([[[0.1, 0.3, 0.3, 0.2, 0.1]]])
+    r = orc.verify_tree(p, p, np.zeros((1, 1), int), parent, None, np.zeros((1, 1)), np.full((1, 1), 0.5), R=4)
+    assert list(r["next_roots"][0]) == [1, 2, 3, 0]
+    assert r["out_tokens"][0, 0] == 2 and r["accept_len"][0] == 0
+
+
+def test_acceptance_rate_definition():
+    # Section 1: alpha = longest accepted draft length / maximum draft length
+    parent = parent_array(1, (1, 1, 1, 1))
+    rng = np.random.default_rng(11)
+    p = _rand_dist(rng, 1, 5, 6)
+    tokens = rng.integers(0, 6, (1, 5))
+    r = orc.verify_tree(p, p.copy(), tokens, parent, None, np.full((1, 5), 0.5), np.full((1, 5), 0.5))
+    assert r["accept_len"][0] / 4 == 1.0
+
+
+def test_decision_margins_flag_uniforms_on_a_threshold():
+    rng = np.random.default_rng(12)
+    parent = parent_array(1, (2,))
+    V = 5
+    p = _rand_dist(rng, 1, 3, V)
+    q = _rand_dist(rng, 1, 3, V)
+    tokens = np.array([[0, 1, 2]])
+    ratio = p[0, 0, 1] / q[0, 0, 1]
+    ua = np.array([[0.5, min(ratio, 0.99), 0.5]])
+    ub = np.full((1, 3), 0.5)
+    m_acc, m_bon = orc.decision_margins(p, q, tokens, parent, None, ua, ub)
+    if ratio < 0.99:
+        assert m_acc[0, 1] < 1e-12
+    assert np.isinf(m_acc[0, 0])
+    # leaves can be stop nodes: their bonus margin is finite
+    assert np.isfinite(m_bon[0, 1]) and np.isfinite(m_bon[0, 2])
