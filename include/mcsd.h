@@ -1,0 +1,172 @@
+/*
+ * mcsd.h -- C ABI of libmcsd: one-pass verification of a candidate token tree
+ * (multi-candidate speculative decoding) on one NVIDIA B200 (sm_100a).
+ *
+ * Three operations make up the verification step of the generation loop in Fig. 1 of
+ * "Improving Multi-candidate Speculative Decoding" (steps 2, 4, 5 and the sampling of step 6):
+ *
+ *   mcsd_build_mask      topology-aware causal mask of the token tree, built once (Sections 2.2, 3.2)
+ *   mcsd_tree_attention  attention of all tree tokens over the prefix KV cache plus the tree's own
+ *                        keys/values under that mask (tree attention, Section 2.2)
+ *   mcsd_verify_tree     multi-candidate accept/reject walk, longest-sequence selection and sampling of
+ *                        the new token (Fig. 1 steps 4-6; Section 3.1 for several target-initialised roots)
+ *
+ * Conventions
+ *   - Every function returns an int status: MCSD_OK (0) or a negative MCSD_ERR_* code.  Nothing throws or
+ *     aborts.  mcsd_status_string() names a code; mcsd_last_cuda_error() returns the cudaError_t behind the
+ *     most recent MCSD_ERR_CUDA of the calling thread.
+ *   - Pointers marked [dev] are device pointers owned by the caller; pointers marked [host] are host
+ *     pointers.  All tensors are dense and contiguous in the stated layout.  These functions never allocate
+ *     or free device memory: kernels that need scratch take a caller-supplied workspace whose size the
+ *     matching *_workspace_bytes() query returns.  A workspace is 256-byte aligned and must be zero-filled
+ *     once before its first use (its first 256 bytes hold a sticky status word, see mcsd_workspace_status).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls only enqueue
+ *     work on that stream and never synchronise, except where stated.
+ *   - Nodes of the tree are in level (BFS) order: parent[n] < n, depth non-decreasing in n, children of a
+ *     node contiguous.  Roots carry parent -1 and form level 0.  With one root the tree is
+ *     draft-initialised and node 0 is the last emitted token; with R > 1 roots it is the
+ *     target-initialised forest of Section 3.1 whose roots are accepted by construction.
+ *   - The dynamic sliced mask of Section 3.2 is a row count: keeping the first gamma draft levels keeps the
+ *     first n_active = level_start[gamma + 1] nodes, and in level order no kept row has a bit beyond them.
+ */
+#ifndef MCSD_H_
+#define MCSD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MCSD_OK                        0
+#define MCSD_ERR_NULL                 -1  /* a required pointer is NULL */
+#define MCSD_ERR_BAD_SHAPE            -2  /* a size or an alignment is out of the supported range */
+#define MCSD_ERR_NOT_BFS              -3  /* parent array is not a level-ordered forest */
+#define MCSD_ERR_BAD_DTYPE            -4
+#define MCSD_ERR_WORKSPACE_TOO_SMALL  -5
+#define MCSD_ERR_CUDA                 -6  /* a CUDA runtime/driver call failed; see mcsd_last_cuda_error() */
+#define MCSD_ERR_TIMEOUT              -7  /* a bounded device-side wait ran out (reported by mcsd_workspace_status) */
+
+#define MCSD_MAX_NODES   192              /* largest tree (roots included) */
+#define MCSD_MAX_WORDS   3                /* 64-bit mask words per node for MCSD_MAX_NODES */
+
+#define MCSD_BF16  0
+#define MCSD_F32   1
+
+const char* mcsd_status_string(int status);
+int mcsd_last_cuda_error(void);
+
+/*
+ * Topology-aware causal mask (Section 2.2; Fig. 1 step 2), built once for the deepest tree (Section 3.2).
+ *
+ *   parent_host      [host] int32[n_nodes], level order, -1 for roots.  Validated on the CPU before anything
+ *                    is launched; a bad array returns MCSD_ERR_NOT_BFS and touches no output.
+ *   anc_dev          [dev]  uint64[n_nodes][words]: bit (j % 64) of word (j / 64) of row n is set iff tree
+ *                    token n may attend to tree token j, i.e. j is n or an ancestor of n.
+ *   words            must be >= ceil(n_nodes / 64) and <= MCSD_MAX_WORDS; unused high words are zeroed.
+ *   depth_dev        [dev]  int32[n_nodes], level of every node (roots 0): position = prefix length + depth.
+ *   level_start_dev  [dev]  int32[n_nodes + 1] capacity; entries 0..*n_levels are written:
+ *                    level_start[l] = index of the first node of level l, level_start[n_levels] = n_nodes.
+ *                    May be NULL.
+ *   level_start_host [host] same content, capacity n_nodes + 1.  May be NULL.
+ *   n_levels         [host] out, number of levels.  May be NULL.
+ *
+ * The tree travels to the kernel as a launch argument, so no host-to-device copy and no synchronisation
+ * takes place; outputs are ready when the work enqueued on `stream` completes.
+ * Errors: MCSD_ERR_NULL, MCSD_ERR_BAD_SHAPE (n_nodes < 1 or > MCSD_MAX_NODES, bad words), MCSD_ERR_NOT_BFS,
+ * MCSD_ERR_CUDA.
+ */
+int mcsd_build_mask(const int32_t* parent_host, int n_nodes,
+                    uint64_t* anc_dev, int words,
+                    int32_t* depth_dev,
+                    int32_t* level_start_dev, int32_t* level_start_host, int* n_levels,
+                    void* stream);
+
+/*
+ * Tree attention (Section 2.2): for every sequence b, head h and active tree token n < n_active[b]
+ *     out[b][h][n] = sum_j softmax_j(softmax_scale * <q[b][h][n], k_j>) v_j
+ * over the prefix keys j = 0 .. seq_lens[b]-1 of the cache and the tree keys j with bit j set in anc[n].
+ * Rows n >= n_active[b] of `out` are not written.
+ *
+ *   q, k_tree, v_tree, out  [dev] [B][H][N][D]
+ *   k_cache, v_cache        [dev] [B][H][L_max][D]; only the first seq_lens[b] rows of sequence b are used
+ *                           (later rows may hold anything, NaN bit patterns included)
+ *   seq_lens                [dev] int32[B], 0 <= seq_lens[b] <= L_max
+ *   n_active                [dev] int32[B], 0 <= n_active[b] <= N (a level-order prefix of the tree), or NULL = N
+ *   anc, words              the mask from mcsd_build_mask for the N-node tree
+ *   D                       64 or 128;  N <= MCSD_MAX_NODES;  B * H <= 65535
+ *   dtype                   MCSD_BF16: bf16 storage, fp32 softmax and accumulation (tensor-core products when
+ *                           D == 128 and all tensors are 16-byte aligned);  MCSD_F32: fp32 throughout
+ *   workspace               [dev] scratch of at least mcsd_tree_attention_workspace_bytes(...) bytes; holds
+ *                           split-KV partial results and the status word.  Calls that may overlap on the
+ *                           device need distinct workspaces.
+ *
+ * Split-KV: the keys of one (b, h) may be processed by several thread blocks, each producing an
+ * unnormalised partial (running maximum, sum, weighted values); a combine pass merges them.
+ * Errors: MCSD_ERR_NULL, MCSD_ERR_BAD_SHAPE, MCSD_ERR_BAD_DTYPE, MCSD_ERR_WORKSPACE_TOO_SMALL, MCSD_ERR_CUDA.
+ * Device-side waits are bounded; one that runs out is reported later by mcsd_workspace_status().
+ */
+size_t mcsd_tree_attention_workspace_bytes(int B, int H, int N, int D, int L_max, int dtype);
+
+int mcsd_tree_attention(const void* q, const void* k_cache, const void* v_cache,
+                        const void* k_tree, const void* v_tree, void* out,
+                        const int32_t* seq_lens, const int32_t* n_active,
+                        const uint64_t* anc, int words,
+                        int B, int H, int N, int D, int L_max, float softmax_scale,
+                        int dtype, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Reads the status word that kernels of mcsd_tree_attention / mcsd_verify_tree leave in `workspace`.
+ * The word is sticky: kernels only ever set it, the caller clears it by zero-filling the first 256 bytes.
+ * Synchronises `stream`.  Returns MCSD_OK, MCSD_ERR_TIMEOUT (a bounded wait ran out; outputs of that call
+ * are invalid) or MCSD_ERR_CUDA.
+ */
+int mcsd_workspace_status(const void* workspace, void* stream);
+
+/*
+ * Multi-candidate accept/reject (Fig. 1 steps 4-6).  For every sequence and every root the walk starts at
+ * the root; at node u the children c_1..c_k are tried in order: child c_i with token x_i is accepted iff
+ *     u_accept[c_i] < min(1, pt(x_i) / q_u(x_i))
+ * where pt starts as p_u and after every rejection becomes norm(max(pt - q_u, 0)).  The first accepted child
+ * becomes the new u (with pt reset to its own row); if none is accepted, or u has no children within the
+ * first gamma[b] draft levels, the walk stops at u and one more token is drawn from the distribution it
+ * stopped with (pt, or p_u at a leaf) by inverse CDF in token-id order: the smallest t with
+ * cumsum(dist)[t] > u_bonus[u] * sum(dist).  The root with the longest accepted path wins (ties: lowest index).
+ *
+ *   p, q          [dev] float[B][N][V]: row n is the target / draft next-token distribution after node n
+ *   tokens        [dev] int32[B][N]: token id of every node (root tokens are never tested)
+ *   parent        [dev] int32[N]: the array given to mcsd_build_mask
+ *   level_start   [dev] int32[n_levels + 1] from mcsd_build_mask
+ *   n_roots       number of level-0 nodes
+ *   gamma         [dev] int32[B], draft levels kept per sequence (0..n_levels-1), or NULL = all
+ *   u_accept      [dev] float[B][N] uniforms, one per candidate node
+ *   u_bonus       [dev] float[B][N] uniforms, one per possible stop node
+ *   accept_len    [dev] int32[B] out: accepted draft tokens of the winning path
+ *   out_tokens    [dev] int32[B][n_levels + 1] out: (token of the winning root if n_roots > 1,) accepted
+ *                 tokens, new token; padded with -1
+ *   out_nodes     [dev] int32[B][n_levels] out: accepted node ids, padded with -1
+ *   best_root     [dev] int32[B] out
+ *   next_roots    [dev] int32[B][R] out or NULL: the R most probable ids of the distribution the new token
+ *                 was drawn from (ties to the smaller id) -- the candidates with which a target-initialised
+ *                 tree (Section 3.1) seeds its next step
+ *   workspace     [dev] >= mcsd_verify_tree_workspace_bytes(B, N, V) bytes
+ *
+ * Errors: MCSD_ERR_NULL, MCSD_ERR_BAD_SHAPE (B, N, V < 1, N > MCSD_MAX_NODES, B > 65535, R < 0 or R > 32,
+ * n_roots or n_levels out of range), MCSD_ERR_WORKSPACE_TOO_SMALL, MCSD_ERR_CUDA.
+ */
+size_t mcsd_verify_tree_workspace_bytes(int B, int N, int V);
+
+int mcsd_verify_tree(const float* p, const float* q,
+                     const int32_t* tokens, const int32_t* parent, const int32_t* level_start,
+                     int n_levels, int n_roots, const int32_t* gamma,
+                     const float* u_accept, const float* u_bonus,
+                     int B, int N, int V,
+                     int32_t* accept_len, int32_t* out_tokens, int32_t* out_nodes,
+                     int32_t* best_root, int32_t* next_roots, int R,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MCSD_H_ */
