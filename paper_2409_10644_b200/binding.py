@@ -1,0 +1,238 @@
+"""ctypes binding of libmcsd.so: argument marshalling only.
+
+Tensors are torch tensors on a CUDA device (torch supplies memory and streams); every function
+passes raw pointers and sizes to the C entry point of the same name (include/mcsd.h) on torch's
+current stream and raises McsdError on a non-zero status.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import NamedTuple, Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libmcsd.so")
+
+MCSD_BF16 = 0
+MCSD_F32 = 1
+MCSD_MAX_NODES = 192
+MCSD_MAX_WORDS = 3
+
+_EXPORTS = (
+    "mcsd_status_string", "mcsd_last_cuda_error", "mcsd_build_mask", "mcsd_tree_attention_workspace_bytes",
+    "mcsd_tree_attention", "mcsd_workspace_status", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree",
+)
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(
+            "libmcsd.so is not built (%s missing). Build it with `python -m paper_2409_10644_b200.build`; "
+            "there is no fallback path." % _LIB_PATH)
+    lib = ctypes.CDLL(_LIB_PATH)
+    c_int, c_void_p, c_size_t, c_float = ctypes.c_int, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_float
+    lib.mcsd_status_string.restype = ctypes.c_char_p
+    lib.mcsd_status_string.argtypes = [c_int]
+    lib.mcsd_last_cuda_error.restype = c_int
+    lib.mcsd_last_cuda_error.argtypes = []
+    lib.mcsd_build_mask.restype = c_int
+    lib.mcsd_build_mask.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
+                                    ctypes.POINTER(c_int), c_void_p]
+    lib.mcsd_tree_attention_workspace_bytes.restype = c_size_t
+    lib.mcsd_tree_attention_workspace_bytes.argtypes = [c_int] * 6
+    lib.mcsd_tree_attention.restype = c_int
+    lib.mcsd_tree_attention.argtypes = [c_void_p] * 9 + [c_int] * 6 + [c_float, c_int, c_void_p, c_size_t, c_void_p]
+    lib.mcsd_workspace_status.restype = c_int
+    lib.mcsd_workspace_status.argtypes = [c_void_p, c_void_p]
+    lib.mcsd_verify_tree_workspace_bytes.restype = c_size_t
+    lib.mcsd_verify_tree_workspace_bytes.argtypes = [c_int] * 3
+    lib.mcsd_verify_tree.restype = c_int
+    lib.mcsd_verify_tree.argtypes = ([c_void_p] * 5 + [c_int, c_int] + [c_void_p] * 3 + [c_int] * 3 +
+                                     [c_void_p] * 5 + [c_int, c_void_p, c_size_t, c_void_p])
+    return lib
+
+
+lib = _load()
+
+
+class McsdError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib.mcsd_status_string(status).decode()
+        if status == -6:
+            msg += " (cudaError %d)" % lib.mcsd_last_cuda_error()
+        super().__init__("%s: %s [%d]" % (where, msg, status))
+
+
+def mcsd_status_string(status: int) -> str:
+    return lib.mcsd_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise McsdError(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dev_tensor(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise ValueError("%s must be a contiguous CUDA tensor of dtype %s" % (name, dtype))
+    return t
+
+
+class TreeMask(NamedTuple):
+    """Outputs of mcsd_build_mask plus the device copy of the parent array the verify step needs."""
+    anc: torch.Tensor            # uint64 bit patterns stored as int64 [N][words]
+    depth: torch.Tensor          # int32 [N]
+    level_start: torch.Tensor    # int32 [N + 1] (first n_levels + 1 entries valid)
+    level_start_host: np.ndarray  # int32 [n_levels + 1]
+    parent: torch.Tensor         # int32 [N]
+    n_nodes: int
+    n_levels: int
+    n_roots: int
+    words: int
+
+
+def mcsd_build_mask(parent, device="cuda", words: Optional[int] = None) -> TreeMask:
+    """Ancestor bitsets, depths and level starts of a level-ordered token tree (built once per tree shape)."""
+    parent = np.ascontiguousarray(np.asarray(parent, dtype=np.int32))
+    n = int(parent.shape[0])
+    if words is None:
+        words = max(1, (n + 63) // 64)
+    dev = torch.device(device)
+    anc = torch.zeros((max(n, 1), words), dtype=torch.int64, device=dev)
+    depth = torch.zeros(max(n, 1), dtype=torch.int32, device=dev)
+    level_start = torch.zeros(max(n, 1) + 1, dtype=torch.int32, device=dev)
+    ls_host = np.zeros(max(n, 1) + 1, dtype=np.int32)
+    n_levels = ctypes.c_int(0)
+    with torch.cuda.device(dev):
+        st = lib.mcsd_build_mask(parent.ctypes.data_as(ctypes.c_void_p), n, _ptr(anc), words, _ptr(depth),
+                                 _ptr(level_start), ls_host.ctypes.data_as(ctypes.c_void_p),
+                                 ctypes.byref(n_levels), _stream())
+    _check(st, "mcsd_build_mask")
+    parent_dev = torch.from_numpy(parent).to(dev)
+    return TreeMask(anc, depth, level_start, ls_host[: n_levels.value + 1].copy(), parent_dev, n, n_levels.value,
+                    int((parent < 0).sum()), words)
+
+
+def n_active_from_gamma(level_start_host, gamma) -> np.ndarray:
+    """Dynamic sliced mask as a row count: keeping gamma draft levels keeps level_start[gamma + 1] nodes."""
+    ls = np.asarray(level_start_host)
+    g = np.clip(np.asarray(gamma, dtype=np.int64), 0, len(ls) - 2)
+    return ls[g + 1].astype(np.int32)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return MCSD_BF16
+    if t.dtype == torch.float32:
+        return MCSD_F32
+    raise ValueError("tree attention takes bf16 or fp32 tensors")
+
+
+def mcsd_tree_attention_workspace_bytes(B, H, N, D, L_max, dtype) -> int:
+    return int(lib.mcsd_tree_attention_workspace_bytes(B, H, N, D, L_max, dtype))
+
+
+def new_workspace(nbytes: int, device) -> torch.Tensor:
+    """Zero-filled, 256-byte aligned scratch buffer (torch's allocator aligns to 512 bytes)."""
+    return torch.zeros(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def mcsd_tree_attention(q, k_cache, v_cache, k_tree, v_tree, seq_lens, n_active, mask: TreeMask,
+                        out: Optional[torch.Tensor] = None, softmax_scale: Optional[float] = None,
+                        workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """out[b][h][n] = attention of tree token n over the prefix cache and its root path (see mcsd.h)."""
+    dt = q.dtype
+    B, H, N, D = q.shape
+    L_max = k_cache.shape[2]
+    for name, t, shape in (("q", q, (B, H, N, D)), ("k_cache", k_cache, (B, H, L_max, D)),
+                           ("v_cache", v_cache, (B, H, L_max, D)), ("k_tree", k_tree, (B, H, N, D)),
+                           ("v_tree", v_tree, (B, H, N, D))):
+        _dev_tensor(t, dt, name)
+        if tuple(t.shape) != shape:
+            raise ValueError("%s has shape %s, expected %s" % (name, tuple(t.shape), shape))
+    _dev_tensor(seq_lens, torch.int32, "seq_lens")
+    if n_active is not None:
+        _dev_tensor(n_active, torch.int32, "n_active")
+    if mask.n_nodes != N:
+        raise ValueError("mask was built for %d nodes, q has %d" % (mask.n_nodes, N))
+    if out is None:
+        out = torch.empty_like(q)
+    code = _dtype_code(q)
+    if softmax_scale is None:
+        softmax_scale = 1.0 / float(np.sqrt(D))
+    need = mcsd_tree_attention_workspace_bytes(B, H, N, D, L_max, code)
+    if workspace is None:
+        workspace = new_workspace(need, q.device)
+    with torch.cuda.device(q.device):
+        st = lib.mcsd_tree_attention(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(k_tree), _ptr(v_tree), _ptr(out),
+                                     _ptr(seq_lens), _ptr(n_active), _ptr(mask.anc), mask.words, B, H, N, D, L_max,
+                                     ctypes.c_float(softmax_scale), code, _ptr(workspace), workspace.numel(), _stream())
+    _check(st, "mcsd_tree_attention")
+    return out
+
+
+def mcsd_workspace_status(workspace: torch.Tensor) -> int:
+    with torch.cuda.device(workspace.device):
+        return int(lib.mcsd_workspace_status(_ptr(workspace), _stream()))
+
+
+def mcsd_verify_tree_workspace_bytes(B, N, V) -> int:
+    return int(lib.mcsd_verify_tree_workspace_bytes(B, N, V))
+
+
+def mcsd_verify_tree(p, q, tokens, mask: TreeMask, gamma, u_accept, u_bonus, R: int = 0,
+                     workspace: Optional[torch.Tensor] = None, out: Optional[dict] = None) -> dict:
+    """Accept/reject walk, longest-path selection and new-token sampling (see mcsd.h). Returns device tensors."""
+    B, N, V = p.shape
+    _dev_tensor(p, torch.float32, "p")
+    _dev_tensor(q, torch.float32, "q")
+    _dev_tensor(tokens, torch.int32, "tokens")
+    _dev_tensor(u_accept, torch.float32, "u_accept")
+    _dev_tensor(u_bonus, torch.float32, "u_bonus")
+    if gamma is not None:
+        _dev_tensor(gamma, torch.int32, "gamma")
+    if mask.n_nodes != N or tuple(q.shape) != (B, N, V) or tuple(tokens.shape) != (B, N):
+        raise ValueError("shape mismatch between p, q, tokens and the tree")
+    dev = p.device
+    nl = mask.n_levels
+    if out is None:
+        out = {
+            "accept_len": torch.empty(B, dtype=torch.int32, device=dev),
+            "out_tokens": torch.empty((B, nl + 1), dtype=torch.int32, device=dev),
+            "out_nodes": torch.empty((B, nl), dtype=torch.int32, device=dev),
+            "best_root": torch.empty(B, dtype=torch.int32, device=dev),
+            "next_roots": torch.empty((B, R), dtype=torch.int32, device=dev) if R > 0 else None,
+        }
+    if workspace is None:
+        workspace = new_workspace(mcsd_verify_tree_workspace_bytes(B, N, V), dev)
+    with torch.cuda.device(dev):
+        st = lib.mcsd_verify_tree(_ptr(p), _ptr(q), _ptr(tokens), _ptr(mask.parent), _ptr(mask.level_start), nl,
+                                  mask.n_roots, _ptr(gamma), _ptr(u_accept), _ptr(u_bonus), B, N, V,
+                                  _ptr(out["accept_len"]), _ptr(out["out_tokens"]), _ptr(out["out_nodes"]),
+                                  _ptr(out["best_root"]), _ptr(out.get("next_roots")), R, _ptr(workspace),
+                                  workspace.numel(), _stream())
+    _check(st, "mcsd_verify_tree")
+    return out
+
+
+def shard_batch(B: int, rank: int, world_size: int):
+    """Sequences [lo, hi) of a batch of B that rank `rank` of `world_size` verifies.
+
+    Sequences are independent in every step of the path, so ranks split the batch and exchange nothing."""
+    if world_size < 1 or not (0 <= rank < world_size):
+        raise ValueError("bad rank/world_size")
+    base, rem = divmod(B, world_size)
+    lo = rank * base + min(rank, rem)
+    return lo, lo + base + (1 if rank < rem else 0)

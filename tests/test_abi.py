@@ -1,0 +1,94 @@
+"""The C ABI library loads, exports every declared symbol, and rejects bad arguments on the host
+before anything is launched (no GPU needed)."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def m():
+    from paper_2409_10644_b200 import build
+    build.build()
+    import paper_2409_10644_b200 as pkg
+    return pkg
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "mcsd.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(mcsd_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(m):
+    names = _declared_functions()
+    assert {"mcsd_build_mask", "mcsd_tree_attention", "mcsd_verify_tree"} <= set(names)
+    for n in names:
+        assert hasattr(m.lib, n), n
+
+
+def test_status_strings(m):
+    seen = {m.mcsd_status_string(s) for s in range(0, -8, -1)}
+    assert len(seen) == 8 and "unknown status" not in seen
+    assert m.mcsd_status_string(-99) == "unknown status"
+
+
+FAKE = ctypes.c_void_p(0x1000)      # never dereferenced: every call below fails its checks first
+
+
+def test_build_mask_rejects_bad_trees_on_the_host(m):
+    def call(parent, n=None, words=1):
+        arr = np.asarray(parent, dtype=np.int32)
+        return m.lib.mcsd_build_mask(arr.ctypes.data_as(ctypes.c_void_p), len(arr) if n is None else n, FAKE, words,
+                                     FAKE, FAKE, None, None, None)
+    assert call([-1, 1]) == -3              # parent not earlier
+    assert call([-1, 0, 1, 0]) == -3        # depth decreases / children not contiguous
+    assert call([-1, -1, 1, 0]) == -3
+    assert call([0, -1]) == -3              # node 0 must be a root
+    assert call([-1, -2]) == -3
+    assert call([-1], n=0) == -2
+    assert call([-1] * 193) == -2
+    assert call([-1] * 65, words=1) == -2   # 65 nodes need two words
+    assert m.lib.mcsd_build_mask(None, 1, FAKE, 1, FAKE, FAKE, None, None, None) == -1
+
+
+def test_attention_argument_checks(m):
+    L = m.lib
+    ws = L.mcsd_tree_attention_workspace_bytes
+    assert ws(1, 4, 15, 64, 128, m.MCSD_F32) >= 256
+    assert ws(1, 4, 15, 96, 128, m.MCSD_F32) == 0          # head_dim must be 64 or 128
+    assert ws(1, 4, 193, 64, 128, m.MCSD_F32) == 0
+    assert ws(1, 4, 15, 64, 128, 7) == 0
+
+    def call(q=FAKE, B=1, H=4, N=15, D=64, Lm=128, dtype=1, wsp=FAKE, wsb=1 << 30, words=1):
+        return L.mcsd_tree_attention(q, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, None, FAKE, words, B, H, N, D, Lm,
+                                     ctypes.c_float(0.125), dtype, wsp, wsb, None)
+    assert call(q=None) == -1
+    assert call(D=96) == -2
+    assert call(N=0) == -2
+    assert call(N=193) == -2
+    assert call(dtype=5) == -4
+    assert call(wsb=16) == -5
+    assert call(wsp=ctypes.c_void_p(0x1010)) == -2      # workspace must be 256-byte aligned
+    assert call(N=100, words=1) == -2
+
+
+def test_verify_argument_checks(m):
+    L = m.lib
+    assert L.mcsd_verify_tree_workspace_bytes(16, 45, 32000) >= 256 + 16 * 45 * 16
+
+    def call(p=FAKE, B=2, N=15, V=100, nl=4, nr=1, R=0, wsb=1 << 20, nxt=None):
+        return L.mcsd_verify_tree(p, FAKE, FAKE, FAKE, FAKE, nl, nr, None, FAKE, FAKE, B, N, V, FAKE, FAKE, FAKE, FAKE,
+                                  nxt, R, FAKE, wsb, None)
+    assert call(p=None) == -1
+    assert call(N=193) == -2
+    assert call(V=0) == -2
+    assert call(nl=0) == -2
+    assert call(nr=0) == -2
+    assert call(R=33, nxt=FAKE) == -2
+    assert call(R=2, nxt=None) == -1
+    assert call(wsb=8) == -5
