@@ -1,0 +1,371 @@
+#!/usr/bin/env python
+"""Benchmark of one-pass token-tree verification (mask slice -> tree attention over all layers -> accept/reject).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One step = one verification pass of the whole path over one batch of the synthetic workload: the tree
+attention of every layer (independent, seeded KV caches resident in HBM) followed by the accept/reject
+walk.  The mask is built once before the timed region (the paper builds it at initialisation, Section 3.2)
+and sliced per sequence by a row count.  The default workload is the long-context one (batch 16, 32 heads
+x 128, 4096-token prefix, tree (1; 4,2,2,1), 32 layers).  With N > 1 (torchrun) every rank verifies its own
+batch of the same size (weak scaling, no data-path collective).
+
+`--impl reference` times the CPU oracle (fp64, numpy) on a bounded sample of the same workload.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "tree_verify_tree_tokens_per_s"
+UNIT = "tree-tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[1]))
+                mx.append(float(r[2]))
+            except Exception:
+                continue
+            for name, col in (("hw_slowdown", 5), ("hw_thermal_slowdown", 6), ("sw_thermal_slowdown", 7),
+                              ("sw_power_cap", 8)):
+                if len(r) > col and r[col].lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def _algorithmic_bytes_attention(H, D, lens, n_act, words, elt):
+    """Bytes one tree-attention call must move: K and V rows of prefix and tree, Q read, O write, mask words."""
+    kv = sum(H * (int(l) + int(n)) * D * 2 * elt for l, n in zip(lens, n_act))
+    qo = sum(H * int(n) * D * 2 * elt for n in n_act)
+    return kv + qo + sum(int(n) * words * 8 for n in n_act)
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle on a bounded sample (reported baseline; also the `--impl reference` arm)
+# ------------------------------------------------------------------------------------------------
+
+def oracle_sample(w, budget_s=12.0, min_pairs=8):
+    """Times the oracle, as it stands, on (sequence, head) attention problems and on verify sequences of
+    workload `w`, and extrapolates to a full step.  Returns (tree-tokens/s, description, threads)."""
+    import torch
+    from mcsd_inputs import attention_inputs, gammas, parent_array, seq_lens, verify_inputs
+    from oracle import mcsd_oracle as orc
+    parent = parent_array(w.n_roots, w.branching)
+    N = len(parent)
+    lens = seq_lens(w)
+    gam = gammas(w)
+    n_act = np.array([orc.n_active_for_gamma(parent, int(g)) for g in gam])
+    scale = 1.0 / np.sqrt(w.D)
+    # attention: one (b, h) problem at a time, drawn with the workload's seeded generator
+    t_attn, pairs = 0.0, 0
+    wb = dataclasses.replace(w, B=1, H=1)
+    while pairs < min_pairs or (t_attn < budget_s and pairs < w.B * w.H * w.n_layers):
+        b = pairs % w.B
+        one = dataclasses.replace(wb, base_seed=w.seed(0, 0) + 7919 * pairs, prefix=(int(lens[b]), int(lens[b])))
+        inp = {k: v.float().numpy() for k, v in attention_inputs(one, 0, "cpu").items()}
+        t0 = time.perf_counter()
+        orc.tree_attention(inp["q"], inp["k_cache"], inp["v_cache"], inp["k_tree"], inp["v_tree"], [int(lens[b])],
+                           [int(n_act[b])], parent, scale)
+        t_attn += time.perf_counter() - t0
+        pairs += 1
+    # verify: whole sequences
+    nseq = min(w.B, 4)
+    vin = verify_inputs(w, 0, "cpu", parent=parent, B=nseq)
+    host = {k: v.numpy() for k, v in vin.items()}
+    t0 = time.perf_counter()
+    orc.verify_tree(host["p"], host["q"], host["tokens"], parent, gam[:nseq], host["u_accept"], host["u_bonus"])
+    t_ver = time.perf_counter() - t0
+    step_s = t_attn / pairs * (w.B * w.H * w.n_layers) + t_ver / nseq * w.B
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([int(i.get("num_threads", 1)) for i in threadpool_info()] or [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    sample = ("%d of %d (sequence, head, layer) attention problems (%.1f s) and %d of %d verify sequences (%.2f s), "
+              "extrapolated to one full step" % (pairs, w.B * w.H * w.n_layers, t_attn, nseq, w.B, t_ver))
+    return float(n_act.sum()) / step_s, sample, threads, step_s
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from mcsd_inputs import workload
+    w = workload(args.workload)
+    vals = []
+    for i in range(args.warmup + args.steps):
+        v, sample, threads, step_s = oracle_sample(w, budget_s=max(2.0, 60.0 / max(1, args.warmup + args.steps)))
+        if i >= args.warmup:
+            vals.append((v, step_s))
+    value = float(np.mean([v for v, _ in vals]))
+    ms = float(np.mean([s for _, s in vals])) * 1e3
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": _config(w, args.gpus),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def _config(w, n_gpus):
+    return {"workload": w.name, "batch_per_gpu": w.B, "heads": w.H, "head_dim": w.D, "prefix": list(w.prefix),
+            "tree": {"n_roots": w.n_roots, "branching": list(w.branching), "nodes": w.n_nodes},
+            "layers": w.n_layers, "vocab": w.V, "parallelism": "batch-sharded x%d, no collective" % n_gpus,
+            "l2": "inputs larger than L2: every layer reads its own %.0f MB KV cache" %
+                  (2 * w.B * w.H * w.L_max * w.D * (4 if w.dtype == "f32" else 2) / 1e6)}
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    import paper_2409_10644_b200 as mcsd
+    from paper_2409_10644_b200.dist import aggregate
+    from mcsd_inputs import attention_inputs, gammas, parent_array, seq_lens, verify_inputs, workload
+
+    w0 = workload(args.workload)
+    w = dataclasses.replace(w0, base_seed=1000 * w0.index + 100000 * rank)
+    parent = parent_array(w.n_roots, w.branching)
+    N = len(parent)
+    elt = 4 if w.dtype == "f32" else 2
+    code = mcsd.MCSD_F32 if w.dtype == "f32" else mcsd.MCSD_BF16
+
+    # ---- init (untimed): mask once, resident KV caches, per-step inputs staged in pinned host memory ----
+    tm = mcsd.mcsd_build_mask(parent, device=dev)
+    lens = seq_lens(w)
+    gam = gammas(w)
+    n_act = mcsd.n_active_from_gamma(tm.level_start_host, gam)
+    lens_d = torch.from_numpy(lens).to(dev)
+    nact_d = torch.from_numpy(n_act).to(dev)
+    gam_d = torch.from_numpy(gam).to(dev)
+    layers = [attention_inputs(w, l, dev) for l in range(w.n_layers)]
+    vin = verify_inputs(w, 0, dev, parent=parent)
+    outs = [torch.empty_like(l["q"]) for l in layers]
+    ws_attn = mcsd.new_workspace(mcsd.mcsd_tree_attention_workspace_bytes(w.B, w.H, N, w.D, w.L_max, code), dev)
+    ws_ver = mcsd.new_workspace(mcsd.mcsd_verify_tree_workspace_bytes(w.B, N, w.V), dev)
+    vout = mcsd.mcsd_verify_tree(vin["p"], vin["q"], vin["tokens"], tm, gam_d, vin["u_accept"], vin["u_bonus"],
+                                 workspace=ws_ver)
+    scale = 1.0 / float(np.sqrt(w.D))
+
+    def step(timed_events=None):
+        for l, (inp, o) in enumerate(zip(layers, outs)):
+            if timed_events is not None:
+                timed_events[l][0].record()
+            mcsd.mcsd_tree_attention(inp["q"], inp["k_cache"], inp["v_cache"], inp["k_tree"], inp["v_tree"], lens_d,
+                                     nact_d, tm, out=o, softmax_scale=scale, workspace=ws_attn)
+            if timed_events is not None:
+                timed_events[l][1].record()
+        mcsd.mcsd_verify_tree(vin["p"], vin["q"], vin["tokens"], tm, gam_d, vin["u_accept"], vin["u_bonus"],
+                              workspace=ws_ver, out=vout)
+
+    def sync_all():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    sync_all()
+    if mcsd.mcsd_workspace_status(ws_attn) != 0 or mcsd.mcsd_workspace_status(ws_ver) != 0:
+        raise SystemExit("a device-side wait timed out during warm-up; results would be invalid")
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in layers]
+          for _ in range(args.steps)]
+    ver_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    launches0 = mcsd.mcsd_launch_count()
+    t_start.record()
+    for k in range(args.steps):
+        step(ev[k])
+        ver_ev[k][1].record()
+    t_end.record()
+    sync_all()
+    launches = mcsd.mcsd_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    ms_local = t_start.elapsed_time(t_end) / args.steps
+    attn_ms = float(np.mean([a.elapsed_time(b) for per in ev for (a, b) in per]))
+    ver_ms = float(np.mean([ev[k][-1][1].elapsed_time(ver_ev[k][1]) for k in range(args.steps)]))
+    if mcsd.mcsd_workspace_status(ws_attn) != 0:
+        raise SystemExit("a device-side wait timed out; results are invalid")
+
+    units, ms = aggregate(float(n_act.sum()), ms_local, device=dev)
+    value = units / (ms * 1e-3)
+
+    # ---- end to end: per-step inputs come from pinned host memory, results go back to the host ----
+    pin = lambda t: t.detach().cpu().pin_memory()
+    h_layers = [{k: pin(l[k]) for k in ("q", "k_tree", "v_tree")} for l in layers]
+    h_vin = {k: pin(v) for k, v in vin.items()}
+    h_lens, h_gam, h_nact = pin(lens_d), pin(gam_d), pin(nact_d)
+    h_outs = [torch.empty(o.shape, dtype=o.dtype).pin_memory() for o in outs]
+    h_vout = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in vout.items() if v is not None}
+    h2d = sum(t.numel() * t.element_size() for l in h_layers for t in l.values()) + \
+        sum(t.numel() * t.element_size() for t in h_vin.values()) + 3 * 4 * w.B
+    d2h = sum(t.numel() * t.element_size() for t in h_outs) + sum(t.numel() * t.element_size() for t in h_vout.values())
+
+    def e2e_step():
+        lens_d.copy_(h_lens, non_blocking=True)
+        gam_d.copy_(h_gam, non_blocking=True)
+        nact_d.copy_(h_nact, non_blocking=True)
+        for l, hl in zip(layers, h_layers):
+            for k, t in hl.items():
+                l[k].copy_(t, non_blocking=True)
+        for k, t in h_vin.items():
+            vin[k].copy_(t, non_blocking=True)
+        step()
+        for o, ho in zip(outs, h_outs):
+            ho.copy_(o, non_blocking=True)
+        for k, t in h_vout.items():
+            t.copy_(vout[k], non_blocking=True)
+
+    e2e_steps = max(2, min(args.steps, 5))
+    e2e_step()
+    sync_all()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    sync_all()
+    e2e_units, e2e_ms = aggregate(float(n_act.sum()), e0.elapsed_time(e1) / e2e_steps, device=dev)
+    e2e_value = e2e_units / (e2e_ms * 1e-3)
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = _peaks()
+    abytes = _algorithmic_bytes_attention(w.H, w.D, lens, n_act, tm.words, elt)
+    achieved = abytes / (attn_ms * 1e-3) / 1e9
+    ver_rows_bytes = int(n_act.sum()) * w.V * 4 * 2
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic", "config": _config(w, world),
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                "ms_per_step": e2e_ms,
+                "note": "per step the tree's q/k/v of every layer, p, q, tokens, uniforms, lengths and gammas are copied "
+                        "from pinned host memory and every layer's attention output plus the verify results are read "
+                        "back; the prefix KV cache is decode state and stays resident in HBM"},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": {"bound": "hbm", "kernel": "tree attention (one layer: main kernel + split-KV combine)",
+                     "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
+                     "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                     "algorithmic_bytes_per_launch": int(abytes), "avg_launch_ms": attn_ms, "traffic": None},
+        "breakdown": {"attention_ms_per_layer": attn_ms, "verify_ms": ver_ms,
+                      "verify_nodes_per_s": float(n_act.sum()) / (ver_ms * 1e-3),
+                      "verify_all_rows_GBs": ver_rows_bytes / (ver_ms * 1e-3) / 1e9,
+                      "tree_tokens_per_s_per_layer": float(n_act.sum()) / (attn_ms * 1e-3),
+                      "mean_accept_len": float(vout["accept_len"].float().mean().item())},
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        v, sample, threads, _ = oracle_sample(w0)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample}
+    print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="long_context_b16")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -58,6 +58,12 @@ const char* mcsd_status_string(int status);
 int mcsd_last_cuda_error(void);
 
 /*
+ * Number of kernels this process has launched through the library so far (all threads, all devices).
+ * Bookkeeping for benchmarks that report how many launches a step of Fig. 1's verification costs.
+ */
+long long mcsd_launch_count(void);
+
+/*
  * Topology-aware causal mask (Section 2.2; Fig. 1 step 2), built once for the deepest tree (Section 3.2).
  *
  *   parent_host      [host] int32[n_nodes], level order, -1 for roots.  Validated on the CPU before anything

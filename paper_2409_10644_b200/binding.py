@@ -22,7 +22,7 @@ MCSD_MAX_NODES = 192
 MCSD_MAX_WORDS = 3
 
 _EXPORTS = (
-    "mcsd_status_string", "mcsd_last_cuda_error", "mcsd_build_mask", "mcsd_tree_attention_workspace_bytes",
+    "mcsd_status_string", "mcsd_last_cuda_error", "mcsd_launch_count", "mcsd_build_mask", "mcsd_tree_attention_workspace_bytes",
     "mcsd_tree_attention", "mcsd_workspace_status", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree",
 )
 
@@ -38,6 +38,8 @@ def _load() -> ctypes.CDLL:
     lib.mcsd_status_string.argtypes = [c_int]
     lib.mcsd_last_cuda_error.restype = c_int
     lib.mcsd_last_cuda_error.argtypes = []
+    lib.mcsd_launch_count.restype = ctypes.c_longlong
+    lib.mcsd_launch_count.argtypes = []
     lib.mcsd_build_mask.restype = c_int
     lib.mcsd_build_mask.argtypes = [c_void_p, c_int, c_void_p, c_int, c_void_p, c_void_p, c_void_p,
                                     ctypes.POINTER(c_int), c_void_p]
@@ -69,6 +71,10 @@ class McsdError(RuntimeError):
 
 def mcsd_status_string(status: int) -> str:
     return lib.mcsd_status_string(int(status)).decode()
+
+
+def mcsd_launch_count() -> int:
+    return int(lib.mcsd_launch_count())
 
 
 def _check(status: int, where: str):

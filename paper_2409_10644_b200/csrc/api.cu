@@ -1,9 +1,13 @@
 // Status reporting of libmcsd.
+#include <atomic>
+
 #include "common.cuh"
 
 namespace mcsd {
 static thread_local int g_last_cuda_error = 0;
 void set_last_cuda_error(cudaError_t e) { g_last_cuda_error = static_cast<int>(e); }
+static std::atomic<long long> g_launches{0};
+void count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 }  // namespace mcsd
 
 extern "C" const char* mcsd_status_string(int status) {
@@ -21,6 +25,8 @@ extern "C" const char* mcsd_status_string(int status) {
 }
 
 extern "C" int mcsd_last_cuda_error(void) { return mcsd::g_last_cuda_error; }
+
+extern "C" long long mcsd_launch_count(void) { return mcsd::g_launches.load(std::memory_order_relaxed); }
 
 extern "C" int mcsd_workspace_status(const void* workspace, void* stream) {
     if (workspace == nullptr) return MCSD_ERR_NULL;

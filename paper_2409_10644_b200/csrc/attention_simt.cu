@@ -192,10 +192,12 @@ static int launch_simt(const AttentionArgs& a, void* scratch, cudaStream_t strea
         static_cast<const T*>(a.k_tree), static_cast<const T*>(a.v_tree), static_cast<T*>(a.out), a.seq_lens,
         a.n_active, a.anc, a.words, a.H, a.N, a.L_max, a.scale, splits, part_ml, part_acc);
     MCSD_CUDA_CHECK(cudaGetLastError());
+    count_launches(1);
     if (splits > 1) {
         tree_attention_simt_combine_kernel<T, D><<<dim3(a.N, a.B * a.H), 32, 0, stream>>>(
             static_cast<T*>(a.out), a.n_active, a.H, a.N, splits, part_ml, part_acc);
         MCSD_CUDA_CHECK(cudaGetLastError());
+        count_launches(1);
     }
     return MCSD_OK;
 }

@@ -17,6 +17,7 @@ struct WorkspaceHeader {
 static_assert(sizeof(WorkspaceHeader) == 256, "workspace header is one 256-byte line");
 
 void set_last_cuda_error(cudaError_t e);
+void count_launches(int n);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

@@ -70,5 +70,6 @@ extern "C" int mcsd_build_mask(const int32_t* parent_host, int n_nodes, uint64_t
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     mcsd::build_mask_kernel<<<1, MCSD_MAX_NODES, 0, s>>>(tree, n_nodes, words, anc_dev, depth_dev, level_start_dev);
     MCSD_CUDA_CHECK(cudaGetLastError());
+    mcsd::count_launches(1);
     return MCSD_OK;
 }

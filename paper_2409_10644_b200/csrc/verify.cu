@@ -330,5 +330,6 @@ extern "C" int mcsd_verify_tree(const float* p, const float* q, const int32_t* t
                                                                  accept_len, out_tokens, out_nodes, best_root,
                                                                  R > 0 ? next_roots : nullptr, R);
     MCSD_CUDA_CHECK(cudaGetLastError());
+    mcsd::count_launches(2);
     return MCSD_OK;
 }

@@ -1,0 +1,312 @@
+"""GPU parity: the CUDA library, called through its C ABI binding, against the CPU oracle on the same seeded inputs.
+
+Bars: mask bits, accepted lengths, node and token ids bit-exact; attention within max-abs 2e-2 for bf16
+tensors (fp32 accumulation) and 1e-4 for fp32 tensors.  Because the bf16 workloads have outputs of
+magnitude ~1e-3, each of them is also run with unit-variance q/k/v under a relative bound, and a "needle"
+input reads the mask out of the attention output directly."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from mcsd_inputs import attention_inputs, gammas, parent_array, seq_lens, verify_inputs, workload
+from oracle import mcsd_oracle as orc
+from tests.helpers import condition_uniforms, oracle_attention_rows, to_np
+
+pytestmark = pytest.mark.gpu
+
+TOL_BF16 = 2e-2
+TOL_F32 = 1e-4
+
+
+@pytest.fixture(scope="module")
+def m():
+    from paper_2409_10644_b200 import build
+    build.build()
+    import paper_2409_10644_b200 as pkg
+    return pkg
+
+
+def _random_bfs_parent(rng, N, n_roots):
+    parent = [-1] * n_roots
+    lo, hi = 0, n_roots
+    while len(parent) < N:
+        start = len(parent)
+        n_new = min(int(rng.integers(1, 3 * (hi - lo) + 1)), N - start)
+        parent.extend(int(x) for x in np.sort(rng.integers(lo, hi, size=n_new)))
+        lo, hi = start, len(parent)
+    return np.asarray(parent[:N], dtype=np.int32)
+
+
+# ----------------------------------------------------------------------------------------------
+# mask
+# ----------------------------------------------------------------------------------------------
+
+def _check_mask(m, parent):
+    tm = m.mcsd_build_mask(parent)
+    torch.cuda.synchronize()
+    depth, ls = orc.tree_levels(parent)
+    bits = orc.pack_bitsets(orc.dense_mask(parent))
+    got = tm.anc.cpu().numpy().view(np.uint64)
+    assert np.array_equal(got[:, :bits.shape[1]], bits)
+    assert not got[:, bits.shape[1]:].any()
+    assert np.array_equal(tm.depth.cpu().numpy(), depth)
+    assert tm.n_levels == len(ls) - 1
+    assert np.array_equal(tm.level_start.cpu().numpy()[:len(ls)], ls)
+    assert np.array_equal(tm.level_start_host, ls)
+    return tm
+
+
+def test_mask_bits_for_all_workload_trees(m):
+    for i in range(1, 6):
+        w = workload(i)
+        _check_mask(m, parent_array(w.n_roots, w.branching))
+    _check_mask(m, parent_array(2, (4, 3, 1, 1)))
+    _check_mask(m, parent_array(16, (1, 1, 1, 1)))
+
+
+@pytest.mark.parametrize("N", [1, 2, 63, 64, 65, 128, 129, 191, 192])
+def test_mask_bits_random_trees(m, N):
+    rng = np.random.default_rng(N)
+    tm = _check_mask(m, _random_bfs_parent(rng, N, int(rng.integers(1, min(N, 9) + 1))))
+    assert tm.words == (N + 63) // 64
+
+
+def test_sliced_mask_is_a_row_count(m):
+    # Section 3.2: rows/columns [0, n_active) of the big mask are the mask of the truncated tree
+    w = workload(3)
+    parent = parent_array(w.n_roots, w.branching)
+    tm = m.mcsd_build_mask(parent)
+    big = tm.anc.cpu().numpy().view(np.uint64)
+    for gamma in range(len(w.branching) + 1):
+        nb = int(m.n_active_from_gamma(tm.level_start_host, [gamma])[0])
+        small = m.mcsd_build_mask(parent_array(w.n_roots, w.branching[:gamma]), words=tm.words)
+        assert np.array_equal(big[:nb], small.anc.cpu().numpy().view(np.uint64))
+
+
+# ----------------------------------------------------------------------------------------------
+# attention
+# ----------------------------------------------------------------------------------------------
+
+def _run_attention(m, w, inp, lens, n_act, parent, scale=None):
+    tm = m.mcsd_build_mask(parent)
+    dev = inp["q"].device
+    lens_d = torch.from_numpy(np.asarray(lens, dtype=np.int32)).to(dev)
+    na_d = None if n_act is None else torch.from_numpy(np.asarray(n_act, dtype=np.int32)).to(dev)
+    B, H, N, D = inp["q"].shape
+    code = m.MCSD_F32 if inp["q"].dtype == torch.float32 else m.MCSD_BF16
+    ws = torch.zeros(m.mcsd_tree_attention_workspace_bytes(B, H, N, D, inp["k_cache"].shape[2], code),
+                     dtype=torch.uint8, device=dev)
+    out = torch.full_like(inp["q"], float("nan"))
+    m.mcsd_tree_attention(inp["q"], inp["k_cache"], inp["v_cache"], inp["k_tree"], inp["v_tree"], lens_d, na_d, tm,
+                          out=out, softmax_scale=scale, workspace=ws)
+    assert m.mcsd_workspace_status(ws) == 0
+    return out
+
+
+def _compare_attention(out, ref_rows, n_act, N, tol_abs, rel=False):
+    worst = 0.0
+    for (b, h), ref in ref_rows.items():
+        nb = N if n_act is None else int(n_act[b])
+        got = to_np(out[b, h]).astype(np.float64)
+        if nb > 0:
+            err = np.abs(got[:nb] - ref[:nb])
+            assert np.isfinite(got[:nb]).all()
+            if rel:
+                scale = np.abs(ref[:nb]).max()
+                assert err.max() <= tol_abs * scale, (b, h, err.max(), scale)
+                rms = np.sqrt((err ** 2).mean()) / np.sqrt((ref[:nb] ** 2).mean())
+                assert rms <= 1e-2, (b, h, rms)
+            else:
+                assert err.max() <= tol_abs, (b, h, err.max())
+            worst = max(worst, err.max())
+        assert np.isnan(got[nb:]).all()          # rows beyond n_active are not written
+    return worst
+
+
+def _all_pairs(B, H):
+    return [(b, h) for b in range(B) for h in range(H)]
+
+
+def _full_attention_case(m, w, std=None, rel=False, lens=None, n_act="gamma", pairs=None, poison=False):
+    parent = parent_array(w.n_roots, w.branching)
+    inp = attention_inputs(w, 0, "cuda", std=std)
+    lens = seq_lens(w) if lens is None else np.asarray(lens, dtype=np.int32)
+    if isinstance(n_act, str):
+        _, ls = orc.tree_levels(parent)
+        n_act = None if w.gamma is None else np.array([orc.n_active_for_gamma(parent, int(g)) for g in gammas(w)])
+    if poison:                                   # cache rows past the prefix may hold anything
+        for b in range(w.B):
+            inp["k_cache"][b, :, int(lens[b]):] = float("nan")
+            inp["v_cache"][b, :, int(lens[b]):] = float("nan")
+    scale = 1.0 / np.sqrt(w.D)
+    out = _run_attention(m, w, inp, lens, n_act, parent, scale)
+    pairs = _all_pairs(w.B, w.H) if pairs is None else pairs
+    ref = oracle_attention_rows(inp, lens, n_act, parent, scale, pairs)
+    tol = TOL_F32 if w.dtype == "f32" else TOL_BF16
+    return _compare_attention(out, ref, n_act, len(parent), tol, rel=rel)
+
+
+def test_attention_tiny_fp32(m):
+    _full_attention_case(m, workload(1))
+
+
+def test_attention_llama7b_b1(m):
+    _full_attention_case(m, workload(2))
+    _full_attention_case(m, workload(2), std=1.0, rel=True)
+
+
+def test_attention_dynamic_slice_reduced(m):
+    # several key tiles plus a ragged tail, per-sequence gamma slices of the 109-node tree
+    w = dataclasses.replace(workload(3), B=3, H=4, prefix=(300, 300))
+    _full_attention_case(m, w, poison=True)
+    _full_attention_case(m, w, std=1.0, rel=True, poison=True)
+
+
+def test_attention_target_init_reduced(m):
+    # ragged prefixes, 8 roots, 160-node tree sliced per sequence
+    w = dataclasses.replace(workload(5), B=4, H=3, prefix=(5, 700))
+    _full_attention_case(m, w, poison=True)
+    _full_attention_case(m, w, std=1.0, rel=True, poison=True)
+
+
+def test_attention_edge_cases(m):
+    w = dataclasses.replace(workload(2), B=4, H=2, prefix=(0, 260))
+    parent = parent_array(w.n_roots, w.branching)
+    N = len(parent)
+    # empty prefix, one-token prefix, exact tile multiple, ragged; empty and one-node trees
+    _full_attention_case(m, w, std=1.0, rel=True, lens=[0, 1, 256, 259], n_act=np.array([N, 5, 0, 1]), poison=True)
+    # head_dim 64 in bf16 and head_dim 128 in fp32 take the CUDA-core kernel
+    _full_attention_case(m, dataclasses.replace(w, D=64), std=1.0, rel=True, lens=[7, 130, 33, 260])
+    w32 = dataclasses.replace(workload(1), D=128, B=2, prefix=(40, 90))
+    _full_attention_case(m, w32, lens=[40, 90])
+    # largest tree
+    wmax = dataclasses.replace(w, n_roots=8, branching=(1, 2, 2, 1, 1, 1, 1), B=2, prefix=(150, 150))
+    assert wmax.n_nodes == 192
+    _full_attention_case(m, wmax, std=1.0, rel=True, n_act=None)
+
+
+def test_attention_needle_reads_out_the_mask(m):
+    # tree keys share one large score and carry one-hot values, the prefix scores 0 and carries zeros:
+    # out[n][j] = 1/(depth(n)+1) exactly where node n may see node j
+    for idx in (2, 3):
+        w = workload(idx)
+        parent = parent_array(w.n_roots, w.branching)
+        N = len(parent)
+        B, H, D, L = 2, 2, 128, 333
+        dev = "cuda"
+        z = lambda *s: torch.zeros(s, dtype=torch.bfloat16, device=dev)
+        q, kc, vc, kt, vt = z(B, H, N, D), z(B, H, L, D), z(B, H, L, D), z(B, H, N, D), z(B, H, N, D)
+        q[..., 0] = 8.0
+        kt[..., 0] = 8.0
+        g = torch.Generator(device=dev).manual_seed(3)
+        kc[..., 1:] = torch.randn((B, H, L, D - 1), generator=g, device=dev).to(torch.bfloat16)
+        for j in range(min(N, D)):
+            vt[:, :, j, j] = 1.0
+        inp = {"q": q, "k_cache": kc, "v_cache": vc, "k_tree": kt, "v_tree": vt}
+        lens = [L, 77]
+        out = _run_attention(m, w, inp, lens, None, parent, scale=1.0)
+        ref = oracle_attention_rows(inp, lens, None, parent, 1.0, _all_pairs(B, H))
+        mask = orc.dense_mask(parent)
+        depth, _ = orc.tree_levels(parent)
+        for (b, h), r in ref.items():
+            got = to_np(out[b, h]).astype(np.float64)
+            assert np.abs(got - r).max() <= 4e-3
+            expect = mask[:, :min(N, D)] / (depth[:, None] + 1.0)
+            assert np.abs(got[:, :min(N, D)] - expect).max() <= 4e-3
+
+
+@pytest.mark.parametrize("idx", [3, 4, 5])
+def test_attention_full_size_sampled(m, idx):
+    # the workload at its full size, in the launch configuration the benchmark times; the oracle
+    # checks a seeded sample of (sequence, head) pairs, every row of each
+    w = workload(idx)
+    rng = np.random.default_rng(idx)
+    pairs = sorted({(int(rng.integers(w.B)), int(rng.integers(w.H))) for _ in range(6)} | {(0, 0), (w.B - 1, w.H - 1)})
+    _full_attention_case(m, w, pairs=pairs)
+    _full_attention_case(m, w, std=1.0, rel=True, pairs=pairs)
+    torch.cuda.empty_cache()
+
+
+# ----------------------------------------------------------------------------------------------
+# accept / reject
+# ----------------------------------------------------------------------------------------------
+
+def _verify_case(m, w, parent=None, B=None, V=None, gamma="workload", R=0, tweak=None, step=0):
+    parent = parent_array(w.n_roots, w.branching) if parent is None else parent
+    vin = verify_inputs(w, step, "cuda", parent=parent, B=B, V=V)
+    B = vin["p"].shape[0]
+    if isinstance(gamma, str):
+        gamma = None if w.gamma is None else gammas(dataclasses.replace(w, B=B), step)
+    if tweak is not None:
+        tweak(vin)
+    host = {k: to_np(v) for k, v in vin.items()}
+    ua, ub = condition_uniforms(host["p"], host["q"], host["tokens"], parent, gamma, host["u_accept"], host["u_bonus"])
+    ref = orc.verify_tree(host["p"], host["q"], host["tokens"], parent, gamma, ua, ub, R=R)
+    tm = m.mcsd_build_mask(parent)
+    dev = vin["p"].device
+    g_d = None if gamma is None else torch.from_numpy(np.asarray(gamma, dtype=np.int32)).to(dev)
+    got = m.mcsd_verify_tree(vin["p"], vin["q"], vin["tokens"], tm, g_d, torch.from_numpy(ua).to(dev),
+                             torch.from_numpy(ub).to(dev), R=R)
+    torch.cuda.synchronize()
+    for k in ("accept_len", "out_tokens", "out_nodes", "best_root"):
+        assert np.array_equal(got[k].cpu().numpy(), ref[k]), k
+    if R > 0:
+        assert np.array_equal(got["next_roots"].cpu().numpy(), ref["next_roots"])
+    return ref
+
+
+def test_verify_tiny_fp32_workload(m):
+    _verify_case(m, workload(1), R=4)
+
+
+def test_verify_llama7b_b1(m):
+    ref = _verify_case(m, workload(2), R=8)
+    assert ref["accept_len"][0] >= 0
+
+
+def test_verify_dynamic_slice(m):
+    _verify_case(m, workload(3))
+    _verify_case(m, workload(3), step=1, R=2)
+
+
+def test_verify_long_context_batch(m):
+    ref = _verify_case(m, workload(4))
+    assert ref["accept_len"].max() > 0          # the workload does accept draft tokens
+
+
+def test_verify_target_initialised_forest(m):
+    ref = _verify_case(m, workload(5), R=8)
+    assert len(set(ref["best_root"].tolist())) > 1
+    torch.cuda.empty_cache()
+
+
+def test_verify_edge_cases(m):
+    w = workload(1)
+    # vocabulary sizes that are not a multiple of four take the scalar-load path
+    for V in (5, 13, 1001):
+        _verify_case(m, w, B=3, V=V, R=3)
+    # gamma = 0: nothing is tested, the new token comes from the root's own row
+    ref = _verify_case(m, w, B=2, gamma=np.array([0, 2]))
+    assert ref["accept_len"][0] == 0
+    # one-node tree
+    _verify_case(m, w, parent=np.array([-1], dtype=np.int32), B=2, R=2)
+    # draft equal to target: every first candidate is accepted down to the leaves
+    def same(vin):
+        vin["q"].copy_(vin["p"])
+    ref = _verify_case(m, w, B=2, tweak=same)
+    assert list(ref["accept_len"]) == [3, 3]
+    # draft mass on a token the target never emits: all rejected, residual equals the target row
+    def disjoint(vin):
+        vin["p"][:, :, 0] = 0.0
+        vin["p"].div_(vin["p"].sum(-1, keepdim=True))
+        vin["q"].zero_()
+        vin["q"][:, :, 0] = 1.0
+        vin["tokens"][:, 1:] = 0
+    ref = _verify_case(m, w, B=2, tweak=disjoint)
+    assert list(ref["accept_len"]) == [0, 0]
+    # fork-shaped tree of Section 3.2 with 16 chains, and the static (2; 4,3,1,1) configuration of Section 4.1
+    w5 = workload(5)
+    _verify_case(m, w5, parent=parent_array(16, (1, 1, 1, 1)), B=4, V=2000, gamma=np.array([4, 1, 2, 0]))
+    _verify_case(m, w5, parent=parent_array(2, (4, 3, 1, 1)), B=4, V=2000, gamma=None, R=2)
