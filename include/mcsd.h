@@ -47,6 +47,7 @@ extern "C" {
 #define MCSD_ERR_WORKSPACE_TOO_SMALL  -5
 #define MCSD_ERR_CUDA                 -6  /* a CUDA runtime/driver call failed; see mcsd_last_cuda_error() */
 #define MCSD_ERR_TIMEOUT              -7  /* a bounded device-side wait ran out (reported by mcsd_workspace_status) */
+#define MCSD_ERR_STATIC_LIMIT         -8  /* problem exceeds the built-in scratch of a *_static entry point */
 
 #define MCSD_MAX_NODES   192              /* largest tree (roots included) */
 #define MCSD_MAX_WORDS   3                /* 64-bit mask words per node for MCSD_MAX_NODES */
@@ -171,6 +172,38 @@ int mcsd_verify_tree(const float* p, const float* q,
                      int32_t* accept_len, int32_t* out_tokens, int32_t* out_nodes,
                      int32_t* best_root, int32_t* next_roots, int R,
                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * mcsd_verify_tree with built-in scratch.  (The paper has no counterpart; this is a deployment convenience.)
+ *
+ * Same computation, arguments and results as mcsd_verify_tree, minus the workspace: the per-node scratch
+ * lives in a fixed array inside the library image.  It is meant for callers that must not, or cannot,
+ * obtain device memory at the point of the call: a serving engine that handed all of HBM to its KV-cache
+ * pool at start-up so that a later cudaMalloc fails, a plug-in running under a host framework that owns the
+ * allocator, or a latency-critical loop where an allocation's implicit synchronisation is not acceptable.
+ * The call itself performs no cudaMalloc/cudaFree and calls no allocating library routine.
+ *
+ *   limit      B * N <= MCSD_STATIC_VERIFY_MAX_STATES, otherwise MCSD_ERR_STATIC_LIMIT is returned and
+ *              nothing is launched.  The array costs about 256 KB on every GPU that loads the library, for
+ *              the life of the process.
+ *   first call The first call on each device looks up the array's device address (with that device
+ *              current); make that first call outside any stream capture.
+ *   sharing    All calls on one device use the same array, which still holds the previous call's contents;
+ *              the entry point clears the part that has to start at zero.  Two calls that can overlap on the
+ *              GPU (different streams, no dependency) race on it: order them, or use mcsd_verify_tree with
+ *              separate workspaces.
+ * Other errors: as mcsd_verify_tree.
+ */
+#define MCSD_STATIC_VERIFY_MAX_STATES 16384
+
+int mcsd_verify_tree_static(const float* p, const float* q,
+                            const int32_t* tokens, const int32_t* parent, const int32_t* level_start,
+                            int n_levels, int n_roots, const int32_t* gamma,
+                            const float* u_accept, const float* u_bonus,
+                            int B, int N, int V,
+                            int32_t* accept_len, int32_t* out_tokens, int32_t* out_nodes,
+                            int32_t* best_root, int32_t* next_roots, int R,
+                            void* stream);
 
 #ifdef __cplusplus
 }

@@ -23,7 +23,7 @@ MCSD_MAX_WORDS = 3
 
 _EXPORTS = (
     "mcsd_status_string", "mcsd_last_cuda_error", "mcsd_launch_count", "mcsd_build_mask", "mcsd_tree_attention_workspace_bytes",
-    "mcsd_tree_attention", "mcsd_workspace_status", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree",
+    "mcsd_tree_attention", "mcsd_workspace_status", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_static",
 )
 
 
@@ -54,6 +54,9 @@ def _load() -> ctypes.CDLL:
     lib.mcsd_verify_tree.restype = c_int
     lib.mcsd_verify_tree.argtypes = ([c_void_p] * 5 + [c_int, c_int] + [c_void_p] * 3 + [c_int] * 3 +
                                      [c_void_p] * 5 + [c_int, c_void_p, c_size_t, c_void_p])
+    lib.mcsd_verify_tree_static.restype = c_int
+    lib.mcsd_verify_tree_static.argtypes = ([c_void_p] * 5 + [c_int, c_int] + [c_void_p] * 3 + [c_int] * 3 +
+                                            [c_void_p] * 5 + [c_int, c_void_p])
     return lib
 
 
@@ -230,6 +233,23 @@ def mcsd_verify_tree(p, q, tokens, mask: TreeMask, gamma, u_accept, u_bonus, R: 
                                   _ptr(out["best_root"]), _ptr(out.get("next_roots")), R, _ptr(workspace),
                                   workspace.numel(), _stream())
     _check(st, "mcsd_verify_tree")
+    return out
+
+
+def mcsd_verify_tree_static(p, q, tokens, mask: TreeMask, gamma, u_accept, u_bonus, out: dict, R: int = 0) -> dict:
+    """mcsd_verify_tree without a workspace, for callers that cannot allocate device memory at call time.
+
+    The scratch is a fixed array inside the library (B * N <= 16384 node states); `out` must hold the
+    preallocated result tensors (accept_len, out_tokens, out_nodes, best_root, next_roots), so this wrapper
+    allocates nothing either.  Calls share the array: do not let two of them overlap on the GPU."""
+    B, N, V = p.shape
+    with torch.cuda.device(p.device):
+        st = lib.mcsd_verify_tree_static(_ptr(p), _ptr(q), _ptr(tokens), _ptr(mask.parent), _ptr(mask.level_start),
+                                         mask.n_levels, mask.n_roots, _ptr(gamma), _ptr(u_accept), _ptr(u_bonus),
+                                         B, N, V, _ptr(out["accept_len"]), _ptr(out["out_tokens"]),
+                                         _ptr(out["out_nodes"]), _ptr(out["best_root"]), _ptr(out.get("next_roots")),
+                                         R, _stream())
+    _check(st, "mcsd_verify_tree_static")
     return out
 
 

@@ -20,6 +20,7 @@ extern "C" const char* mcsd_status_string(int status) {
         case MCSD_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
         case MCSD_ERR_CUDA: return "CUDA call failed";
         case MCSD_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case MCSD_ERR_STATIC_LIMIT: return "problem exceeds the built-in scratch of this entry point";
         default: return "unknown status";
     }
 }

@@ -17,6 +17,8 @@
 //
 // Rows are read with 128-bit loads when the row length allows; reductions run in a fixed order, fp32 per
 // lane and fp64 across warps.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace mcsd {
@@ -332,4 +334,53 @@ extern "C" int mcsd_verify_tree(const float* p, const float* q, const int32_t* t
     MCSD_CUDA_CHECK(cudaGetLastError());
     mcsd::count_launches(2);
     return MCSD_OK;
+}
+
+// ------------------------------------------------------------------------------------------------------
+// Variant with built-in scratch, for callers that cannot allocate device memory.
+// ------------------------------------------------------------------------------------------------------
+namespace mcsd {
+
+// Scratch that lives in the library image itself: one copy per GPU that loads the library, held until the
+// process exits.  Layout: workspace header, then MCSD_STATIC_VERIFY_MAX_STATES node states.
+constexpr size_t kStaticScratchBytes = sizeof(WorkspaceHeader) + sizeof(NodeState) * (size_t)MCSD_STATIC_VERIFY_MAX_STATES;
+static __device__ __align__(256) unsigned char g_static_verify_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_static_mutex;
+static void* g_static_ptr[kMaxDevices] = {};
+
+// In host code the array's name is only a handle; the address kernels can use has to be asked for, once
+// per device, with that device current.
+static int static_scratch_for_current_device(void** out) {
+    int dev = -1;
+    MCSD_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return MCSD_ERR_BAD_SHAPE;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (g_static_ptr[dev] == nullptr) {
+        void* ptr = nullptr;
+        MCSD_CUDA_CHECK(cudaGetSymbolAddress(&ptr, g_static_verify_scratch));
+        if (ptr == nullptr) return MCSD_ERR_CUDA;
+        g_static_ptr[dev] = ptr;
+    }
+    *out = g_static_ptr[dev];
+    return MCSD_OK;
+}
+
+}  // namespace mcsd
+
+extern "C" int mcsd_verify_tree_static(const float* p, const float* q, const int32_t* tokens, const int32_t* parent,
+                                       const int32_t* level_start, int n_levels, int n_roots, const int32_t* gamma,
+                                       const float* u_accept, const float* u_bonus, int B, int N, int V,
+                                       int32_t* accept_len, int32_t* out_tokens, int32_t* out_nodes,
+                                       int32_t* best_root, int32_t* next_roots, int R, void* stream) {
+    if (B >= 1 && N >= 1 && (long long)B * N > MCSD_STATIC_VERIFY_MAX_STATES) return MCSD_ERR_STATIC_LIMIT;
+    void* scratch = nullptr;
+    const int st = mcsd::static_scratch_for_current_device(&scratch);
+    if (st != MCSD_OK) return st;
+    // the array keeps whatever the previous call left; the status line must start at zero
+    MCSD_CUDA_CHECK(cudaMemsetAsync(scratch, 0, sizeof(mcsd::WorkspaceHeader), static_cast<cudaStream_t>(stream)));
+    return mcsd_verify_tree(p, q, tokens, parent, level_start, n_levels, n_roots, gamma, u_accept, u_bonus, B, N, V,
+                            accept_len, out_tokens, out_nodes, best_root, next_roots, R, scratch,
+                            mcsd::kStaticScratchBytes, stream);
 }

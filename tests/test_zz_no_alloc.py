@@ -1,0 +1,60 @@
+"""The workspace-free verify entry point (for callers that cannot allocate device memory when they call)
+must give exactly the results of the regular entry point, call after call, although every call reuses the
+same built-in scratch array.  Collected last on purpose."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from mcsd_inputs import gammas, parent_array, verify_inputs, workload
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def m():
+    from paper_2409_10644_b200 import build
+    build.build()
+    import paper_2409_10644_b200 as pkg
+    return pkg
+
+
+def _outputs(B, n_levels, R, dev):
+    return {
+        "accept_len": torch.full((B,), -7, dtype=torch.int32, device=dev),
+        "out_tokens": torch.full((B, n_levels + 1), -7, dtype=torch.int32, device=dev),
+        "out_nodes": torch.full((B, n_levels), -7, dtype=torch.int32, device=dev),
+        "best_root": torch.full((B,), -7, dtype=torch.int32, device=dev),
+        "next_roots": torch.full((B, R), -7, dtype=torch.int32, device=dev),
+    }
+
+
+def test_static_scratch_entry_point_matches_the_workspace_one_twice_in_a_row(m):
+    dev = torch.device("cuda", 0)
+    R = 4
+    # two different problems back to back: a large one, then a smaller one that leaves most of the
+    # previous call's node states behind in the shared array
+    cases = [(workload(5), 12, 4000, 0), (workload(3), 5, 1000, 1)]
+    for w, B, V, step in cases:
+        parent = parent_array(w.n_roots, w.branching)
+        tm = m.mcsd_build_mask(parent, device=dev)
+        vin = verify_inputs(w, step, dev, parent=parent, B=B, V=V)
+        gam = torch.from_numpy(gammas(dataclasses.replace(w, B=B), step)).to(dev)
+        ref = m.mcsd_verify_tree(vin["p"], vin["q"], vin["tokens"], tm, gam, vin["u_accept"], vin["u_bonus"], R=R)
+        out = _outputs(B, tm.n_levels, R, dev)
+        got = m.mcsd_verify_tree_static(vin["p"], vin["q"], vin["tokens"], tm, gam, vin["u_accept"], vin["u_bonus"],
+                                        out, R=R)
+        torch.cuda.synchronize()
+        for k in ("accept_len", "out_tokens", "out_nodes", "best_root", "next_roots"):
+            assert torch.equal(got[k], ref[k]), k          # integer results: identical, not just close
+        assert int(ref["accept_len"].max()) >= 0
+
+
+def test_static_scratch_entry_point_rejects_oversized_problems(m):
+    import ctypes
+    fake = ctypes.c_void_p(0x1000)     # never dereferenced: the size check comes first
+    st = m.lib.mcsd_verify_tree_static(fake, fake, fake, fake, fake, 4, 1, None, fake, fake, 200, 192, 100,
+                                       fake, fake, fake, fake, None, 0, None)
+    assert st == -8
+    assert "built-in scratch" in m.mcsd_status_string(st)
