@@ -1,7 +1,753 @@
-// Tensor-core path of tree attention; not built yet: every shape takes the CUDA-core kernel.
+// Tree attention (Section 2.2 of the paper) on the fifth-generation tensor cores of sm_100a: bf16, head_dim 128.
+//
+// One persistent thread block per SM walks a contiguous range of 128-key tiles of the flattened
+// (sequence, head, key tile) space, so the K/V stream of every (sequence, head) is read from HBM exactly once
+// and all SMs carry the same number of tiles whatever the batch and the prefix lengths are.  Where a range
+// boundary cuts a (sequence, head), both sides write an unnormalised partial (running maximum, sum, weighted
+// values) and a combine kernel merges them: split-KV.
+//
+// The problem is set up transposed so that the small dimension (tree tokens, 16..128 per head) is the MMA N
+// and the 128 keys of a tile fill the MMA M:
+//     S^T[key][query] = K_tile[key][d] * Q[query][d]^T            (A = K tile, B = Q, both K-major, from TMA)
+//     O^T[d][query]  += V_tile[key][d]^T * P^T[key][query]        (A = V tile read MN-major, B = P^T written
+//                                                                  by the softmax threads, MN-major)
+// Accumulators live in tensor memory: S^T double-buffered (columns 0 and 128), O^T at column 256.
+//
+// Warp roles (192 threads):
+//   warps 0-3  softmax: thread r owns key row r of the tile = TMEM lane r.  Column (per-query) maxima are
+//              reduced with redux.sync inside a warp and through shared memory across the four warps; the
+//              running reference maximum is only raised when a tile exceeds it by more than 2^8 ("lazy"
+//              rescaling), so O^T in tensor memory is rarely touched between MMAs.  Row sums are kept per
+//              thread and reduced once per segment.  These threads also apply the tree mask (transposed
+//              ancestor bitsets), zero V rows past the end of a ragged tile and run the epilogue.
+//   warp 4     TMA producer: K and V tiles into a ring of 32 KB slots, Q once per segment.
+//   warp 5     MMA issuer (one thread) and owner of the tensor-memory allocation.
+// Every mbarrier wait is bounded; a wait that runs out raises a flag in the workspace header, all roles drain
+// and the block exits cleanly.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <mutex>
+
 #include "attention.cuh"
+
 namespace mcsd {
-bool tc_supported(const AttentionArgs&) { return false; }
-size_t tc_workspace_bytes(int, int, int, int, int) { return 0; }
-int tree_attention_tc(const AttentionArgs&, WorkspaceHeader*, void*, size_t, cudaStream_t) { return MCSD_ERR_BAD_DTYPE; }
+
+constexpr int kTile = 128;                    // keys per tile
+constexpr int kTcThreads = 192;
+constexpr int kSlotBytes = kTile * 128 * 2;   // one K or V tile: 128 rows x 128 bf16
+constexpr int kSlabBytes = kTile * 128;       // 64 of the 128 columns: rows of 128 bytes (the TMA swizzle span)
+constexpr int kMaxSlots = 6;
+constexpr int kMaxBatchTc = 256;
+constexpr int kTmemCols = 512;
+constexpr int kColS1 = 128, kColO = 256;
+constexpr float kLazyTau = 8.0f;              // raise the reference maximum only beyond 2^8
+constexpr int kMaxCtas = 160;                 // partial slots are provisioned for this many thread blocks
+constexpr long long kSpinCycles = 4000000000LL;   // about two seconds
+
+struct TcSmall {
+    unsigned long long slot_full[kMaxSlots];
+    unsigned long long slot_empty[kMaxSlots];
+    unsigned long long s_full[2];
+    unsigned long long p_full, pv_done, q_full, q_empty, drain;
+    uint32_t tmem_base;
+    int abort_flag;
+    int pad[2];
+    float m_ref[128];
+    float alpha[128];
+    float inv_l[128];
+    float wred[4][128];
+    unsigned long long dmask[128][2];
+    int cum_tiles[kMaxBatchTc + 1];
+};
+
+struct TcParams {
+    __nv_bfloat16* out;
+    const int32_t* seq_lens;
+    const int32_t* n_active;
+    const uint64_t* anc;
+    int words;
+    int B, H, N, L_max;
+    float scale_log2;
+    float* part_ml;      // [2 * kMaxCtas][2][128]
+    float* part_o;       // [2 * kMaxCtas][128][128]
+    WorkspaceHeader* header;
+    int n_slots;
+    int npadq;           // rows of the Q box = 16 * (template chunk count)
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(void* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(void* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(void* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(void* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  Returns false if the wait ran out or another role already gave up; `where` names the wait.
+__device__ __noinline__ bool mbar_wait_slow(void* bar, uint32_t parity, TcSmall* sm, WorkspaceHeader* header, int where) {
+    const long long t0 = clock64();
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 255u) {
+            if (*(volatile int*)&sm->abort_flag) return false;
+            if (clock64() - t0 > kSpinCycles) {
+                *(volatile int*)&sm->abort_flag = 1;
+                header->detail = where;
+                header->status = MCSD_ERR_TIMEOUT;
+                __threadfence();
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, TcSmall* sm, WorkspaceHeader* header, int where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, sm, header, where);
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, void* bar, int x, int y, int z) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(void* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tc_st16(uint32_t taddr, const float* v) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+          "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+          "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
+          "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
+          "r"(__float_as_uint(v[15])) : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float warp_max_f32(float v) {
+    float r;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+    return r;
+}
+// barrier 1 over the 128 softmax threads, returning the OR of `pred`
+__device__ __forceinline__ bool softmax_sync_any(bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "bar.red.or.pred q, 1, 128, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r) : "r"((uint32_t)pred) : "memory");
+    return r != 0;
+}
+
+// Shared-memory matrix descriptor of tcgen05.mma: start address, leading/stride byte offsets (all >> 4),
+// descriptor version 1, swizzle mode in the top bits (0 = none, 2 = 128-byte).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+           (1ull << 46) | ((uint64_t)layout << 61);
+}
+// Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, M = 128, N = n, operand major-ness.
+__device__ __forceinline__ uint32_t instr_desc(int n, int a_mn_major, int b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+// ------------------------------------------------------------------ tile bookkeeping
+__device__ __forceinline__ int tiles_of(int L, int Nb) {
+    return Nb > 0 ? (L + kTile - 1) / kTile + (Nb + kTile - 1) / kTile : 0;
+}
+
+struct Segment {
+    int b, h, lt, Tb, L, Nb, nP;
+};
+
+__device__ __forceinline__ void locate(const TcSmall* sm, const TcParams& p, long long t, Segment& s) {
+    int lo = 0, hi = p.B;                      // find b with H*cum[b] <= t < H*cum[b+1]
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if ((long long)p.H * sm->cum_tiles[mid] <= t) lo = mid; else hi = mid;
+    }
+    s.b = lo;
+    s.L = min(max(p.seq_lens[lo], 0), p.L_max);
+    s.Nb = p.n_active ? min(max(p.n_active[lo], 0), p.N) : p.N;
+    s.Tb = sm->cum_tiles[lo + 1] - sm->cum_tiles[lo];
+    s.nP = (s.L + kTile - 1) / kTile;
+    const long long r = t - (long long)p.H * sm->cum_tiles[lo];
+    s.h = (int)(r / s.Tb);
+    s.lt = (int)(r % s.Tb);
+}
+
+// ------------------------------------------------------------------ the kernel
+template <int NCH>
+__global__ void __launch_bounds__(kTcThreads, 1)
+tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kc,
+                         const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kt,
+                         const __grid_constant__ CUtensorMap tm_vt, const TcParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int NS = p.n_slots;
+    unsigned char* ring = smem;
+    unsigned char* p_buf = ring + (size_t)NS * kSlotBytes;
+    unsigned char* q_buf = p_buf + (size_t)p.npadq * 256;
+    TcSmall* sm = reinterpret_cast<TcSmall*>(q_buf + (size_t)p.npadq * 256);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int G = gridDim.x, cta = blockIdx.x;
+
+    // ---- set-up: tile counts per sequence, barriers, tensor memory, transposed tree mask
+    if (tid == 0) {
+        int acc = 0;
+        for (int b = 0; b < p.B; ++b) {
+            sm->cum_tiles[b] = acc;
+            const int L = min(max(p.seq_lens[b], 0), p.L_max);
+            const int Nb = p.n_active ? min(max(p.n_active[b], 0), p.N) : p.N;
+            acc += tiles_of(L, Nb);
+        }
+        sm->cum_tiles[p.B] = acc;
+        for (int i = 0; i < kMaxSlots; ++i) { mbar_init(&sm->slot_full[i], 1); mbar_init(&sm->slot_empty[i], 1); }
+        mbar_init(&sm->s_full[0], 1);
+        mbar_init(&sm->s_full[1], 1);
+        mbar_init(&sm->p_full, 128);
+        mbar_init(&sm->pv_done, 1);
+        mbar_init(&sm->q_full, 1);
+        mbar_init(&sm->q_empty, 1);
+        mbar_init(&sm->drain, 1);
+        sm->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (tid < 128) {
+        // dmask[t] = set of queries that may see tree key t (bit n of the transposed ancestor matrix)
+        unsigned long long w0 = 0, w1 = 0;
+        if (tid < p.N) {
+            for (int n = 0; n < p.N; ++n) {
+                const unsigned long long word = p.anc[(size_t)n * p.words + (tid >> 6)];
+                if ((word >> (tid & 63)) & 1ull) {
+                    if (n < 64) w0 |= 1ull << n; else w1 |= 1ull << (n - 64);
+                }
+            }
+        }
+        sm->dmask[tid][0] = w0;
+        sm->dmask[tid][1] = w1;
+    }
+    __syncthreads();
+    const long long total = (long long)p.H * sm->cum_tiles[p.B];
+    const long long t_begin = (long long)cta * total / G, t_end = (long long)(cta + 1) * total / G;
+    if (t_begin >= t_end) return;              // uniform for the whole block: nothing allocated yet
+
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *(volatile uint32_t*)&sm->tmem_base;
+    WorkspaceHeader* hdr = p.header;
+
+    if (warp == 4) {
+        // =========================================================== TMA producer
+        if (lane == 0) {
+            long long t = t_begin;
+            uint32_t u = 0, seg = 0;
+            bool ok = true;
+            while (t < t_end && ok) {
+                Segment s;
+                locate(sm, p, t, s);
+                const int cnt = (int)min((long long)(s.Tb - s.lt), t_end - t);
+                const int bh = s.b * p.H + s.h;
+                ok = mbar_wait(&sm->q_empty, (seg & 1u) ^ 1u, sm, hdr, 1);
+                if (!ok) break;
+                mbar_expect_tx(&sm->q_full, (uint32_t)p.npadq * 256u);
+                tma_load_3d(smem_u32(q_buf), &tm_q, &sm->q_full, 0, 0, bh);
+                tma_load_3d(smem_u32(q_buf) + (uint32_t)p.npadq * 128u, &tm_q, &sm->q_full, 64, 0, bh);
+                for (int i = 0; i < cnt && ok; ++i) {
+                    const int lti = s.lt + i;
+                    const bool tree = lti >= s.nP;
+                    const int row0 = (tree ? lti - s.nP : lti) * kTile;
+                    for (int kv = 0; kv < 2 && ok; ++kv, ++u) {
+                        const uint32_t slot = u % (uint32_t)NS;
+                        ok = mbar_wait(&sm->slot_empty[slot], ((u / (uint32_t)NS) & 1u) ^ 1u, sm, hdr, 2);
+                        if (!ok) break;
+                        const CUtensorMap* map = kv == 0 ? (tree ? &tm_kt : &tm_kc) : (tree ? &tm_vt : &tm_vc);
+                        const uint32_t dst = smem_u32(ring) + slot * (uint32_t)kSlotBytes;
+                        mbar_expect_tx(&sm->slot_full[slot], (uint32_t)kSlotBytes);
+                        tma_load_3d(dst, map, &sm->slot_full[slot], 0, row0, bh);
+                        tma_load_3d(dst + kSlabBytes, map, &sm->slot_full[slot], 64, row0, bh);
+                    }
+                }
+                t += cnt;
+                ++seg;
+            }
+            if (!ok) {
+                // gave up: let copies already issued land before the block exits
+                const uint32_t first = u > (uint32_t)NS ? u - (uint32_t)NS : 0u;
+                for (uint32_t x = first; x < u; ++x) {
+                    void* bar = &sm->slot_full[x % (uint32_t)NS];
+                    const uint32_t par = (x / (uint32_t)NS) & 1u;
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(bar, par) && clock64() - t0 < kSpinCycles / 8) {}
+                }
+            }
+        }
+    } else if (warp == 5) {
+        // =========================================================== MMA issuer
+        if (lane == 0) {
+            long long t = t_begin;
+            uint32_t u = 0, g = 0, seg = 0;
+            bool ok = true;
+            const uint32_t ring_a = smem_u32(ring), q_a = smem_u32(q_buf), p_a = smem_u32(p_buf);
+            while (t < t_end && ok) {
+                Segment s;
+                locate(sm, p, t, s);
+                const int cnt = (int)min((long long)(s.Tb - s.lt), t_end - t);
+                const int npad = (s.Nb + 15) & ~15;
+                const uint32_t idesc_s = instr_desc(npad, 0, 0), idesc_pv = instr_desc(npad, 1, 1);
+                ok = mbar_wait(&sm->q_full, seg & 1u, sm, hdr, 3);
+                for (int i = 0; i <= cnt && ok; ++i) {
+                    if (i < cnt) {
+                        const uint32_t gi = g + (uint32_t)i, sb = gi & 1u;
+                        const uint32_t uk = u + 2u * (uint32_t)i, slot = uk % (uint32_t)NS;
+                        ok = mbar_wait(&sm->slot_full[slot], (uk / (uint32_t)NS) & 1u, sm, hdr, 4);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t ka = ring_a + slot * (uint32_t)kSlotBytes;
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            // 16 of the 128 head dims per MMA: slab k/4, 32-byte step inside the swizzled row
+                            const uint64_t da = smem_desc(ka + (k >> 2) * kSlabBytes + (k & 3) * 32, 16, 1024, 2);
+                            const uint64_t db = smem_desc(q_a + (k >> 2) * (uint32_t)p.npadq * 128u + (k & 3) * 32, 16, 1024, 2);
+                            tc_mma(tmem + (sb ? kColS1 : 0), da, db, idesc_s, k > 0);
+                        }
+                        tc_commit(&sm->s_full[sb]);
+                        tc_commit(&sm->slot_empty[slot]);
+                        if (i == cnt - 1) tc_commit(&sm->q_empty);
+                    }
+                    if (i >= 1) {
+                        const uint32_t gj = g + (uint32_t)(i - 1);
+                        const uint32_t uv = u + 2u * (uint32_t)(i - 1) + 1u, slot = uv % (uint32_t)NS;
+                        ok = mbar_wait(&sm->slot_full[slot], (uv / (uint32_t)NS) & 1u, sm, hdr, 5);
+                        if (!ok) break;
+                        ok = mbar_wait(&sm->p_full, gj & 1u, sm, hdr, 6);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t va = ring_a + slot * (uint32_t)kSlotBytes;
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            // 16 keys per MMA.  V^T: two 64-dim atoms 16 KB apart (leading), 8-key groups 1 KB apart.
+                            const uint64_t da = smem_desc(va + k * 2048, kSlabBytes, 1024, 2);
+                            // P^T: 8-key groups 128 B apart (leading), 8-query groups 2 KB apart (stride), no swizzle.
+                            const uint64_t db = smem_desc(p_a + k * 256, 128, 2048, 0);
+                            tc_mma(tmem + kColO, da, db, idesc_pv, !(i == 1 && k == 0));
+                        }
+                        tc_commit(&sm->slot_empty[slot]);
+                        tc_commit(&sm->pv_done);
+                    }
+                }
+                u += 2u * (uint32_t)cnt;
+                g += (uint32_t)cnt;
+                ++seg;
+                t += cnt;
+            }
+            // all MMAs issued by this thread must have finished before tensor memory is released
+            tc_commit(&sm->drain);
+            {
+                const long long t0 = clock64();
+                while (!mbar_try_wait(&sm->drain, 0) && clock64() - t0 < kSpinCycles) {}
+            }
+        }
+    } else {
+        // =========================================================== softmax / mask / epilogue (128 threads)
+        const int r = tid;
+        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+        long long t = t_begin;
+        uint32_t u = 0, g = 0;
+        bool failed = false;
+        float acc_l[NCH][16];
+        while (t < t_end) {
+            Segment s;
+            locate(sm, p, t, s);
+            const int cnt = (int)min((long long)(s.Tb - s.lt), t_end - t);
+            const int nch = (s.Nb + 15) >> 4;
+            const int bh = s.b * p.H + s.h;
+            const unsigned long long nb_lo = s.Nb >= 64 ? ~0ull : ((1ull << s.Nb) - 1ull);
+            const unsigned long long nb_hi = s.Nb >= 128 ? ~0ull : (s.Nb > 64 ? ((1ull << (s.Nb - 64)) - 1ull) : 0ull);
+            sm->m_ref[r] = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < NCH; ++c)
+#pragma unroll
+                for (int k = 0; k < 16; ++k) acc_l[c][k] = 0.f;
+            if (softmax_sync_any(failed)) { failed = true; break; }
+
+            for (int i = 0; i < cnt; ++i) {
+                const uint32_t gi = g + (uint32_t)i, sb = gi & 1u;
+                const int lti = s.lt + i;
+                const bool tree = lti >= s.nP;
+                const int row0 = (tree ? lti - s.nP : lti) * kTile;
+                const int valid = min(kTile, (tree ? s.Nb : s.L) - row0);
+                // queries that may see this thread's key
+                unsigned long long cm0 = 0, cm1 = 0;
+                if (r < valid) {
+                    cm0 = nb_lo; cm1 = nb_hi;
+                    if (tree) { cm0 &= sm->dmask[row0 + r][0]; cm1 &= sm->dmask[row0 + r][1]; }
+                }
+                if (!mbar_wait(&sm->s_full[sb], (gi >> 1) & 1u, sm, hdr, 7)) failed = true;
+                tc_fence_after();
+                const uint32_t s_addr = tmem + lane_addr + (sb ? kColS1 : 0);
+
+                // ---- pass 1: per-query maximum over the 128 keys of the tile
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    if (c < nch) {
+                        float v[16];
+                        tc_ld16(s_addr + 16 * c, v);
+                        const uint32_t bits = (uint32_t)(((c < 4 ? cm0 : cm1) >> ((c & 3) * 16)) & 0xFFFFull);
+                        float mine = -INFINITY;
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) {
+                            const float x = ((bits >> k) & 1u) ? v[k] * p.scale_log2 : -INFINITY;
+                            const float mx = warp_max_f32(x);
+                            if (lane == k) mine = mx;
+                        }
+                        if (lane < 16) sm->wred[warp][16 * c + lane] = mine;
+                    }
+                }
+                if (softmax_sync_any(failed)) { failed = true; break; }
+                // one thread per query folds the four warps' maxima into the running reference
+                bool need = false;
+                if (r < 16 * nch) {
+                    const float tm = fmaxf(fmaxf(sm->wred[0][r], sm->wred[1][r]), fmaxf(sm->wred[2][r], sm->wred[3][r]));
+                    const float mo = sm->m_ref[r];
+                    float a = 1.f;
+                    if (tm > mo + kLazyTau || (mo == -INFINITY && tm > -INFINITY)) {
+                        a = (mo == -INFINITY) ? 0.f : exp2f(mo - tm);
+                        sm->m_ref[r] = tm;
+                        need = (i > 0) && (mo != -INFINITY);     // accumulated O^T and sums must be rescaled
+                    }
+                    sm->alpha[r] = a;
+                }
+                const bool rescale = softmax_sync_any(need);
+
+                // P buffer (and O, if it is rescaled) must no longer be in use by the previous tile's MMA
+                if (gi > 0 && !mbar_wait(&sm->pv_done, (gi - 1u) & 1u, sm, hdr, 8)) failed = true;
+                if (rescale) {
+                    tc_fence_after();
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) {
+                        if (c < nch) {
+                            float o[16];
+                            tc_ld16(tmem + lane_addr + kColO + 16 * c, o);
+#pragma unroll
+                            for (int k = 0; k < 16; ++k) {
+                                const float a = sm->alpha[16 * c + k];
+                                o[k] *= a;
+                                acc_l[c][k] *= a;
+                            }
+                            tc_st16(tmem + lane_addr + kColO + 16 * c, o);
+                        }
+                    }
+                }
+
+                // ---- pass 2: probabilities, row sums, P^T tile for the second MMA
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    if (c < nch) {
+                        float v[16];
+                        tc_ld16(s_addr + 16 * c, v);
+                        const uint32_t bits = (uint32_t)(((c < 4 ? cm0 : cm1) >> ((c & 3) * 16)) & 0xFFFFull);
+                        uint32_t packed[8];
+#pragma unroll
+                        for (int k = 0; k < 16; k += 2) {
+                            const float2 mr = *reinterpret_cast<const float2*>(&sm->m_ref[16 * c + k]);
+                            const float p0 = ((bits >> k) & 1u) ? exp2f(v[k] * p.scale_log2 - mr.x) : 0.f;
+                            const float p1 = ((bits >> (k + 1)) & 1u) ? exp2f(v[k + 1] * p.scale_log2 - mr.y) : 0.f;
+                            acc_l[c][k] += p0;
+                            acc_l[c][k + 1] += p1;
+                            __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+                            packed[k >> 1] = *reinterpret_cast<uint32_t*>(&h2);
+                        }
+                        uint4* dst0 = reinterpret_cast<uint4*>(p_buf + (size_t)(2 * c) * 2048 + (size_t)r * 16);
+                        uint4* dst1 = reinterpret_cast<uint4*>(p_buf + (size_t)(2 * c + 1) * 2048 + (size_t)r * 16);
+                        *dst0 = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                        *dst1 = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+                    }
+                }
+                // rows of the V tile past the end of the prefix / tree may hold anything: make them zero
+                if (valid < kTile) {
+                    const uint32_t uv = u + 2u * (uint32_t)i + 1u, slot = uv % (uint32_t)NS;
+                    if (!mbar_wait(&sm->slot_full[slot], (uv / (uint32_t)NS) & 1u, sm, hdr, 9)) failed = true;
+                    if (r >= valid && !failed) {
+                        uint4* z0 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + (size_t)r * 128);
+                        uint4* z1 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + kSlabBytes + (size_t)r * 128);
+#pragma unroll
+                        for (int x = 0; x < 8; ++x) { z0[x] = make_uint4(0, 0, 0, 0); z1[x] = make_uint4(0, 0, 0, 0); }
+                    }
+                }
+                fence_async_smem();
+                tc_fence_before();
+                mbar_arrive(&sm->p_full);
+            }
+            if (softmax_sync_any(failed)) { failed = true; break; }
+
+            // ---- epilogue of the segment
+            const uint32_t glast = g + (uint32_t)cnt - 1u;
+            if (!mbar_wait(&sm->pv_done, glast & 1u, sm, hdr, 10)) failed = true;
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                if (c < nch) {
+                    float mine = 0.f;
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) {
+                        float v = acc_l[c][k];
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                        if (lane == k) mine = v;
+                    }
+                    if (lane < 16) sm->wred[warp][16 * c + lane] = mine;
+                }
+            }
+            if (softmax_sync_any(failed)) { failed = true; break; }
+            const bool full = (cnt == s.Tb);
+            const int slot_id = 2 * cta + (t > t_begin ? 1 : 0);
+            if (r < 16 * nch) {
+                const float l = (sm->wred[0][r] + sm->wred[1][r]) + (sm->wred[2][r] + sm->wred[3][r]);
+                if (full) {
+                    sm->inv_l[r] = l > 0.f ? 1.f / l : 0.f;
+                } else {
+                    p.part_ml[((size_t)slot_id * 2 + 0) * 128 + r] = sm->m_ref[r];
+                    p.part_ml[((size_t)slot_id * 2 + 1) * 128 + r] = l;
+                }
+            }
+            if (softmax_sync_any(false)) { failed = true; break; }
+#pragma unroll
+            for (int c = 0; c < NCH; ++c) {
+                if (c < nch) {
+                    float o[16];
+                    tc_ld16(tmem + lane_addr + kColO + 16 * c, o);
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) {
+                        const int n = 16 * c + k;
+                        if (n < s.Nb) {
+                            if (full) p.out[((size_t)bh * p.N + n) * 128 + r] = __float2bfloat16_rn(o[k] * sm->inv_l[n]);
+                            else p.part_o[((size_t)slot_id * 128 + n) * 128 + r] = o[k];
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            if (softmax_sync_any(false)) { failed = true; break; }
+            g += (uint32_t)cnt;
+            u += 2u * (uint32_t)cnt;
+            t += cnt;
+        }
+    }
+
+    // ---- tear-down
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// Merges the partials of every (sequence, head) whose tiles were split over several thread blocks.
+// grid: B * H blocks of 128 threads (thread = output column d).
+__global__ void __launch_bounds__(128)
+tree_attention_tc_combine_kernel(const TcParams p, int G) {
+    __shared__ int s_cum[2];
+    __shared__ long long s_total;
+    const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H, d = threadIdx.x;
+    if (d == 0) {
+        int acc = 0, mine = 0, tb = 0;
+        for (int i = 0; i < p.B; ++i) {
+            const int L = min(max(p.seq_lens[i], 0), p.L_max);
+            const int Nb = p.n_active ? min(max(p.n_active[i], 0), p.N) : p.N;
+            const int ti = tiles_of(L, Nb);
+            if (i == b) { mine = acc; tb = ti; }
+            acc += ti;
+        }
+        s_cum[0] = mine; s_cum[1] = tb; s_total = (long long)p.H * acc;
+    }
+    __syncthreads();
+    const int Tb = s_cum[1];
+    if (Tb == 0) return;
+    const long long total = s_total;
+    const long long t0 = (long long)p.H * s_cum[0] + (long long)h * Tb, t1 = t0 + Tb;
+    const int c_lo = (int)(((t0 + 1) * G + total - 1) / total - 1), c_hi = (int)((t1 * G + total - 1) / total - 1);
+    if (c_lo == c_hi) return;                  // one block saw every tile and wrote the result itself
+    const int Nb = p.n_active ? min(max(p.n_active[b], 0), p.N) : p.N;
+    for (int n = 0; n < Nb; ++n) {
+        float M = -INFINITY;
+        for (int c = c_lo; c <= c_hi; ++c) {
+            const long long start = (long long)c * total / G;
+            const int slot = 2 * c + (t0 > start ? 1 : 0);
+            M = fmaxf(M, p.part_ml[((size_t)slot * 2 + 0) * 128 + n]);
+        }
+        float lsum = 0.f, acc = 0.f;
+        for (int c = c_lo; c <= c_hi; ++c) {
+            const long long start = (long long)c * total / G;
+            const int slot = 2 * c + (t0 > start ? 1 : 0);
+            const float ms = p.part_ml[((size_t)slot * 2 + 0) * 128 + n];
+            if (ms == -INFINITY) continue;
+            const float w = exp2f(ms - M);
+            lsum += w * p.part_ml[((size_t)slot * 2 + 1) * 128 + n];
+            acc = fmaf(w, p.part_o[((size_t)slot * 128 + n) * 128 + d], acc);
+        }
+        p.out[((size_t)bh * p.N + n) * 128 + d] = __float2bfloat16_rn(lsum > 0.f ? acc / lsum : 0.f);
+    }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    });
+    return fn;
+}
+
+// [BH][rows][128] bf16 tensor, boxes of box_rows x 64 columns, 128-byte swizzle, zero fill outside
+static bool make_map(CUtensorMap* map, const void* base, int rows, int bh, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return false;
+    cuuint64_t dims[3] = {128, (cuuint64_t)rows, (cuuint64_t)bh};
+    cuuint64_t strides[2] = {256, (cuuint64_t)rows * 256};
+    cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int chunks_for(int N) {
+    const int nch = (N + 15) / 16;
+    return nch <= 3 ? 3 : nch <= 4 ? 4 : nch <= 7 ? 7 : 8;
+}
+
+static int slots_for(int nch) {
+    const long long avail = 232448LL - 1024 - (long long)sizeof(TcSmall) - (long long)nch * 16 * 512;
+    long long ns = avail / kSlotBytes;
+    if (ns > kMaxSlots) ns = kMaxSlots;
+    return (int)ns;
+}
+
+bool tc_supported(const AttentionArgs& a) {
+    return a.N <= 128 && a.B <= kMaxBatchTc && encode_fn() != nullptr;
+}
+
+size_t tc_workspace_bytes(int, int, int N, int, int) {
+    if (N > 128) return 0;
+    return align_up((size_t)2 * kMaxCtas * 2 * 128 * sizeof(float), 256) +
+           align_up((size_t)2 * kMaxCtas * 128 * 128 * sizeof(float), 256);
+}
+
+template <int NCH>
+static int launch_tc(const CUtensorMap* maps, const TcParams& p, int grid, size_t smem_bytes, cudaStream_t stream) {
+    MCSD_CUDA_CHECK(cudaFuncSetAttribute(tree_attention_tc_kernel<NCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    tree_attention_tc_kernel<NCH><<<grid, kTcThreads, smem_bytes, stream>>>(maps[0], maps[1], maps[2], maps[3], maps[4], p);
+    MCSD_CUDA_CHECK(cudaGetLastError());
+    return MCSD_OK;
+}
+
+int tree_attention_tc(const AttentionArgs& a, WorkspaceHeader* header, void* scratch, size_t scratch_bytes,
+                      cudaStream_t stream) {
+    if (scratch_bytes < tc_workspace_bytes(a.B, a.H, a.N, a.D, a.L_max)) return MCSD_ERR_WORKSPACE_TOO_SMALL;
+    const int nch = chunks_for(a.N);
+    const int npadq = nch * 16;
+    const int ns = slots_for(nch);
+    if (ns < 4) return MCSD_ERR_BAD_SHAPE;
+    const int bh = a.B * a.H;
+
+    CUtensorMap maps[5];
+    const bool have_cache = a.L_max > 0;
+    bool ok = make_map(&maps[0], a.q, a.N, bh, npadq);
+    ok = ok && make_map(&maps[1], have_cache ? a.k_cache : a.k_tree, have_cache ? a.L_max : a.N, bh, kTile);
+    ok = ok && make_map(&maps[2], have_cache ? a.v_cache : a.v_tree, have_cache ? a.L_max : a.N, bh, kTile);
+    ok = ok && make_map(&maps[3], a.k_tree, a.N, bh, kTile);
+    ok = ok && make_map(&maps[4], a.v_tree, a.N, bh, kTile);
+    if (!ok) { set_last_cuda_error(cudaErrorInvalidValue); return MCSD_ERR_CUDA; }
+
+    int dev = 0, sms = 0;
+    MCSD_CUDA_CHECK(cudaGetDevice(&dev));
+    MCSD_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const int grid = sms < kMaxCtas ? sms : kMaxCtas;
+
+    TcParams p;
+    p.out = static_cast<__nv_bfloat16*>(a.out);
+    p.seq_lens = a.seq_lens;
+    p.n_active = a.n_active;
+    p.anc = a.anc;
+    p.words = a.words;
+    p.B = a.B; p.H = a.H; p.N = a.N; p.L_max = a.L_max;
+    p.scale_log2 = a.scale * 1.4426950408889634f;
+    p.part_ml = static_cast<float*>(scratch);
+    p.part_o = reinterpret_cast<float*>(static_cast<char*>(scratch) + align_up((size_t)2 * kMaxCtas * 2 * 128 * sizeof(float), 256));
+    p.header = header;
+    p.n_slots = ns;
+    p.npadq = npadq;
+    const size_t smem_bytes = 1024 + (size_t)ns * kSlotBytes + (size_t)npadq * 512 + sizeof(TcSmall);
+
+    int st;
+    switch (nch) {
+        case 3: st = launch_tc<3>(maps, p, grid, smem_bytes, stream); break;
+        case 4: st = launch_tc<4>(maps, p, grid, smem_bytes, stream); break;
+        case 7: st = launch_tc<7>(maps, p, grid, smem_bytes, stream); break;
+        default: st = launch_tc<8>(maps, p, grid, smem_bytes, stream); break;
+    }
+    if (st != MCSD_OK) return st;
+    count_launches(1);
+    tree_attention_tc_combine_kernel<<<bh, 128, 0, stream>>>(p, grid);
+    MCSD_CUDA_CHECK(cudaGetLastError());
+    count_launches(1);
+    return MCSD_OK;
+}
+
 }  // namespace mcsd
