@@ -200,6 +200,10 @@ def run_ours(args):
     from mcsd_inputs import attention_inputs, gammas, parent_array, seq_lens, verify_inputs, workload
 
     w0 = workload(args.workload)
+    if args.batch > 0:
+        w0 = dataclasses.replace(w0, B=args.batch)
+    if args.layers > 0:
+        w0 = dataclasses.replace(w0, n_layers=args.layers)
     w = dataclasses.replace(w0, base_seed=1000 * w0.index + 100000 * rank)
     parent = parent_array(w.n_roots, w.branching)
     N = len(parent)
@@ -358,6 +362,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="long_context_b16")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling of a smaller case only)")
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling only)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
