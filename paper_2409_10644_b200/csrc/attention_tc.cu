@@ -13,15 +13,16 @@
 //                                                                  by the softmax threads, MN-major)
 // Accumulators live in tensor memory: S^T double-buffered (columns 0 and 128), O^T at column 256.
 //
-// Warp roles (192 threads):
-//   warps 0-3  softmax: thread r owns key row r of the tile = TMEM lane r.  Column (per-query) maxima are
-//              reduced with redux.sync inside a warp and through shared memory across the four warps; the
-//              running reference maximum is only raised when a tile exceeds it by more than 2^8 ("lazy"
-//              rescaling), so O^T in tensor memory is rarely touched between MMAs.  Row sums are kept per
-//              thread and reduced once per segment.  These threads also apply the tree mask (transposed
-//              ancestor bitsets), zero V rows past the end of a ragged tile and run the epilogue.
-//   warp 4     TMA producer: K and V tiles into a ring of 32 KB slots, Q once per segment.
-//   warp 5     MMA issuer (one thread) and owner of the tensor-memory allocation.
+// Warp roles (320 threads):
+//   warps 0-7  softmax, two warpgroups that split the query columns of each tile: thread r of a group owns
+//              key row r of the tile = TMEM lane r.  The running reference maximum of a query is only raised
+//              when a score exceeds it by more than 2^8 ("lazy" rescaling): the common tile costs one vote,
+//              and only then are exact column maxima reduced (redux.sync inside a warp, shared memory across
+//              warps) and O^T in tensor memory rescaled.  Row sums are kept per thread and reduced once per
+//              segment.  These threads also apply the tree mask (transposed ancestor bitsets), zero V rows
+//              past the end of a ragged tile and run the epilogue.
+//   warp 8     TMA producer: K and V tiles into a ring of 32 KB slots, Q once per segment.
+//   warp 9     MMA issuer (one thread) and owner of the tensor-memory allocation.
 // Every mbarrier wait is bounded; a wait that runs out raises a flag in the workspace header, all roles drain
 // and the block exits cleanly.
 #include <cuda.h>
@@ -34,7 +35,9 @@
 namespace mcsd {
 
 constexpr int kTile = 128;                    // keys per tile
-constexpr int kTcThreads = 192;
+constexpr int kSoftmaxGroups = 2;              // warpgroups that split the query columns of every tile
+constexpr int kProducerWarp = 4 * kSoftmaxGroups, kMmaWarp = kProducerWarp + 1;
+constexpr int kTcThreads = 32 * (kMmaWarp + 1);
 constexpr int kSlotBytes = kTile * 128 * 2;   // one K or V tile: 128 rows x 128 bf16
 constexpr int kSlabBytes = kTile * 128;       // 64 of the 128 columns: rows of 128 bytes (the TMA swizzle span)
 constexpr int kMaxSlots = 6;
@@ -52,12 +55,11 @@ struct TcSmall {
     unsigned long long p_full, pv_done, q_full, q_empty, drain;
     uint32_t tmem_base;
     int abort_flag;
-    int pad[2];
-    float m_ref[128];
-    float alpha[128];
-    float inv_l[128];
-    float wred[4][128];
-    unsigned long long dmask[128][2];
+    alignas(16) float m_ref[128];
+    alignas(16) float alpha[128];
+    alignas(16) float inv_l[128];
+    alignas(16) float wred[kSoftmaxGroups][4][64];
+    alignas(16) unsigned long long dmask[128][2];
     int cum_tiles[kMaxBatchTc + 1];
 };
 
@@ -140,41 +142,44 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t desc_a, uint64_
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
 }
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
-    uint32_t r[16];
+// eight consecutive fp32 columns of this thread's TMEM lane; the caller waits with tc_wait_ld()
+__device__ __forceinline__ void tc_ld8(uint32_t taddr, float* v) {
+    uint32_t r[8];
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
         : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
-__device__ __forceinline__ void tc_st16(uint32_t taddr, const float* v) {
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_st8(uint32_t taddr, const float* v) {
     asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
         ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
           "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
-          "r"(__float_as_uint(v[7])), "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])),
-          "r"(__float_as_uint(v[11])), "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])),
-          "r"(__float_as_uint(v[15])) : "memory");
-    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+          "r"(__float_as_uint(v[7])) : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
 __device__ __forceinline__ float warp_max_f32(float v) {
     float r;
     asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
     return r;
 }
-// barrier 1 over the 128 softmax threads, returning the OR of `pred`
-__device__ __forceinline__ bool softmax_sync_any(bool pred) {
+// named barrier `id` over the 128 threads of one softmax warpgroup, returning the OR of `pred`
+__device__ __forceinline__ bool group_sync_any(int id, bool pred) {
     uint32_t r;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 p, %1, 0;\n\t"
-        "bar.red.or.pred q, 1, 128, p;\n\t"
+        "setp.ne.u32 p, %2, 0;\n\t"
+        "bar.red.or.pred q, %1, 128, p;\n\t"
         "selp.u32 %0, 1, 0, q;\n\t}"
-        : "=r"(r) : "r"((uint32_t)pred) : "memory");
+        : "=r"(r) : "r"(id), "r"((uint32_t)pred) : "memory");
     return r != 0;
 }
 
@@ -245,7 +250,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         for (int i = 0; i < kMaxSlots; ++i) { mbar_init(&sm->slot_full[i], 1); mbar_init(&sm->slot_empty[i], 1); }
         mbar_init(&sm->s_full[0], 1);
         mbar_init(&sm->s_full[1], 1);
-        mbar_init(&sm->p_full, 128);
+        mbar_init(&sm->p_full, 128 * kSoftmaxGroups);
         mbar_init(&sm->pv_done, 1);
         mbar_init(&sm->q_full, 1);
         mbar_init(&sm->q_empty, 1);
@@ -272,7 +277,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     const long long t_begin = (long long)cta * total / G, t_end = (long long)(cta + 1) * total / G;
     if (t_begin >= t_end) return;              // uniform for the whole block: nothing allocated yet
 
-    if (warp == 5) {
+    if (warp == kMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -282,7 +287,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     const uint32_t tmem = *(volatile uint32_t*)&sm->tmem_base;
     WorkspaceHeader* hdr = p.header;
 
-    if (warp == 4) {
+    if (warp == kProducerWarp) {
         // =========================================================== TMA producer
         if (lane == 0) {
             long long t = t_begin;
@@ -327,7 +332,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 }
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == kMmaWarp) {
         // =========================================================== MMA issuer
         if (lane == 0) {
             long long t = t_begin;
@@ -394,27 +399,39 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             }
         }
     } else {
-        // =========================================================== softmax / mask / epilogue (128 threads)
-        const int r = tid;
-        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+        // =========================================================== softmax / mask / epilogue
+        // Two warpgroups work on the same tile and split its query columns in groups of eight; thread r of
+        // either group owns key row r (TMEM lane r).  Per tile the common case is one pass: load S^T, subtract
+        // the running reference, check that nothing exceeds it by more than 2^kLazyTau (one vote per group),
+        // exponentiate, add to the per-thread row sums and store P^T.  Only when the vote fires (always on the
+        // first tile of a segment) are exact column maxima computed and O^T rescaled.
+        constexpr int CPT = NCH;                       // 8-column groups per thread (two groups share 16*NCH columns)
+        constexpr bool KEEP = CPT <= 4;                // keep the shifted scores in registers between the passes
+        const int wg = warp >> 2, wq = warp & 3;
+        const int r = tid & 127;
+        const int bar_id = 1 + wg;
+        const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
         long long t = t_begin;
         uint32_t u = 0, g = 0;
         bool failed = false;
-        float acc_l[NCH][16];
+        float acc_l[CPT][8];
         while (t < t_end) {
             Segment s;
             locate(sm, p, t, s);
             const int cnt = (int)min((long long)(s.Tb - s.lt), t_end - t);
-            const int nch = (s.Nb + 15) >> 4;
             const int bh = s.b * p.H + s.h;
+            const int ng8 = (s.Nb + 7) >> 3;
+            const int g0 = wg * CPT;
+            const int ncg = max(0, min(CPT, ng8 - g0));          // 8-column groups of this thread in this segment
+            const int col0 = g0 * 8;
             const unsigned long long nb_lo = s.Nb >= 64 ? ~0ull : ((1ull << s.Nb) - 1ull);
             const unsigned long long nb_hi = s.Nb >= 128 ? ~0ull : (s.Nb > 64 ? ((1ull << (s.Nb - 64)) - 1ull) : 0ull);
-            sm->m_ref[r] = -INFINITY;
+            if (r < ncg * 8) sm->m_ref[col0 + r] = -INFINITY;
 #pragma unroll
-            for (int c = 0; c < NCH; ++c)
+            for (int j = 0; j < CPT; ++j)
 #pragma unroll
-                for (int k = 0; k < 16; ++k) acc_l[c][k] = 0.f;
-            if (softmax_sync_any(failed)) { failed = true; break; }
+                for (int k = 0; k < 8; ++k) acc_l[j][k] = 0.f;
+            if (group_sync_any(bar_id, failed)) { failed = true; break; }
 
             for (int i = 0; i < cnt; ++i) {
                 const uint32_t gi = g + (uint32_t)i, sb = gi & 1u;
@@ -422,95 +439,166 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 const bool tree = lti >= s.nP;
                 const int row0 = (tree ? lti - s.nP : lti) * kTile;
                 const int valid = min(kTile, (tree ? s.Nb : s.L) - row0);
-                // queries that may see this thread's key
-                unsigned long long cm0 = 0, cm1 = 0;
-                if (r < valid) {
-                    cm0 = nb_lo; cm1 = nb_hi;
-                    if (tree) { cm0 &= sm->dmask[row0 + r][0]; cm1 &= sm->dmask[row0 + r][1]; }
+                const bool full_tile = !tree && valid == kTile;   // every key visible to every query: no masking
+                // queries that may see this thread's key (bit n), shifted to this thread's first column
+                unsigned long long cm = 0;
+                if (!full_tile && r < valid) {
+                    unsigned long long c0 = nb_lo, c1 = nb_hi;
+                    if (tree) { c0 &= sm->dmask[row0 + r][0]; c1 &= sm->dmask[row0 + r][1]; }
+                    cm = col0 >= 64 ? (c1 >> (col0 - 64)) : (col0 == 0 ? c0 : ((c0 >> col0) | (c1 << (64 - col0))));
                 }
                 if (!mbar_wait(&sm->s_full[sb], (gi >> 1) & 1u, sm, hdr, 7)) failed = true;
                 tc_fence_after();
-                const uint32_t s_addr = tmem + lane_addr + (sb ? kColS1 : 0);
+                const uint32_t s_addr = tmem + lane_addr + (sb ? kColS1 : 0) + col0;
 
-                // ---- pass 1: per-query maximum over the 128 keys of the tile
+                // ---- pass A: scores minus the running reference, and the largest excess
+                float y[KEEP ? CPT : 1][8];
+                float dmax = -INFINITY;
+                if (KEEP) {
 #pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    if (c < nch) {
-                        float v[16];
-                        tc_ld16(s_addr + 16 * c, v);
-                        const uint32_t bits = (uint32_t)(((c < 4 ? cm0 : cm1) >> ((c & 3) * 16)) & 0xFFFFull);
-                        float mine = -INFINITY;
+                    for (int j = 0; j < CPT; ++j)
+                        if (j < ncg) tc_ld8(s_addr + 8 * j, y[KEEP ? j : 0]);
+                    tc_wait_ld();
+                }
 #pragma unroll
-                        for (int k = 0; k < 16; ++k) {
-                            const float x = ((bits >> k) & 1u) ? v[k] * p.scale_log2 : -INFINITY;
-                            const float mx = warp_max_f32(x);
-                            if (lane == k) mine = mx;
+                for (int j = 0; j < CPT; ++j) {
+                    if (j < ncg) {
+                        float v[8];
+                        if (KEEP) {
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) v[k] = y[KEEP ? j : 0][k];
+                        } else {
+                            tc_ld8(s_addr + 8 * j, v);
+                            tc_wait_ld();
                         }
-                        if (lane < 16) sm->wred[warp][16 * c + lane] = mine;
+                        const float4 m0 = *reinterpret_cast<const float4*>(&sm->m_ref[col0 + 8 * j]);
+                        const float4 m1 = *reinterpret_cast<const float4*>(&sm->m_ref[col0 + 8 * j + 4]);
+                        const float mr[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+                        const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            float yy = fmaf(v[k], p.scale_log2, -mr[k]);
+                            if (!full_tile && !((bits >> k) & 1u)) yy = -INFINITY;
+                            dmax = fmaxf(dmax, yy);
+                            if (KEEP) y[KEEP ? j : 0][k] = yy;
+                        }
                     }
                 }
-                if (softmax_sync_any(failed)) { failed = true; break; }
-                // one thread per query folds the four warps' maxima into the running reference
-                bool need = false;
-                if (r < 16 * nch) {
-                    const float tm = fmaxf(fmaxf(sm->wred[0][r], sm->wred[1][r]), fmaxf(sm->wred[2][r], sm->wred[3][r]));
-                    const float mo = sm->m_ref[r];
-                    float a = 1.f;
-                    if (tm > mo + kLazyTau || (mo == -INFINITY && tm > -INFINITY)) {
-                        a = (mo == -INFINITY) ? 0.f : exp2f(mo - tm);
-                        sm->m_ref[r] = tm;
-                        need = (i > 0) && (mo != -INFINITY);     // accumulated O^T and sums must be rescaled
-                    }
-                    sm->alpha[r] = a;
-                }
-                const bool rescale = softmax_sync_any(need);
-
-                // P buffer (and O, if it is rescaled) must no longer be in use by the previous tile's MMA
-                if (gi > 0 && !mbar_wait(&sm->pv_done, (gi - 1u) & 1u, sm, hdr, 8)) failed = true;
-                if (rescale) {
-                    tc_fence_after();
+                if (group_sync_any(bar_id, dmax > kLazyTau || failed)) {
+                    if (*(volatile int*)&sm->abort_flag) { failed = true; break; }
+                    // ---- slow path: exact per-query maxima of this tile, new reference, rescale what was accumulated
 #pragma unroll
-                    for (int c = 0; c < NCH; ++c) {
-                        if (c < nch) {
-                            float o[16];
-                            tc_ld16(tmem + lane_addr + kColO + 16 * c, o);
+                    for (int j = 0; j < CPT; ++j) {
+                        if (j < ncg) {
+                            float v[8];
+                            tc_ld8(s_addr + 8 * j, v);
+                            tc_wait_ld();
+                            const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
+                            float mine = -INFINITY;
 #pragma unroll
-                            for (int k = 0; k < 16; ++k) {
-                                const float a = sm->alpha[16 * c + k];
-                                o[k] *= a;
-                                acc_l[c][k] *= a;
+                            for (int k = 0; k < 8; ++k) {
+                                const float x = (full_tile || ((bits >> k) & 1u)) ? v[k] * p.scale_log2 : -INFINITY;
+                                const float mx = warp_max_f32(x);
+                                if (lane == k) mine = mx;
                             }
-                            tc_st16(tmem + lane_addr + kColO + 16 * c, o);
+                            if (lane < 8) sm->wred[wg][wq][8 * j + lane] = mine;
+                        }
+                    }
+                    group_sync_any(bar_id, false);
+                    bool need = false;
+                    if (r < ncg * 8) {
+                        const float tm = fmaxf(fmaxf(sm->wred[wg][0][r], sm->wred[wg][1][r]),
+                                               fmaxf(sm->wred[wg][2][r], sm->wred[wg][3][r]));
+                        const float mo = sm->m_ref[col0 + r];
+                        float a = 1.f;
+                        if (tm > mo) {
+                            a = (mo == -INFINITY) ? 0.f : exp2f(mo - tm);
+                            sm->m_ref[col0 + r] = tm;
+                            need = (i > 0) && (mo != -INFINITY);
+                        }
+                        sm->alpha[col0 + r] = a;
+                    }
+                    const bool rescale = group_sync_any(bar_id, need);
+                    if (gi > 0 && !mbar_wait(&sm->pv_done, (gi - 1u) & 1u, sm, hdr, 8)) failed = true;
+                    if (rescale) {
+                        tc_fence_after();
+#pragma unroll
+                        for (int j = 0; j < CPT; ++j) {
+                            if (j < ncg) {
+                                float o[8];
+                                tc_ld8(tmem + lane_addr + kColO + col0 + 8 * j, o);
+                                tc_wait_ld();
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) {
+                                    const float a = sm->alpha[col0 + 8 * j + k];
+                                    o[k] *= a;
+                                    acc_l[j][k] *= a;
+                                }
+                                tc_st8(tmem + lane_addr + kColO + col0 + 8 * j, o);
+                            }
+                        }
+                        tc_wait_st();
+                    }
+                    if (KEEP) {
+#pragma unroll
+                        for (int j = 0; j < CPT; ++j) {
+                            if (j < ncg) {
+                                float v[8];
+                                tc_ld8(s_addr + 8 * j, v);
+                                tc_wait_ld();
+                                const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) {
+                                    float yy = fmaf(v[k], p.scale_log2, -sm->m_ref[col0 + 8 * j + k]);
+                                    if (!full_tile && !((bits >> k) & 1u)) yy = -INFINITY;
+                                    y[KEEP ? j : 0][k] = yy;
+                                }
+                            }
                         }
                     }
                 }
 
-                // ---- pass 2: probabilities, row sums, P^T tile for the second MMA
+                // P buffer must no longer be read by the previous tile's MMA; this wait also keeps every thread
+                // within one phase of the p_full barrier
+                if (gi > 0 && !mbar_wait(&sm->pv_done, (gi - 1u) & 1u, sm, hdr, 8)) failed = true;
+
+                // ---- pass B: probabilities, row sums, P^T for the second MMA
 #pragma unroll
-                for (int c = 0; c < NCH; ++c) {
-                    if (c < nch) {
-                        float v[16];
-                        tc_ld16(s_addr + 16 * c, v);
-                        const uint32_t bits = (uint32_t)(((c < 4 ? cm0 : cm1) >> ((c & 3) * 16)) & 0xFFFFull);
-                        uint32_t packed[8];
+                for (int j = 0; j < CPT; ++j) {
+                    if (j < ncg) {
+                        float yy[8];
+                        if (KEEP) {
 #pragma unroll
-                        for (int k = 0; k < 16; k += 2) {
-                            const float2 mr = *reinterpret_cast<const float2*>(&sm->m_ref[16 * c + k]);
-                            const float p0 = ((bits >> k) & 1u) ? exp2f(v[k] * p.scale_log2 - mr.x) : 0.f;
-                            const float p1 = ((bits >> (k + 1)) & 1u) ? exp2f(v[k + 1] * p.scale_log2 - mr.y) : 0.f;
-                            acc_l[c][k] += p0;
-                            acc_l[c][k + 1] += p1;
+                            for (int k = 0; k < 8; ++k) yy[k] = y[KEEP ? j : 0][k];
+                        } else {
+                            float v[8];
+                            tc_ld8(s_addr + 8 * j, v);
+                            tc_wait_ld();
+                            const float4 m0 = *reinterpret_cast<const float4*>(&sm->m_ref[col0 + 8 * j]);
+                            const float4 m1 = *reinterpret_cast<const float4*>(&sm->m_ref[col0 + 8 * j + 4]);
+                            const float mr[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+                            const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                yy[k] = fmaf(v[k], p.scale_log2, -mr[k]);
+                                if (!full_tile && !((bits >> k) & 1u)) yy[k] = -INFINITY;
+                            }
+                        }
+                        uint32_t packed[4];
+#pragma unroll
+                        for (int k = 0; k < 8; k += 2) {
+                            const float p0 = ex2_approx(yy[k]), p1 = ex2_approx(yy[k + 1]);   // 2^-inf = 0 for masked entries
+                            acc_l[j][k] += p0;
+                            acc_l[j][k + 1] += p1;
                             __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
                             packed[k >> 1] = *reinterpret_cast<uint32_t*>(&h2);
                         }
-                        uint4* dst0 = reinterpret_cast<uint4*>(p_buf + (size_t)(2 * c) * 2048 + (size_t)r * 16);
-                        uint4* dst1 = reinterpret_cast<uint4*>(p_buf + (size_t)(2 * c + 1) * 2048 + (size_t)r * 16);
-                        *dst0 = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-                        *dst1 = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+                        *reinterpret_cast<uint4*>(p_buf + (size_t)(g0 + j) * 2048 + (size_t)r * 16) =
+                            make_uint4(packed[0], packed[1], packed[2], packed[3]);
                     }
                 }
                 // rows of the V tile past the end of the prefix / tree may hold anything: make them zero
-                if (valid < kTile) {
+                if (wg == 0 && valid < kTile) {
                     const uint32_t uv = u + 2u * (uint32_t)i + 1u, slot = uv % (uint32_t)NS;
                     if (!mbar_wait(&sm->slot_full[slot], (uv / (uint32_t)NS) & 1u, sm, hdr, 9)) failed = true;
                     if (r >= valid && !failed) {
@@ -524,47 +612,48 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 tc_fence_before();
                 mbar_arrive(&sm->p_full);
             }
-            if (softmax_sync_any(failed)) { failed = true; break; }
+            if (group_sync_any(bar_id, failed)) { failed = true; break; }
 
-            // ---- epilogue of the segment
+            // ---- epilogue of the segment: each group finishes its own query columns
             const uint32_t glast = g + (uint32_t)cnt - 1u;
             if (!mbar_wait(&sm->pv_done, glast & 1u, sm, hdr, 10)) failed = true;
             tc_fence_after();
 #pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-                if (c < nch) {
+            for (int j = 0; j < CPT; ++j) {
+                if (j < ncg) {
                     float mine = 0.f;
 #pragma unroll
-                    for (int k = 0; k < 16; ++k) {
-                        float v = acc_l[c][k];
+                    for (int k = 0; k < 8; ++k) {
+                        float v = acc_l[j][k];
 #pragma unroll
                         for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
                         if (lane == k) mine = v;
                     }
-                    if (lane < 16) sm->wred[warp][16 * c + lane] = mine;
+                    if (lane < 8) sm->wred[wg][wq][8 * j + lane] = mine;
                 }
             }
-            if (softmax_sync_any(failed)) { failed = true; break; }
+            if (group_sync_any(bar_id, failed)) { failed = true; break; }
             const bool full = (cnt == s.Tb);
             const int slot_id = 2 * cta + (t > t_begin ? 1 : 0);
-            if (r < 16 * nch) {
-                const float l = (sm->wred[0][r] + sm->wred[1][r]) + (sm->wred[2][r] + sm->wred[3][r]);
+            if (r < ncg * 8) {
+                const float l = (sm->wred[wg][0][r] + sm->wred[wg][1][r]) + (sm->wred[wg][2][r] + sm->wred[wg][3][r]);
                 if (full) {
-                    sm->inv_l[r] = l > 0.f ? 1.f / l : 0.f;
+                    sm->inv_l[col0 + r] = l > 0.f ? 1.f / l : 0.f;
                 } else {
-                    p.part_ml[((size_t)slot_id * 2 + 0) * 128 + r] = sm->m_ref[r];
-                    p.part_ml[((size_t)slot_id * 2 + 1) * 128 + r] = l;
+                    p.part_ml[((size_t)slot_id * 2 + 0) * 128 + col0 + r] = sm->m_ref[col0 + r];
+                    p.part_ml[((size_t)slot_id * 2 + 1) * 128 + col0 + r] = l;
                 }
             }
-            if (softmax_sync_any(false)) { failed = true; break; }
+            group_sync_any(bar_id, false);
 #pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-                if (c < nch) {
-                    float o[16];
-                    tc_ld16(tmem + lane_addr + kColO + 16 * c, o);
+            for (int j = 0; j < CPT; ++j) {
+                if (j < ncg) {
+                    float o[8];
+                    tc_ld8(tmem + lane_addr + kColO + col0 + 8 * j, o);
+                    tc_wait_ld();
 #pragma unroll
-                    for (int k = 0; k < 16; ++k) {
-                        const int n = 16 * c + k;
+                    for (int k = 0; k < 8; ++k) {
+                        const int n = col0 + 8 * j + k;
                         if (n < s.Nb) {
                             if (full) p.out[((size_t)bh * p.N + n) * 128 + r] = __float2bfloat16_rn(o[k] * sm->inv_l[n]);
                             else p.part_o[((size_t)slot_id * 128 + n) * 128 + r] = o[k];
@@ -573,7 +662,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 }
             }
             tc_fence_before();
-            if (softmax_sync_any(false)) { failed = true; break; }
+            group_sync_any(bar_id, false);
             g += (uint32_t)cnt;
             u += 2u * (uint32_t)cnt;
             t += cnt;
@@ -583,7 +672,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     // ---- tear-down
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == kMmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
