@@ -237,16 +237,13 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = gridDim.x, cta = blockIdx.x;
 
-    // ---- set-up: tile counts per sequence, barriers, tensor memory, transposed tree mask
+    // ---- set-up: tile counts per sequence, barriers, tensor memory
+    for (int b = tid; b < p.B; b += kTcThreads) {
+        const int L = min(max(p.seq_lens[b], 0), p.L_max);
+        const int Nb = p.n_active ? min(max(p.n_active[b], 0), p.N) : p.N;
+        sm->cum_tiles[b + 1] = tiles_of(L, Nb);
+    }
     if (tid == 0) {
-        int acc = 0;
-        for (int b = 0; b < p.B; ++b) {
-            sm->cum_tiles[b] = acc;
-            const int L = min(max(p.seq_lens[b], 0), p.L_max);
-            const int Nb = p.n_active ? min(max(p.n_active[b], 0), p.N) : p.N;
-            acc += tiles_of(L, Nb);
-        }
-        sm->cum_tiles[p.B] = acc;
         for (int i = 0; i < kMaxSlots; ++i) { mbar_init(&sm->slot_full[i], 1); mbar_init(&sm->slot_empty[i], 1); }
         mbar_init(&sm->s_full[0], 1);
         mbar_init(&sm->s_full[1], 1);
@@ -258,19 +255,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (tid < 128) {
-        // dmask[t] = set of queries that may see tree key t (bit n of the transposed ancestor matrix)
-        unsigned long long w0 = 0, w1 = 0;
-        if (tid < p.N) {
-            for (int n = 0; n < p.N; ++n) {
-                const unsigned long long word = p.anc[(size_t)n * p.words + (tid >> 6)];
-                if ((word >> (tid & 63)) & 1ull) {
-                    if (n < 64) w0 |= 1ull << n; else w1 |= 1ull << (n - 64);
-                }
-            }
-        }
-        sm->dmask[tid][0] = w0;
-        sm->dmask[tid][1] = w1;
+    __syncthreads();
+    if (tid == 0) {
+        int acc = 0;
+        sm->cum_tiles[0] = 0;
+        for (int b = 1; b <= p.B; ++b) { acc += sm->cum_tiles[b]; sm->cum_tiles[b] = acc; }
     }
     __syncthreads();
     const long long total = (long long)p.H * sm->cum_tiles[p.B];
@@ -410,6 +399,23 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         const int wg = warp >> 2, wq = warp & 3;
         const int r = tid & 127;
         const int bar_id = 1 + wg;
+        if (wg == 0) {
+            // dmask[t] = set of queries that may see tree key t: the ancestor bitsets transposed.  Built while
+            // the first tiles are in flight; first read at a tree tile, after several group barriers.
+            unsigned long long w0 = 0, w1 = 0;
+            if (r < p.N) {
+#pragma unroll 8
+                for (int n = 0; n < p.N; ++n) {
+                    const unsigned long long word = p.anc[(size_t)n * p.words + (r >> 6)];
+                    const unsigned long long bit = (word >> (r & 63)) & 1ull;
+                    if (n < 64) w0 |= bit << n; else w1 |= bit << (n - 64);
+                }
+            }
+            sm->dmask[r][0] = w0;
+            sm->dmask[r][1] = w1;
+        }
+        // both groups read dmask: order its writes before any tile is processed
+        asm volatile("bar.sync 3, 256;" ::: "memory");
         const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
         long long t = t_begin;
         uint32_t u = 0, g = 0;
@@ -679,47 +685,71 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
 }
 
 // Merges the partials of every (sequence, head) whose tiles were split over several thread blocks.
-// grid: B * H blocks of 128 threads (thread = output column d).
-__global__ void __launch_bounds__(128)
+// grid: B * H blocks of 128 x kCombineRows threads: thread (d, y) produces output column d of queries
+// y, y + kCombineRows, ...  All loads of one query are independent, so a block costs a few memory latencies.
+constexpr int kCombineRows = 8;
+constexpr int kCombineMaxParts = 8;
+
+__global__ void __launch_bounds__(128 * kCombineRows)
 tree_attention_tc_combine_kernel(const TcParams p, int G) {
-    __shared__ int s_cum[2];
+    __shared__ int s_tiles[kMaxBatchTc];
+    __shared__ int s_info[2];
     __shared__ long long s_total;
-    const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H, d = threadIdx.x;
-    if (d == 0) {
-        int acc = 0, mine = 0, tb = 0;
-        for (int i = 0; i < p.B; ++i) {
-            const int L = min(max(p.seq_lens[i], 0), p.L_max);
-            const int Nb = p.n_active ? min(max(p.n_active[i], 0), p.N) : p.N;
-            const int ti = tiles_of(L, Nb);
-            if (i == b) { mine = acc; tb = ti; }
-            acc += ti;
-        }
-        s_cum[0] = mine; s_cum[1] = tb; s_total = (long long)p.H * acc;
+    const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H, d = threadIdx.x, y = threadIdx.y;
+    const int flat = y * 128 + d;
+    for (int i = flat; i < p.B; i += 128 * kCombineRows) {
+        const int L = min(max(p.seq_lens[i], 0), p.L_max);
+        const int Nb = p.n_active ? min(max(p.n_active[i], 0), p.N) : p.N;
+        s_tiles[i] = tiles_of(L, Nb);
     }
     __syncthreads();
-    const int Tb = s_cum[1];
+    if (flat == 0) {
+        int acc = 0, mine = 0;
+        for (int i = 0; i < p.B; ++i) { if (i == b) mine = acc; acc += s_tiles[i]; }
+        s_info[0] = mine; s_info[1] = s_tiles[b]; s_total = (long long)p.H * acc;
+    }
+    __syncthreads();
+    const int Tb = s_info[1];
     if (Tb == 0) return;
     const long long total = s_total;
-    const long long t0 = (long long)p.H * s_cum[0] + (long long)h * Tb, t1 = t0 + Tb;
+    const long long t0 = (long long)p.H * s_info[0] + (long long)h * Tb, t1 = t0 + Tb;
     const int c_lo = (int)(((t0 + 1) * G + total - 1) / total - 1), c_hi = (int)((t1 * G + total - 1) / total - 1);
     if (c_lo == c_hi) return;                  // one block saw every tile and wrote the result itself
     const int Nb = p.n_active ? min(max(p.n_active[b], 0), p.N) : p.N;
-    for (int n = 0; n < Nb; ++n) {
+    for (int n = y; n < Nb; n += kCombineRows) {
         float M = -INFINITY;
-        for (int c = c_lo; c <= c_hi; ++c) {
-            const long long start = (long long)c * total / G;
-            const int slot = 2 * c + (t0 > start ? 1 : 0);
-            M = fmaxf(M, p.part_ml[((size_t)slot * 2 + 0) * 128 + n]);
+        for (int c0 = c_lo; c0 <= c_hi; c0 += kCombineMaxParts) {
+            float ms[kCombineMaxParts];
+#pragma unroll
+            for (int i = 0; i < kCombineMaxParts; ++i) {
+                const int c = c0 + i;
+                const long long start = (long long)c * total / G;
+                const int slot = 2 * c + (t0 > start ? 1 : 0);
+                ms[i] = c <= c_hi ? p.part_ml[((size_t)slot * 2 + 0) * 128 + n] : -INFINITY;
+            }
+#pragma unroll
+            for (int i = 0; i < kCombineMaxParts; ++i) M = fmaxf(M, ms[i]);
         }
         float lsum = 0.f, acc = 0.f;
-        for (int c = c_lo; c <= c_hi; ++c) {
-            const long long start = (long long)c * total / G;
-            const int slot = 2 * c + (t0 > start ? 1 : 0);
-            const float ms = p.part_ml[((size_t)slot * 2 + 0) * 128 + n];
-            if (ms == -INFINITY) continue;
-            const float w = exp2f(ms - M);
-            lsum += w * p.part_ml[((size_t)slot * 2 + 1) * 128 + n];
-            acc = fmaf(w, p.part_o[((size_t)slot * 128 + n) * 128 + d], acc);
+        for (int c0 = c_lo; c0 <= c_hi; c0 += kCombineMaxParts) {
+            float ms[kCombineMaxParts], ls[kCombineMaxParts], os[kCombineMaxParts];
+#pragma unroll
+            for (int i = 0; i < kCombineMaxParts; ++i) {
+                const int c = c0 + i;
+                const long long start = (long long)c * total / G;
+                const int slot = 2 * c + (t0 > start ? 1 : 0);
+                const bool on = c <= c_hi;
+                ms[i] = on ? p.part_ml[((size_t)slot * 2 + 0) * 128 + n] : -INFINITY;
+                ls[i] = on ? p.part_ml[((size_t)slot * 2 + 1) * 128 + n] : 0.f;
+                os[i] = on ? p.part_o[((size_t)slot * 128 + n) * 128 + d] : 0.f;
+            }
+#pragma unroll
+            for (int i = 0; i < kCombineMaxParts; ++i) {
+                if (ms[i] == -INFINITY) continue;
+                const float w = exp2f(ms[i] - M);
+                lsum = fmaf(w, ls[i], lsum);
+                acc = fmaf(w, os[i], acc);
+            }
         }
         p.out[((size_t)bh * p.N + n) * 128 + d] = __float2bfloat16_rn(lsum > 0.f ? acc / lsum : 0.f);
     }
@@ -833,7 +863,7 @@ int tree_attention_tc(const AttentionArgs& a, WorkspaceHeader* header, void* scr
     }
     if (st != MCSD_OK) return st;
     count_launches(1);
-    tree_attention_tc_combine_kernel<<<bh, 128, 0, stream>>>(p, grid);
+    tree_attention_tc_combine_kernel<<<bh, dim3(128, kCombineRows), 0, stream>>>(p, grid);
     MCSD_CUDA_CHECK(cudaGetLastError());
     count_launches(1);
     return MCSD_OK;
