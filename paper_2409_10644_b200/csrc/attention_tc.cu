@@ -688,7 +688,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
 // grid: B * H blocks of 128 x kCombineRows threads: thread (d, y) produces output column d of queries
 // y, y + kCombineRows, ...  All loads of one query are independent, so a block costs a few memory latencies.
 constexpr int kCombineRows = 8;
-constexpr int kCombineMaxParts = 8;
+constexpr int kCombineMaxParts = 64;           // a (sequence, head) has at most 34 tiles, so at most 35 pieces
 
 __global__ void __launch_bounds__(128 * kCombineRows)
 tree_attention_tc_combine_kernel(const TcParams p, int G) {
@@ -716,40 +716,29 @@ tree_attention_tc_combine_kernel(const TcParams p, int G) {
     const int c_lo = (int)(((t0 + 1) * G + total - 1) / total - 1), c_hi = (int)((t1 * G + total - 1) / total - 1);
     if (c_lo == c_hi) return;                  // one block saw every tile and wrote the result itself
     const int Nb = p.n_active ? min(max(p.n_active[b], 0), p.N) : p.N;
+    // partial slot of every thread block that saw a piece of this (sequence, head): worked out once
+    __shared__ int s_slot[kCombineMaxParts];
+    const int nparts = min(c_hi - c_lo + 1, kCombineMaxParts);
+    if (flat < nparts) {
+        const int c = c_lo + flat;
+        const long long start = (long long)c * total / G;
+        s_slot[flat] = 2 * c + (t0 > start ? 1 : 0);
+    }
+    __syncthreads();
     for (int n = y; n < Nb; n += kCombineRows) {
         float M = -INFINITY;
-        for (int c0 = c_lo; c0 <= c_hi; c0 += kCombineMaxParts) {
-            float ms[kCombineMaxParts];
-#pragma unroll
-            for (int i = 0; i < kCombineMaxParts; ++i) {
-                const int c = c0 + i;
-                const long long start = (long long)c * total / G;
-                const int slot = 2 * c + (t0 > start ? 1 : 0);
-                ms[i] = c <= c_hi ? p.part_ml[((size_t)slot * 2 + 0) * 128 + n] : -INFINITY;
-            }
-#pragma unroll
-            for (int i = 0; i < kCombineMaxParts; ++i) M = fmaxf(M, ms[i]);
-        }
+#pragma unroll 4
+        for (int i = 0; i < nparts; ++i) M = fmaxf(M, p.part_ml[((size_t)s_slot[i] * 2 + 0) * 128 + n]);
         float lsum = 0.f, acc = 0.f;
-        for (int c0 = c_lo; c0 <= c_hi; c0 += kCombineMaxParts) {
-            float ms[kCombineMaxParts], ls[kCombineMaxParts], os[kCombineMaxParts];
-#pragma unroll
-            for (int i = 0; i < kCombineMaxParts; ++i) {
-                const int c = c0 + i;
-                const long long start = (long long)c * total / G;
-                const int slot = 2 * c + (t0 > start ? 1 : 0);
-                const bool on = c <= c_hi;
-                ms[i] = on ? p.part_ml[((size_t)slot * 2 + 0) * 128 + n] : -INFINITY;
-                ls[i] = on ? p.part_ml[((size_t)slot * 2 + 1) * 128 + n] : 0.f;
-                os[i] = on ? p.part_o[((size_t)slot * 128 + n) * 128 + d] : 0.f;
-            }
-#pragma unroll
-            for (int i = 0; i < kCombineMaxParts; ++i) {
-                if (ms[i] == -INFINITY) continue;
-                const float w = exp2f(ms[i] - M);
-                lsum = fmaf(w, ls[i], lsum);
-                acc = fmaf(w, os[i], acc);
-            }
+#pragma unroll 4
+        for (int i = 0; i < nparts; ++i) {
+            const int slot = s_slot[i];
+            const float ms = p.part_ml[((size_t)slot * 2 + 0) * 128 + n];
+            const float ls = p.part_ml[((size_t)slot * 2 + 1) * 128 + n];
+            const float os = p.part_o[((size_t)slot * 128 + n) * 128 + d];
+            const float w = ms == -INFINITY ? 0.f : exp2f(ms - M);
+            lsum = fmaf(w, ls, lsum);
+            acc = fmaf(w, os, acc);
         }
         p.out[((size_t)bh * p.N + n) * 128 + d] = __float2bfloat16_rn(lsum > 0.f ? acc / lsum : 0.f);
     }
