@@ -3,8 +3,8 @@
 // One persistent thread block per SM walks a contiguous range of 128-key tiles of the flattened
 // (sequence, head, key tile) space, so the K/V stream of every (sequence, head) is read from HBM exactly once
 // and all SMs carry the same number of tiles whatever the batch and the prefix lengths are.  Where a range
-// boundary cuts a (sequence, head), both sides write an unnormalised partial (running maximum, sum, weighted
-// values) and a combine kernel merges them: split-KV.
+// boundary cuts a (sequence, head), every side writes an unnormalised partial (running maximum, sum, weighted
+// values) and takes a ticket; the block that arrives last combines the partials: split-KV.
 //
 // The problem is set up transposed so that the small dimension (tree tokens, 16..128 per head) is the MMA N
 // and the 128 keys of a tile fill the MMA M:
@@ -45,6 +45,7 @@ constexpr int kMaxBatchTc = 256;
 constexpr int kTmemCols = 512;
 constexpr int kColS1 = 128, kColO = 256;
 constexpr float kLazyTau = 8.0f;              // raise the reference maximum only beyond 2^8
+constexpr int kMaxParts = 64;                 // a (sequence, head) has at most 34 tiles, so at most 35 pieces
 constexpr int kMaxCtas = 160;                 // partial slots are provisioned for this many thread blocks
 constexpr long long kSpinCycles = 4000000000LL;   // about two seconds
 
@@ -55,6 +56,8 @@ struct TcSmall {
     unsigned long long p_full, pv_done, q_full, q_empty, drain;
     uint32_t tmem_base;
     int abort_flag;
+    int merge_parts[kSoftmaxGroups];   // > 0: this block finished a split (sequence, head) last and merges it
+    int merge_slot[kSoftmaxGroups][kMaxParts];
     alignas(16) float m_ref[128];
     alignas(16) float alpha[128];
     alignas(16) float inv_l[128];
@@ -73,6 +76,7 @@ struct TcParams {
     float scale_log2;
     float* part_ml;      // [2 * kMaxCtas][2][128]
     float* part_o;       // [2 * kMaxCtas][128][128]
+    int* counters;       // [B * H][softmax group] arrivals per split (sequence, head); zero between launches
     WorkspaceHeader* header;
     int n_slots;
     int npadq;           // rows of the Q box = 16 * (template chunk count)
@@ -235,7 +239,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     TcSmall* sm = reinterpret_cast<TcSmall*>(q_buf + (size_t)p.npadq * 256);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int G = gridDim.x, cta = blockIdx.x;
+    const int cta = blockIdx.x;
 
     // ---- set-up: tile counts per sequence, barriers, tensor memory
     for (int b = tid; b < p.B; b += kTcThreads) {
@@ -263,8 +267,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     }
     __syncthreads();
     const long long total = (long long)p.H * sm->cum_tiles[p.B];
+    // With fewer tiles than thread blocks only the first `total` blocks work, so every working block owns at
+    // least one tile and the blocks that share a (sequence, head) are consecutive.
+    const int G = (int)min((long long)gridDim.x, total);
+    if (cta >= G) return;                      // uniform for the whole block: nothing allocated yet
     const long long t_begin = (long long)cta * total / G, t_end = (long long)(cta + 1) * total / G;
-    if (t_begin >= t_end) return;              // uniform for the whole block: nothing allocated yet
 
     if (warp == kMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)), "r"(kTmemCols) : "memory");
@@ -668,6 +675,73 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 }
             }
             tc_fence_before();
+            if (!full) {
+                // Split-KV combine: every block that finished a piece of this (sequence, head) takes a ticket;
+                // the last one merges all pieces (its own included) into the output.  The two softmax groups own
+                // disjoint query columns and run this protocol independently of each other.
+                __threadfence();
+                group_sync_any(bar_id, false);
+                if (r == 0) {
+                    const long long t0 = t - s.lt, t1 = t0 + s.Tb;
+                    const int c_lo = (int)(((t0 + 1) * G + total - 1) / total - 1);
+                    const int c_hi = (int)((t1 * G + total - 1) / total - 1);
+                    const int nparts = min(c_hi - c_lo + 1, kMaxParts);
+                    int* counter = p.counters + (size_t)bh * kSoftmaxGroups + wg;
+                    const int old = atomicAdd(counter, 1);
+                    int mine = 0;
+                    if (old == nparts - 1) {
+                        atomicExch(counter, 0);                   // ready for the next launch
+                        __threadfence();
+                        mine = nparts;
+                        for (int i = 0; i < nparts; ++i) {
+                            const long long start = (long long)(c_lo + i) * total / G;
+                            sm->merge_slot[wg][i] = 2 * (c_lo + i) + (t0 > start ? 1 : 0);
+                        }
+                    }
+                    sm->merge_parts[wg] = mine;
+                }
+                group_sync_any(bar_id, false);
+                const int nparts = sm->merge_parts[wg];
+                if (nparts > 0) {
+#pragma unroll
+                    for (int j = 0; j < CPT; ++j) {
+                        if (j < ncg) {
+                            float M[8], lsum[8], acc[8];
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) { M[k] = -INFINITY; lsum[k] = 0.f; acc[k] = 0.f; }
+                            for (int i = 0; i < nparts; ++i) {
+                                const int slot = sm->merge_slot[wg][i];
+                                const float* pm = p.part_ml + ((size_t)slot * 2 + 0) * 128 + col0 + 8 * j;
+                                const float* pl = p.part_ml + ((size_t)slot * 2 + 1) * 128 + col0 + 8 * j;
+                                const float* po = p.part_o + ((size_t)slot * 128 + col0 + 8 * j) * 128 + r;
+                                float ms[8], ls[8], os[8];
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) {
+                                    const bool on = col0 + 8 * j + k < s.Nb;
+                                    ms[k] = on ? __ldcg(pm + k) : -INFINITY;
+                                    ls[k] = on ? __ldcg(pl + k) : 0.f;
+                                    os[k] = on ? __ldcg(po + (size_t)k * 128) : 0.f;
+                                }
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) {
+                                    const float mn = fmaxf(M[k], ms[k]);
+                                    if (mn == -INFINITY) continue;
+                                    const float a = exp2f(M[k] - mn), w = exp2f(ms[k] - mn);
+                                    lsum[k] = fmaf(lsum[k], a, w * ls[k]);
+                                    acc[k] = fmaf(acc[k], a, w * os[k]);
+                                    M[k] = mn;
+                                }
+                            }
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const int n = col0 + 8 * j + k;
+                                if (n < s.Nb)
+                                    p.out[((size_t)bh * p.N + n) * 128 + r] = __float2bfloat16_rn(lsum[k] > 0.f ? acc[k] / lsum[k] : 0.f);
+                            }
+                        }
+                    }
+                }
+            }
             group_sync_any(bar_id, false);
             g += (uint32_t)cnt;
             u += 2u * (uint32_t)cnt;
@@ -681,66 +755,6 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     if (warp == kMmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
-    }
-}
-
-// Merges the partials of every (sequence, head) whose tiles were split over several thread blocks.
-// grid: B * H blocks of 128 x kCombineRows threads: thread (d, y) produces output column d of queries
-// y, y + kCombineRows, ...  All loads of one query are independent, so a block costs a few memory latencies.
-constexpr int kCombineRows = 8;
-constexpr int kCombineMaxParts = 64;           // a (sequence, head) has at most 34 tiles, so at most 35 pieces
-
-__global__ void __launch_bounds__(128 * kCombineRows)
-tree_attention_tc_combine_kernel(const TcParams p, int G) {
-    __shared__ int s_tiles[kMaxBatchTc];
-    __shared__ int s_info[2];
-    __shared__ long long s_total;
-    const int bh = blockIdx.x, b = bh / p.H, h = bh % p.H, d = threadIdx.x, y = threadIdx.y;
-    const int flat = y * 128 + d;
-    for (int i = flat; i < p.B; i += 128 * kCombineRows) {
-        const int L = min(max(p.seq_lens[i], 0), p.L_max);
-        const int Nb = p.n_active ? min(max(p.n_active[i], 0), p.N) : p.N;
-        s_tiles[i] = tiles_of(L, Nb);
-    }
-    __syncthreads();
-    if (flat == 0) {
-        int acc = 0, mine = 0;
-        for (int i = 0; i < p.B; ++i) { if (i == b) mine = acc; acc += s_tiles[i]; }
-        s_info[0] = mine; s_info[1] = s_tiles[b]; s_total = (long long)p.H * acc;
-    }
-    __syncthreads();
-    const int Tb = s_info[1];
-    if (Tb == 0) return;
-    const long long total = s_total;
-    const long long t0 = (long long)p.H * s_info[0] + (long long)h * Tb, t1 = t0 + Tb;
-    const int c_lo = (int)(((t0 + 1) * G + total - 1) / total - 1), c_hi = (int)((t1 * G + total - 1) / total - 1);
-    if (c_lo == c_hi) return;                  // one block saw every tile and wrote the result itself
-    const int Nb = p.n_active ? min(max(p.n_active[b], 0), p.N) : p.N;
-    // partial slot of every thread block that saw a piece of this (sequence, head): worked out once
-    __shared__ int s_slot[kCombineMaxParts];
-    const int nparts = min(c_hi - c_lo + 1, kCombineMaxParts);
-    if (flat < nparts) {
-        const int c = c_lo + flat;
-        const long long start = (long long)c * total / G;
-        s_slot[flat] = 2 * c + (t0 > start ? 1 : 0);
-    }
-    __syncthreads();
-    for (int n = y; n < Nb; n += kCombineRows) {
-        float M = -INFINITY;
-#pragma unroll 4
-        for (int i = 0; i < nparts; ++i) M = fmaxf(M, p.part_ml[((size_t)s_slot[i] * 2 + 0) * 128 + n]);
-        float lsum = 0.f, acc = 0.f;
-#pragma unroll 4
-        for (int i = 0; i < nparts; ++i) {
-            const int slot = s_slot[i];
-            const float ms = p.part_ml[((size_t)slot * 2 + 0) * 128 + n];
-            const float ls = p.part_ml[((size_t)slot * 2 + 1) * 128 + n];
-            const float os = p.part_o[((size_t)slot * 128 + n) * 128 + d];
-            const float w = ms == -INFINITY ? 0.f : exp2f(ms - M);
-            lsum = fmaf(w, ls, lsum);
-            acc = fmaf(w, os, acc);
-        }
-        p.out[((size_t)bh * p.N + n) * 128 + d] = __float2bfloat16_rn(lsum > 0.f ? acc / lsum : 0.f);
     }
 }
 
@@ -794,7 +808,7 @@ bool tc_supported(const AttentionArgs& a) {
 size_t tc_workspace_bytes(int, int, int N, int, int) {
     if (N > 128) return 0;
     return align_up((size_t)2 * kMaxCtas * 2 * 128 * sizeof(float), 256) +
-           align_up((size_t)2 * kMaxCtas * 128 * 128 * sizeof(float), 256);
+           align_up((size_t)2 * kMaxCtas * 128 * 128 * sizeof(float), 256) + (size_t)65536 * kSoftmaxGroups * sizeof(int);
 }
 
 template <int NCH>
@@ -838,6 +852,7 @@ int tree_attention_tc(const AttentionArgs& a, WorkspaceHeader* header, void* scr
     p.scale_log2 = a.scale * 1.4426950408889634f;
     p.part_ml = static_cast<float*>(scratch);
     p.part_o = reinterpret_cast<float*>(static_cast<char*>(scratch) + align_up((size_t)2 * kMaxCtas * 2 * 128 * sizeof(float), 256));
+    p.counters = reinterpret_cast<int*>(reinterpret_cast<char*>(p.part_o) + align_up((size_t)2 * kMaxCtas * 128 * 128 * sizeof(float), 256));
     p.header = header;
     p.n_slots = ns;
     p.npadq = npadq;
@@ -851,9 +866,6 @@ int tree_attention_tc(const AttentionArgs& a, WorkspaceHeader* header, void* scr
         default: st = launch_tc<8>(maps, p, grid, smem_bytes, stream); break;
     }
     if (st != MCSD_OK) return st;
-    count_launches(1);
-    tree_attention_tc_combine_kernel<<<bh, dim3(128, kCombineRows), 0, stream>>>(p, grid);
-    MCSD_CUDA_CHECK(cudaGetLastError());
     count_launches(1);
     return MCSD_OK;
 }
