@@ -35,6 +35,25 @@ UNIT = "tree-tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 
 
+# DRAM traffic of the attention kernel from an `ncu --set full` capture (profiles/tree_attention_tc_b4_ncu_full.md):
+# dram__bytes_read.sum + dram__bytes_write.sum per launch on a 4-sequence case; traffic grows in proportion to the
+# batch.  The figure only holds for the kernel source it was taken on.
+_TRAFFIC_CAPTURE = {"source_sha1_12": "a30cefe10883", "bytes_per_launch": 282_763_776, "batch": 4,
+                    "workload": "long_context_b16"}
+
+
+def _traffic_for(w):
+    import hashlib
+    src = os.path.join(ROOT, "paper_2409_10644_b200", "csrc", "attention_tc.cu")
+    try:
+        sha = hashlib.sha1(open(src, "rb").read()).hexdigest()[:12]
+    except OSError:
+        return None
+    if sha != _TRAFFIC_CAPTURE["source_sha1_12"] or w.name != _TRAFFIC_CAPTURE["workload"]:
+        return None
+    return int(_TRAFFIC_CAPTURE["bytes_per_launch"] * w.B / _TRAFFIC_CAPTURE["batch"])
+
+
 def _peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -338,7 +357,7 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "kernel": "tree attention (one layer: main kernel + split-KV combine)",
                      "achieved": achieved, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s",
                      "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                     "algorithmic_bytes_per_launch": int(abytes), "avg_launch_ms": attn_ms, "traffic": None},
+                     "algorithmic_bytes_per_launch": int(abytes), "avg_launch_ms": attn_ms, "traffic": _traffic_for(w0)},
         "breakdown": {"attention_ms_per_layer": attn_ms, "verify_ms": ver_ms,
                       "verify_nodes_per_s": float(n_act.sum()) / (ver_ms * 1e-3),
                       "verify_all_rows_GBs": ver_rows_bytes / (ver_ms * 1e-3) / 1e9,
