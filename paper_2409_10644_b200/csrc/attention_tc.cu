@@ -35,6 +35,7 @@
 namespace mcsd {
 
 constexpr int kTile = 128;                    // keys per tile
+constexpr int kQBlock = 128;                  // queries per work item
 constexpr int kSoftmaxGroups = 2;              // warpgroups that split the query columns of every tile
 constexpr int kProducerWarp = 4 * kSoftmaxGroups, kMmaWarp = kProducerWarp + 1;
 constexpr int kTcThreads = 32 * (kMmaWarp + 1);
@@ -62,7 +63,7 @@ struct TcSmall {
     alignas(16) float alpha[128];
     alignas(16) float inv_l[128];
     alignas(16) float wred[kSoftmaxGroups][4][64];
-    alignas(16) unsigned long long dmask[128][2];
+    alignas(16) unsigned long long dmask[MCSD_MAX_NODES][3];
     int cum_tiles[kMaxBatchTc + 1];
 };
 
@@ -76,7 +77,7 @@ struct TcParams {
     float scale_log2;
     float* part_ml;      // [2 * kMaxCtas][2][128]
     float* part_o;       // [2 * kMaxCtas][128][128]
-    int* counters;       // [B * H][softmax group] arrivals per split (sequence, head); zero between launches
+    int* counters;       // [B * H][query block][softmax group] arrivals per split work item; zero between launches
     WorkspaceHeader* header;
     int n_slots;
     int npadq;           // rows of the Q box = 16 * (template chunk count)
@@ -200,12 +201,18 @@ __device__ __forceinline__ uint32_t instr_desc(int n, int a_mn_major, int b_mn_m
 }
 
 // ------------------------------------------------------------------ tile bookkeeping
-__device__ __forceinline__ int tiles_of(int L, int Nb) {
+// Queries are processed in blocks of at most 128 (the tensor-memory budget); a tree with more nodes makes
+// each (sequence, head) two work items that read the same keys.  Tiles per work item: prefix tiles, then tree tiles.
+__device__ __forceinline__ int kv_tiles_of(int L, int Nb) {
     return Nb > 0 ? (L + kTile - 1) / kTile + (Nb + kTile - 1) / kTile : 0;
+}
+__device__ __forceinline__ int tiles_of(int L, int Nb) {
+    return kv_tiles_of(L, Nb) * ((Nb + kQBlock - 1) / kQBlock);
 }
 
 struct Segment {
     int b, h, lt, Tb, L, Nb, nP;
+    int qb, q0, Nq, Tkv;      // query block, its first query, its query count, tiles per query block
 };
 
 __device__ __forceinline__ void locate(const TcSmall* sm, const TcParams& p, long long t, Segment& s) {
@@ -221,7 +228,12 @@ __device__ __forceinline__ void locate(const TcSmall* sm, const TcParams& p, lon
     s.nP = (s.L + kTile - 1) / kTile;
     const long long r = t - (long long)p.H * sm->cum_tiles[lo];
     s.h = (int)(r / s.Tb);
-    s.lt = (int)(r % s.Tb);
+    const int rem = (int)(r % s.Tb);
+    s.Tkv = kv_tiles_of(s.L, s.Nb);
+    s.qb = rem / s.Tkv;
+    s.lt = rem % s.Tkv;
+    s.q0 = s.qb * kQBlock;
+    s.Nq = min(kQBlock, s.Nb - s.q0);
 }
 
 // ------------------------------------------------------------------ the kernel
@@ -292,13 +304,13 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             while (t < t_end && ok) {
                 Segment s;
                 locate(sm, p, t, s);
-                const int cnt = (int)min((long long)(s.Tb - s.lt), t_end - t);
+                const int cnt = (int)min((long long)(s.Tkv - s.lt), t_end - t);
                 const int bh = s.b * p.H + s.h;
                 ok = mbar_wait(&sm->q_empty, (seg & 1u) ^ 1u, sm, hdr, 1);
                 if (!ok) break;
                 mbar_expect_tx(&sm->q_full, (uint32_t)p.npadq * 256u);
-                tma_load_3d(smem_u32(q_buf), &tm_q, &sm->q_full, 0, 0, bh);
-                tma_load_3d(smem_u32(q_buf) + (uint32_t)p.npadq * 128u, &tm_q, &sm->q_full, 64, 0, bh);
+                tma_load_3d(smem_u32(q_buf), &tm_q, &sm->q_full, 0, s.q0, bh);
+                tma_load_3d(smem_u32(q_buf) + (uint32_t)p.npadq * 128u, &tm_q, &sm->q_full, 64, s.q0, bh);
                 for (int i = 0; i < cnt && ok; ++i) {
                     const int lti = s.lt + i;
                     const bool tree = lti >= s.nP;
@@ -338,8 +350,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             while (t < t_end && ok) {
                 Segment s;
                 locate(sm, p, t, s);
-                const int cnt = (int)min((long long)(s.Tb - s.lt), t_end - t);
-                const int npad = (s.Nb + 15) & ~15;
+                const int cnt = (int)min((long long)(s.Tkv - s.lt), t_end - t);
+                const int npad = (s.Nq + 15) & ~15;
                 const uint32_t idesc_s = instr_desc(npad, 0, 0), idesc_pv = instr_desc(npad, 1, 1);
                 ok = mbar_wait(&sm->q_full, seg & 1u, sm, hdr, 3);
                 for (int i = 0; i <= cnt && ok; ++i) {
@@ -406,20 +418,21 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         const int wg = warp >> 2, wq = warp & 3;
         const int r = tid & 127;
         const int bar_id = 1 + wg;
-        if (wg == 0) {
+        if (tid < MCSD_MAX_NODES) {
             // dmask[t] = set of queries that may see tree key t: the ancestor bitsets transposed.  Built while
             // the first tiles are in flight; first read at a tree tile, after several group barriers.
-            unsigned long long w0 = 0, w1 = 0;
-            if (r < p.N) {
-#pragma unroll 8
+            unsigned long long w0 = 0, w1 = 0, w2 = 0;
+            if (tid < p.N) {
+#pragma unroll 4
                 for (int n = 0; n < p.N; ++n) {
-                    const unsigned long long word = p.anc[(size_t)n * p.words + (r >> 6)];
-                    const unsigned long long bit = (word >> (r & 63)) & 1ull;
-                    if (n < 64) w0 |= bit << n; else w1 |= bit << (n - 64);
+                    const unsigned long long word = p.anc[(size_t)n * p.words + (tid >> 6)];
+                    const unsigned long long bit = (word >> (tid & 63)) & 1ull;
+                    if (n < 64) w0 |= bit << n; else if (n < 128) w1 |= bit << (n - 64); else w2 |= bit << (n - 128);
                 }
             }
-            sm->dmask[r][0] = w0;
-            sm->dmask[r][1] = w1;
+            sm->dmask[tid][0] = w0;
+            sm->dmask[tid][1] = w1;
+            sm->dmask[tid][2] = w2;
         }
         // both groups read dmask: order its writes before any tile is processed
         asm volatile("bar.sync 3, 256;" ::: "memory");
@@ -431,14 +444,14 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         while (t < t_end) {
             Segment s;
             locate(sm, p, t, s);
-            const int cnt = (int)min((long long)(s.Tb - s.lt), t_end - t);
+            const int cnt = (int)min((long long)(s.Tkv - s.lt), t_end - t);
             const int bh = s.b * p.H + s.h;
-            const int ng8 = (s.Nb + 7) >> 3;
+            const int ng8 = (s.Nq + 7) >> 3;
             const int g0 = wg * CPT;
             const int ncg = max(0, min(CPT, ng8 - g0));          // 8-column groups of this thread in this segment
             const int col0 = g0 * 8;
-            const unsigned long long nb_lo = s.Nb >= 64 ? ~0ull : ((1ull << s.Nb) - 1ull);
-            const unsigned long long nb_hi = s.Nb >= 128 ? ~0ull : (s.Nb > 64 ? ((1ull << (s.Nb - 64)) - 1ull) : 0ull);
+            const unsigned long long nb_lo = s.Nq >= 64 ? ~0ull : ((1ull << s.Nq) - 1ull);
+            const unsigned long long nb_hi = s.Nq >= 128 ? ~0ull : (s.Nq > 64 ? ((1ull << (s.Nq - 64)) - 1ull) : 0ull);
             if (r < ncg * 8) sm->m_ref[col0 + r] = -INFINITY;
 #pragma unroll
             for (int j = 0; j < CPT; ++j)
@@ -457,7 +470,10 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 unsigned long long cm = 0;
                 if (!full_tile && r < valid) {
                     unsigned long long c0 = nb_lo, c1 = nb_hi;
-                    if (tree) { c0 &= sm->dmask[row0 + r][0]; c1 &= sm->dmask[row0 + r][1]; }
+                    if (tree) {                     // bits q0 .. q0+127 of the key's row of the transposed mask
+                        c0 &= sm->dmask[row0 + r][s.qb ? 2 : 0];
+                        c1 &= s.qb ? 0ull : sm->dmask[row0 + r][1];
+                    }
                     cm = col0 >= 64 ? (c1 >> (col0 - 64)) : (col0 == 0 ? c0 : ((c0 >> col0) | (c1 << (64 - col0))));
                 }
                 if (!mbar_wait(&sm->s_full[sb], (gi >> 1) & 1u, sm, hdr, 7)) failed = true;
@@ -646,7 +662,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 }
             }
             if (group_sync_any(bar_id, failed)) { failed = true; break; }
-            const bool full = (cnt == s.Tb);
+            const bool full = (cnt == s.Tkv);
             const int slot_id = 2 * cta + (t > t_begin ? 1 : 0);
             if (r < ncg * 8) {
                 const float l = (sm->wred[wg][0][r] + sm->wred[wg][1][r]) + (sm->wred[wg][2][r] + sm->wred[wg][3][r]);
@@ -667,8 +683,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
 #pragma unroll
                     for (int k = 0; k < 8; ++k) {
                         const int n = col0 + 8 * j + k;
-                        if (n < s.Nb) {
-                            if (full) p.out[((size_t)bh * p.N + n) * 128 + r] = __float2bfloat16_rn(o[k] * sm->inv_l[n]);
+                        if (n < s.Nq) {
+                            if (full) p.out[((size_t)bh * p.N + s.q0 + n) * 128 + r] = __float2bfloat16_rn(o[k] * sm->inv_l[n]);
                             else p.part_o[((size_t)slot_id * 128 + n) * 128 + r] = o[k];
                         }
                     }
@@ -682,11 +698,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 __threadfence();
                 group_sync_any(bar_id, false);
                 if (r == 0) {
-                    const long long t0 = t - s.lt, t1 = t0 + s.Tb;
+                    const long long t0 = t - s.lt, t1 = t0 + s.Tkv;
                     const int c_lo = (int)(((t0 + 1) * G + total - 1) / total - 1);
                     const int c_hi = (int)((t1 * G + total - 1) / total - 1);
                     const int nparts = min(c_hi - c_lo + 1, kMaxParts);
-                    int* counter = p.counters + (size_t)bh * kSoftmaxGroups + wg;
+                    int* counter = p.counters + ((size_t)bh * 2 + s.qb) * kSoftmaxGroups + wg;
                     const int old = atomicAdd(counter, 1);
                     int mine = 0;
                     if (old == nparts - 1) {
@@ -717,7 +733,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                                 float ms[8], ls[8], os[8];
 #pragma unroll
                                 for (int k = 0; k < 8; ++k) {
-                                    const bool on = col0 + 8 * j + k < s.Nb;
+                                    const bool on = col0 + 8 * j + k < s.Nq;
                                     ms[k] = on ? __ldcg(pm + k) : -INFINITY;
                                     ls[k] = on ? __ldcg(pl + k) : 0.f;
                                     os[k] = on ? __ldcg(po + (size_t)k * 128) : 0.f;
@@ -735,8 +751,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
 #pragma unroll
                             for (int k = 0; k < 8; ++k) {
                                 const int n = col0 + 8 * j + k;
-                                if (n < s.Nb)
-                                    p.out[((size_t)bh * p.N + n) * 128 + r] = __float2bfloat16_rn(lsum[k] > 0.f ? acc[k] / lsum[k] : 0.f);
+                                if (n < s.Nq)
+                                    p.out[((size_t)bh * p.N + s.q0 + n) * 128 + r] = __float2bfloat16_rn(lsum[k] > 0.f ? acc[k] / lsum[k] : 0.f);
                             }
                         }
                     }
@@ -790,7 +806,7 @@ static bool make_map(CUtensorMap* map, const void* base, int rows, int bh, int b
 }
 
 static int chunks_for(int N) {
-    const int nch = (N + 15) / 16;
+    const int nch = ((N < kQBlock ? N : kQBlock) + 15) / 16;
     return nch <= 3 ? 3 : nch <= 4 ? 4 : nch <= 7 ? 7 : 8;
 }
 
@@ -802,13 +818,13 @@ static int slots_for(int nch) {
 }
 
 bool tc_supported(const AttentionArgs& a) {
-    return a.N <= 128 && a.B <= kMaxBatchTc && encode_fn() != nullptr;
+    return a.N <= MCSD_MAX_NODES && a.B <= kMaxBatchTc && encode_fn() != nullptr;
 }
 
 size_t tc_workspace_bytes(int, int, int N, int, int) {
-    if (N > 128) return 0;
+    if (N > MCSD_MAX_NODES) return 0;
     return align_up((size_t)2 * kMaxCtas * 2 * 128 * sizeof(float), 256) +
-           align_up((size_t)2 * kMaxCtas * 128 * 128 * sizeof(float), 256) + (size_t)65536 * kSoftmaxGroups * sizeof(int);
+           align_up((size_t)2 * kMaxCtas * 128 * 128 * sizeof(float), 256) + (size_t)65536 * 2 * kSoftmaxGroups * sizeof(int);
 }
 
 template <int NCH>
