@@ -14,7 +14,8 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libmcsd.so")
+# MCSD_LIB selects another build of the same library (A/B timing of kernel variants)
+_LIB_PATH = os.environ.get("MCSD_LIB") or os.path.join(_HERE, "libmcsd.so")
 
 MCSD_BF16 = 0
 MCSD_F32 = 1
