@@ -300,6 +300,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         if (lane == 0) {
             long long t = t_begin;
             uint32_t u = 0, seg = 0;
+            uint32_t slot = 0, phase = 0;              // ring position of use u (kept incrementally: no divisions)
             bool ok = true;
             while (t < t_end && ok) {
                 Segment s;
@@ -316,14 +317,14 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     const bool tree = lti >= s.nP;
                     const int row0 = (tree ? lti - s.nP : lti) * kTile;
                     for (int kv = 0; kv < 2 && ok; ++kv, ++u) {
-                        const uint32_t slot = u % (uint32_t)NS;
-                        ok = mbar_wait(&sm->slot_empty[slot], ((u / (uint32_t)NS) & 1u) ^ 1u, sm, hdr, 2);
+                        ok = mbar_wait(&sm->slot_empty[slot], phase ^ 1u, sm, hdr, 2);
                         if (!ok) break;
                         const CUtensorMap* map = kv == 0 ? (tree ? &tm_kt : &tm_kc) : (tree ? &tm_vt : &tm_vc);
                         const uint32_t dst = smem_u32(ring) + slot * (uint32_t)kSlotBytes;
                         mbar_expect_tx(&sm->slot_full[slot], (uint32_t)kSlotBytes);
                         tma_load_3d(dst, map, &sm->slot_full[slot], 0, row0, bh);
                         tma_load_3d(dst + kSlabBytes, map, &sm->slot_full[slot], 64, row0, bh);
+                        if (++slot == (uint32_t)NS) { slot = 0; phase ^= 1u; }
                     }
                 }
                 t += cnt;
@@ -344,7 +345,10 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         // =========================================================== MMA issuer
         if (lane == 0) {
             long long t = t_begin;
-            uint32_t u = 0, g = 0, seg = 0;
+            uint32_t g = 0, seg = 0;
+            // ring positions of the next K tile (uses 0, 2, 4, ...) and the next V tile (uses 1, 3, 5, ...), kept
+            // incrementally: this thread is the pacing one, divisions by the slot count would cost it a tenth
+            uint32_t kslot = 0, kphase = 0, vslot = 1u % (uint32_t)NS, vphase = (1u / (uint32_t)NS) & 1u;
             bool ok = true;
             const uint32_t ring_a = smem_u32(ring), q_a = smem_u32(q_buf), p_a = smem_u32(p_buf);
             while (t < t_end && ok) {
@@ -357,9 +361,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 for (int i = 0; i <= cnt && ok; ++i) {
                     if (i < cnt) {
                         const uint32_t gi = g + (uint32_t)i, sb = gi & 1u;
-                        const uint32_t uk = u + 2u * (uint32_t)i, slot = uk % (uint32_t)NS;
-                        ok = mbar_wait(&sm->slot_full[slot], (uk / (uint32_t)NS) & 1u, sm, hdr, 4);
+                        const uint32_t slot = kslot;
+                        ok = mbar_wait(&sm->slot_full[slot], kphase, sm, hdr, 4);
                         if (!ok) break;
+                        kslot += 2u;
+                        if (kslot >= (uint32_t)NS) { kslot -= (uint32_t)NS; kphase ^= 1u; }
                         tc_fence_after();
                         const uint32_t ka = ring_a + slot * (uint32_t)kSlotBytes;
 #pragma unroll
@@ -375,9 +381,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     }
                     if (i >= 1) {
                         const uint32_t gj = g + (uint32_t)(i - 1);
-                        const uint32_t uv = u + 2u * (uint32_t)(i - 1) + 1u, slot = uv % (uint32_t)NS;
-                        ok = mbar_wait(&sm->slot_full[slot], (uv / (uint32_t)NS) & 1u, sm, hdr, 5);
+                        const uint32_t slot = vslot;
+                        ok = mbar_wait(&sm->slot_full[slot], vphase, sm, hdr, 5);
                         if (!ok) break;
+                        vslot += 2u;
+                        if (vslot >= (uint32_t)NS) { vslot -= (uint32_t)NS; vphase ^= 1u; }
                         ok = mbar_wait(&sm->p_full, gj & 1u, sm, hdr, 6);
                         if (!ok) break;
                         tc_fence_after();
@@ -394,7 +402,6 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                         tc_commit(&sm->pv_done);
                     }
                 }
-                u += 2u * (uint32_t)cnt;
                 g += (uint32_t)cnt;
                 ++seg;
                 t += cnt;
