@@ -425,24 +425,29 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         const int wg = warp >> 2, wq = warp & 3;
         const int r = tid & 127;
         const int bar_id = 1 + wg;
-        if (tid < MCSD_MAX_NODES) {
-            // dmask[t] = set of queries that may see tree key t: the ancestor bitsets transposed.  Built while
-            // the first tiles are in flight; first read at a tree tile, after several group barriers.
-            unsigned long long w0 = 0, w1 = 0, w2 = 0;
-            if (tid < p.N) {
-#pragma unroll 4
-                for (int n = 0; n < p.N; ++n) {
-                    const unsigned long long word = p.anc[(size_t)n * p.words + (tid >> 6)];
-                    const unsigned long long bit = (word >> (tid & 63)) & 1ull;
-                    if (n < 64) w0 |= bit << n; else if (n < 128) w1 |= bit << (n - 64); else w2 |= bit << (n - 128);
+        // dmask[t] = set of queries that may see tree key t: the ancestor bitsets transposed.  The bitsets are
+        // first copied to shared memory in one coalesced round trip (the P^T buffer is free until the first tile
+        // is finished), then every thread transposes one key's column out of shared memory.
+        {
+            unsigned long long* anc_s = reinterpret_cast<unsigned long long*>(p_buf);
+            const int n_words = p.N * p.words;                   // at most 192 * 3 words = 4.5 KB
+            for (int i = tid; i < n_words; i += 256) anc_s[i] = p.anc[i];
+            asm volatile("bar.sync 3, 256;" ::: "memory");
+            if (tid < MCSD_MAX_NODES) {
+                unsigned long long w0 = 0, w1 = 0, w2 = 0;
+                if (tid < p.N) {
+                    for (int n = 0; n < p.N; ++n) {
+                        const unsigned long long bit = (anc_s[n * p.words + (tid >> 6)] >> (tid & 63)) & 1ull;
+                        if (n < 64) w0 |= bit << n; else if (n < 128) w1 |= bit << (n - 64); else w2 |= bit << (n - 128);
+                    }
                 }
+                sm->dmask[tid][0] = w0;
+                sm->dmask[tid][1] = w1;
+                sm->dmask[tid][2] = w2;
             }
-            sm->dmask[tid][0] = w0;
-            sm->dmask[tid][1] = w1;
-            sm->dmask[tid][2] = w2;
+            // both groups read dmask and will overwrite the staging copy: order both before any tile is processed
+            asm volatile("bar.sync 3, 256;" ::: "memory");
         }
-        // both groups read dmask: order its writes before any tile is processed
-        asm volatile("bar.sync 3, 256;" ::: "memory");
         const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
         long long t = t_begin;
         uint32_t u = 0, g = 0;
