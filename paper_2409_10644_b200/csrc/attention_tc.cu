@@ -657,30 +657,68 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
 
             // ---- epilogue of the segment: each group finishes its own query columns
             const uint32_t glast = g + (uint32_t)cnt - 1u;
+            const bool full = (cnt == s.Tkv);
+            const int slot_id = 2 * cta + (t > t_begin ? 1 : 0);
+            if (!full && r == 0) {
+                // which blocks hold the other pieces of this work item (worked out while the last MMA drains)
+                const long long t0 = t - s.lt, t1 = t0 + s.Tkv;
+                const int c_lo = (int)(((t0 + 1) * G + total - 1) / total - 1);
+                const int c_hi = (int)((t1 * G + total - 1) / total - 1);
+                const int nparts = min(c_hi - c_lo + 1, kMaxParts);
+                int others = 0;
+                for (int i = 0; i < nparts; ++i) {
+                    if (c_lo + i == cta) continue;
+                    const long long start = (long long)(c_lo + i) * total / G;
+                    sm->merge_slot[wg][others++] = 2 * (c_lo + i) + (t0 > start ? 1 : 0);
+                }
+                sm->merge_parts[wg] = nparts;
+            }
             if (!mbar_wait(&sm->pv_done, glast & 1u, sm, hdr, 10)) failed = true;
             tc_fence_after();
+            // Row sums: every thread holds a partial sum per query; reduce the 8 sums of a column group across the
+            // warp by recursive halving (9 shuffles instead of 40): after the three exchange steps lane L holds the
+            // sum of column (L >> 2) & 7 over its exchange partners, two more steps finish the reduction.
 #pragma unroll
             for (int j = 0; j < CPT; ++j) {
                 if (j < ncg) {
-                    float mine = 0.f;
+                    float v4[4], v2[2], v1;
+                    {
+                        const bool up = lane & 16;
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        float v = acc_l[j][k];
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                        if (lane == k) mine = v;
+                        for (int k = 0; k < 4; ++k) {
+                            const float send = up ? acc_l[j][k] : acc_l[j][k + 4];
+                            const float keep = up ? acc_l[j][k + 4] : acc_l[j][k];
+                            v4[k] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+                        }
                     }
-                    if (lane < 8) sm->wred[wg][wq][8 * j + lane] = mine;
+                    {
+                        const bool up = lane & 8;
+#pragma unroll
+                        for (int k = 0; k < 2; ++k) {
+                            const float send = up ? v4[k] : v4[k + 2];
+                            const float keep = up ? v4[k + 2] : v4[k];
+                            v2[k] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+                        }
+                    }
+                    {
+                        const bool up = lane & 4;
+                        const float send = up ? v2[0] : v2[1];
+                        const float keep = up ? v2[1] : v2[0];
+                        v1 = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+                    }
+                    v1 += __shfl_xor_sync(0xffffffffu, v1, 2);
+                    v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
+                    // lane bits 4,3,2 select column 4*b4 + 2*b3 + b2
+                    if ((lane & 3) == 0) sm->wred[wg][wq][8 * j + ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1)] = v1;
                 }
             }
             if (group_sync_any(bar_id, failed)) { failed = true; break; }
-            const bool full = (cnt == s.Tkv);
-            const int slot_id = 2 * cta + (t > t_begin ? 1 : 0);
             if (r < ncg * 8) {
                 const float l = (sm->wred[wg][0][r] + sm->wred[wg][1][r]) + (sm->wred[wg][2][r] + sm->wred[wg][3][r]);
                 if (full) {
                     sm->inv_l[col0 + r] = l > 0.f ? 1.f / l : 0.f;
                 } else {
+                    sm->inv_l[col0 + r] = l;                   // kept for the merge below
                     p.part_ml[((size_t)slot_id * 2 + 0) * 128 + col0 + r] = sm->m_ref[col0 + r];
                     p.part_ml[((size_t)slot_id * 2 + 1) * 128 + col0 + r] = l;
                 }
@@ -704,68 +742,81 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             }
             tc_fence_before();
             if (!full) {
-                // Split-KV combine: every block that finished a piece of this (sequence, head) takes a ticket;
-                // the last one merges all pieces (its own included) into the output.  The two softmax groups own
-                // disjoint query columns and run this protocol independently of each other.
+                // Split-KV combine: every block that finished a piece of this work item takes a ticket; the last
+                // one merges the other pieces (read back from the workspace) with its own, which is still in
+                // tensor memory.  The two softmax groups own disjoint query columns and run this protocol independently.
                 __threadfence();
                 group_sync_any(bar_id, false);
                 if (r == 0) {
-                    const long long t0 = t - s.lt, t1 = t0 + s.Tkv;
-                    const int c_lo = (int)(((t0 + 1) * G + total - 1) / total - 1);
-                    const int c_hi = (int)((t1 * G + total - 1) / total - 1);
-                    const int nparts = min(c_hi - c_lo + 1, kMaxParts);
                     int* counter = p.counters + ((size_t)bh * 2 + s.qb) * kSoftmaxGroups + wg;
+                    const int nparts = sm->merge_parts[wg];
                     const int old = atomicAdd(counter, 1);
-                    int mine = 0;
                     if (old == nparts - 1) {
                         atomicExch(counter, 0);                   // ready for the next launch
                         __threadfence();
-                        mine = nparts;
-                        for (int i = 0; i < nparts; ++i) {
-                            const long long start = (long long)(c_lo + i) * total / G;
-                            sm->merge_slot[wg][i] = 2 * (c_lo + i) + (t0 > start ? 1 : 0);
-                        }
+                    } else {
+                        sm->merge_parts[wg] = 0;                  // not the last: nothing more to do
                     }
-                    sm->merge_parts[wg] = mine;
                 }
                 group_sync_any(bar_id, false);
                 const int nparts = sm->merge_parts[wg];
                 if (nparts > 0) {
+                    // JB column groups are merged at a time: all of them when they fit in registers
+                    constexpr int JB = 1;
 #pragma unroll
-                    for (int j = 0; j < CPT; ++j) {
-                        if (j < ncg) {
-                            float M[8], lsum[8], acc[8];
+                    for (int j0 = 0; j0 < CPT; j0 += JB) {
+                        if (j0 < ncg) {
+                            float M[JB][8], lsum[JB][8], o_keep[JB][8];
 #pragma unroll
-                            for (int k = 0; k < 8; ++k) { M[k] = -INFINITY; lsum[k] = 0.f; acc[k] = 0.f; }
-                            for (int i = 0; i < nparts; ++i) {
+                            for (int jj = 0; jj < JB; ++jj) {
+                                if (j0 + jj < ncg) tc_ld8(tmem + lane_addr + kColO + col0 + 8 * (j0 + jj), o_keep[jj]);
+                            }
+                            tc_wait_ld();
+#pragma unroll
+                            for (int jj = 0; jj < JB; ++jj)
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) {
+                                    const int n = col0 + 8 * (j0 + jj) + k;
+                                    const bool on = j0 + jj < ncg && n < s.Nq;
+                                    M[jj][k] = on ? sm->m_ref[n] : -INFINITY;
+                                    lsum[jj][k] = on ? sm->inv_l[n] : 0.f;
+                                    if (!on) o_keep[jj][k] = 0.f;
+                                }
+                            for (int i = 0; i < nparts - 1; ++i) {
                                 const int slot = sm->merge_slot[wg][i];
-                                const float* pm = p.part_ml + ((size_t)slot * 2 + 0) * 128 + col0 + 8 * j;
-                                const float* pl = p.part_ml + ((size_t)slot * 2 + 1) * 128 + col0 + 8 * j;
-                                const float* po = p.part_o + ((size_t)slot * 128 + col0 + 8 * j) * 128 + r;
-                                float ms[8], ls[8], os[8];
+                                float ms[JB][8], ls[JB][8], os[JB][8];
+                                // all loads of one piece are issued before any is used: one memory round trip
 #pragma unroll
-                                for (int k = 0; k < 8; ++k) {
-                                    const bool on = col0 + 8 * j + k < s.Nq;
-                                    ms[k] = on ? __ldcg(pm + k) : -INFINITY;
-                                    ls[k] = on ? __ldcg(pl + k) : 0.f;
-                                    os[k] = on ? __ldcg(po + (size_t)k * 128) : 0.f;
-                                }
+                                for (int jj = 0; jj < JB; ++jj)
 #pragma unroll
-                                for (int k = 0; k < 8; ++k) {
-                                    const float mn = fmaxf(M[k], ms[k]);
-                                    if (mn == -INFINITY) continue;
-                                    const float a = exp2f(M[k] - mn), w = exp2f(ms[k] - mn);
-                                    lsum[k] = fmaf(lsum[k], a, w * ls[k]);
-                                    acc[k] = fmaf(acc[k], a, w * os[k]);
-                                    M[k] = mn;
-                                }
+                                    for (int k = 0; k < 8; ++k) {
+                                        const int n = col0 + 8 * (j0 + jj) + k;
+                                        const bool on = j0 + jj < ncg && n < s.Nq;
+                                        ms[jj][k] = on ? __ldcg(p.part_ml + ((size_t)slot * 2 + 0) * 128 + n) : -INFINITY;
+                                        ls[jj][k] = on ? __ldcg(p.part_ml + ((size_t)slot * 2 + 1) * 128 + n) : 0.f;
+                                        os[jj][k] = on ? __ldcg(p.part_o + ((size_t)slot * 128 + n) * 128 + r) : 0.f;
+                                    }
+#pragma unroll
+                                for (int jj = 0; jj < JB; ++jj)
+#pragma unroll
+                                    for (int k = 0; k < 8; ++k) {
+                                        const float mn = fmaxf(M[jj][k], ms[jj][k]);
+                                        if (mn == -INFINITY) continue;
+                                        const float a = exp2f(M[jj][k] - mn), w = exp2f(ms[jj][k] - mn);
+                                        lsum[jj][k] = fmaf(lsum[jj][k], a, w * ls[jj][k]);
+                                        o_keep[jj][k] = fmaf(o_keep[jj][k], a, w * os[jj][k]);
+                                        M[jj][k] = mn;
+                                    }
                             }
 #pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                const int n = col0 + 8 * j + k;
-                                if (n < s.Nq)
-                                    p.out[((size_t)bh * p.N + s.q0 + n) * 128 + r] = __float2bfloat16_rn(lsum[k] > 0.f ? acc[k] / lsum[k] : 0.f);
-                            }
+                            for (int jj = 0; jj < JB; ++jj)
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) {
+                                    const int n = col0 + 8 * (j0 + jj) + k;
+                                    if (j0 + jj < ncg && n < s.Nq)
+                                        p.out[((size_t)bh * p.N + s.q0 + n) * 128 + r] =
+                                            __float2bfloat16_rn(lsum[jj][k] > 0.f ? o_keep[jj][k] / lsum[jj][k] : 0.f);
+                                }
                         }
                     }
                 }
