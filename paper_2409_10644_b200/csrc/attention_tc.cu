@@ -724,18 +724,27 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 }
             }
             group_sync_any(bar_id, false);
+            // O^T rows of this thread, up to four column groups per tensor-memory round trip
+            constexpr int EB = CPT < 4 ? CPT : 4;
 #pragma unroll
-            for (int j = 0; j < CPT; ++j) {
-                if (j < ncg) {
-                    float o[8];
-                    tc_ld8(tmem + lane_addr + kColO + col0 + 8 * j, o);
+            for (int j0 = 0; j0 < CPT; j0 += EB) {
+                if (j0 < ncg) {
+                    float o[EB][8];
+#pragma unroll
+                    for (int jj = 0; jj < EB; ++jj)
+                        if (j0 + jj < CPT && j0 + jj < ncg) tc_ld8(tmem + lane_addr + kColO + col0 + 8 * (j0 + jj), o[jj]);
                     tc_wait_ld();
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        const int n = col0 + 8 * j + k;
-                        if (n < s.Nq) {
-                            if (full) p.out[((size_t)bh * p.N + s.q0 + n) * 128 + r] = __float2bfloat16_rn(o[k] * sm->inv_l[n]);
-                            else p.part_o[((size_t)slot_id * 128 + n) * 128 + r] = o[k];
+                    for (int jj = 0; jj < EB; ++jj) {
+                        if (j0 + jj < CPT && j0 + jj < ncg) {
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const int n = col0 + 8 * (j0 + jj) + k;
+                                if (n < s.Nq) {
+                                    if (full) p.out[((size_t)bh * p.N + s.q0 + n) * 128 + r] = __float2bfloat16_rn(o[jj][k] * sm->inv_l[n]);
+                                    else p.part_o[((size_t)slot_id * 128 + n) * 128 + r] = o[jj][k];
+                                }
+                            }
                         }
                     }
                 }
@@ -752,8 +761,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     const int nparts = sm->merge_parts[wg];
                     const int old = atomicAdd(counter, 1);
                     if (old == nparts - 1) {
-                        atomicExch(counter, 0);                   // ready for the next launch
-                        __threadfence();
+                        *(volatile int*)counter = 0;              // nobody else arrives in this launch: ready for the next one
+                        __threadfence();                          // acquire: the other pieces' partials are visible
                     } else {
                         sm->merge_parts[wg] = 0;                  // not the last: nothing more to do
                     }
