@@ -864,8 +864,37 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
+// Tensor maps depend only on (base pointer, rows, B*H, box rows).  A decode loop calls with the same few
+// buffers every step, so the encoded maps are kept in a small per-thread table (round-robin replacement).
+struct MapKey {
+    const void* base;
+    int rows, bh, box_rows;
+};
+constexpr int kMapCacheSize = 256;
+struct MapCache {
+    MapKey key[kMapCacheSize];
+    CUtensorMap map[kMapCacheSize];
+    int used = 0, next = 0;
+};
+static thread_local MapCache g_map_cache;
+
+static bool encode_map(CUtensorMap* map, const void* base, int rows, int bh, int box_rows);
+
 // [BH][rows][128] bf16 tensor, boxes of box_rows x 64 columns, 128-byte swizzle, zero fill outside
 static bool make_map(CUtensorMap* map, const void* base, int rows, int bh, int box_rows) {
+    MapCache& c = g_map_cache;
+    for (int i = 0; i < c.used; ++i) {
+        const MapKey& k = c.key[i];
+        if (k.base == base && k.rows == rows && k.bh == bh && k.box_rows == box_rows) { *map = c.map[i]; return true; }
+    }
+    if (!encode_map(map, base, rows, bh, box_rows)) return false;
+    const int slot = c.used < kMapCacheSize ? c.used++ : (c.next = (c.next + 1) % kMapCacheSize);
+    c.key[slot] = MapKey{base, rows, bh, box_rows};
+    c.map[slot] = *map;
+    return true;
+}
+
+static bool encode_map(CUtensorMap* map, const void* base, int rows, int bh, int box_rows) {
     EncodeTiledFn fn = encode_fn();
     if (fn == nullptr) return false;
     cuuint64_t dims[3] = {128, (cuuint64_t)rows, (cuuint64_t)bh};
@@ -901,7 +930,16 @@ size_t tc_workspace_bytes(int, int, int N, int, int) {
 
 template <int NCH>
 static int launch_tc(const CUtensorMap* maps, const TcParams& p, int grid, size_t smem_bytes, cudaStream_t stream) {
-    MCSD_CUDA_CHECK(cudaFuncSetAttribute(tree_attention_tc_kernel<NCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    // the opt-in to large dynamic shared memory is per device: done on the first launch on each device
+    static std::mutex mu;
+    static bool done[64] = {};
+    int dev = 0;
+    MCSD_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64 || !done[dev]) {
+        std::lock_guard<std::mutex> lock(mu);
+        MCSD_CUDA_CHECK(cudaFuncSetAttribute(tree_attention_tc_kernel<NCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+        if (dev >= 0 && dev < 64) done[dev] = true;
+    }
     tree_attention_tc_kernel<NCH><<<grid, kTcThreads, smem_bytes, stream>>>(maps[0], maps[1], maps[2], maps[3], maps[4], p);
     MCSD_CUDA_CHECK(cudaGetLastError());
     return MCSD_OK;
@@ -927,7 +965,12 @@ int tree_attention_tc(const AttentionArgs& a, WorkspaceHeader* header, void* scr
 
     int dev = 0, sms = 0;
     MCSD_CUDA_CHECK(cudaGetDevice(&dev));
-    MCSD_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    static thread_local int sms_dev = -1, sms_cached = 0;
+    if (sms_dev != dev) {
+        MCSD_CUDA_CHECK(cudaDeviceGetAttribute(&sms_cached, cudaDevAttrMultiProcessorCount, dev));
+        sms_dev = dev;
+    }
+    sms = sms_cached;
     const int grid = sms < kMaxCtas ? sms : kMaxCtas;
 
     TcParams p;
