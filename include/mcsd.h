@@ -174,6 +174,27 @@ int mcsd_verify_tree(const float* p, const float* q,
                      void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * KV-cache update after acceptance (Fig. 1 step 6): "update the input IDs, key-value cache".  For every layer and
+ * sequence b the keys/values of the winning root (node best_root[b]; with a single root that is node 0, the last
+ * emitted token, which is not in the prefix cache yet) and of the accepted nodes out_nodes[b][0 .. accept_len[b]-1]
+ * are copied from the tree tensors to cache rows seq_lens[b], seq_lens[b]+1, ..., then seq_lens[b] grows by
+ * 1 + accept_len[b].  Rows that would fall beyond L_max are dropped and the length saturates at L_max.
+ *
+ *   k_cache_layers, v_cache_layers  [dev] arrays of n_layers device pointers, each a cache [B][H][L_max][D] (in/out)
+ *   k_tree_layers, v_tree_layers    [dev] arrays of n_layers device pointers, each [B][H][N][D]
+ *   seq_lens                        [dev] int32[B], in/out
+ *   accept_len, out_nodes, best_root  [dev] outputs of mcsd_verify_tree (out_nodes is [B][n_levels])
+ *   dtype                           MCSD_BF16 or MCSD_F32; D is 64 or 128; all tensors 16-byte aligned
+ *
+ * Two launches on `stream` for all layers together; no workspace.  Errors: MCSD_ERR_NULL, MCSD_ERR_BAD_SHAPE,
+ * MCSD_ERR_BAD_DTYPE, MCSD_ERR_CUDA.
+ */
+int mcsd_commit_kv(void* const* k_cache_layers, void* const* v_cache_layers,
+                   const void* const* k_tree_layers, const void* const* v_tree_layers, int n_layers,
+                   int32_t* seq_lens, const int32_t* accept_len, const int32_t* out_nodes, const int32_t* best_root,
+                   int n_levels, int B, int H, int N, int D, int L_max, int dtype, void* stream);
+
+/*
  * mcsd_verify_tree with built-in scratch.  (The paper has no counterpart; this is a deployment convenience.)
  *
  * Same computation, arguments and results as mcsd_verify_tree, minus the workspace: the per-node scratch

@@ -317,3 +317,29 @@ def decision_margins(p, q, tokens, parent, gamma, u_accept, u_bonus):
             lo = cs[t - 1] if t > 0 else -np.inf
             m_bon[b, u] = min(target - lo, cs[t] - target) / z
     return m_acc, m_bon
+
+
+# ----------------------------------------------------------------------------
+# KV-cache update after acceptance (Fig. 1 step 6)
+# ----------------------------------------------------------------------------
+
+def commit_kv(k_cache, v_cache, k_tree, v_tree, seq_lens, accept_len, out_nodes, best_root):
+    """Append the keys/values of the accepted tokens to the prefix cache (in place) and return the new lengths.
+
+    For sequence b the committed tree tokens are the winning root (with a single root that is node 0, the last
+    emitted token, whose K/V is not in the prefix yet) followed by the accepted nodes out_nodes[b][:accept_len[b]],
+    written to cache rows seq_lens[b], seq_lens[b]+1, ...  Rows that would fall beyond L_max are dropped and the
+    length saturates at L_max.  k_cache, v_cache: [B][H][L_max][D]; k_tree, v_tree: [B][H][N][D].
+    """
+    B, H, L_max, D = k_cache.shape
+    new_lens = np.array(seq_lens, dtype=np.int32).copy()
+    for b in range(B):
+        nodes = [int(best_root[b])] + [int(n) for n in out_nodes[b][: int(accept_len[b])]]
+        L = int(seq_lens[b])
+        for i, n in enumerate(nodes):
+            if L + i >= L_max:
+                break
+            k_cache[b, :, L + i, :] = k_tree[b, :, n, :]
+            v_cache[b, :, L + i, :] = v_tree[b, :, n, :]
+        new_lens[b] = min(L_max, L + len(nodes))
+    return new_lens

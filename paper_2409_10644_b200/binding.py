@@ -24,7 +24,7 @@ MCSD_MAX_WORDS = 3
 
 _EXPORTS = (
     "mcsd_status_string", "mcsd_last_cuda_error", "mcsd_launch_count", "mcsd_build_mask", "mcsd_tree_attention_workspace_bytes",
-    "mcsd_tree_attention", "mcsd_workspace_status", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_static",
+    "mcsd_tree_attention", "mcsd_workspace_status", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_static", "mcsd_commit_kv",
 )
 
 
@@ -58,6 +58,8 @@ def _load() -> ctypes.CDLL:
     lib.mcsd_verify_tree_static.restype = c_int
     lib.mcsd_verify_tree_static.argtypes = ([c_void_p] * 5 + [c_int, c_int] + [c_void_p] * 3 + [c_int] * 3 +
                                             [c_void_p] * 5 + [c_int, c_void_p])
+    lib.mcsd_commit_kv.restype = c_int
+    lib.mcsd_commit_kv.argtypes = [c_void_p] * 4 + [c_int] + [c_void_p] * 4 + [c_int] * 7 + [c_void_p]
     return lib
 
 
@@ -252,6 +254,29 @@ def mcsd_verify_tree_static(p, q, tokens, mask: TreeMask, gamma, u_accept, u_bon
                                          R, _stream())
     _check(st, "mcsd_verify_tree_static")
     return out
+
+
+def layer_pointer_table(tensors) -> torch.Tensor:
+    """Device array of the data pointers of per-layer tensors (int64), as mcsd_commit_kv takes them."""
+    dev = tensors[0].device
+    return torch.tensor([t.data_ptr() for t in tensors], dtype=torch.int64, device=dev)
+
+
+def mcsd_commit_kv(k_cache_ptrs, v_cache_ptrs, k_tree_ptrs, v_tree_ptrs, seq_lens, verify_out, mask: TreeMask,
+                   B: int, H: int, D: int, L_max: int, dtype: torch.dtype) -> None:
+    """Append the accepted tokens' K/V to every layer's prefix cache and grow seq_lens (see mcsd.h).
+
+    The four `*_ptrs` arguments are device int64 tensors from layer_pointer_table(); `verify_out` is the dict
+    returned by mcsd_verify_tree."""
+    n_layers = int(k_cache_ptrs.numel())
+    code = MCSD_BF16 if dtype == torch.bfloat16 else MCSD_F32
+    _dev_tensor(seq_lens, torch.int32, "seq_lens")
+    with torch.cuda.device(seq_lens.device):
+        st = lib.mcsd_commit_kv(_ptr(k_cache_ptrs), _ptr(v_cache_ptrs), _ptr(k_tree_ptrs), _ptr(v_tree_ptrs), n_layers,
+                                _ptr(seq_lens), _ptr(verify_out["accept_len"]), _ptr(verify_out["out_nodes"]),
+                                _ptr(verify_out["best_root"]), mask.n_levels, B, H, mask.n_nodes, D, L_max, code,
+                                _stream())
+    _check(st, "mcsd_commit_kv")
 
 
 def shard_batch(B: int, rank: int, world_size: int):

@@ -92,3 +92,16 @@ def test_verify_argument_checks(m):
     assert call(R=33, nxt=FAKE) == -2
     assert call(R=2, nxt=None) == -1
     assert call(wsb=8) == -5
+
+
+def test_commit_kv_argument_checks(m):
+    L = m.lib
+
+    def call(kc=FAKE, n_layers=2, B=2, H=2, N=15, D=64, Lm=64, dtype=1, nl=4):
+        return L.mcsd_commit_kv(kc, FAKE, FAKE, FAKE, n_layers, FAKE, FAKE, FAKE, FAKE, nl, B, H, N, D, Lm, dtype, None)
+    assert call(kc=None) == -1
+    assert call(n_layers=0) == -2
+    assert call(D=96) == -2
+    assert call(N=193) == -2
+    assert call(nl=0) == -2
+    assert call(dtype=3) == -4

@@ -310,3 +310,39 @@ def test_verify_edge_cases(m):
     w5 = workload(5)
     _verify_case(m, w5, parent=parent_array(16, (1, 1, 1, 1)), B=4, V=2000, gamma=np.array([4, 1, 2, 0]))
     _verify_case(m, w5, parent=parent_array(2, (4, 3, 1, 1)), B=4, V=2000, gamma=None, R=2)
+
+
+# ----------------------------------------------------------------------------------------------
+# KV-cache update after acceptance
+# ----------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("idx,dtype_D", [(5, None), (3, None), (1, None)])
+def test_commit_kv_matches_oracle(m, idx, dtype_D):
+    w = dataclasses.replace(workload(idx), B=4, H=3, prefix=(30, 60), n_layers=3)
+    parent = parent_array(w.n_roots, w.branching)
+    N = len(parent)
+    tm = m.mcsd_build_mask(parent)
+    dev = "cuda"
+    layers = [attention_inputs(w, l, dev) for l in range(w.n_layers)]
+    lens = np.array([30, 41, 57, 60][: w.B], dtype=np.int32)          # the last two run out of cache rows
+    vin = verify_inputs(w, 0, dev, parent=parent, V=500)
+    gam = None if w.gamma is None else torch.from_numpy(gammas(w)).to(dev)
+    vout = m.mcsd_verify_tree(vin["p"], vin["q"], vin["tokens"], tm, gam, vin["u_accept"], vin["u_bonus"])
+    torch.cuda.synchronize()
+    host_layers = [{k: to_np(v).copy() for k, v in l.items()} for l in layers]
+    hv = {k: v.cpu().numpy() for k, v in vout.items() if v is not None}
+    lens_d = torch.from_numpy(lens).to(dev)
+    kc = m.layer_pointer_table([l["k_cache"] for l in layers])
+    vc = m.layer_pointer_table([l["v_cache"] for l in layers])
+    kt = m.layer_pointer_table([l["k_tree"] for l in layers])
+    vt = m.layer_pointer_table([l["v_tree"] for l in layers])
+    m.mcsd_commit_kv(kc, vc, kt, vt, lens_d, vout, tm, w.B, w.H, w.D, w.L_max, w.torch_dtype)
+    torch.cuda.synchronize()
+    new_ref = None
+    for l, hl in zip(layers, host_layers):
+        new_ref = orc.commit_kv(hl["k_cache"], hl["v_cache"], hl["k_tree"], hl["v_tree"], lens, hv["accept_len"],
+                                hv["out_nodes"], hv["best_root"])
+        assert np.array_equal(to_np(l["k_cache"]), hl["k_cache"])         # copies: bit-exact
+        assert np.array_equal(to_np(l["v_cache"]), hl["v_cache"])
+    assert np.array_equal(lens_d.cpu().numpy(), new_ref)
+    assert (new_ref > lens).any()

@@ -477,3 +477,41 @@ def test_decision_margins_flag_uniforms_on_a_threshold():
     assert np.isinf(m_acc[0, 0])
     # leaves can be stop nodes: their bonus margin is finite
     assert np.isfinite(m_bon[0, 1]) and np.isfinite(m_bon[0, 2])
+
+
+def test_commit_kv_turns_the_accepted_path_into_ordinary_prefix():
+    """Fig. 1 step 6: after the cache update the accepted tokens are plain prefix tokens, so causal attention of the
+    deepest accepted token over the updated cache equals its tree-attention output before the update."""
+    rng = np.random.default_rng(21)
+    parent = parent_array(2, (2, 2, 1))
+    N = len(parent)
+    B, H, D, L_max = 3, 2, 8, 20
+    q, kc, vc, kt, vt = _rand_attn(rng, B, H, N, D, L_max)
+    lens = np.array([5, 11, 18], dtype=np.int32)            # the last sequence runs out of cache rows
+    scale = 0.4
+    before = orc.tree_attention(q, kc, vc, kt, vt, lens, None, parent, scale)
+    mask = orc.dense_mask(parent)
+    leaves = [n for n in range(N) if not np.any(parent == n)]
+    best_root, accept_len, out_nodes = [], [], np.full((B, 4), -1)
+    for b in range(B):
+        leaf = leaves[int(rng.integers(len(leaves)))]
+        path = [n for n in range(N) if mask[leaf, n]]
+        cut = int(rng.integers(1, len(path) + 1))           # accept a prefix of the root path
+        best_root.append(path[0]); accept_len.append(cut - 1); out_nodes[b, :cut - 1] = path[1:cut]
+    kc2, vc2 = kc.copy(), vc.copy()
+    new_lens = orc.commit_kv(kc2, vc2, kt, vt, lens, accept_len, out_nodes, best_root)
+    for b in range(B):
+        cnt = 1 + accept_len[b]
+        assert new_lens[b] == min(L_max, lens[b] + cnt)
+        assert np.array_equal(kc2[b, :, :lens[b]], kc[b, :, :lens[b]])          # old prefix untouched
+        if lens[b] + cnt > L_max:
+            continue
+        last = best_root[b] if accept_len[b] == 0 else out_nodes[b, accept_len[b] - 1]
+        for h in range(H):
+            T = new_lens[b]
+            q_seq = np.zeros((T, D)); q_seq[-1] = q[b, h, last]
+            ref = _sdpa_causal_last(q_seq, kc2[b, h, :T], vc2[b, h, :T], scale)[-1]
+            np.testing.assert_allclose(ref, before[b, h, last], rtol=0, atol=1e-12)
+    # rows past the updated length keep their old content
+    b = 0
+    assert np.array_equal(kc2[b, :, new_lens[b]:], kc[b, :, new_lens[b]:])
