@@ -13,7 +13,7 @@
 //                                                                  by the softmax threads, MN-major)
 // Accumulators live in tensor memory: S^T double-buffered (columns 0 and 128), O^T at column 256.
 //
-// Warp roles (320 threads):
+// Warp roles (352 threads):
 //   warps 0-7  softmax, two warpgroups that split the query columns of each tile: thread r of a group owns
 //              key row r of the tile = TMEM lane r.  The running reference maximum of a query is only raised
 //              when a score exceeds it by more than 2^8 ("lazy" rescaling): the common tile costs one vote,
@@ -23,6 +23,7 @@
 //              past the end of a ragged tile and run the epilogue.
 //   warp 8     TMA producer: K and V tiles into a ring of 32 KB slots, Q once per segment.
 //   warp 9     MMA issuer (one thread) and owner of the tensor-memory allocation.
+//   warp 10    bookkeeping (one thread): which other blocks share a work item with this one.
 // Every mbarrier wait is bounded; a wait that runs out raises a flag in the workspace header, all roles drain
 // and the block exits cleanly.
 #include <cuda.h>
@@ -37,8 +38,8 @@ namespace mcsd {
 constexpr int kTile = 128;                    // keys per tile
 constexpr int kQBlock = 128;                  // queries per work item
 constexpr int kSoftmaxGroups = 2;              // warpgroups that split the query columns of every tile
-constexpr int kProducerWarp = 4 * kSoftmaxGroups, kMmaWarp = kProducerWarp + 1;
-constexpr int kTcThreads = 32 * (kMmaWarp + 1);
+constexpr int kProducerWarp = 4 * kSoftmaxGroups, kMmaWarp = kProducerWarp + 1, kHelperWarp = kMmaWarp + 1;
+constexpr int kTcThreads = 32 * (kHelperWarp + 1);
 constexpr int kSlotBytes = kTile * 128 * 2;   // one K or V tile: 128 rows x 128 bf16
 constexpr int kSlabBytes = kTile * 128;       // 64 of the 128 columns: rows of 128 bytes (the TMA swizzle span)
 constexpr int kMaxSlots = 6;
@@ -54,18 +55,25 @@ struct TcSmall {
     unsigned long long slot_full[kMaxSlots];
     unsigned long long slot_empty[kMaxSlots];
     unsigned long long s_full[2];
-    unsigned long long p_full, pv_done, q_full, q_empty, drain;
+    unsigned long long p_full, pv_done, q_full, q_empty, drain, info_ready;
     uint32_t tmem_base;
     int abort_flag;
     int merge_parts[kSoftmaxGroups];   // > 0: this block finished a split (sequence, head) last and merges it
-    int merge_slot[kSoftmaxGroups][kMaxParts];
+    // pieces of the (at most two) work items this block shares with others: [0] the segment at the start of its
+    // range, [1] the one at the end.  Worked out once by the bookkeeping warp.
+    int piece_parts[2];
+    int piece_slot[2][kMaxParts];
+    long long range[2];                // first and one-past-last tile of this block
+    int n_blocks;                      // blocks that got tiles
     alignas(16) float m_ref[128];
-    alignas(16) float alpha[128];
-    alignas(16) float inv_l[128];
+    alignas(16) float alpha[128];      // rescale factors of a slow-path tile; in the epilogue: 1/l (or l) per query
     alignas(16) float wred[kSoftmaxGroups][4][64];
     alignas(16) unsigned long long dmask[MCSD_MAX_NODES][3];
-    int cum_tiles[kMaxBatchTc + 1];
+    unsigned short cum_tiles[kMaxBatchTc + 2];   // tiles per head of the sequences before b (at most 256 * 68)
+    int cum_w[kMaxBatchTc + 1];        // the same in cost units (see tile_weight)
 };
+// the small state must leave room for six 32 KB ring slots next to Q and P^T of a 48-query launch
+static_assert(sizeof(TcSmall) <= 232448 - 1024 - 6 * 32768 - 48 * 512, "TcSmall grew: the 6-slot ring no longer fits");
 
 struct TcParams {
     __nv_bfloat16* out;
@@ -236,6 +244,63 @@ __device__ __forceinline__ void locate(const TcSmall* sm, const TcParams& p, lon
     s.Nq = min(kQBlock, s.Nb - s.q0);
 }
 
+// Cost of one tile in units of about 100 cycles, measured on this kernel: flat up to 32 queries, then growing with
+// the number of query columns the softmax threads and the MMAs have to cover.  Thread blocks get equal cost, not
+// equal tile counts, so that sequences with deep trees do not make their blocks finish late.
+__device__ __forceinline__ int tile_weight(int Nq) {
+    return 24 + (max(0, Nq - 32) * 9) / 32;
+}
+// Fixed cost of a work item (pipeline drain, row-sum reduction, output of Nq columns), carried by its first tile.
+__device__ __forceinline__ int item_weight(int Nq) {
+    return 30 + (Nq * 5) / 8;
+}
+__device__ __forceinline__ int head_weight(int L, int Nb) {        // cost of one (sequence, head): all query blocks
+    const int tkv = kv_tiles_of(L, Nb);
+    int w = 0;
+    for (int q0 = 0; q0 < Nb; q0 += kQBlock) w += tkv * tile_weight(min(kQBlock, Nb - q0)) + item_weight(min(kQBlock, Nb - q0));
+    return w;
+}
+// cumulative cost of the tiles before the one a Segment points at
+__device__ __forceinline__ long long weight_before(const TcSmall* sm, const TcParams& p, const Segment& s) {
+    long long w = (long long)p.H * sm->cum_w[s.b] + (long long)s.h * (sm->cum_w[s.b + 1] - sm->cum_w[s.b]);
+    if (s.qb) w += (long long)s.Tkv * tile_weight(kQBlock) + item_weight(kQBlock);
+    return w + (long long)s.lt * tile_weight(s.Nq) + (s.lt > 0 ? item_weight(s.Nq) : 0);
+}
+// Tile t belongs to block floor(weight_before(t) * G / total_w).  First tile of block c: the first tile whose
+// cumulative cost reaches ceil(c * total_w / G).
+__device__ __forceinline__ long long first_tile_of_block(const TcSmall* sm, const TcParams& p, int c, int G, long long total_w,
+                                                         long long total_tiles) {
+    const long long wt = ((long long)c * total_w + G - 1) / G;
+    if (wt >= total_w) return total_tiles;
+    int lo = 0, hi = p.B;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if ((long long)p.H * sm->cum_w[mid] <= wt) lo = mid; else hi = mid;
+    }
+    const int L = min(max(p.seq_lens[lo], 0), p.L_max);
+    const int Nb = p.n_active ? min(max(p.n_active[lo], 0), p.N) : p.N;
+    const int tkv = kv_tiles_of(L, Nb);
+    const int wh = sm->cum_w[lo + 1] - sm->cum_w[lo], tb = sm->cum_tiles[lo + 1] - sm->cum_tiles[lo];
+    const long long rem = wt - (long long)p.H * sm->cum_w[lo];
+    const int h = (int)(rem / wh);
+    int r2 = (int)(rem % wh);
+    long long t = (long long)p.H * sm->cum_tiles[lo] + (long long)h * tb;
+    // inside a work item the tiles start at cost 0, f + w, f + 2w, ... (f = fixed cost on the first tile)
+    const int w0 = tile_weight(min(kQBlock, Nb)), f0 = item_weight(min(kQBlock, Nb));
+    if (r2 >= tkv * w0 + f0 && Nb > kQBlock) {         // inside the second query block
+        r2 -= tkv * w0 + f0;
+        t += tkv;
+        const int w1 = tile_weight(Nb - kQBlock), f1 = item_weight(Nb - kQBlock);
+        return r2 == 0 ? t : t + max(1, (r2 - f1 + w1 - 1) / w1);
+    }
+    return r2 == 0 ? t : t + max(1, (r2 - f0 + w0 - 1) / w0);
+}
+__device__ __forceinline__ int block_of_tile(const TcSmall* sm, const TcParams& p, long long t, int G, long long total_w) {
+    Segment s;
+    locate(sm, p, t, s);
+    return (int)min((long long)G - 1, weight_before(sm, p, s) * G / total_w);
+}
+
 // ------------------------------------------------------------------ the kernel
 template <int NCH>
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -257,7 +322,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     for (int b = tid; b < p.B; b += kTcThreads) {
         const int L = min(max(p.seq_lens[b], 0), p.L_max);
         const int Nb = p.n_active ? min(max(p.n_active[b], 0), p.N) : p.N;
-        sm->cum_tiles[b + 1] = tiles_of(L, Nb);
+        sm->cum_tiles[b + 1] = (unsigned short)tiles_of(L, Nb);
+        sm->cum_w[b + 1] = head_weight(L, Nb);
     }
     if (tid == 0) {
         for (int i = 0; i < kMaxSlots; ++i) { mbar_init(&sm->slot_full[i], 1); mbar_init(&sm->slot_empty[i], 1); }
@@ -268,22 +334,37 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         mbar_init(&sm->q_full, 1);
         mbar_init(&sm->q_empty, 1);
         mbar_init(&sm->drain, 1);
+        mbar_init(&sm->info_ready, 1);
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
     if (tid == 0) {
-        int acc = 0;
+        int acc = 0, accw = 0;
         sm->cum_tiles[0] = 0;
-        for (int b = 1; b <= p.B; ++b) { acc += sm->cum_tiles[b]; sm->cum_tiles[b] = acc; }
+        sm->cum_w[0] = 0;
+        for (int b = 1; b <= p.B; ++b) {
+            acc += sm->cum_tiles[b]; sm->cum_tiles[b] = (unsigned short)acc;
+            accw += sm->cum_w[b]; sm->cum_w[b] = accw;
+        }
+        // No block's share of the cost may be smaller than the heaviest tile, so that consecutive tiles never skip
+        // a block: every working block then owns at least one tile and the blocks sharing a work item are consecutive.
+        const long long tot_w = (long long)p.H * accw;
+        const int nb = (int)max(1LL, min((long long)gridDim.x, tot_w / (tile_weight(kQBlock) + item_weight(kQBlock))));
+        sm->n_blocks = nb;
+    }
+    __syncthreads();
+    if (tid == 0 || tid == 32) {               // the two ends of this block's range, side by side
+        const long long tot = (long long)p.H * sm->cum_tiles[p.B], tot_w = (long long)p.H * sm->cum_w[p.B];
+        const int nb = sm->n_blocks, which = tid >> 5;
+        sm->range[which] = (tot > 0 && cta < nb) ? first_tile_of_block(sm, p, cta + which, nb, tot_w, tot) : 0;
     }
     __syncthreads();
     const long long total = (long long)p.H * sm->cum_tiles[p.B];
-    // With fewer tiles than thread blocks only the first `total` blocks work, so every working block owns at
-    // least one tile and the blocks that share a (sequence, head) are consecutive.
-    const int G = (int)min((long long)gridDim.x, total);
-    if (cta >= G) return;                      // uniform for the whole block: nothing allocated yet
-    const long long t_begin = (long long)cta * total / G, t_end = (long long)(cta + 1) * total / G;
+    const long long total_w = (long long)p.H * sm->cum_w[p.B];
+    const int G = sm->n_blocks;
+    const long long t_begin = sm->range[0], t_end = sm->range[1];
+    if (t_begin >= t_end) return;              // uniform for the whole block: nothing allocated yet
 
     if (warp == kMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)), "r"(kTmemCols) : "memory");
@@ -340,6 +421,32 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     while (!mbar_try_wait(bar, par) && clock64() - t0 < kSpinCycles / 8) {}
                 }
             }
+        }
+    } else if (warp == kHelperWarp) {
+        // =========================================================== bookkeeping, off everybody's critical path
+        if (lane == 0) {
+            // which blocks hold the other pieces of the work items this block shares with its neighbours
+            for (int which = 0; which < 2; ++which) {
+                Segment sp;
+                locate(sm, p, which == 0 ? t_begin : t_end - 1, sp);
+                const long long at = which == 0 ? t_begin : t_end - 1;
+                const long long t0 = at - sp.lt, t1 = t0 + sp.Tkv;
+                int nparts = 0;
+                const bool shared = which == 0 ? (t0 < t_begin || t1 > t_end) : (t0 > t_begin && t1 > t_end);
+                if (shared) {
+                    const int c_lo = block_of_tile(sm, p, t0, G, total_w);
+                    const int c_hi = block_of_tile(sm, p, t1 - 1, G, total_w);
+                    nparts = min(c_hi - c_lo + 1, kMaxParts);
+                    int others = 0;
+                    for (int i = 0; i < nparts; ++i) {
+                        if (c_lo + i == cta) continue;
+                        const long long start = first_tile_of_block(sm, p, c_lo + i, G, total_w, total);
+                        sm->piece_slot[which][others++] = 2 * (c_lo + i) + (t0 > start ? 1 : 0);
+                    }
+                }
+                sm->piece_parts[which] = nparts;
+            }
+            mbar_arrive(&sm->info_ready);
         }
     } else if (warp == kMmaWarp) {
         // =========================================================== MMA issuer
@@ -659,20 +766,6 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             const uint32_t glast = g + (uint32_t)cnt - 1u;
             const bool full = (cnt == s.Tkv);
             const int slot_id = 2 * cta + (t > t_begin ? 1 : 0);
-            if (!full && r == 0) {
-                // which blocks hold the other pieces of this work item (worked out while the last MMA drains)
-                const long long t0 = t - s.lt, t1 = t0 + s.Tkv;
-                const int c_lo = (int)(((t0 + 1) * G + total - 1) / total - 1);
-                const int c_hi = (int)((t1 * G + total - 1) / total - 1);
-                const int nparts = min(c_hi - c_lo + 1, kMaxParts);
-                int others = 0;
-                for (int i = 0; i < nparts; ++i) {
-                    if (c_lo + i == cta) continue;
-                    const long long start = (long long)(c_lo + i) * total / G;
-                    sm->merge_slot[wg][others++] = 2 * (c_lo + i) + (t0 > start ? 1 : 0);
-                }
-                sm->merge_parts[wg] = nparts;
-            }
             if (!mbar_wait(&sm->pv_done, glast & 1u, sm, hdr, 10)) failed = true;
             tc_fence_after();
             // Row sums: every thread holds a partial sum per query; reduce the 8 sums of a column group across the
@@ -716,9 +809,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             if (r < ncg * 8) {
                 const float l = (sm->wred[wg][0][r] + sm->wred[wg][1][r]) + (sm->wred[wg][2][r] + sm->wred[wg][3][r]);
                 if (full) {
-                    sm->inv_l[col0 + r] = l > 0.f ? 1.f / l : 0.f;
+                    sm->alpha[col0 + r] = l > 0.f ? 1.f / l : 0.f;
                 } else {
-                    sm->inv_l[col0 + r] = l;                   // kept for the merge below
+                    sm->alpha[col0 + r] = l;                   // kept for the merge below
                     p.part_ml[((size_t)slot_id * 2 + 0) * 128 + col0 + r] = sm->m_ref[col0 + r];
                     p.part_ml[((size_t)slot_id * 2 + 1) * 128 + col0 + r] = l;
                 }
@@ -741,7 +834,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                             for (int k = 0; k < 8; ++k) {
                                 const int n = col0 + 8 * (j0 + jj) + k;
                                 if (n < s.Nq) {
-                                    if (full) p.out[((size_t)bh * p.N + s.q0 + n) * 128 + r] = __float2bfloat16_rn(o[jj][k] * sm->inv_l[n]);
+                                    if (full) p.out[((size_t)bh * p.N + s.q0 + n) * 128 + r] = __float2bfloat16_rn(o[jj][k] * sm->alpha[n]);
                                     else p.part_o[((size_t)slot_id * 128 + n) * 128 + r] = o[jj][k];
                                 }
                             }
@@ -756,9 +849,12 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 // tensor memory.  The two softmax groups own disjoint query columns and run this protocol independently.
                 __threadfence();
                 group_sync_any(bar_id, false);
+                const int which = slot_id & 1;
                 if (r == 0) {
+                    if (!mbar_wait(&sm->info_ready, 0, sm, hdr, 12)) failed = true;
                     int* counter = p.counters + ((size_t)bh * 2 + s.qb) * kSoftmaxGroups + wg;
-                    const int nparts = sm->merge_parts[wg];
+                    const int nparts = sm->piece_parts[which];
+                    sm->merge_parts[wg] = nparts;
                     const int old = atomicAdd(counter, 1);
                     if (old == nparts - 1) {
                         *(volatile int*)counter = 0;              // nobody else arrives in this launch: ready for the next one
@@ -788,11 +884,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                                     const int n = col0 + 8 * (j0 + jj) + k;
                                     const bool on = j0 + jj < ncg && n < s.Nq;
                                     M[jj][k] = on ? sm->m_ref[n] : -INFINITY;
-                                    lsum[jj][k] = on ? sm->inv_l[n] : 0.f;
+                                    lsum[jj][k] = on ? sm->alpha[n] : 0.f;
                                     if (!on) o_keep[jj][k] = 0.f;
                                 }
                             for (int i = 0; i < nparts - 1; ++i) {
-                                const int slot = sm->merge_slot[wg][i];
+                                const int slot = sm->piece_slot[which][i];
                                 float ms[JB][8], ls[JB][8], os[JB][8];
                                 // all loads of one piece are issued before any is used: one memory round trip
 #pragma unroll
