@@ -16,6 +16,9 @@ What each function follows:
   to the whole prefix plus the tree tokens its mask row allows.  The method
   reaches exactly softmax(scale * q k^T) v over that key set, so the oracle is
   that definition written out.
+* ``softmax_temperature``, ``verify_tree_logits``, ``verify_tree_greedy`` --
+  Fig. 1 step 4 (next-token logits become distributions) at the two sampling
+  temperatures of Section 4.1: 0.7 (probabilistic) and 0 (greedy).
 * ``verify_tree`` -- Fig. 1 steps 4-6: per-sibling acceptance with probability
   min(1, p/q) (the speculative-sampling rule the paper inherits, Section 2.1),
   on rejection the target distribution becomes norm(max(p - q, 0)) and the next
@@ -317,6 +320,97 @@ def decision_margins(p, q, tokens, parent, gamma, u_accept, u_bonus):
             lo = cs[t - 1] if t > 0 else -np.inf
             m_bon[b, u] = min(target - lo, cs[t] - target) / z
     return m_acc, m_bon
+
+
+# ----------------------------------------------------------------------------
+# verification from next-token logits (Fig. 1 step 4; temperatures of Section 4.1)
+# ----------------------------------------------------------------------------
+
+def softmax_temperature(logits, temperature):
+    """Next-token distribution exp(z_v / T) / sum_w exp(z_w / T) over the last axis, fp64, T > 0.
+
+    Fig. 1 step 4 turns the target's next-token logits into distributions; the
+    experiments sample at temperature 0.7.  The row maximum is subtracted
+    before the exponential, which changes nothing mathematically.
+    """
+    if not temperature > 0.0:
+        raise ValueError("temperature must be positive; temperature 0 is verify_tree_greedy")
+    z = np.asarray(logits, dtype=np.float64) / float(temperature)
+    z = z - z.max(axis=-1, keepdims=True)
+    e = np.exp(z)
+    return e / e.sum(axis=-1, keepdims=True)
+
+
+def verify_tree_logits(target_logits, draft_logits, temperature, tokens, parent, gamma, u_accept, u_bonus, R=0,
+                       trace: Optional[list] = None):
+    """verify_tree on p = softmax(target_logits / T), q = softmax(draft_logits / T) (both models sample at T)."""
+    p = softmax_temperature(target_logits, temperature)
+    q = softmax_temperature(draft_logits, temperature)
+    return verify_tree(p, q, tokens, parent, gamma, u_accept, u_bonus, R, trace)
+
+
+def argmax_lowest(row):
+    """Index of the largest entry; among equal largest entries the lowest id."""
+    row = np.asarray(row, dtype=np.float64)
+    best = 0
+    for v in range(1, len(row)):
+        if row[v] > row[best]:
+            best = v
+    return best
+
+
+def verify_tree_greedy(target_logits, tokens, parent, gamma, R=0):
+    """Temperature 0 (greedy sampling, Section 4.1): the target distribution is the point mass on its argmax.
+
+    A child is accepted iff its token is the argmax of the target logits at its
+    parent (min(1, p/q) is 1 there and 0 elsewhere, and the residual of a point
+    mass is the same point mass); the new token at the stop node is that node's
+    argmax.  No random numbers are involved.  next_roots lists the R largest
+    logits of the stop node (ties: lower id first).
+    """
+    parent = np.asarray(parent, dtype=np.int64)
+    depth, level_start = tree_levels(parent)
+    n_levels = len(level_start) - 1
+    N = len(parent)
+    zt = np.asarray(target_logits, dtype=np.float64)
+    B = zt.shape[0]
+    roots = [n for n in range(N) if parent[n] < 0]
+    n_roots = len(roots)
+    accept_len = np.zeros(B, dtype=np.int32)
+    out_tokens = np.full((B, n_levels + 1), -1, dtype=np.int32)
+    out_nodes = np.full((B, n_levels), -1, dtype=np.int32)
+    best_root = np.zeros(B, dtype=np.int32)
+    next_roots = np.full((B, max(R, 0)), -1, dtype=np.int32)
+    for b in range(B):
+        g = n_levels - 1 if gamma is None else int(gamma[b])
+        best = None
+        for r in roots:
+            u = r
+            path: List[int] = []
+            while depth[u] < g:
+                top = argmax_lowest(zt[b, u])
+                nxt = None
+                for c in _children(parent, u):
+                    if int(tokens[b, c]) == top:
+                        nxt = c
+                        break
+                if nxt is None:
+                    break
+                path.append(nxt)
+                u = nxt
+            if best is None or len(path) > len(best[1]):
+                best = (r, path, u)
+        r, path, stop = best
+        accept_len[b] = len(path)
+        best_root[b] = r
+        toks = ([int(tokens[b, r])] if n_roots > 1 else []) + [int(tokens[b, c]) for c in path]
+        toks.append(argmax_lowest(zt[b, stop]))
+        out_tokens[b, :len(toks)] = toks
+        out_nodes[b, :len(path)] = path
+        if R > 0:
+            next_roots[b, :] = np.argsort(-zt[b, stop], kind="stable")[:R]
+    return {"accept_len": accept_len, "out_tokens": out_tokens, "out_nodes": out_nodes,
+            "best_root": best_root, "next_roots": next_roots}
 
 
 # ----------------------------------------------------------------------------

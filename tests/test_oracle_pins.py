@@ -515,3 +515,175 @@ def test_commit_kv_turns_the_accepted_path_into_ordinary_prefix():
     # rows past the updated length keep their old content
     b = 0
     assert np.array_equal(kc2[b, :, new_lens[b]:], kc[b, :, new_lens[b]:])
+
+
+# ----------------------------------------------------------------------------
+# verification from logits: temperature and greedy (Fig. 1 step 4, Section 4.1)
+# ----------------------------------------------------------------------------
+
+def test_softmax_temperature_against_library_and_identities():
+    import scipy.special
+    rng = np.random.default_rng(20)
+    z = rng.normal(0, 3, (2, 3, 17))
+    for T in (1.0, 0.7, 2.5):
+        s = orc.softmax_temperature(z, T)
+        np.testing.assert_allclose(s, scipy.special.softmax(z / T, axis=-1), rtol=1e-13, atol=0)
+        np.testing.assert_allclose(s.sum(-1), 1.0, rtol=1e-14)
+        # adding a constant to a row changes nothing; log-ratios are logit differences over T
+        np.testing.assert_allclose(orc.softmax_temperature(z + 123.0, T), s, rtol=1e-12)
+        np.testing.assert_allclose(np.log(s[..., 3] / s[..., 5]), (z[..., 3] - z[..., 5]) / T, rtol=1e-11)
+    # temperature T is the T = 1 distribution raised to 1/T and renormalised
+    s1 = orc.softmax_temperature(z, 1.0)
+    pw = s1 ** (1.0 / 0.7)
+    np.testing.assert_allclose(orc.softmax_temperature(z, 0.7), pw / pw.sum(-1, keepdims=True), rtol=1e-12)
+    # large logits must not overflow
+    big = np.array([[1000.0, 999.0, -1000.0]])
+    np.testing.assert_allclose(orc.softmax_temperature(big, 1.0)[0, :2], [1 / (1 + np.exp(-1)), 1 / (1 + np.exp(1))], rtol=1e-13)
+    with pytest.raises(ValueError):
+        orc.softmax_temperature(z, 0.0)
+
+
+@pytest.mark.parametrize("T", [0.7, 1.0])
+def test_exact_enumeration_output_distribution_is_tempered_target(T):
+    """One node, two sibling candidates drawn i.i.d. from softmax(draft / T): the emitted token is distributed as
+    softmax(target / T), written here with the library routine, not the oracle's own softmax."""
+    import scipy.special
+    V, k = 4, 2
+    rng = np.random.default_rng(21)
+    zt = rng.normal(0, 2, (1, 1 + k, V))
+    zd = zt + rng.normal(0, 1.5, (1, 1 + k, V))
+    q0 = scipy.special.softmax(zd[0, 0] / T)
+    parent = parent_array(1, (k,))
+    emitted = np.zeros(V)
+    for xs in itertools.product(range(V), repeat=k):
+        w = np.prod([q0[x] for x in xs])
+        tokens = np.array([[0] + list(xs)])
+        # acceptance probabilities of the two stages, from an all-rejected traced run
+        trace = []
+        ua = np.full((1, 1 + k), 1.0)
+        ub = np.full((1, 1 + k), 0.5)
+        orc.verify_tree_logits(zt, zd, T, tokens, parent, None, ua, ub, trace=trace)
+        a = [t["a"] for t in trace if "child" in t]
+        stop = [t for t in trace if "stop" in t][0]
+        reach = 1.0
+        for i in range(k):
+            emitted[xs[i]] += w * reach * a[i]
+            reach *= 1.0 - a[i]
+        emitted += w * reach * stop["dist"] / stop["dist"].sum()
+    np.testing.assert_allclose(emitted, scipy.special.softmax(zt[0, 0] / T), rtol=0, atol=1e-12)
+
+
+def _toy_model_logits(seq, V):
+    """A deterministic toy 'target model': next-token logits as a function of the whole token sequence."""
+    rng = np.random.default_rng(abs(hash(tuple(int(t) for t in seq))) % (2 ** 32))
+    return rng.normal(0, 1, V)
+
+
+def _toy_tree(parent, V, prefix, seed, hit_rate):
+    """Tokens for every node (a child repeats the model's argmax with probability hit_rate) and, for every
+    node, the toy model's logits after prefix + the node's root path."""
+    rng = np.random.default_rng(seed)
+    N = len(parent)
+    tokens = np.zeros(N, dtype=np.int64)
+    paths = [None] * N
+    logits = np.zeros((N, V))
+    for n in range(N):
+        if parent[n] < 0:
+            tokens[n] = rng.integers(0, V)
+            paths[n] = list(prefix) + [tokens[n]]
+        else:
+            top = int(np.argmax(logits[parent[n]]))
+            tokens[n] = top if rng.random() < hit_rate else rng.integers(0, V)
+            paths[n] = paths[parent[n]] + [tokens[n]]
+        logits[n] = _toy_model_logits(paths[n], V)
+    return tokens, logits, paths
+
+
+@pytest.mark.parametrize("n_roots,branching", [(1, (3, 2, 1)), (1, (1, 1, 1, 1)), (2, (2, 2, 1)), (3, (2, 1))])
+def test_greedy_verification_reproduces_autoregressive_greedy_decoding(n_roots, branching):
+    """Temperature 0: what verification emits after a root is exactly what the target would have produced
+    token by token (speculative decoding does not change greedy output), and it stops at the first level where no
+    candidate carries the target's argmax."""
+    V = 7
+    parent = parent_array(n_roots, branching)
+    depth, level_start = orc.tree_levels(parent)
+    hits = 0
+    for seed in range(40):
+        prefix = [seed % V, (3 * seed) % V]
+        tokens, logits, paths = _toy_tree(parent, V, prefix, seed, 0.7)
+        r = orc.verify_tree_greedy(logits[None], tokens[None], parent, None, R=2)
+        ln = int(r["accept_len"][0])
+        root = int(r["best_root"][0])
+        emitted = [int(t) for t in r["out_tokens"][0] if t >= 0]
+        assert len(emitted) == ln + 1 + (1 if n_roots > 1 else 0)
+        # autoregressive greedy decode of the toy model from prefix + chosen root token
+        seq = list(prefix) + [int(tokens[root])]
+        want = [int(tokens[root])] if n_roots > 1 else []
+        for _ in range(ln + 1):
+            nxt = int(np.argmax(_toy_model_logits(seq, V)))
+            want.append(nxt)
+            seq.append(nxt)
+        assert emitted == want
+        # accepted nodes form a root path of the chosen root
+        u = root
+        for i in range(ln):
+            c = int(r["out_nodes"][0, i])
+            assert parent[c] == u and tokens[c] == emitted[i + (1 if n_roots > 1 else 0)]
+            u = c
+        # the walk could not have gone further: no child of the stop node carries its argmax (or the tree ends)
+        kids = [c for c in range(len(parent)) if parent[c] == u]
+        assert all(tokens[c] != emitted[-1] for c in kids)
+        # no other root gets further (brute force over all root paths)
+        for n in range(len(parent)):
+            path = []
+            v = n
+            while v >= 0:
+                path.append(v)
+                v = parent[v]
+            path = path[::-1]
+            # siblings are tried in order, so of several siblings with the argmax token the first is followed
+            def first_hit(par):
+                top = int(np.argmax(logits[par]))
+                hit = [c for c in range(len(parent)) if parent[c] == par and tokens[c] == top]
+                return hit[0] if hit else -1
+            ok = all(path[i + 1] == first_hit(path[i]) for i in range(len(path) - 1))
+            if ok:
+                assert len(path) - 1 <= ln
+                if len(path) - 1 == ln:
+                    assert path[0] >= root
+        assert list(r["next_roots"][0]) == list(np.argsort(-logits[u], kind="stable")[:2])
+        hits += ln
+    assert hits > 0                                     # the cases do accept something
+
+
+def test_greedy_is_the_low_temperature_limit_and_honours_gamma_and_ties():
+    rng = np.random.default_rng(23)
+    V = 9
+    parent = parent_array(2, (2, 2, 1))
+    N = len(parent)
+    for trial in range(20):
+        zt = rng.normal(0, 1, (3, N, V))
+        zt[np.arange(3)[:, None], np.arange(N)[None, :], rng.integers(0, V, (3, N))] += 2.0   # a clear winner
+        zd = zt + rng.normal(0, 0.5, (3, N, V))
+        # a cold draft only ever proposes its own most likely token; some of those agree with the target
+        tokens = rng.integers(0, V, (3, N))
+        for c in range(N):
+            if parent[c] >= 0:
+                src = zt if rng.random() < 0.6 else zd
+                tokens[:, c] = np.argmax(src[:, parent[c]], axis=-1)
+        gamma = rng.integers(0, 4, 3)
+        ua = rng.uniform(0.01, 0.99, (3, N))
+        ub = rng.uniform(0.01, 0.99, (3, N))
+        cold = orc.verify_tree_logits(zt, zd, 1e-3, tokens, parent, gamma, ua, ub, R=1)
+        greedy = orc.verify_tree_greedy(zt, tokens, parent, gamma, R=1)
+        for key in ("accept_len", "out_tokens", "out_nodes", "best_root", "next_roots"):
+            assert np.array_equal(cold[key], greedy[key]), key
+        assert np.all(greedy["accept_len"] <= gamma)
+    # equal largest logits: the lowest id wins, for acceptance and for the new token
+    z = np.zeros((1, 3, 4))
+    z[0, 0] = [1.0, 5.0, 5.0, 0.0]
+    z[0, 1] = [2.0, 2.0, 2.0, 2.0]
+    r = orc.verify_tree_greedy(z, np.array([[0, 2, 1]]), parent_array(1, (2,)), None, R=3)
+    assert r["accept_len"][0] == 1 and r["out_nodes"][0, 0] == 2
+    assert list(r["out_tokens"][0]) == [1, 0, -1] and list(r["next_roots"][0]) == [0, 1, 2]
+    assert orc.argmax_lowest([3.0, 7.0, 7.0]) == 1
