@@ -174,6 +174,35 @@ int mcsd_verify_tree(const float* p, const float* q,
                      void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * mcsd_verify_tree from next-token logits (Fig. 1 step 4: the target's logits are turned into distributions;
+ * Section 4.1: temperature 0.7 for probabilistic and 0 for greedy sampling).
+ *
+ *   temperature > 0   p = softmax(target_logits / temperature), q = softmax(draft_logits / temperature), then exactly
+ *                     the procedure of mcsd_verify_tree.  p and q are formed on the fly from the logits (one extra
+ *                     pass per visited node for the row maxima and normalisers) and never written to memory.
+ *   temperature == 0  greedy: a candidate is accepted iff its token is the id of the largest target logit at its
+ *                     parent (ties: lowest id; of several siblings with that token the first), the new token is
+ *                     the largest target logit of the stop node, and next_roots lists the R largest target logits
+ *                     there (ties: lower id first).  draft_logits, u_accept and u_bonus are not read and may be NULL.
+ *
+ *   target_logits, draft_logits   [dev] dtype[B][N][V]: row n holds the logits of the token that follows node n
+ *   dtype                         MCSD_F32 or MCSD_BF16 (bf16 logits are widened to fp32 exactly)
+ *   temperature                   0, or 1e-3 <= temperature <= 1e6
+ *   all other arguments           as for mcsd_verify_tree; the workspace size is mcsd_verify_tree_workspace_bytes(B, N, V)
+ *
+ * Arithmetic: exponentials and row sums in fp32 per lane, fp64 across warps and for the acceptance ratio.
+ * Errors: as mcsd_verify_tree, plus MCSD_ERR_BAD_DTYPE and MCSD_ERR_BAD_SHAPE for a temperature out of range.
+ */
+int mcsd_verify_tree_logits(const void* target_logits, const void* draft_logits, int dtype, float temperature,
+                            const int32_t* tokens, const int32_t* parent, const int32_t* level_start,
+                            int n_levels, int n_roots, const int32_t* gamma,
+                            const float* u_accept, const float* u_bonus,
+                            int B, int N, int V,
+                            int32_t* accept_len, int32_t* out_tokens, int32_t* out_nodes,
+                            int32_t* best_root, int32_t* next_roots, int R,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * KV-cache update after acceptance (Fig. 1 step 6): "update the input IDs, key-value cache".  For every layer and
  * sequence b the keys/values of the winning root (node best_root[b]; with a single root that is node 0, the last
  * emitted token, which is not in the prefix cache yet) and of the accepted nodes out_nodes[b][0 .. accept_len[b]-1]

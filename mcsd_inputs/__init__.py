@@ -28,7 +28,7 @@ import torch
 
 __all__ = [
     "Workload", "WORKLOADS", "workload", "parent_array", "fork_parent_array",
-    "seq_lens", "gammas", "attention_inputs", "verify_inputs", "UNIFORM_MARGIN",
+    "seq_lens", "gammas", "attention_inputs", "verify_inputs", "verify_logit_inputs", "UNIFORM_MARGIN",
 ]
 
 # Uniforms are kept inside [UNIFORM_MARGIN, 1 - UNIFORM_MARGIN].
@@ -235,3 +235,57 @@ def verify_inputs(w: Workload, step: int = 0, device="cpu", parent: Optional[np.
     u_accept = torch.rand((B, N), generator=ga, device=device, dtype=torch.float32).clamp_(lo, hi)
     u_bonus = torch.rand((B, N), generator=gb, device=device, dtype=torch.float32).clamp_(lo, hi)
     return {"p": p, "q": q, "tokens": tokens.to(torch.int32), "u_accept": u_accept, "u_bonus": u_bonus}
+
+
+def verify_logit_inputs(w: Workload, temperature: float, dtype=torch.float32, step: int = 0, device="cpu",
+                        parent: Optional[np.ndarray] = None, B: Optional[int] = None, V: Optional[int] = None):
+    """target_logits, draft_logits ``[B][N][V]`` in `dtype`, tokens ``[B][N]`` int32, u_accept, u_bonus ``[B][N]`` fp32.
+
+    The logits are those behind ``verify_inputs`` (draft = target + noise), rounded to `dtype`.  What the draft
+    proposes depends on how it samples: at temperature > 0 a node's children are independent draws from
+    softmax(draft logits of the parent / temperature); at temperature 0 they are the parent's largest draft
+    logits, one per child.  Roots are as in ``verify_inputs``.
+    """
+    if parent is None:
+        parent = parent_array(w.n_roots, w.branching)
+    B = w.B if B is None else B
+    V = w.V if V is None else V
+    N = len(parent)
+    n_roots = int((parent < 0).sum())
+
+    gt = _gen(device, w.seed(step, _S_LOGIT_T))
+    gd = _gen(device, w.seed(step, _S_LOGIT_D))
+    logit_t = torch.randn((B, N, V), generator=gt, device=device, dtype=torch.float32) * w.sigma_target
+    logit_d = logit_t + torch.randn((B, N, V), generator=gd, device=device, dtype=torch.float32) * w.sigma_draft
+    logit_t = logit_t.to(dtype)
+    logit_d = logit_d.to(dtype)
+
+    gk = _gen(device, w.seed(step, _S_TOK))
+    tokens = torch.zeros((B, N), dtype=torch.int64, device=device)
+    if n_roots == 1:
+        tokens[:, 0] = torch.randint(0, V, (B,), generator=gk, device=device)
+    else:
+        gr = _gen(device, w.seed(step, _S_ROOT))
+        root_row = torch.randn((B, V), generator=gr, device=device) * w.sigma_target
+        tokens[:, :n_roots] = torch.topk(root_row, n_roots, dim=-1).indices
+    c = n_roots
+    while c < N:
+        u = int(parent[c])
+        e = c
+        while e < N and parent[e] == u:
+            e += 1
+        row = logit_d[:, u, :].float()
+        if temperature > 0:
+            tokens[:, c:e] = torch.multinomial(torch.softmax(row / temperature, dim=-1), e - c, replacement=True,
+                                               generator=gk)
+        else:
+            tokens[:, c:e] = torch.topk(row, e - c, dim=-1).indices
+        c = e
+
+    ga = _gen(device, w.seed(step, _S_UACC))
+    gb = _gen(device, w.seed(step, _S_UBON))
+    lo, hi = UNIFORM_MARGIN, 1.0 - UNIFORM_MARGIN
+    u_accept = torch.rand((B, N), generator=ga, device=device, dtype=torch.float32).clamp_(lo, hi)
+    u_bonus = torch.rand((B, N), generator=gb, device=device, dtype=torch.float32).clamp_(lo, hi)
+    return {"target_logits": logit_t, "draft_logits": logit_d, "tokens": tokens.to(torch.int32),
+            "u_accept": u_accept, "u_bonus": u_bonus}

@@ -24,7 +24,7 @@ MCSD_MAX_WORDS = 3
 
 _EXPORTS = (
     "mcsd_status_string", "mcsd_last_cuda_error", "mcsd_launch_count", "mcsd_build_mask", "mcsd_tree_attention_workspace_bytes",
-    "mcsd_tree_attention", "mcsd_workspace_status", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_static", "mcsd_commit_kv",
+    "mcsd_tree_attention", "mcsd_workspace_status", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_logits", "mcsd_verify_tree_static", "mcsd_commit_kv",
 )
 
 
@@ -55,6 +55,10 @@ def _load() -> ctypes.CDLL:
     lib.mcsd_verify_tree.restype = c_int
     lib.mcsd_verify_tree.argtypes = ([c_void_p] * 5 + [c_int, c_int] + [c_void_p] * 3 + [c_int] * 3 +
                                      [c_void_p] * 5 + [c_int, c_void_p, c_size_t, c_void_p])
+    lib.mcsd_verify_tree_logits.restype = c_int
+    lib.mcsd_verify_tree_logits.argtypes = ([c_void_p, c_void_p, c_int, c_float] + [c_void_p] * 3 + [c_int, c_int] +
+                                            [c_void_p] * 3 + [c_int] * 3 + [c_void_p] * 5 +
+                                            [c_int, c_void_p, c_size_t, c_void_p])
     lib.mcsd_verify_tree_static.restype = c_int
     lib.mcsd_verify_tree_static.argtypes = ([c_void_p] * 5 + [c_int, c_int] + [c_void_p] * 3 + [c_int] * 3 +
                                             [c_void_p] * 5 + [c_int, c_void_p])
@@ -236,6 +240,52 @@ def mcsd_verify_tree(p, q, tokens, mask: TreeMask, gamma, u_accept, u_bonus, R: 
                                   _ptr(out["best_root"]), _ptr(out.get("next_roots")), R, _ptr(workspace),
                                   workspace.numel(), _stream())
     _check(st, "mcsd_verify_tree")
+    return out
+
+
+def mcsd_verify_tree_logits(target_logits, draft_logits, temperature: float, tokens, mask: TreeMask, gamma,
+                            u_accept, u_bonus, R: int = 0, workspace: Optional[torch.Tensor] = None,
+                            out: Optional[dict] = None) -> dict:
+    """mcsd_verify_tree on softmax(logits / temperature), formed inside the kernels; temperature 0 is greedy
+    verification, for which draft_logits, u_accept and u_bonus may be None (see mcsd.h)."""
+    B, N, V = target_logits.shape
+    dt = target_logits.dtype
+    if dt not in (torch.float32, torch.bfloat16):
+        raise ValueError("logits must be float32 or bfloat16")
+    _dev_tensor(target_logits, dt, "target_logits")
+    _dev_tensor(tokens, torch.int32, "tokens")
+    if draft_logits is not None:
+        _dev_tensor(draft_logits, dt, "draft_logits")
+        if tuple(draft_logits.shape) != (B, N, V):
+            raise ValueError("shape mismatch between target and draft logits")
+    if u_accept is not None:
+        _dev_tensor(u_accept, torch.float32, "u_accept")
+    if u_bonus is not None:
+        _dev_tensor(u_bonus, torch.float32, "u_bonus")
+    if gamma is not None:
+        _dev_tensor(gamma, torch.int32, "gamma")
+    if mask.n_nodes != N or tuple(tokens.shape) != (B, N):
+        raise ValueError("shape mismatch between logits, tokens and the tree")
+    dev = target_logits.device
+    nl = mask.n_levels
+    if out is None:
+        out = {
+            "accept_len": torch.empty(B, dtype=torch.int32, device=dev),
+            "out_tokens": torch.empty((B, nl + 1), dtype=torch.int32, device=dev),
+            "out_nodes": torch.empty((B, nl), dtype=torch.int32, device=dev),
+            "best_root": torch.empty(B, dtype=torch.int32, device=dev),
+            "next_roots": torch.empty((B, R), dtype=torch.int32, device=dev) if R > 0 else None,
+        }
+    if workspace is None:
+        workspace = new_workspace(mcsd_verify_tree_workspace_bytes(B, N, V), dev)
+    code = MCSD_BF16 if dt == torch.bfloat16 else MCSD_F32
+    with torch.cuda.device(dev):
+        st = lib.mcsd_verify_tree_logits(_ptr(target_logits), _ptr(draft_logits), code, float(temperature), _ptr(tokens),
+                                         _ptr(mask.parent), _ptr(mask.level_start), nl, mask.n_roots, _ptr(gamma),
+                                         _ptr(u_accept), _ptr(u_bonus), B, N, V, _ptr(out["accept_len"]),
+                                         _ptr(out["out_tokens"]), _ptr(out["out_nodes"]), _ptr(out["best_root"]),
+                                         _ptr(out.get("next_roots")), R, _ptr(workspace), workspace.numel(), _stream())
+    _check(st, "mcsd_verify_tree_logits")
     return out
 
 

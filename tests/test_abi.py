@@ -94,6 +94,26 @@ def test_verify_argument_checks(m):
     assert call(wsb=8) == -5
 
 
+def test_verify_logits_argument_checks(m):
+    L = m.lib
+
+    def call(zt=FAKE, zd=FAKE, dtype=1, T=0.7, ua=FAKE, B=2, N=15, V=100, nl=4, nr=1, R=0, wsb=1 << 20, nxt=None):
+        return L.mcsd_verify_tree_logits(zt, zd, dtype, ctypes.c_float(T), FAKE, FAKE, FAKE, nl, nr, None, ua, FAKE,
+                                         B, N, V, FAKE, FAKE, FAKE, FAKE, nxt, R, FAKE, wsb, None)
+    assert call(zt=None) == -1
+    assert call(zd=None) == -1                   # the draft logits are needed unless the temperature is 0
+    assert call(ua=None) == -1
+    assert call(T=-1.0) == -2
+    assert call(T=float("nan")) == -2
+    assert call(T=1e-5) == -2
+    assert call(dtype=9) == -4
+    assert call(N=193) == -2
+    assert call(V=0) == -2
+    assert call(R=2, nxt=None) == -1
+    assert call(wsb=8) == -5
+    assert call(T=0.0, zd=None, ua=None, wsb=8) == -5    # greedy passes the pointer checks without draft and uniforms
+
+
 def test_commit_kv_argument_checks(m):
     L = m.lib
 

@@ -10,7 +10,8 @@ import numpy as np
 import pytest
 import torch
 
-from mcsd_inputs import attention_inputs, gammas, parent_array, seq_lens, verify_inputs, workload
+from mcsd_inputs import (attention_inputs, gammas, parent_array, seq_lens, verify_inputs, verify_logit_inputs,
+                         workload)
 from oracle import mcsd_oracle as orc
 from tests.helpers import condition_uniforms, oracle_attention_rows, to_np
 
@@ -310,6 +311,128 @@ def test_verify_edge_cases(m):
     w5 = workload(5)
     _verify_case(m, w5, parent=parent_array(16, (1, 1, 1, 1)), B=4, V=2000, gamma=np.array([4, 1, 2, 0]))
     _verify_case(m, w5, parent=parent_array(2, (4, 3, 1, 1)), B=4, V=2000, gamma=None, R=2)
+
+
+# ----------------------------------------------------------------------------------------------
+# accept / reject from logits: temperature > 0 and greedy (temperature 0)
+# ----------------------------------------------------------------------------------------------
+
+def _verify_logits_case(m, w, T, dtype, parent=None, B=None, V=None, gamma="workload", R=0, tweak=None, step=0):
+    parent = parent_array(w.n_roots, w.branching) if parent is None else parent
+    vin = verify_logit_inputs(w, T, dtype, step, "cuda", parent=parent, B=B, V=V)
+    B = vin["target_logits"].shape[0]
+    if isinstance(gamma, str):
+        gamma = None if w.gamma is None else gammas(dataclasses.replace(w, B=B), step)
+    if tweak is not None:
+        tweak(vin)
+    host = {k: to_np(v) for k, v in vin.items()}
+    zt, zd = host["target_logits"], host["draft_logits"]
+    ua, ub = host["u_accept"].copy(), host["u_bonus"].copy()
+    keys = ("accept_len", "out_tokens", "out_nodes", "best_root", "next_roots")
+    parts = []
+    for b in range(B):                                   # sequences are independent; one at a time bounds the fp64 memory
+        g = None if gamma is None else gamma[b:b + 1]
+        if T > 0:
+            pb = orc.softmax_temperature(zt[b:b + 1], T)
+            qb = orc.softmax_temperature(zd[b:b + 1], T)
+            ua[b:b + 1], ub[b:b + 1] = condition_uniforms(pb, qb, host["tokens"][b:b + 1], parent, g, ua[b:b + 1],
+                                                          ub[b:b + 1], seed=777 + b)
+            del pb, qb
+            parts.append(orc.verify_tree_logits(zt[b:b + 1], zd[b:b + 1], T, host["tokens"][b:b + 1], parent, g,
+                                                ua[b:b + 1], ub[b:b + 1], R=R))
+        else:
+            parts.append(orc.verify_tree_greedy(zt[b:b + 1], host["tokens"][b:b + 1], parent, g, R=R))
+    ref = {k: np.concatenate([p_[k] for p_ in parts], axis=0) for k in keys}
+    tm = m.mcsd_build_mask(parent)
+    dev = vin["target_logits"].device
+    g_d = None if gamma is None else torch.from_numpy(np.asarray(gamma, dtype=np.int32)).to(dev)
+    if T > 0:
+        got = m.mcsd_verify_tree_logits(vin["target_logits"], vin["draft_logits"], T, vin["tokens"], tm, g_d,
+                                        torch.from_numpy(ua).to(dev), torch.from_numpy(ub).to(dev), R=R)
+    else:
+        got = m.mcsd_verify_tree_logits(vin["target_logits"], None, 0.0, vin["tokens"], tm, g_d, None, None, R=R)
+    torch.cuda.synchronize()
+    for k in ("accept_len", "out_tokens", "out_nodes", "best_root"):
+        assert np.array_equal(got[k].cpu().numpy(), ref[k]), k
+    if R > 0:
+        assert np.array_equal(got["next_roots"].cpu().numpy(), ref["next_roots"])
+    return ref
+
+
+@pytest.mark.parametrize("T", [0.7, 1.0])
+def test_verify_logits_tiny_fp32_workload(m, T):
+    _verify_logits_case(m, workload(1), T, torch.float32, R=4)
+    _verify_logits_case(m, workload(1), T, torch.bfloat16, B=3, R=4, step=1)
+
+
+def test_verify_logits_llama_shapes_bf16(m):
+    ref = _verify_logits_case(m, workload(2), 0.7, torch.bfloat16, R=8)
+    assert ref["accept_len"][0] >= 0
+    ref = _verify_logits_case(m, workload(4), 0.7, torch.bfloat16)
+    assert ref["accept_len"].max() > 0
+
+
+def test_verify_logits_dynamic_slice_and_forest(m):
+    _verify_logits_case(m, workload(3), 0.7, torch.float32, R=2)
+    ref = _verify_logits_case(m, workload(5), 1.0, torch.bfloat16, B=8, R=8)
+    assert len(set(ref["best_root"].tolist())) > 1
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_verify_greedy_workloads(m, dtype):
+    _verify_logits_case(m, workload(1), 0.0, dtype, R=4)
+    ref = _verify_logits_case(m, workload(4), 0.0, dtype, R=2)
+    assert ref["accept_len"].max() > 0
+    _verify_logits_case(m, workload(3), 0.0, dtype, step=1)
+    _verify_logits_case(m, workload(5), 0.0, dtype, B=8, R=8)
+    torch.cuda.empty_cache()
+
+
+def test_verify_logits_edge_cases(m):
+    w = workload(1)
+    for T in (0.7, 0.0):
+        for dtype in (torch.float32, torch.bfloat16):
+            # vocabulary sizes that are not a multiple of the vector width take the scalar-load path
+            for V in (5, 13, 1001):
+                _verify_logits_case(m, w, T, dtype, B=3, V=V, R=3)
+            ref = _verify_logits_case(m, w, T, dtype, B=2, gamma=np.array([0, 2]))
+            assert ref["accept_len"][0] == 0
+            _verify_logits_case(m, w, T, dtype, parent=np.array([-1], dtype=np.int32), B=2, R=2)
+    # ids the models can never emit (logit -inf), in different places for target and draft
+    def masked(vin):
+        vin["target_logits"][:, :, 0:40] = float("-inf")
+        vin["draft_logits"][:, :, 20:60] = float("-inf")
+        vin["tokens"][:, 1:3] = 5                          # candidates the target can never emit
+    ref = _verify_logits_case(m, w, 0.7, torch.float32, B=2, tweak=masked, R=3)
+    assert ref["out_tokens"].max() >= 40
+    # draft equal to target: every first candidate is accepted down to the leaves
+    def same(vin):
+        vin["draft_logits"].copy_(vin["target_logits"])
+    ref = _verify_logits_case(m, w, 1.0, torch.float32, B=2, tweak=same)
+    assert list(ref["accept_len"]) == [3, 3]
+    # greedy with equal largest logits: the lowest id wins; of two siblings with that token the first is followed
+    def ties(vin):
+        z = vin["target_logits"]
+        z.clamp_(max=2.0)
+        z[:, :, 700] = 4.0
+        z[:, :, 300] = 4.0
+        vin["tokens"][:, 1] = 700
+        vin["tokens"][:, 2] = 300
+        vin["tokens"][:, 5] = 300
+        vin["tokens"][:, 6] = 300
+    ref = _verify_logits_case(m, w, 0.0, torch.float32, B=2, tweak=ties, R=3)
+    assert list(ref["out_nodes"][0][:2]) == [2, 5] and list(ref["next_roots"][0][:2]) == [300, 700]
+    # large logits and a high temperature stay finite
+    def big(vin):
+        vin["target_logits"].mul_(30.0)
+        vin["draft_logits"].mul_(30.0)
+    _verify_logits_case(m, w, 50.0, torch.float32, B=2, tweak=big, R=2)
+    w5 = workload(5)
+    _verify_logits_case(m, w5, 0.7, torch.bfloat16, parent=parent_array(16, (1, 1, 1, 1)), B=4, V=2000,
+                        gamma=np.array([4, 1, 2, 0]))
+    _verify_logits_case(m, w5, 0.7, torch.float32, parent=parent_array(2, (4, 3, 1, 1)), B=4, V=2000, gamma=None, R=2)
+    _verify_logits_case(m, w5, 0.0, torch.bfloat16, parent=parent_array(2, (4, 3, 1, 1)), B=4, V=2000, gamma=None, R=2)
 
 
 # ----------------------------------------------------------------------------------------------
