@@ -26,7 +26,10 @@
 
 namespace mcsd {
 
-constexpr int kVerifyThreads = 1024;
+#ifndef MCSD_VERIFY_THREADS
+#define MCSD_VERIFY_THREADS 512
+#endif
+constexpr int kVerifyThreads = MCSD_VERIFY_THREADS;
 constexpr int kVerifyWarps = kVerifyThreads / 32;
 
 struct NodeState {
