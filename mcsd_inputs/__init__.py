@@ -65,6 +65,7 @@ class Workload:
     sigma_draft: float = 1.0
     n_layers: int = 1
     base_seed: Optional[int] = None
+    early_stop: Optional[float] = None   # threshold beta of a synthetic early-stop process that sets gamma
 
     @property
     def L_max(self) -> int:
@@ -95,6 +96,12 @@ WORKLOADS: Dict[str, Workload] = {
                  _INV_SQRT_128, n_layers=32),
         Workload("target_init_b32", 5, "bf16", 32, 32, 128, (256, 4096), 8, (1, 2, 2, 1, 1, 1), (1, 6), 32000,
                  _INV_SQRT_128, sigma_draft=1.5),
+        # the paper's own tree shapes (Section 4.1): the static target-initialised configuration (2; 4,3,1,1) and
+        # the fork of width 16 and depth 5 hanging off the last emitted token, cut by an early stop (beta = 0.4)
+        Workload("paper_static_2_4_3_1_1", 6, "bf16", 16, 32, 128, (512, 2048), 2, (4, 3, 1, 1), None, 32000,
+                 _INV_SQRT_128),
+        Workload("paper_fork_w16_d5", 7, "bf16", 16, 32, 128, (512, 2048), 1, (16, 1, 1, 1, 1), (1, 5), 32000,
+                 _INV_SQRT_128, early_stop=0.4),
     )
 }
 
@@ -157,7 +164,28 @@ def gammas(w: Workload, step: int = 0) -> np.ndarray:
         return np.full(w.B, full, dtype=np.int32)
     lo, hi = w.gamma
     g = _gen("cpu", w.seed(step, _S_GAMMA))
+    if w.early_stop is not None:
+        return _early_stop_gammas(w, g, lo, hi)
     return torch.randint(lo, hi + 1, (w.B,), generator=g).numpy().astype(np.int32)
+
+
+def _early_stop_gammas(w: Workload, g: torch.Generator, lo: int, hi: int) -> np.ndarray:
+    """Stand-in for the decision model of Section 3.3, which is not part of the verification path.
+
+    Every draft turn gives each of the W candidate sequences a score in (0, 1) (here uniform); a sequence's
+    predicted chance of being accepted so far is the product of its scores; drafting stops after the first turn
+    at which every sequence is below the threshold, else at the maximum depth.  gamma = turns drafted.
+    """
+    W = w.n_roots if w.n_roots > 1 else w.branching[0]
+    score = torch.rand((w.B, hi, W), generator=g, dtype=torch.float64).cumprod(dim=1)
+    alive = (score.max(dim=2).values >= w.early_stop).numpy()          # [B][turn]
+    out = np.full(w.B, hi, dtype=np.int32)
+    for b in range(w.B):
+        for t in range(hi):
+            if not alive[b, t]:
+                out[b] = t + 1
+                break
+    return np.clip(out, lo, hi).astype(np.int32)
 
 
 def attention_inputs(w: Workload, layer: int = 0, device="cpu", std: Optional[float] = None):

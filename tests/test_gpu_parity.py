@@ -218,7 +218,7 @@ def test_attention_needle_reads_out_the_mask(m):
             assert np.abs(got[:, :min(N, D)] - expect).max() <= 4e-3
 
 
-@pytest.mark.parametrize("idx", [3, 4, 5])
+@pytest.mark.parametrize("idx", [3, 4, 5, 6, 7])
 def test_attention_full_size_sampled(m, idx):
     # the workload at its full size, in the launch configuration the benchmark times; the oracle
     # checks a seeded sample of (sequence, head) pairs, every row of each
@@ -433,6 +433,17 @@ def test_verify_logits_edge_cases(m):
                         gamma=np.array([4, 1, 2, 0]))
     _verify_logits_case(m, w5, 0.7, torch.float32, parent=parent_array(2, (4, 3, 1, 1)), B=4, V=2000, gamma=None, R=2)
     _verify_logits_case(m, w5, 0.0, torch.bfloat16, parent=parent_array(2, (4, 3, 1, 1)), B=4, V=2000, gamma=None, R=2)
+
+
+def test_verify_paper_shaped_workloads(m):
+    # the static (2; 4,3,1,1) forest and the early-stopped fork W = 16, D = 5 of Section 4.1, all three verify modes
+    for idx in (6, 7):
+        w = workload(idx)
+        ref = _verify_case(m, w, R=2)
+        assert ref["accept_len"].max() > 0
+        _verify_logits_case(m, w, 0.7, torch.bfloat16, R=2, step=1)
+        _verify_logits_case(m, w, 0.0, torch.bfloat16, R=2, step=1)
+        torch.cuda.empty_cache()
 
 
 # ----------------------------------------------------------------------------------------------

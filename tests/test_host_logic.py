@@ -96,3 +96,23 @@ def test_two_rank_batch_sharding_over_gloo(m):
         assert p.exitcode == 0
     assert ok
     assert units == 5 * 7 and ms == 20.0      # units add up over ranks, time is the slowest rank's
+
+
+def test_paper_shaped_workloads_and_early_stop_gammas():
+    """Section 4.1: the static configuration (2; 4,3,1,1) has 82 nodes; the fork W = 16, D = 5 hangs 80 draft tokens
+    off the last emitted token.  The early-stop stand-in gives reproducible draft lengths in 1..D that do vary."""
+    from mcsd_inputs import gammas, parent_array, workload
+    w6, w7 = workload("paper_static_2_4_3_1_1"), workload("paper_fork_w16_d5")
+    assert w6.n_nodes == 2 + 2 * 40 and w6.n_roots == 2
+    p7 = parent_array(w7.n_roots, w7.branching)
+    assert len(p7) == 1 + 16 * 5 and int((p7 == 0).sum()) == 16
+    for n in range(17, len(p7)):                      # every deeper node continues exactly one chain
+        assert int((p7 == p7[n]).sum()) == 1
+    assert list(gammas(w6)) == [4] * w6.B
+    seen = set()
+    for step in range(6):
+        g = gammas(w7, step)
+        assert np.array_equal(g, gammas(w7, step))
+        assert g.min() >= 1 and g.max() <= 5
+        seen |= set(g.tolist())
+    assert len(seen) >= 3
