@@ -30,6 +30,7 @@
 #include <cuda_bf16.h>
 
 #include <mutex>
+#include <type_traits>
 
 #include "attention.cuh"
 
@@ -45,7 +46,7 @@ constexpr int kSlabBytes = kTile * 128;       // 64 of the 128 columns: rows of 
 constexpr int kMaxSlots = 6;
 constexpr int kMaxBatchTc = 256;
 constexpr int kTmemCols = 512;
-constexpr int kColS1 = 128, kColO = 256;
+constexpr int kColS1 = 128, kColO = 256, kColL = 384;   // tensor-memory columns: S^T twice, O^T, row sums
 constexpr float kLazyTau = 8.0f;              // raise the reference maximum only beyond 2^8
 constexpr int kMaxParts = 64;                 // a (sequence, head) has at most 34 tiles, so at most 35 pieces
 constexpr int kMaxCtas = 160;                 // partial slots are provisioned for this many thread blocks
@@ -62,7 +63,7 @@ struct TcSmall {
     // pieces of the (at most two) work items this block shares with others: [0] the segment at the start of its
     // range, [1] the one at the end.  Worked out once by the bookkeeping warp.
     int piece_parts[2];
-    int piece_slot[2][kMaxParts];
+    unsigned short piece_slot[2][kMaxParts];
     long long range[2];                // first and one-past-last tile of this block
     int n_blocks;                      // blocks that got tiles
     alignas(16) float m_ref[128];
@@ -71,6 +72,7 @@ struct TcSmall {
     alignas(16) unsigned long long dmask[MCSD_MAX_NODES][3];
     unsigned short cum_tiles[kMaxBatchTc + 2];   // tiles per head of the sequences before b (at most 256 * 68)
     int cum_w[kMaxBatchTc + 1];        // the same in cost units (see tile_weight)
+    alignas(128) __nv_bfloat16 ones[256];   // 16 x 16 matrix of ones: B operand of the row-sum product (wide launches)
 };
 // the small state must leave room for six 32 KB ring slots next to Q and P^T of a 48-query launch
 static_assert(sizeof(TcSmall) <= 232448 - 1024 - 6 * 32768 - 48 * 512, "TcSmall grew: the 6-slot ring no longer fits");
@@ -165,7 +167,35 @@ __device__ __forceinline__ void tc_ld8(uint32_t taddr, float* v) {
 #pragma unroll
     for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ float tc_ld1(uint32_t taddr) {
+    float v;
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=f"(v) : "r"(taddr) : "memory");
+    return v;
+}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Calls f(j, values of 8-column group j) for the first ncg of a thread's column groups, reading tensor memory
+// MCSD_SWEEP_BATCH groups per round trip (larger batches cost registers the wide kernels do not have).  ncg is
+// uniform per warp.
+#ifndef MCSD_SWEEP_BATCH
+#define MCSD_SWEEP_BATCH 1
+#endif
+template <int CPT, typename F>
+__device__ __forceinline__ void sweep_groups(uint32_t taddr, int ncg, F&& f) {
+    constexpr int SB = MCSD_SWEEP_BATCH;
+#pragma unroll
+    for (int j0 = 0; j0 < CPT; j0 += SB) {
+        if (j0 < ncg) {
+            float buf[SB][8];
+#pragma unroll
+            for (int jj = 0; jj < SB; ++jj)
+                if (j0 + jj < CPT && j0 + jj < ncg) tc_ld8(taddr + 8 * (j0 + jj), buf[jj]);
+            tc_wait_ld();
+#pragma unroll
+            for (int jj = 0; jj < SB; ++jj)
+                if (j0 + jj < CPT && j0 + jj < ncg) f(j0 + jj, buf[jj]);
+        }
+    }
+}
 __device__ __forceinline__ void tc_st8(uint32_t taddr, const float* v) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
@@ -319,6 +349,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     const int cta = blockIdx.x;
 
     // ---- set-up: tile counts per sequence, barriers, tensor memory
+    constexpr bool WIDE = NCH > 4;              // many query columns: row sums come from the tensor cores (see below)
+    if (WIDE && tid < 256) {
+        sm->ones[tid] = __float2bfloat16_rn(1.0f);
+        fence_async_smem();                      // read by the tensor cores through the async proxy
+    }
     for (int b = tid; b < p.B; b += kTcThreads) {
         const int L = min(max(p.seq_lens[b], 0), p.L_max);
         const int Nb = p.n_active ? min(max(p.n_active[b], 0), p.N) : p.N;
@@ -441,7 +476,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     for (int i = 0; i < nparts; ++i) {
                         if (c_lo + i == cta) continue;
                         const long long start = first_tile_of_block(sm, p, c_lo + i, G, total_w, total);
-                        sm->piece_slot[which][others++] = 2 * (c_lo + i) + (t0 > start ? 1 : 0);
+                        sm->piece_slot[which][others++] = (unsigned short)(2 * (c_lo + i) + (t0 > start ? 1 : 0));
                     }
                 }
                 sm->piece_parts[which] = nparts;
@@ -505,6 +540,17 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                             const uint64_t db = smem_desc(p_a + k * 256, 128, 2048, 0);
                             tc_mma(tmem + kColO, da, db, idesc_pv, !(i == 1 && k == 0));
                         }
+                        if (WIDE) {
+                            // Row sums of this tile's probabilities: L[query][.] = P[query][key] * ones[key][.], P^T read
+                            // as the A operand (queries on the accumulator's lanes), not accumulated across tiles.
+                            const uint32_t idesc_l = instr_desc(16, 1, 0);
+                            const uint64_t d1 = smem_desc(smem_u32(sm->ones), 128, 256, 0);
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const uint64_t dp = smem_desc(p_a + k * 256, 128, 2048, 0);
+                                tc_mma(tmem + kColL, dp, d1, idesc_l, k > 0);
+                            }
+                        }
                         tc_commit(&sm->slot_empty[slot]);
                         tc_commit(&sm->pv_done);
                     }
@@ -532,6 +578,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         const int wg = warp >> 2, wq = warp & 3;
         const int r = tid & 127;
         const int bar_id = 1 + wg;
+        // Reference maxima and rescale factors of this group's own query columns, indexed from the group's first
+        // column: the split of the columns between the groups changes with the segment's query count, and one group
+        // may already be in the next segment while the other still finishes this one.
+        float* const mref = sm->m_ref + 64 * wg;
+        float* const alph = sm->alpha + 64 * wg;
         // dmask[t] = set of queries that may see tree key t: the ancestor bitsets transposed.  The bitsets are
         // first copied to shared memory in one coalesced round trip (the P^T buffer is free until the first tile
         // is finished), then every thread transposes one key's column out of shared memory.
@@ -559,23 +610,27 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         long long t = t_begin;
         uint32_t u = 0, g = 0;
         bool failed = false;
-        float acc_l[CPT][8];
+        float acc_l[KEEP ? CPT : 1][8];
+        float l_run = 0.f;                              // wide launches: row sum of query r (this thread's lane) so far
         while (t < t_end) {
             Segment s;
             locate(sm, p, t, s);
             const int cnt = (int)min((long long)(s.Tkv - s.lt), t_end - t);
             const int bh = s.b * p.H + s.h;
             const int ng8 = (s.Nq + 7) >> 3;
-            const int g0 = wg * CPT;
-            const int ncg = max(0, min(CPT, ng8 - g0));          // 8-column groups of this thread in this segment
+            const int half = (ng8 + 1) >> 1;                     // the two groups split the columns evenly
+            const int g0 = wg * half;
+            const int ncg = wg == 0 ? half : ng8 - half;         // 8-column groups of this thread in this segment
             const int col0 = g0 * 8;
             const unsigned long long nb_lo = s.Nq >= 64 ? ~0ull : ((1ull << s.Nq) - 1ull);
             const unsigned long long nb_hi = s.Nq >= 128 ? ~0ull : (s.Nq > 64 ? ((1ull << (s.Nq - 64)) - 1ull) : 0ull);
-            if (r < ncg * 8) sm->m_ref[col0 + r] = -INFINITY;
+            if (r < ncg * 8) mref[r] = -INFINITY;
 #pragma unroll
-            for (int j = 0; j < CPT; ++j)
+            for (int j = 0; j < (KEEP ? CPT : 1); ++j)
 #pragma unroll
                 for (int k = 0; k < 8; ++k) acc_l[j][k] = 0.f;
+            l_run = 0.f;
+            const bool own = r >= col0 && r < col0 + 8 * ncg;    // wide launches: query r is one of this group's
             if (group_sync_any(bar_id, failed)) { failed = true; break; }
 
             for (int i = 0; i < cnt; ++i) {
@@ -598,39 +653,61 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 if (!mbar_wait(&sm->s_full[sb], (gi >> 1) & 1u, sm, hdr, 7)) failed = true;
                 tc_fence_after();
                 const uint32_t s_addr = tmem + lane_addr + (sb ? kColS1 : 0) + col0;
+                bool l_taken = false;                   // wide launches: previous tile's row sum already added
 
                 // ---- pass A: scores minus the running reference, and the largest excess
                 float y[KEEP ? CPT : 1][8];
+                uint32_t pk[KEEP ? 1 : CPT][4];
                 float dmax = -INFINITY;
+                auto wide_pass = [&](auto masked_tag) {
+                    constexpr bool MASKED = decltype(masked_tag)::value;
+                    sweep_groups<CPT>(s_addr, ncg, [&](int j, const float* v) {
+                        const float4 m0 = *reinterpret_cast<const float4*>(&mref[8 * j]);
+                        const float4 m1 = *reinterpret_cast<const float4*>(&mref[8 * j + 4]);
+                        const float mr[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+                        const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
+                        float yy[8];
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            yy[k] = fmaf(v[k], p.scale_log2, -mr[k]);
+                            if (MASKED && !((bits >> k) & 1u)) yy[k] = -INFINITY;
+                            dmax = fmaxf(dmax, yy[k]);
+                        }
+#pragma unroll
+                        for (int k = 0; k < 8; k += 2) {
+                            __nv_bfloat162 h2 = __floats2bfloat162_rn(ex2_approx(yy[k]), ex2_approx(yy[k + 1]));
+                            pk[KEEP ? 0 : j][k >> 1] = *reinterpret_cast<uint32_t*>(&h2);
+                        }
+                    });
+                };
                 if (KEEP) {
 #pragma unroll
                     for (int j = 0; j < CPT; ++j)
                         if (j < ncg) tc_ld8(s_addr + 8 * j, y[KEEP ? j : 0]);
                     tc_wait_ld();
                 }
+                if (KEEP) {
 #pragma unroll
-                for (int j = 0; j < CPT; ++j) {
-                    if (j < ncg) {
-                        float v[8];
-                        if (KEEP) {
+                    for (int j = 0; j < CPT; ++j) {
+                        if (j < ncg) {
+                            const float4 m0 = *reinterpret_cast<const float4*>(&mref[8 * j]);
+                            const float4 m1 = *reinterpret_cast<const float4*>(&mref[8 * j + 4]);
+                            const float mr[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+                            const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
 #pragma unroll
-                            for (int k = 0; k < 8; ++k) v[k] = y[KEEP ? j : 0][k];
-                        } else {
-                            tc_ld8(s_addr + 8 * j, v);
-                            tc_wait_ld();
-                        }
-                        const float4 m0 = *reinterpret_cast<const float4*>(&sm->m_ref[col0 + 8 * j]);
-                        const float4 m1 = *reinterpret_cast<const float4*>(&sm->m_ref[col0 + 8 * j + 4]);
-                        const float mr[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
-                        const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            float yy = fmaf(v[k], p.scale_log2, -mr[k]);
-                            if (!full_tile && !((bits >> k) & 1u)) yy = -INFINITY;
-                            dmax = fmaxf(dmax, yy);
-                            if (KEEP) y[KEEP ? j : 0][k] = yy;
+                            for (int k = 0; k < 8; ++k) {
+                                float yy = fmaf(y[KEEP ? j : 0][k], p.scale_log2, -mr[k]);
+                                if (!full_tile && !((bits >> k) & 1u)) yy = -INFINITY;
+                                dmax = fmaxf(dmax, yy);
+                                y[KEEP ? j : 0][k] = yy;
+                            }
                         }
                     }
+                } else {
+                    // wide launches: one sweep gives the largest excess and, optimistically, the probabilities
+                    // themselves (packed bf16, kept in registers until the P^T buffer is free); row sums come
+                    // from the tensor cores, so nothing is accumulated here that a raised reference would spoil
+                    if (full_tile) wide_pass(std::false_type{}); else wide_pass(std::true_type{});
                 }
                 if (group_sync_any(bar_id, dmax > kLazyTau || failed)) {
                     if (*(volatile int*)&sm->abort_flag) { failed = true; break; }
@@ -657,17 +734,24 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     if (r < ncg * 8) {
                         const float tm = fmaxf(fmaxf(sm->wred[wg][0][r], sm->wred[wg][1][r]),
                                                fmaxf(sm->wred[wg][2][r], sm->wred[wg][3][r]));
-                        const float mo = sm->m_ref[col0 + r];
+                        const float mo = mref[r];
                         float a = 1.f;
                         if (tm > mo) {
                             a = (mo == -INFINITY) ? 0.f : exp2f(mo - tm);
-                            sm->m_ref[col0 + r] = tm;
+                            mref[r] = tm;
                             need = (i > 0) && (mo != -INFINITY);
                         }
-                        sm->alpha[col0 + r] = a;
+                        alph[r] = a;
                     }
                     const bool rescale = group_sync_any(bar_id, need);
                     if (gi > 0 && !mbar_wait(&sm->pv_done, (gi - 1u) & 1u, sm, hdr, 8)) failed = true;
+                    if (WIDE) {
+                        // the previous tile's row sum belongs to the old reference: take it in before rescaling
+                        tc_fence_after();
+                        if (i > 0) { const float lp = tc_ld1(tmem + lane_addr + kColL); tc_wait_ld(); l_run += lp; }
+                        l_taken = true;
+                        if (own) l_run *= alph[r - col0];
+                    }
                     if (rescale) {
                         tc_fence_after();
 #pragma unroll
@@ -678,9 +762,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                                 tc_wait_ld();
 #pragma unroll
                                 for (int k = 0; k < 8; ++k) {
-                                    const float a = sm->alpha[col0 + 8 * j + k];
+                                    const float a = alph[8 * j + k];
                                     o[k] *= a;
-                                    acc_l[j][k] *= a;
+                                    if (KEEP) acc_l[KEEP ? j : 0][k] *= a;
                                 }
                                 tc_st8(tmem + lane_addr + kColO + col0 + 8 * j, o);
                             }
@@ -697,12 +781,14 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                                 const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
 #pragma unroll
                                 for (int k = 0; k < 8; ++k) {
-                                    float yy = fmaf(v[k], p.scale_log2, -sm->m_ref[col0 + 8 * j + k]);
+                                    float yy = fmaf(v[k], p.scale_log2, -mref[8 * j + k]);
                                     if (!full_tile && !((bits >> k) & 1u)) yy = -INFINITY;
                                     y[KEEP ? j : 0][k] = yy;
                                 }
                             }
                         }
+                    } else {
+                        if (full_tile) wide_pass(std::false_type{}); else wide_pass(std::true_type{});
                     }
                 }
 
@@ -711,39 +797,37 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 if (gi > 0 && !mbar_wait(&sm->pv_done, (gi - 1u) & 1u, sm, hdr, 8)) failed = true;
 
                 // ---- pass B: probabilities, row sums, P^T for the second MMA
+                if (KEEP) {
 #pragma unroll
-                for (int j = 0; j < CPT; ++j) {
-                    if (j < ncg) {
-                        float yy[8];
-                        if (KEEP) {
+                    for (int j = 0; j < CPT; ++j) {
+                        if (j < ncg) {
+                            uint32_t packed[4];
 #pragma unroll
-                            for (int k = 0; k < 8; ++k) yy[k] = y[KEEP ? j : 0][k];
-                        } else {
-                            float v[8];
-                            tc_ld8(s_addr + 8 * j, v);
-                            tc_wait_ld();
-                            const float4 m0 = *reinterpret_cast<const float4*>(&sm->m_ref[col0 + 8 * j]);
-                            const float4 m1 = *reinterpret_cast<const float4*>(&sm->m_ref[col0 + 8 * j + 4]);
-                            const float mr[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
-                            const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                yy[k] = fmaf(v[k], p.scale_log2, -mr[k]);
-                                if (!full_tile && !((bits >> k) & 1u)) yy[k] = -INFINITY;
+                            for (int k = 0; k < 8; k += 2) {
+                                // 2^-inf = 0 for masked entries
+                                const float p0 = ex2_approx(y[KEEP ? j : 0][k]), p1 = ex2_approx(y[KEEP ? j : 0][k + 1]);
+                                acc_l[KEEP ? j : 0][k] += p0;
+                                acc_l[KEEP ? j : 0][k + 1] += p1;
+                                __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+                                packed[k >> 1] = *reinterpret_cast<uint32_t*>(&h2);
                             }
+                            *reinterpret_cast<uint4*>(p_buf + (size_t)(g0 + j) * 2048 + (size_t)r * 16) =
+                                make_uint4(packed[0], packed[1], packed[2], packed[3]);
                         }
-                        uint32_t packed[4];
-#pragma unroll
-                        for (int k = 0; k < 8; k += 2) {
-                            const float p0 = ex2_approx(yy[k]), p1 = ex2_approx(yy[k + 1]);   // 2^-inf = 0 for masked entries
-                            acc_l[j][k] += p0;
-                            acc_l[j][k + 1] += p1;
-                            __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-                            packed[k >> 1] = *reinterpret_cast<uint32_t*>(&h2);
-                        }
-                        *reinterpret_cast<uint4*>(p_buf + (size_t)(g0 + j) * 2048 + (size_t)r * 16) =
-                            make_uint4(packed[0], packed[1], packed[2], packed[3]);
                     }
+                } else {
+                    // the previous tile's row sum (its product has finished: pv_done) before the next one replaces it
+                    if (!l_taken && i > 0) {
+                        tc_fence_after();
+                        const float lp = tc_ld1(tmem + lane_addr + kColL);
+                        tc_wait_ld();
+                        l_run += lp;
+                    }
+#pragma unroll
+                    for (int j = 0; j < CPT; ++j)
+                        if (j < ncg)
+                            *reinterpret_cast<uint4*>(p_buf + (size_t)(g0 + j) * 2048 + (size_t)r * 16) =
+                                make_uint4(pk[KEEP ? 0 : j][0], pk[KEEP ? 0 : j][1], pk[KEEP ? 0 : j][2], pk[KEEP ? 0 : j][3]);
                 }
                 // rows of the V tile past the end of the prefix / tree may hold anything: make them zero
                 if (wg == 0 && valid < kTile) {
@@ -768,6 +852,22 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             const int slot_id = 2 * cta + (t > t_begin ? 1 : 0);
             if (!mbar_wait(&sm->pv_done, glast & 1u, sm, hdr, 10)) failed = true;
             tc_fence_after();
+            if (WIDE) {
+                // Row sums came from the tensor cores, query by lane: add the last tile's and hand the sum of each of
+                // this group's queries to the threads that finish its columns.
+                const float lp = tc_ld1(tmem + lane_addr + kColL);
+                tc_wait_ld();
+                const float l = l_run + lp;
+                if (own) {
+                    if (full) {
+                        alph[r - col0] = l > 0.f ? 1.f / l : 0.f;
+                    } else {
+                        alph[r - col0] = l;            // kept for the merge below
+                        p.part_ml[((size_t)slot_id * 2 + 0) * 128 + r] = mref[r - col0];
+                        p.part_ml[((size_t)slot_id * 2 + 1) * 128 + r] = l;
+                    }
+                }
+            } else {
             // Row sums: every thread holds a partial sum per query; reduce the 8 sums of a column group across the
             // warp by recursive halving (9 shuffles instead of 40): after the three exchange steps lane L holds the
             // sum of column (L >> 2) & 7 over its exchange partners, two more steps finish the reduction.
@@ -779,8 +879,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                         const bool up = lane & 16;
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
-                            const float send = up ? acc_l[j][k] : acc_l[j][k + 4];
-                            const float keep = up ? acc_l[j][k + 4] : acc_l[j][k];
+                            const float send = up ? acc_l[KEEP ? j : 0][k] : acc_l[KEEP ? j : 0][k + 4];
+                            const float keep = up ? acc_l[KEEP ? j : 0][k + 4] : acc_l[KEEP ? j : 0][k];
                             v4[k] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
                         }
                     }
@@ -809,12 +909,13 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             if (r < ncg * 8) {
                 const float l = (sm->wred[wg][0][r] + sm->wred[wg][1][r]) + (sm->wred[wg][2][r] + sm->wred[wg][3][r]);
                 if (full) {
-                    sm->alpha[col0 + r] = l > 0.f ? 1.f / l : 0.f;
+                    alph[r] = l > 0.f ? 1.f / l : 0.f;
                 } else {
-                    sm->alpha[col0 + r] = l;                   // kept for the merge below
-                    p.part_ml[((size_t)slot_id * 2 + 0) * 128 + col0 + r] = sm->m_ref[col0 + r];
+                    alph[r] = l;                   // kept for the merge below
+                    p.part_ml[((size_t)slot_id * 2 + 0) * 128 + col0 + r] = mref[r];
                     p.part_ml[((size_t)slot_id * 2 + 1) * 128 + col0 + r] = l;
                 }
+            }
             }
             group_sync_any(bar_id, false);
             // O^T rows of this thread, up to four column groups per tensor-memory round trip
@@ -834,7 +935,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                             for (int k = 0; k < 8; ++k) {
                                 const int n = col0 + 8 * (j0 + jj) + k;
                                 if (n < s.Nq) {
-                                    if (full) p.out[((size_t)bh * p.N + s.q0 + n) * 128 + r] = __float2bfloat16_rn(o[jj][k] * sm->alpha[n]);
+                                    if (full) p.out[((size_t)bh * p.N + s.q0 + n) * 128 + r] = __float2bfloat16_rn(o[jj][k] * alph[n - col0]);
                                     else p.part_o[((size_t)slot_id * 128 + n) * 128 + r] = o[jj][k];
                                 }
                             }
@@ -883,8 +984,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                                 for (int k = 0; k < 8; ++k) {
                                     const int n = col0 + 8 * (j0 + jj) + k;
                                     const bool on = j0 + jj < ncg && n < s.Nq;
-                                    M[jj][k] = on ? sm->m_ref[n] : -INFINITY;
-                                    lsum[jj][k] = on ? sm->alpha[n] : 0.f;
+                                    M[jj][k] = on ? mref[n - col0] : -INFINITY;
+                                    lsum[jj][k] = on ? alph[n - col0] : 0.f;
                                     if (!on) o_keep[jj][k] = 0.f;
                                 }
                             for (int i = 0; i < nparts - 1; ++i) {
