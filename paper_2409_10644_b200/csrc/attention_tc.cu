@@ -173,26 +173,18 @@ __device__ __forceinline__ float tc_ld1(uint32_t taddr) {
     return v;
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-// Calls f(j, values of 8-column group j) for the first ncg of a thread's column groups, reading tensor memory
-// MCSD_SWEEP_BATCH groups per round trip (larger batches cost registers the wide kernels do not have).  ncg is
+// Calls f(j, values of 8-column group j) for the first ncg of a thread's column groups, one tensor-memory round
+// trip per group (larger batches cost registers the wide kernels do not have and measured no faster).  ncg is
 // uniform per warp.
-#ifndef MCSD_SWEEP_BATCH
-#define MCSD_SWEEP_BATCH 1
-#endif
 template <int CPT, typename F>
 __device__ __forceinline__ void sweep_groups(uint32_t taddr, int ncg, F&& f) {
-    constexpr int SB = MCSD_SWEEP_BATCH;
 #pragma unroll
-    for (int j0 = 0; j0 < CPT; j0 += SB) {
-        if (j0 < ncg) {
-            float buf[SB][8];
-#pragma unroll
-            for (int jj = 0; jj < SB; ++jj)
-                if (j0 + jj < CPT && j0 + jj < ncg) tc_ld8(taddr + 8 * (j0 + jj), buf[jj]);
+    for (int j = 0; j < CPT; ++j) {
+        if (j < ncg) {
+            float buf[8];
+            tc_ld8(taddr + 8 * j, buf);
             tc_wait_ld();
-#pragma unroll
-            for (int jj = 0; jj < SB; ++jj)
-                if (j0 + jj < CPT && j0 + jj < ncg) f(j0 + jj, buf[jj]);
+            f(j, buf);
         }
     }
 }
@@ -274,27 +266,31 @@ __device__ __forceinline__ void locate(const TcSmall* sm, const TcParams& p, lon
     s.Nq = min(kQBlock, s.Nb - s.q0);
 }
 
-// Cost of one tile in units of about 100 cycles, measured on this kernel: flat up to 32 queries, then growing with
-// the number of query columns the softmax threads and the MMAs have to cover.  Thread blocks get equal cost, not
-// equal tile counts, so that sequences with deep trees do not make their blocks finish late.
-__device__ __forceinline__ int tile_weight(int Nq) {
-    return 24 + (max(0, Nq - 32) * 9) / 32;
+// Cost of one tile in units of about 100 cycles, measured on this kernel.  Launches for up to 64 query columns:
+// flat up to 32 queries (the key/value stream sets the pace), then growing with the columns the softmax threads
+// cover.  Wide launches: nearly flat, set by the 24 tensor-core instructions per tile and the shallower ring.
+// Thread blocks get equal cost, not equal tile counts, so that sequences with deep trees do not make their blocks
+// finish late.
+__device__ __forceinline__ int tile_weight(int Nq, bool wide) {
+    return wide ? 27 + Nq / 19 : 24 + (max(0, Nq - 32) * 9) / 32;
 }
-// Fixed cost of a work item (pipeline drain, row-sum reduction, output of Nq columns), carried by its first tile.
-__device__ __forceinline__ int item_weight(int Nq) {
-    return 30 + (Nq * 5) / 8;
+// Fixed cost of a work item (pipeline fill and drain, first-tile reference search, row sums, output of Nq columns),
+// carried by its first tile.
+__device__ __forceinline__ int item_weight(int Nq, bool wide) {
+    return (wide ? 100 : 30) + (Nq * 5) / 8;
 }
-__device__ __forceinline__ int head_weight(int L, int Nb) {        // cost of one (sequence, head): all query blocks
+__device__ __forceinline__ int head_weight(int L, int Nb, bool wide) {        // cost of one (sequence, head): all query blocks
     const int tkv = kv_tiles_of(L, Nb);
     int w = 0;
-    for (int q0 = 0; q0 < Nb; q0 += kQBlock) w += tkv * tile_weight(min(kQBlock, Nb - q0)) + item_weight(min(kQBlock, Nb - q0));
+    for (int q0 = 0; q0 < Nb; q0 += kQBlock) w += tkv * tile_weight(min(kQBlock, Nb - q0), wide) + item_weight(min(kQBlock, Nb - q0), wide);
     return w;
 }
 // cumulative cost of the tiles before the one a Segment points at
 __device__ __forceinline__ long long weight_before(const TcSmall* sm, const TcParams& p, const Segment& s) {
+    const bool wide = p.npadq > 64;
     long long w = (long long)p.H * sm->cum_w[s.b] + (long long)s.h * (sm->cum_w[s.b + 1] - sm->cum_w[s.b]);
-    if (s.qb) w += (long long)s.Tkv * tile_weight(kQBlock) + item_weight(kQBlock);
-    return w + (long long)s.lt * tile_weight(s.Nq) + (s.lt > 0 ? item_weight(s.Nq) : 0);
+    if (s.qb) w += (long long)s.Tkv * tile_weight(kQBlock, wide) + item_weight(kQBlock, wide);
+    return w + (long long)s.lt * tile_weight(s.Nq, wide) + (s.lt > 0 ? item_weight(s.Nq, wide) : 0);
 }
 // Tile t belongs to block floor(weight_before(t) * G / total_w).  First tile of block c: the first tile whose
 // cumulative cost reaches ceil(c * total_w / G).
@@ -316,11 +312,12 @@ __device__ __forceinline__ long long first_tile_of_block(const TcSmall* sm, cons
     int r2 = (int)(rem % wh);
     long long t = (long long)p.H * sm->cum_tiles[lo] + (long long)h * tb;
     // inside a work item the tiles start at cost 0, f + w, f + 2w, ... (f = fixed cost on the first tile)
-    const int w0 = tile_weight(min(kQBlock, Nb)), f0 = item_weight(min(kQBlock, Nb));
+    const bool wide = p.npadq > 64;
+    const int w0 = tile_weight(min(kQBlock, Nb), wide), f0 = item_weight(min(kQBlock, Nb), wide);
     if (r2 >= tkv * w0 + f0 && Nb > kQBlock) {         // inside the second query block
         r2 -= tkv * w0 + f0;
         t += tkv;
-        const int w1 = tile_weight(Nb - kQBlock), f1 = item_weight(Nb - kQBlock);
+        const int w1 = tile_weight(Nb - kQBlock, wide), f1 = item_weight(Nb - kQBlock, wide);
         return r2 == 0 ? t : t + max(1, (r2 - f1 + w1 - 1) / w1);
     }
     return r2 == 0 ? t : t + max(1, (r2 - f0 + w0 - 1) / w0);
@@ -358,7 +355,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         const int L = min(max(p.seq_lens[b], 0), p.L_max);
         const int Nb = p.n_active ? min(max(p.n_active[b], 0), p.N) : p.N;
         sm->cum_tiles[b + 1] = (unsigned short)tiles_of(L, Nb);
-        sm->cum_w[b + 1] = head_weight(L, Nb);
+        sm->cum_w[b + 1] = head_weight(L, Nb, NCH > 4);
     }
     if (tid == 0) {
         for (int i = 0; i < kMaxSlots; ++i) { mbar_init(&sm->slot_full[i], 1); mbar_init(&sm->slot_empty[i], 1); }
@@ -385,7 +382,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         // No block's share of the cost may be smaller than the heaviest tile, so that consecutive tiles never skip
         // a block: every working block then owns at least one tile and the blocks sharing a work item are consecutive.
         const long long tot_w = (long long)p.H * accw;
-        const int nb = (int)max(1LL, min((long long)gridDim.x, tot_w / (tile_weight(kQBlock) + item_weight(kQBlock))));
+        const int nb = (int)max(1LL, min((long long)gridDim.x, tot_w / (tile_weight(kQBlock, NCH > 4) + item_weight(kQBlock, NCH > 4))));
         sm->n_blocks = nb;
     }
     __syncthreads();
@@ -585,23 +582,28 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         float* const alph = sm->alpha + 64 * wg;
         // dmask[t] = set of queries that may see tree key t: the ancestor bitsets transposed.  The bitsets are
         // first copied to shared memory in one coalesced round trip (the P^T buffer is free until the first tile
-        // is finished), then every thread transposes one key's column out of shared memory.
+        // is finished), then the warps transpose them key by key.
         {
             unsigned long long* anc_s = reinterpret_cast<unsigned long long*>(p_buf);
             const int n_words = p.N * p.words;                   // at most 192 * 3 words = 4.5 KB
             for (int i = tid; i < n_words; i += 256) anc_s[i] = p.anc[i];
             asm volatile("bar.sync 3, 256;" ::: "memory");
-            if (tid < MCSD_MAX_NODES) {
-                unsigned long long w0 = 0, w1 = 0, w2 = 0;
-                if (tid < p.N) {
-                    for (int n = 0; n < p.N; ++n) {
-                        const unsigned long long bit = (anc_s[n * p.words + (tid >> 6)] >> (tid & 63)) & 1ull;
-                        if (n < 64) w0 |= bit << n; else if (n < 128) w1 |= bit << (n - 64); else w2 |= bit << (n - 128);
-                    }
+            // Transposition, one 32-query piece of one key's row per thread and step (consecutive threads take
+            // consecutive keys, so a warp reads the same word of 32 bitsets in turn: broadcasts, no bank conflicts).
+            // Rows for keys beyond the tree are never read.
+            const int n_chunks = (p.N + 31) >> 5;
+            const uint32_t* anc32 = reinterpret_cast<const uint32_t*>(anc_s);
+            for (int idx = tid; idx < p.N * 6; idx += 32 * 4 * kSoftmaxGroups) {
+                const int c = idx / p.N, t = idx - c * p.N;
+                uint32_t piece = 0;
+                if (c < n_chunks) {
+                    const uint32_t* col = anc32 + (t >> 5);          // 32-bit half of the 64-bit word that holds bit t
+                    const int n_end = min(32, p.N - 32 * c);
+#pragma unroll 8
+                    for (int i = 0; i < n_end; ++i)
+                        piece |= ((col[(size_t)(32 * c + i) * p.words * 2] >> (t & 31)) & 1u) << i;
                 }
-                sm->dmask[tid][0] = w0;
-                sm->dmask[tid][1] = w1;
-                sm->dmask[tid][2] = w2;
+                reinterpret_cast<uint32_t*>(&sm->dmask[t][0])[c] = piece;
             }
             // both groups read dmask and will overwrite the staging copy: order both before any tile is processed
             asm volatile("bar.sync 3, 256;" ::: "memory");
