@@ -16,6 +16,8 @@ What each function follows:
   to the whole prefix plus the tree tokens its mask row allows.  The method
   reaches exactly softmax(scale * q k^T) v over that key set, so the oracle is
   that definition written out.
+* ``sample_without_replacement``, ``sample_roots`` -- Section 3.1: several new
+  tokens, not one, are sampled from the target side to start the next tree.
 * ``softmax_temperature``, ``verify_tree_logits``, ``verify_tree_greedy`` --
   Fig. 1 step 4 (next-token logits become distributions) at the two sampling
   temperatures of Section 4.1: 0.7 (probabilistic) and 0 (greedy).
@@ -320,6 +322,58 @@ def decision_margins(p, q, tokens, parent, gamma, u_accept, u_bonus):
             lo = cs[t - 1] if t > 0 else -np.inf
             m_bon[b, u] = min(target - lo, cs[t] - target) / z
     return m_acc, m_bon
+
+
+# ----------------------------------------------------------------------------
+# several new tokens from the target side (Section 3.1)
+# ----------------------------------------------------------------------------
+
+def sample_without_replacement(dist, uniforms):
+    """R distinct token ids drawn one after the other from an unnormalised distribution.
+
+    Section 3.1 samples several tokens, not one, from the target's distribution to start the next candidate
+    tree.  Reading taken here (the paper does not say how): the tokens are distinct; draw i is an inverse-CDF draw
+    in token-id order (uniform uniforms[i]) from the distribution restricted to the ids not drawn yet, which is the
+    usual sequential sampling without replacement.  When no mass is left the remaining entries are -1.
+    """
+    rest = np.array(dist, dtype=np.float64, copy=True)
+    out = np.full(len(uniforms), -1, dtype=np.int32)
+    for i, u in enumerate(uniforms):
+        if not rest.sum() > 0.0:
+            break
+        t = inverse_cdf(rest, float(u))
+        out[i] = t
+        rest[t] = 0.0
+    return out
+
+
+def stop_distribution(p, q, tokens, parent, gamma_b, u_accept, b, verify_out):
+    """Unnormalised distribution the new token of sequence b is drawn from: the target row of the stop node of the
+    winning path, residualised once per candidate rejected there (Fig. 1 steps 4-6)."""
+    parent = np.asarray(parent, dtype=np.int64)
+    depth, level_start = tree_levels(parent)
+    n_levels = len(level_start) - 1
+    g = n_levels - 1 if gamma_b is None else int(gamma_b)
+    ln = int(verify_out["accept_len"][b])
+    stop = int(verify_out["out_nodes"][b, ln - 1]) if ln > 0 else int(verify_out["best_root"][b])
+    kids = _children(parent, stop)
+    dist = np.asarray(p[b, stop], dtype=np.float64)
+    if depth[stop] < g and kids:
+        idx, res = node_decision(p[b, stop], q[b, stop], [tokens[b, c] for c in kids], [u_accept[b, c] for c in kids])
+        assert idx is None, "the winning path stops where every candidate was rejected"
+        dist = res
+    return stop, dist
+
+
+def sample_roots(p, q, tokens, parent, gamma, u_accept, verify_out, u_roots):
+    """next_roots[b][:] = R distinct ids drawn from the stop distribution of every sequence (see above)."""
+    B = p.shape[0]
+    R = u_roots.shape[1]
+    out = np.full((B, R), -1, dtype=np.int32)
+    for b in range(B):
+        _, dist = stop_distribution(p, q, tokens, parent, None if gamma is None else gamma[b], u_accept, b, verify_out)
+        out[b] = sample_without_replacement(dist, u_roots[b])
+    return out
 
 
 # ----------------------------------------------------------------------------

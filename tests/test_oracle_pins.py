@@ -687,3 +687,79 @@ def test_greedy_is_the_low_temperature_limit_and_honours_gamma_and_ties():
     assert r["accept_len"][0] == 1 and r["out_nodes"][0, 0] == 2
     assert list(r["out_tokens"][0]) == [1, 0, -1] and list(r["next_roots"][0]) == [0, 1, 2]
     assert orc.argmax_lowest([3.0, 7.0, 7.0]) == 1
+
+
+# ----------------------------------------------------------------------------
+# several target-side tokens for the next tree (Section 3.1)
+# ----------------------------------------------------------------------------
+
+def test_sampling_without_replacement_follows_the_sequential_law():
+    """Pairs (t1, t2) drawn with a fine grid of uniforms occur with frequency P(t1) * P(t2) / (1 - P(t1)), the law of
+    sequential sampling without replacement, written out here independently of the oracle's own routine."""
+    dist = np.array([0.5, 0.0, 1.5, 1.0, 2.0])            # unnormalised, one id without mass
+    P = dist / dist.sum()
+    G = 240
+    grid = (np.arange(G) + 0.5) / G
+    counts = np.zeros((5, 5))
+    for u1 in grid:
+        for u2 in grid:
+            t = orc.sample_without_replacement(dist, [u1, u2])
+            assert t[0] != t[1]
+            counts[t[0], t[1]] += 1
+    freq = counts / G ** 2
+    want = np.zeros((5, 5))
+    for a in range(5):
+        for b in range(5):
+            if a != b and P[a] > 0 and P[b] > 0:
+                want[a, b] = P[a] * P[b] / (1.0 - P[a])
+    assert np.abs(freq - want).max() < 2.5 / G
+    assert counts[1].sum() == 0 and counts[:, 1].sum() == 0
+
+
+def test_sampling_without_replacement_special_cases():
+    dist = np.array([0.2, 0.3, 0.5])
+    # all ids drawn: a permutation; with more draws than ids with mass, the rest is -1
+    t = orc.sample_without_replacement(dist, [0.9, 0.1, 0.5, 0.5])
+    assert sorted(t[:3]) == [0, 1, 2] and t[3] == -1
+    assert list(t[:3]) == [2, 0, 1]                        # 0.9 -> id 2; then {0.2, 0.3}: 0.1 -> id 0; then id 1
+    # in token-id order with a strict comparison: a uniform exactly on a CDF edge takes the next id
+    assert orc.sample_without_replacement(np.array([1.0, 1.0]), [0.5])[0] == 1
+    # point mass
+    assert list(orc.sample_without_replacement(np.array([0.0, 3.0, 0.0]), [0.7, 0.7])) == [1, -1]
+
+
+def test_sample_roots_draws_from_the_residual_of_the_stop_node():
+    rng = np.random.default_rng(31)
+    V = 6
+    parent = parent_array(1, (2, 1))
+    N = len(parent)
+    p = _rand_dist(rng, 2, N, V)
+    q = _rand_dist(rng, 2, N, V)
+    tokens = rng.integers(0, V, (2, N))
+    ua = np.ones((2, N))                                    # reject everything: stop at the root after two rejections
+    ub = np.full((2, N), 0.5)
+    v = orc.verify_tree(p, q, tokens, parent, None, ua, ub)
+    assert list(v["accept_len"]) == [0, 0]
+    ur = rng.uniform(0.05, 0.95, (2, 3))
+    roots = orc.sample_roots(p, q, tokens, parent, None, ua, v, ur)
+    for b in range(2):
+        r1 = np.maximum(p[b, 0] - q[b, 0], 0.0); r1 /= r1.sum()          # residual after the first rejection
+        r2 = np.maximum(r1 - q[b, 0], 0.0)                                # and after the second
+        if r2.sum() > 0:
+            r2 /= r2.sum()
+        else:
+            r2 = p[b, 0]
+        stop, dist = orc.stop_distribution(p, q, tokens, parent, None, ua, b, v)
+        assert stop == 0
+        np.testing.assert_allclose(dist / dist.sum(), r2 / r2.sum(), atol=1e-12)
+        n_pos = int((r2 > 0).sum())
+        got = [int(t) for t in roots[b] if t >= 0]
+        assert len(got) == min(3, n_pos) and len(set(got)) == len(got) and all(r2[t] > 0 for t in got)
+        assert all(t == -1 for t in roots[b][len(got):])
+    # an accepted path: the distribution is the target row of the deepest accepted node
+    ua0 = np.zeros((2, N))
+    v2 = orc.verify_tree(p, q, tokens, parent, None, ua0, ub)
+    for b in range(2):
+        stop, dist = orc.stop_distribution(p, q, tokens, parent, None, ua0, b, v2)
+        assert stop == int(v2["out_nodes"][b, v2["accept_len"][b] - 1])
+        np.testing.assert_allclose(dist, p[b, stop], atol=0)
