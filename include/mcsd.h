@@ -203,6 +203,35 @@ int mcsd_verify_tree_logits(const void* target_logits, const void* draft_logits,
                             void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Several new tokens for a target-initialised tree (Section 3.1: instead of one token, several are sampled from the
+ * target side and become the roots of the next candidate tree).  To be called after mcsd_verify_tree (or
+ * mcsd_verify_tree_logits with temperature > 0) on the same rows, results and workspace: for every sequence it draws
+ * R distinct ids from the distribution the winning path stopped with -- the target row of the stop node, residualised
+ * once per candidate rejected there -- one after the other: draw i is an inverse-CDF draw in token-id order with
+ * uniform u_roots[b][i] over the ids not drawn before.  (The paper does not say how the tokens are drawn; distinct
+ * tokens by sequential sampling without replacement is the reading taken here.  next_roots of mcsd_verify_tree
+ * lists the most probable ids instead.)
+ *
+ *   p, q / target_logits, draft_logits, dtype, temperature   the rows given to the verify call
+ *   accept_len, out_nodes, best_root   [dev] its results (out_nodes is [B][n_levels])
+ *   u_roots        [dev] float[B][R] uniforms
+ *   next_roots     [dev] int32[B][R] out; -1 where fewer than R ids carry mass
+ *   workspace      [dev] the workspace the verify call used (read only here)
+ *
+ * One launch on `stream`.  Errors: MCSD_ERR_NULL, MCSD_ERR_BAD_SHAPE (sizes as for mcsd_verify_tree, R < 1 or R > 32,
+ * temperature outside [1e-3, 1e6]), MCSD_ERR_BAD_DTYPE, MCSD_ERR_WORKSPACE_TOO_SMALL, MCSD_ERR_CUDA.
+ */
+int mcsd_sample_roots(const float* p, const float* q,
+                      const int32_t* accept_len, const int32_t* out_nodes, const int32_t* best_root, int n_levels,
+                      const float* u_roots, int B, int N, int V, int R, int32_t* next_roots,
+                      const void* workspace, size_t workspace_bytes, void* stream);
+
+int mcsd_sample_roots_logits(const void* target_logits, const void* draft_logits, int dtype, float temperature,
+                             const int32_t* accept_len, const int32_t* out_nodes, const int32_t* best_root, int n_levels,
+                             const float* u_roots, int B, int N, int V, int R, int32_t* next_roots,
+                             const void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * KV-cache update after acceptance (Fig. 1 step 6): "update the input IDs, key-value cache".  For every layer and
  * sequence b the keys/values of the winning root (node best_root[b]; with a single root that is node 0, the last
  * emitted token, which is not in the prefix cache yet) and of the accepted nodes out_nodes[b][0 .. accept_len[b]-1]

@@ -24,7 +24,8 @@ MCSD_MAX_WORDS = 3
 
 _EXPORTS = (
     "mcsd_status_string", "mcsd_last_cuda_error", "mcsd_launch_count", "mcsd_build_mask", "mcsd_tree_attention_workspace_bytes",
-    "mcsd_tree_attention", "mcsd_workspace_status", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_logits", "mcsd_verify_tree_static", "mcsd_commit_kv",
+    "mcsd_tree_attention", "mcsd_workspace_status", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_logits", "mcsd_verify_tree_static", "mcsd_commit_kv", "mcsd_sample_roots",
+    "mcsd_sample_roots_logits",
 )
 
 
@@ -59,6 +60,11 @@ def _load() -> ctypes.CDLL:
     lib.mcsd_verify_tree_logits.argtypes = ([c_void_p, c_void_p, c_int, c_float] + [c_void_p] * 3 + [c_int, c_int] +
                                             [c_void_p] * 3 + [c_int] * 3 + [c_void_p] * 5 +
                                             [c_int, c_void_p, c_size_t, c_void_p])
+    lib.mcsd_sample_roots.restype = c_int
+    lib.mcsd_sample_roots.argtypes = [c_void_p] * 5 + [c_int, c_void_p] + [c_int] * 4 + [c_void_p, c_void_p, c_size_t, c_void_p]
+    lib.mcsd_sample_roots_logits.restype = c_int
+    lib.mcsd_sample_roots_logits.argtypes = ([c_void_p, c_void_p, c_int, c_float] + [c_void_p] * 3 + [c_int, c_void_p] +
+                                             [c_int] * 4 + [c_void_p, c_void_p, c_size_t, c_void_p])
     lib.mcsd_verify_tree_static.restype = c_int
     lib.mcsd_verify_tree_static.argtypes = ([c_void_p] * 5 + [c_int, c_int] + [c_void_p] * 3 + [c_int] * 3 +
                                             [c_void_p] * 5 + [c_int, c_void_p])
@@ -286,6 +292,33 @@ def mcsd_verify_tree_logits(target_logits, draft_logits, temperature: float, tok
                                          _ptr(out["out_tokens"]), _ptr(out["out_nodes"]), _ptr(out["best_root"]),
                                          _ptr(out.get("next_roots")), R, _ptr(workspace), workspace.numel(), _stream())
     _check(st, "mcsd_verify_tree_logits")
+    return out
+
+
+def mcsd_sample_roots(p, q, verify_out: dict, mask: TreeMask, u_roots, workspace: torch.Tensor,
+                      temperature: Optional[float] = None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """R distinct new tokens per sequence from the distribution the winning path stopped with (see mcsd.h).
+
+    `p`, `q` are the probability rows given to mcsd_verify_tree, or -- with `temperature` -- the target and draft
+    logits given to mcsd_verify_tree_logits; `verify_out` and `workspace` are that call's results and workspace."""
+    B, N, V = p.shape
+    _dev_tensor(u_roots, torch.float32, "u_roots")
+    R = int(u_roots.shape[1])
+    if out is None:
+        out = torch.empty((B, R), dtype=torch.int32, device=p.device)
+    args = (_ptr(verify_out["accept_len"]), _ptr(verify_out["out_nodes"]), _ptr(verify_out["best_root"]), mask.n_levels,
+            _ptr(u_roots), B, N, V, R, _ptr(out), _ptr(workspace), workspace.numel(), _stream())
+    with torch.cuda.device(p.device):
+        if temperature is None:
+            _dev_tensor(p, torch.float32, "p")
+            _dev_tensor(q, torch.float32, "q")
+            st = lib.mcsd_sample_roots(_ptr(p), _ptr(q), *args)
+        else:
+            code = MCSD_BF16 if p.dtype == torch.bfloat16 else MCSD_F32
+            _dev_tensor(p, p.dtype, "target_logits")
+            _dev_tensor(q, p.dtype, "draft_logits")
+            st = lib.mcsd_sample_roots_logits(_ptr(p), _ptr(q), code, float(temperature), *args)
+    _check(st, "mcsd_sample_roots")
     return out
 
 

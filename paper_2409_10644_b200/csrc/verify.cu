@@ -37,6 +37,24 @@ extern "C" int mcsd_verify_tree(const float* p, const float* q, const int32_t* t
     return MCSD_OK;
 }
 
+extern "C" int mcsd_sample_roots(const float* p, const float* q, const int32_t* accept_len, const int32_t* out_nodes,
+                                 const int32_t* best_root, int n_levels, const float* u_roots, int B, int N, int V,
+                                 int R, int32_t* next_roots, const void* workspace, size_t workspace_bytes,
+                                 void* stream) {
+    if (!p || !q || !accept_len || !out_nodes || !best_root || !u_roots || !next_roots || !workspace) return MCSD_ERR_NULL;
+    if (B < 1 || N < 1 || V < 1 || N > MCSD_MAX_NODES || B > 65535) return MCSD_ERR_BAD_SHAPE;
+    if (n_levels < 1 || n_levels > N || R < 1 || R > 32) return MCSD_ERR_BAD_SHAPE;
+    if (workspace_bytes < mcsd_verify_tree_workspace_bytes(B, N, V)) return MCSD_ERR_WORKSPACE_TOO_SMALL;
+    const auto* state = reinterpret_cast<const mcsd::NodeState*>(static_cast<const char*>(workspace) +
+                                                                sizeof(mcsd::WorkspaceHeader));
+    const mcsd::ProbRows rows{p, q};
+    mcsd::sample_roots_kernel<mcsd::ProbRows><<<B, mcsd::kVerifyThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+        rows, state, accept_len, out_nodes, best_root, n_levels, u_roots, N, V, R, next_roots);
+    MCSD_CUDA_CHECK(cudaGetLastError());
+    mcsd::count_launches(1);
+    return MCSD_OK;
+}
+
 // ------------------------------------------------------------------------------------------------------
 // Variant with built-in scratch, for callers that cannot allocate device memory.
 // ------------------------------------------------------------------------------------------------------

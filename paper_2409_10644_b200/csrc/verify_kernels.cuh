@@ -439,41 +439,30 @@ __device__ void top_ids(const Load& load, int V, int R, int32_t* __restrict__ ds
     }
 }
 
-template <typename Rows>
-__global__ void __launch_bounds__(kVerifyThreads)
-verify_select_kernel(Rows rows, const int32_t* __restrict__ tokens, const NodeState* __restrict__ state,
-                     int n_levels, int n_roots, const float* __restrict__ u_bonus, int N, int V,
-                     int32_t* __restrict__ accept_len, int32_t* __restrict__ out_tokens,
-                     int32_t* __restrict__ out_nodes, int32_t* __restrict__ best_root,
-                     int32_t* __restrict__ next_roots, int R) {
-    using Dist = typename Rows::Dist;
-    constexpr int E = Dist::E;
+// Inverse CDF in token-id order over the unnormalised distribution `load` hands out E ids at a time: the smallest
+// id t whose running sum exceeds u * total; if rounding lets nothing exceed it, the last id with mass (V - 1 if
+// there is none).  Every thread of the block must call it; all get the id, and *total_out the total mass.
+// pass 1: every warp sums one contiguous range of ids; pass 2: one warp locates the crossing, starting in the
+// range where the running sum passes u * total.
+struct CdfScratch {
+    double tot[kVerifyWarps];
+    int last[kVerifyWarps];
+    int found;
+    double total;
+};
+template <int E, typename Load>
+__device__ int block_inverse_cdf(const Load& load, float u, int V, CdfScratch* sc, double* total_out) {
     constexpr int kStride = 32 * E;             // ids one warp covers per step
-    __shared__ int s_len[MCSD_MAX_NODES];
-    __shared__ int s_stop, s_slot;
-    __shared__ VerifyScratch s_scratch;
-    __shared__ double s_tot[kVerifyWarps];
-    __shared__ int s_last[kVerifyWarps];
-    __shared__ float s_bv[kVerifyWarps];
-    __shared__ int s_bi[kVerifyWarps];
-    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const NodeState* st = state + (size_t)b * N;
-
-    select_path(st, tokens, b, n_levels, n_roots, N, accept_len, out_tokens, out_nodes, best_root, s_len, &s_stop, &s_slot);
-    const int u = s_stop;
-    Dist d = rows.open(b, u, N, V, &s_scratch);
-    d.set_c(st[u].c);
-
-    // ---- new token: inverse CDF over dist_v = max(p_v - c q_v, 0) in token-id order ----
-    // pass 1: every warp sums one contiguous range of ids
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int span = ((V + kVerifyWarps - 1) / kVerifyWarps + kStride - 1) / kStride * kStride;
+    __syncthreads();                            // the scratch may still be read from a previous call
     {
         const int lo = warp * span, hi = min(V, lo + span);
         float acc = 0.f;
         int last = -1;
         for (int idx = lo + lane * E; idx < hi; idx += kStride) {
             float r[E];
-            d.load(idx, r);
+            load(idx, r);
             acc += tree_sum<E>(r);
 #pragma unroll
             for (int i = 0; i < E; ++i)
@@ -482,18 +471,17 @@ verify_select_kernel(Rows rows, const int32_t* __restrict__ tokens, const NodeSt
         acc = warp_sum(acc);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
-        if (lane == 0) { s_tot[warp] = (double)acc; s_last[warp] = last; }
+        if (lane == 0) { sc->tot[warp] = (double)acc; sc->last[warp] = last; }
     }
     __syncthreads();
-    // pass 2: one warp locates the crossing, starting in the range where the running sum passes u * Z
     if (warp == 0) {
         double total = 0.0;
         int last_pos = -1;
-        for (int w = 0; w < kVerifyWarps; ++w) { total += s_tot[w]; last_pos = max(last_pos, s_last[w]); }
-        const double target = (double)u_bonus[(size_t)b * N + u] * total;
+        for (int w = 0; w < kVerifyWarps; ++w) { total += sc->tot[w]; last_pos = max(last_pos, sc->last[w]); }
+        const double target = (double)u * total;
         double base = 0.0;
         int w0 = 0;
-        while (w0 < kVerifyWarps && !(base + s_tot[w0] > target)) { base += s_tot[w0]; ++w0; }
+        while (w0 < kVerifyWarps && !(base + sc->tot[w0] > target)) { base += sc->tot[w0]; ++w0; }
         int found = -1;
         for (int w = w0; w < kVerifyWarps && found < 0; ++w) {
             const int lo = w * span, hi = min(V, lo + span);
@@ -502,7 +490,7 @@ verify_select_kernel(Rows rows, const int32_t* __restrict__ tokens, const NodeSt
                 float r[E];
 #pragma unroll
                 for (int i = 0; i < E; ++i) r[i] = 0.f;
-                if (idx < hi) d.load(idx, r);
+                if (idx < hi) load(idx, r);
                 const float ls = tree_sum<E>(r);
                 float incl = ls;
 #pragma unroll
@@ -534,13 +522,85 @@ verify_select_kernel(Rows rows, const int32_t* __restrict__ tokens, const NodeSt
             }
         }
         if (found < 0) found = last_pos >= 0 ? last_pos : V - 1;
-        if (lane == 0) out_tokens[(size_t)b * (n_levels + 1) + s_slot] = found;
+        if (lane == 0) { sc->found = found; sc->total = total; }
     }
+    __syncthreads();
+    *total_out = sc->total;
+    return sc->found;
+}
+
+template <typename Rows>
+__global__ void __launch_bounds__(kVerifyThreads)
+verify_select_kernel(Rows rows, const int32_t* __restrict__ tokens, const NodeState* __restrict__ state,
+                     int n_levels, int n_roots, const float* __restrict__ u_bonus, int N, int V,
+                     int32_t* __restrict__ accept_len, int32_t* __restrict__ out_tokens,
+                     int32_t* __restrict__ out_nodes, int32_t* __restrict__ best_root,
+                     int32_t* __restrict__ next_roots, int R) {
+    using Dist = typename Rows::Dist;
+    constexpr int E = Dist::E;
+    __shared__ int s_len[MCSD_MAX_NODES];
+    __shared__ int s_stop, s_slot;
+    __shared__ VerifyScratch s_scratch;
+    __shared__ CdfScratch s_cdf;
+    __shared__ float s_bv[kVerifyWarps];
+    __shared__ int s_bi[kVerifyWarps];
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const NodeState* st = state + (size_t)b * N;
+
+    select_path(st, tokens, b, n_levels, n_roots, N, accept_len, out_tokens, out_nodes, best_root, s_len, &s_stop, &s_slot);
+    const int u = s_stop;
+    Dist d = rows.open(b, u, N, V, &s_scratch);
+    d.set_c(st[u].c);
+
+    // ---- new token: inverse CDF over dist_v = max(p_v - c q_v, 0) in token-id order ----
+    auto load = [&d](int idx, float (&r)[E]) { d.load(idx, r); };
+    double total;
+    const int found = block_inverse_cdf<E>(load, u_bonus[(size_t)b * N + u], V, &s_cdf, &total);
+    if (tid == 0) out_tokens[(size_t)b * (n_levels + 1) + s_slot] = found;
 
     // ---- optional: the R most probable ids of the same distribution ----
-    if (next_roots != nullptr && R > 0) {
-        auto load = [&d](int idx, float (&r)[E]) { d.load(idx, r); };
-        top_ids<E>(load, V, R, next_roots + (size_t)b * R, s_bv, s_bi);
+    if (next_roots != nullptr && R > 0) top_ids<E>(load, V, R, next_roots + (size_t)b * R, s_bv, s_bi);
+}
+
+// Several distinct new tokens from the distribution the winning path stopped with (Section 3.1 samples more than
+// one token from the target side to start the next candidate tree): one thread block per sequence, draw i by
+// inverse CDF with uniform u_roots[b][i] over the ids not drawn before.  Runs after the two verify kernels on the
+// same workspace, from which it takes the stop node's residual coefficient.
+template <typename Rows>
+__global__ void __launch_bounds__(kVerifyThreads)
+sample_roots_kernel(Rows rows, const NodeState* __restrict__ state, const int32_t* __restrict__ accept_len,
+                    const int32_t* __restrict__ out_nodes, const int32_t* __restrict__ best_root, int n_levels,
+                    const float* __restrict__ u_roots, int N, int V, int R, int32_t* __restrict__ next_roots) {
+    using Dist = typename Rows::Dist;
+    constexpr int E = Dist::E;
+    __shared__ VerifyScratch s_scratch;
+    __shared__ CdfScratch s_cdf;
+    __shared__ int s_pick[32];
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int ln = min(max(accept_len[b], 0), n_levels);
+    int u = ln > 0 ? out_nodes[(size_t)b * n_levels + ln - 1] : best_root[b];
+    u = min(max(u, 0), N - 1);
+    Dist d = rows.open(b, u, N, V, &s_scratch);
+    d.set_c(state[(size_t)b * N + u].c);
+    for (int i = 0; i < R; ++i) {
+        const int* picks = s_pick;
+        auto load = [&d, i, picks](int idx, float (&r)[E]) {
+            d.load(idx, r);
+            for (int j = 0; j < i; ++j) {                    // ids already drawn carry no mass any more
+                const int e = picks[j] - idx;
+#pragma unroll
+                for (int k = 0; k < E; ++k)
+                    if (e == k) r[k] = 0.f;
+            }
+        };
+        double total;
+        int tok = block_inverse_cdf<E>(load, u_roots[(size_t)b * R + i], V, &s_cdf, &total);
+        if (!(total > 0.0)) {                                 // nothing left: the rest of the list is empty
+            for (int j = i + tid; j < R; j += kVerifyThreads) next_roots[(size_t)b * R + j] = -1;
+            break;
+        }
+        if (tid == 0) { s_pick[i] = tok; next_roots[(size_t)b * R + i] = tok; }
+        __syncthreads();
     }
 }
 

@@ -146,3 +146,35 @@ extern "C" int mcsd_verify_tree_logits(const void* target_logits, const void* dr
                                               n_levels, n_roots, gamma, u_accept, u_bonus, B, N, V, accept_len, out_tokens,
                                               out_nodes, best_root, roots, R, state, s);
 }
+
+extern "C" int mcsd_sample_roots_logits(const void* target_logits, const void* draft_logits, int dtype, float temperature,
+                                        const int32_t* accept_len, const int32_t* out_nodes, const int32_t* best_root,
+                                        int n_levels, const float* u_roots, int B, int N, int V, int R,
+                                        int32_t* next_roots, const void* workspace, size_t workspace_bytes,
+                                        void* stream) {
+    if (!target_logits || !draft_logits || !accept_len || !out_nodes || !best_root || !u_roots || !next_roots ||
+        !workspace)
+        return MCSD_ERR_NULL;
+    if (!(temperature >= 1e-3f) || !(temperature <= 1e6f)) return MCSD_ERR_BAD_SHAPE;      // also rejects NaN and 0
+    if (dtype != MCSD_BF16 && dtype != MCSD_F32) return MCSD_ERR_BAD_DTYPE;
+    if (B < 1 || N < 1 || V < 1 || N > MCSD_MAX_NODES || B > 65535) return MCSD_ERR_BAD_SHAPE;
+    if (n_levels < 1 || n_levels > N || R < 1 || R > 32) return MCSD_ERR_BAD_SHAPE;
+    if (workspace_bytes < mcsd_verify_tree_workspace_bytes(B, N, V)) return MCSD_ERR_WORKSPACE_TOO_SMALL;
+    const auto* state = reinterpret_cast<const mcsd::NodeState*>(static_cast<const char*>(workspace) +
+                                                                sizeof(mcsd::WorkspaceHeader));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const float k = 1.4426950408889634f / temperature;
+    if (dtype == MCSD_F32) {
+        const mcsd::LogitRows<float> rows{static_cast<const float*>(target_logits), static_cast<const float*>(draft_logits), k};
+        mcsd::sample_roots_kernel<mcsd::LogitRows<float>><<<B, mcsd::kVerifyThreads, 0, s>>>(
+            rows, state, accept_len, out_nodes, best_root, n_levels, u_roots, N, V, R, next_roots);
+    } else {
+        const mcsd::LogitRows<__nv_bfloat16> rows{static_cast<const __nv_bfloat16*>(target_logits),
+                                                  static_cast<const __nv_bfloat16*>(draft_logits), k};
+        mcsd::sample_roots_kernel<mcsd::LogitRows<__nv_bfloat16>><<<B, mcsd::kVerifyThreads, 0, s>>>(
+            rows, state, accept_len, out_nodes, best_root, n_levels, u_roots, N, V, R, next_roots);
+    }
+    MCSD_CUDA_CHECK(cudaGetLastError());
+    mcsd::count_launches(1);
+    return MCSD_OK;
+}

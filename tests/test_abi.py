@@ -114,6 +114,28 @@ def test_verify_logits_argument_checks(m):
     assert call(T=0.0, zd=None, ua=None, wsb=8) == -5    # greedy passes the pointer checks without draft and uniforms
 
 
+def test_sample_roots_argument_checks(m):
+    L = m.lib
+
+    def call(p=FAKE, B=2, N=15, V=100, nl=4, R=2, wsb=1 << 20, u=FAKE):
+        return L.mcsd_sample_roots(p, FAKE, FAKE, FAKE, FAKE, nl, u, B, N, V, R, FAKE, FAKE, wsb, None)
+    assert call(p=None) == -1
+    assert call(u=None) == -1
+    assert call(R=0) == -2
+    assert call(R=33) == -2
+    assert call(N=193) == -2
+    assert call(nl=0) == -2
+    assert call(wsb=8) == -5
+
+    def call_l(T=0.7, dtype=1, zd=FAKE):
+        return L.mcsd_sample_roots_logits(FAKE, zd, dtype, ctypes.c_float(T), FAKE, FAKE, FAKE, 4, FAKE, 2, 15, 100, 2,
+                                          FAKE, FAKE, 8, None)
+    assert call_l() == -5
+    assert call_l(T=0.0) == -2                  # greedy verification has nothing to sample
+    assert call_l(dtype=7) == -4
+    assert call_l(zd=None) == -1
+
+
 def test_commit_kv_argument_checks(m):
     L = m.lib
 

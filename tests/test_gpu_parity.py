@@ -446,6 +446,100 @@ def test_verify_paper_shaped_workloads(m):
         torch.cuda.empty_cache()
 
 
+def _roots_margin_ok(dist, picks, us, margin=2e-5):
+    """True if every draw's uniform keeps `margin` (relative to the remaining mass) from the CDF edges of its id.
+    The kernel forms the running sums in fp32 per lane and fp64 across warps (relative error around 1e-6); after the
+    heaviest ids have been drawn the remaining ones are too light for the 1e-4 used elsewhere."""
+    rest = np.array(dist, dtype=np.float64, copy=True)
+    for t, u in zip(picks, us):
+        if t < 0:
+            break
+        cs = np.cumsum(rest)
+        z = cs[-1]
+        lo = cs[t - 1] if t > 0 else -np.inf
+        if min(u * z - lo, cs[t] - u * z) / z < margin:
+            return False
+        rest[t] = 0.0
+    return True
+
+
+@pytest.mark.parametrize("idx,R", [(1, 4), (5, 8), (7, 3)])
+def test_sample_roots_matches_oracle(m, idx, R):
+    w = workload(idx)
+    parent = parent_array(w.n_roots, w.branching)
+    B = min(w.B, 8)
+    dev = "cuda"
+    gam = None if w.gamma is None else gammas(dataclasses.replace(w, B=B))
+    tm = m.mcsd_build_mask(parent)
+    g_d = None if gam is None else torch.from_numpy(gam).to(dev)
+    rng = np.random.default_rng(50 + idx)
+    for mode in ("prob", "logits"):
+        if mode == "prob":
+            vin = verify_inputs(w, 0, dev, parent=parent, B=B)
+            host = {k: to_np(v) for k, v in vin.items()}
+            ph, qh = host["p"], host["q"]
+        else:
+            vin = verify_logit_inputs(w, 0.7, torch.bfloat16, 0, dev, parent=parent, B=B)
+            host = {k: to_np(v) for k, v in vin.items()}
+            ph = np.concatenate([orc.softmax_temperature(host["target_logits"][b:b + 1], 0.7) for b in range(B)])
+            qh = np.concatenate([orc.softmax_temperature(host["draft_logits"][b:b + 1], 0.7) for b in range(B)])
+        ua, ub = condition_uniforms(ph, qh, host["tokens"], parent, gam, host["u_accept"], host["u_bonus"])
+        ref_v = orc.verify_tree(ph, qh, host["tokens"], parent, gam, ua, ub)
+        # uniforms for the roots, redrawn (seeded) until none sits on a CDF edge the oracle evaluates
+        ur = rng.uniform(0.001, 0.999, (B, R)).astype(np.float32)
+        for b in range(B):
+            _, dist = orc.stop_distribution(ph, qh, host["tokens"], parent, None if gam is None else gam[b], ua, b, ref_v)
+            for _ in range(400):
+                picks = orc.sample_without_replacement(dist, ur[b])
+                if _roots_margin_ok(dist, picks, ur[b]):
+                    break
+                ur[b] = rng.uniform(0.001, 0.999, R).astype(np.float32)
+            else:
+                raise RuntimeError("could not move the root uniforms away from the thresholds")
+        ref = orc.sample_roots(ph, qh, host["tokens"], parent, gam, ua, ref_v, ur)
+        ws = m.new_workspace(m.mcsd_verify_tree_workspace_bytes(B, len(parent), w.V), dev)
+        ua_d, ub_d, ur_d = (torch.from_numpy(x).to(dev) for x in (ua, ub, ur))
+        if mode == "prob":
+            vout = m.mcsd_verify_tree(vin["p"], vin["q"], vin["tokens"], tm, g_d, ua_d, ub_d, workspace=ws)
+            got = m.mcsd_sample_roots(vin["p"], vin["q"], vout, tm, ur_d, ws)
+        else:
+            vout = m.mcsd_verify_tree_logits(vin["target_logits"], vin["draft_logits"], 0.7, vin["tokens"], tm, g_d, ua_d,
+                                             ub_d, workspace=ws)
+            got = m.mcsd_sample_roots(vin["target_logits"], vin["draft_logits"], vout, tm, ur_d, ws, temperature=0.7)
+        torch.cuda.synchronize()
+        assert np.array_equal(vout["accept_len"].cpu().numpy(), ref_v["accept_len"])
+        assert np.array_equal(got.cpu().numpy(), ref), mode
+        for b in range(B):
+            row = [t for t in ref[b] if t >= 0]
+            assert len(set(row)) == len(row)
+        del vin
+        torch.cuda.empty_cache()
+
+
+def test_sample_roots_runs_out_of_mass(m):
+    # a target row with mass on three ids only: the fourth and fifth root are -1
+    w = workload(1)
+    parent = np.array([-1], dtype=np.int32)
+    dev = "cuda"
+    V = 50
+    p = torch.zeros((2, 1, V), device=dev)
+    p[:, 0, 7] = 0.5
+    p[:, 0, 20] = 0.25
+    p[:, 0, 41] = 0.25
+    q = torch.full((2, 1, V), 1.0 / V, device=dev)
+    tm = m.mcsd_build_mask(parent)
+    tokens = torch.zeros((2, 1), dtype=torch.int32, device=dev)
+    half = torch.full((2, 1), 0.5, device=dev)
+    ws = m.new_workspace(m.mcsd_verify_tree_workspace_bytes(2, 1, V), dev)
+    vout = m.mcsd_verify_tree(p, q, tokens, tm, None, half, half, workspace=ws)
+    ur = torch.tensor([[0.9, 0.1, 0.5, 0.5, 0.5], [0.1, 0.9, 0.5, 0.5, 0.5]], device=dev)
+    got = m.mcsd_sample_roots(p, q, vout, tm, ur, ws).cpu().numpy()
+    ref = np.stack([orc.sample_without_replacement(to_np(p[b, 0]), to_np(ur[b])) for b in range(2)])
+    assert np.array_equal(got, ref)
+    assert list(got[0]) == [41, 7, 20, -1, -1] and list(got[1]) == [7, 41, 20, -1, -1]
+    del w
+
+
 # ----------------------------------------------------------------------------------------------
 # KV-cache update after acceptance
 # ----------------------------------------------------------------------------------------------

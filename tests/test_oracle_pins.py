@@ -698,7 +698,7 @@ def test_sampling_without_replacement_follows_the_sequential_law():
     sequential sampling without replacement, written out here independently of the oracle's own routine."""
     dist = np.array([0.5, 0.0, 1.5, 1.0, 2.0])            # unnormalised, one id without mass
     P = dist / dist.sum()
-    G = 240
+    G = 160
     grid = (np.arange(G) + 0.5) / G
     counts = np.zeros((5, 5))
     for u1 in grid:
