@@ -188,6 +188,19 @@ def test_attention_edge_cases(m):
     _full_attention_case(m, wmax, std=1.0, rel=True, n_act=None)
 
 
+def test_attention_query_split_changes_between_segments(m):
+    # Many short sequences of the 192-node tree with a different number of active nodes each: consecutive work
+    # items of a thread block then split their query columns between the two softmax groups differently, and one
+    # group may be a segment ahead of the other.  Run several times: a race would not fail every time.
+    w = dataclasses.replace(workload(2), n_roots=8, branching=(1, 2, 2, 1, 1, 1, 1), B=12, H=3, prefix=(5, 300))
+    assert w.n_nodes == 192
+    rng = np.random.default_rng(7)
+    lens = rng.integers(5, 301, w.B).astype(np.int32)
+    n_act = np.array([192, 64, 17, 130, 8, 100, 192, 33, 160, 72, 129, 1], dtype=np.int32)
+    for _ in range(3):
+        _full_attention_case(m, w, std=1.0, rel=True, lens=lens, n_act=n_act, poison=True)
+
+
 def test_attention_needle_reads_out_the_mask(m):
     # tree keys share one large score and carry one-hot values, the prefix scores 0 and carries zeros:
     # out[n][j] = 1/(depth(n)+1) exactly where node n may see node j
