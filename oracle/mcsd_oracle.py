@@ -162,6 +162,24 @@ def tree_attention(q, k_cache, v_cache, k_tree, v_tree, seq_lens, n_active, pare
     return out
 
 
+def tree_attention_gqa(q, k_cache, v_cache, k_tree, v_tree, seq_lens, n_active, parent, scale):
+    """Tree attention (Section 2.2) for a target whose query heads share key/value heads (grouped-query attention).
+
+    q is [B][H_q][N][D], the key/value tensors have H_kv heads, H_q = G * H_kv, and query head h reads key/value
+    head h // G; everything else is tree_attention.  The paper's targets are multi-head models (G = 1).
+    """
+    Hq, Hkv = q.shape[1], k_tree.shape[1]
+    if Hq % Hkv:
+        raise ValueError("the number of query heads must be a multiple of the number of key/value heads")
+    G = Hq // Hkv
+    out = np.zeros(q.shape, dtype=np.float64)
+    for h in range(Hq):
+        kv = h // G
+        out[:, h:h + 1] = tree_attention(q[:, h:h + 1], k_cache[:, kv:kv + 1], v_cache[:, kv:kv + 1],
+                                         k_tree[:, kv:kv + 1], v_tree[:, kv:kv + 1], seq_lens, n_active, parent, scale)
+    return out
+
+
 # ----------------------------------------------------------------------------
 # multi-candidate accept / reject (Fig. 1 steps 4-6, Section 3.1)
 # ----------------------------------------------------------------------------

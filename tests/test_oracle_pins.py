@@ -763,3 +763,25 @@ def test_sample_roots_draws_from_the_residual_of_the_stop_node():
         stop, dist = orc.stop_distribution(p, q, tokens, parent, None, ua0, b, v2)
         assert stop == int(v2["out_nodes"][b, v2["accept_len"][b] - 1])
         np.testing.assert_allclose(dist, p[b, stop], atol=0)
+
+
+def test_grouped_query_attention_is_attention_with_repeated_kv_heads():
+    rng = np.random.default_rng(41)
+    B, Hkv, G, D, L = 2, 2, 3, 8, 11
+    parent = parent_array(1, (2, 2))
+    N = len(parent)
+    q = rng.normal(size=(B, Hkv * G, N, D))
+    kc, vc = rng.normal(size=(B, Hkv, L, D)), rng.normal(size=(B, Hkv, L, D))
+    kt, vt = rng.normal(size=(B, Hkv, N, D)), rng.normal(size=(B, Hkv, N, D))
+    lens, nact = [11, 4], [N, 3]
+    got = orc.tree_attention_gqa(q, kc, vc, kt, vt, lens, nact, parent, 0.3)
+    rep = lambda x: np.repeat(x, G, axis=1)                 # head h reads key/value head h // G
+    want = orc.tree_attention(q, rep(kc), rep(vc), rep(kt), rep(vt), lens, nact, parent, 0.3)
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-14)
+    # heads of one group differ only through their queries
+    q2 = q.copy()
+    q2[:, 1] = q2[:, 0]
+    got2 = orc.tree_attention_gqa(q2, kc, vc, kt, vt, lens, nact, parent, 0.3)
+    np.testing.assert_allclose(got2[:, 1], got2[:, 0], rtol=0, atol=0)
+    with pytest.raises(ValueError):
+        orc.tree_attention_gqa(q[:, :5], kc, vc, kt, vt, lens, nact, parent, 0.3)
