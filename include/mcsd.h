@@ -124,6 +124,29 @@ int mcsd_tree_attention(const void* q, const void* k_cache, const void* v_cache,
                         int dtype, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * mcsd_tree_attention for a target with grouped-query attention: q and out have H_q heads, the four key/value
+ * tensors H_kv heads, H_q = G * H_kv, and query head h reads key/value head h / G (the paper's targets are
+ * multi-head models, G = 1; Section 2.2 defines the attention itself).  Everything else as mcsd_tree_attention.
+ * With bf16 and head_dim 128 the tensor-core kernel stacks the queries of S heads of a group into one work unit
+ * (S the largest of 8, 4, 2 that divides G with S * N <= MCSD_MAX_NODES, else 1), so that a key/value head is
+ * streamed G / S times instead of G times.
+ *
+ *   q, out                  [dev] dtype[B][H_q][N][D]
+ *   k_cache, v_cache        [dev] dtype[B][H_kv][L_max][D]
+ *   k_tree, v_tree          [dev] dtype[B][H_kv][N][D]
+ *   workspace               >= mcsd_tree_attention_workspace_bytes(B, H_q, N, D, L_max, dtype) bytes, zero-filled once
+ *
+ * Errors: as mcsd_tree_attention, plus MCSD_ERR_BAD_SHAPE when H_q is not a multiple of H_kv.
+ */
+int mcsd_tree_attention_gqa(const void* q, const void* k_cache, const void* v_cache,
+                            const void* k_tree, const void* v_tree, void* out,
+                            const int32_t* seq_lens, const int32_t* n_active,
+                            const uint64_t* anc, int words,
+                            int B, int H_q, int H_kv, int N, int D, int L_max,
+                            float softmax_scale, int dtype,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Reads the status word that kernels of mcsd_tree_attention / mcsd_verify_tree leave in `workspace`.
  * The word is sticky: kernels only ever set it, the caller clears it by zero-filling the first 256 bytes.
  * Synchronises `stream`.  Returns MCSD_OK, MCSD_ERR_TIMEOUT (a bounded wait ran out; outputs of that call

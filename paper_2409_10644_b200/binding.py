@@ -24,7 +24,7 @@ MCSD_MAX_WORDS = 3
 
 _EXPORTS = (
     "mcsd_status_string", "mcsd_last_cuda_error", "mcsd_launch_count", "mcsd_build_mask", "mcsd_tree_attention_workspace_bytes",
-    "mcsd_tree_attention", "mcsd_workspace_status", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_logits", "mcsd_verify_tree_static", "mcsd_commit_kv", "mcsd_sample_roots",
+    "mcsd_tree_attention", "mcsd_tree_attention_gqa", "mcsd_workspace_status", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_logits", "mcsd_verify_tree_static", "mcsd_commit_kv", "mcsd_sample_roots",
     "mcsd_sample_roots_logits",
 )
 
@@ -49,6 +49,8 @@ def _load() -> ctypes.CDLL:
     lib.mcsd_tree_attention_workspace_bytes.argtypes = [c_int] * 6
     lib.mcsd_tree_attention.restype = c_int
     lib.mcsd_tree_attention.argtypes = [c_void_p] * 9 + [c_int] * 6 + [c_float, c_int, c_void_p, c_size_t, c_void_p]
+    lib.mcsd_tree_attention_gqa.restype = c_int
+    lib.mcsd_tree_attention_gqa.argtypes = [c_void_p] * 9 + [c_int] * 7 + [c_float, c_int, c_void_p, c_size_t, c_void_p]
     lib.mcsd_workspace_status.restype = c_int
     lib.mcsd_workspace_status.argtypes = [c_void_p, c_void_p]
     lib.mcsd_verify_tree_workspace_bytes.restype = c_size_t
@@ -174,13 +176,18 @@ def new_workspace(nbytes: int, device) -> torch.Tensor:
 def mcsd_tree_attention(q, k_cache, v_cache, k_tree, v_tree, seq_lens, n_active, mask: TreeMask,
                         out: Optional[torch.Tensor] = None, softmax_scale: Optional[float] = None,
                         workspace: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """out[b][h][n] = attention of tree token n over the prefix cache and its root path (see mcsd.h)."""
+    """out[b][h][n] = attention of tree token n over the prefix cache and its root path (see mcsd.h).
+
+    Key/value tensors with fewer heads than q select grouped-query attention (query head h reads head h // G)."""
     dt = q.dtype
     B, H, N, D = q.shape
     L_max = k_cache.shape[2]
-    for name, t, shape in (("q", q, (B, H, N, D)), ("k_cache", k_cache, (B, H, L_max, D)),
-                           ("v_cache", v_cache, (B, H, L_max, D)), ("k_tree", k_tree, (B, H, N, D)),
-                           ("v_tree", v_tree, (B, H, N, D))):
+    H_kv = k_tree.shape[1]
+    if H_kv < 1 or H % H_kv:
+        raise ValueError("q has %d heads, the key/value tensors %d" % (H, H_kv))
+    for name, t, shape in (("q", q, (B, H, N, D)), ("k_cache", k_cache, (B, H_kv, L_max, D)),
+                           ("v_cache", v_cache, (B, H_kv, L_max, D)), ("k_tree", k_tree, (B, H_kv, N, D)),
+                           ("v_tree", v_tree, (B, H_kv, N, D))):
         _dev_tensor(t, dt, name)
         if tuple(t.shape) != shape:
             raise ValueError("%s has shape %s, expected %s" % (name, tuple(t.shape), shape))
@@ -198,9 +205,16 @@ def mcsd_tree_attention(q, k_cache, v_cache, k_tree, v_tree, seq_lens, n_active,
     if workspace is None:
         workspace = new_workspace(need, q.device)
     with torch.cuda.device(q.device):
-        st = lib.mcsd_tree_attention(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(k_tree), _ptr(v_tree), _ptr(out),
-                                     _ptr(seq_lens), _ptr(n_active), _ptr(mask.anc), mask.words, B, H, N, D, L_max,
-                                     ctypes.c_float(softmax_scale), code, _ptr(workspace), workspace.numel(), _stream())
+        if H_kv == H:
+            st = lib.mcsd_tree_attention(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(k_tree), _ptr(v_tree), _ptr(out),
+                                         _ptr(seq_lens), _ptr(n_active), _ptr(mask.anc), mask.words, B, H, N, D, L_max,
+                                         ctypes.c_float(softmax_scale), code, _ptr(workspace), workspace.numel(),
+                                         _stream())
+        else:
+            st = lib.mcsd_tree_attention_gqa(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(k_tree), _ptr(v_tree), _ptr(out),
+                                             _ptr(seq_lens), _ptr(n_active), _ptr(mask.anc), mask.words, B, H, H_kv, N, D,
+                                             L_max, ctypes.c_float(softmax_scale), code, _ptr(workspace),
+                                             workspace.numel(), _stream())
     _check(st, "mcsd_tree_attention")
     return out
 

@@ -31,14 +31,14 @@ extern "C" size_t mcsd_tree_attention_workspace_bytes(int B, int H, int N, int D
     return sizeof(mcsd::WorkspaceHeader) + mcsd::align_up(scratch, 256);
 }
 
-extern "C" int mcsd_tree_attention(const void* q, const void* k_cache, const void* v_cache, const void* k_tree,
-                                   const void* v_tree, void* out, const int32_t* seq_lens, const int32_t* n_active,
-                                   const uint64_t* anc, int words, int B, int H, int N, int D, int L_max,
-                                   float softmax_scale, int dtype, void* workspace, size_t workspace_bytes,
-                                   void* stream) {
+static int run_attention(const void* q, const void* k_cache, const void* v_cache, const void* k_tree, const void* v_tree,
+                         void* out, const int32_t* seq_lens, const int32_t* n_active, const uint64_t* anc, int words,
+                         int B, int H, int G, int N, int D, int L_max, float softmax_scale, int dtype, void* workspace,
+                         size_t workspace_bytes, void* stream) {
     if (!q || !k_tree || !v_tree || !out || !seq_lens || !anc || !workspace) return MCSD_ERR_NULL;
     const int st = check_shape(B, H, N, D, L_max, dtype);
     if (st != MCSD_OK) return st;
+    if (G < 1 || H % G != 0) return MCSD_ERR_BAD_SHAPE;
     if (L_max > 0 && (!k_cache || !v_cache)) return MCSD_ERR_NULL;
     if (words < (N + 63) / 64 || words > MCSD_MAX_WORDS) return MCSD_ERR_BAD_SHAPE;
     if (workspace_bytes < mcsd_tree_attention_workspace_bytes(B, H, N, D, L_max, dtype))
@@ -46,11 +46,30 @@ extern "C" int mcsd_tree_attention(const void* q, const void* k_cache, const voi
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MCSD_ERR_BAD_SHAPE;
 
     mcsd::AttentionArgs a{q, k_cache, v_cache, k_tree, v_tree, out, seq_lens, n_active, anc, words,
-                          B, H, N, D, L_max, softmax_scale, dtype};
+                          B, H, N, D, L_max, softmax_scale, dtype, G};
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     auto* header = static_cast<mcsd::WorkspaceHeader*>(workspace);
     void* scratch = static_cast<char*>(workspace) + sizeof(mcsd::WorkspaceHeader);
     const size_t scratch_bytes = workspace_bytes - sizeof(mcsd::WorkspaceHeader);
     if (mcsd::use_tc(a)) return mcsd::tree_attention_tc(a, header, scratch, scratch_bytes, s);
     return mcsd::tree_attention_simt(a, scratch, s);
+}
+
+extern "C" int mcsd_tree_attention(const void* q, const void* k_cache, const void* v_cache, const void* k_tree,
+                                   const void* v_tree, void* out, const int32_t* seq_lens, const int32_t* n_active,
+                                   const uint64_t* anc, int words, int B, int H, int N, int D, int L_max,
+                                   float softmax_scale, int dtype, void* workspace, size_t workspace_bytes,
+                                   void* stream) {
+    return run_attention(q, k_cache, v_cache, k_tree, v_tree, out, seq_lens, n_active, anc, words, B, H, 1, N, D, L_max,
+                         softmax_scale, dtype, workspace, workspace_bytes, stream);
+}
+
+extern "C" int mcsd_tree_attention_gqa(const void* q, const void* k_cache, const void* v_cache, const void* k_tree,
+                                       const void* v_tree, void* out, const int32_t* seq_lens, const int32_t* n_active,
+                                       const uint64_t* anc, int words, int B, int H_q, int H_kv, int N, int D, int L_max,
+                                       float softmax_scale, int dtype, void* workspace, size_t workspace_bytes,
+                                       void* stream) {
+    if (H_kv < 1 || H_q < H_kv || H_q % H_kv != 0) return MCSD_ERR_BAD_SHAPE;
+    return run_attention(q, k_cache, v_cache, k_tree, v_tree, out, seq_lens, n_active, anc, words, B, H_q, H_q / H_kv, N,
+                         D, L_max, softmax_scale, dtype, workspace, workspace_bytes, stream);
 }

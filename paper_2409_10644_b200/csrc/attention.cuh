@@ -16,9 +16,10 @@ struct AttentionArgs {
     const int32_t* n_active;
     const uint64_t* anc;
     int words;
-    int B, H, N, D, L_max;
+    int B, H, N, D, L_max;   // H: query heads
     float scale;
     int dtype;
+    int G;                   // query heads per key/value head (1: multi-head attention); key/value tensors have H / G heads
 };
 
 // CUDA-core path (fp32, or bf16 shapes the tensor-core kernel does not take)

@@ -30,7 +30,7 @@ __global__ void __launch_bounds__(kSimtThreads)
 tree_attention_simt_kernel(const T* __restrict__ q, const T* __restrict__ k_cache, const T* __restrict__ v_cache,
                            const T* __restrict__ k_tree, const T* __restrict__ v_tree, T* __restrict__ out,
                            const int32_t* __restrict__ seq_lens, const int32_t* __restrict__ n_active,
-                           const uint64_t* __restrict__ anc, int words, int H, int N, int L_max, float scale,
+                           const uint64_t* __restrict__ anc, int words, int H, int G, int N, int L_max, float scale,
                            int splits, float* __restrict__ part_ml, float* __restrict__ part_acc) {
     constexpr int DL = D / 32;                            // output columns per lane
     __shared__ float s_q[kSimtQBlock][D];
@@ -52,10 +52,11 @@ tree_attention_simt_kernel(const T* __restrict__ q, const T* __restrict__ k_cach
         const int r = i / D, d = i % D;
         s_q[r][d] = (q0 + r < Nb) ? to_f32(qb[(size_t)(q0 + r) * D + d]) : 0.f;
     }
-    const T* kc = k_cache + (size_t)bh * L_max * D;
-    const T* vc = v_cache + (size_t)bh * L_max * D;
-    const T* kt = k_tree + (size_t)bh * N * D;
-    const T* vt = v_tree + (size_t)bh * N * D;
+    const size_t bkv = (size_t)b * (H / G) + (bh % H) / G;   // query head h reads key/value head h / G
+    const T* kc = k_cache + bkv * L_max * D;
+    const T* vc = v_cache + bkv * L_max * D;
+    const T* kt = k_tree + bkv * N * D;
+    const T* vt = v_tree + bkv * N * D;
 
     float m[kSimtQPerWarp], l[kSimtQPerWarp], o[kSimtQPerWarp][DL];
 #pragma unroll
@@ -190,7 +191,7 @@ static int launch_simt(const AttentionArgs& a, void* scratch, cudaStream_t strea
     tree_attention_simt_kernel<T, D><<<grid, kSimtThreads, 0, stream>>>(
         static_cast<const T*>(a.q), static_cast<const T*>(a.k_cache), static_cast<const T*>(a.v_cache),
         static_cast<const T*>(a.k_tree), static_cast<const T*>(a.v_tree), static_cast<T*>(a.out), a.seq_lens,
-        a.n_active, a.anc, a.words, a.H, a.N, a.L_max, a.scale, splits, part_ml, part_acc);
+        a.n_active, a.anc, a.words, a.H, a.G, a.N, a.L_max, a.scale, splits, part_ml, part_acc);
     MCSD_CUDA_CHECK(cudaGetLastError());
     count_launches(1);
     if (splits > 1) {

@@ -83,7 +83,11 @@ struct TcParams {
     const int32_t* n_active;
     const uint64_t* anc;
     int words;
-    int B, H, N, L_max;
+    int B, H, N, L_max;      // H: work units per sequence = query heads / G; N tree nodes (= tree keys)
+    int G, g_shift;          // query heads stacked into one work unit (1, 2, 4 or 8 = 1 << g_shift): its G * N queries
+                             // are taken node-major, query j = head j % G of the unit, node j / G
+    int Hkv, group;          // key/value heads, and query heads per key/value head (a multiple of G): unit u of a
+                             // sequence reads key/value head u * G / group
     float scale_log2;
     float* part_ml;      // [2 * kMaxCtas][2][128]
     float* part_o;       // [2 * kMaxCtas][128][128]
@@ -143,6 +147,11 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z) : "memory");
 }
 
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, void* bar, int x, int y, int z, int w) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -236,8 +245,8 @@ __device__ __forceinline__ uint32_t instr_desc(int n, int a_mn_major, int b_mn_m
 __device__ __forceinline__ int kv_tiles_of(int L, int Nb) {
     return Nb > 0 ? (L + kTile - 1) / kTile + (Nb + kTile - 1) / kTile : 0;
 }
-__device__ __forceinline__ int tiles_of(int L, int Nb) {
-    return kv_tiles_of(L, Nb) * ((Nb + kQBlock - 1) / kQBlock);
+__device__ __forceinline__ int tiles_of(int L, int Nb, int G) {
+    return kv_tiles_of(L, Nb) * ((Nb * G + kQBlock - 1) / kQBlock);
 }
 
 struct Segment {
@@ -263,7 +272,7 @@ __device__ __forceinline__ void locate(const TcSmall* sm, const TcParams& p, lon
     s.qb = rem / s.Tkv;
     s.lt = rem % s.Tkv;
     s.q0 = s.qb * kQBlock;
-    s.Nq = min(kQBlock, s.Nb - s.q0);
+    s.Nq = min(kQBlock, s.Nb * p.G - s.q0);
 }
 
 // Cost of one tile in units of about 100 cycles, measured on this kernel.  Launches for up to 64 query columns:
@@ -279,8 +288,9 @@ __device__ __forceinline__ int tile_weight(int Nq, bool wide) {
 __device__ __forceinline__ int item_weight(int Nq, bool wide) {
     return (wide ? 100 : 30) + (Nq * 5) / 8;
 }
-__device__ __forceinline__ int head_weight(int L, int Nb, bool wide) {        // cost of one (sequence, head): all query blocks
-    const int tkv = kv_tiles_of(L, Nb);
+__device__ __forceinline__ int head_weight(int L, int Nk, int G, bool wide) {  // cost of one (sequence, head): all query blocks
+    const int tkv = kv_tiles_of(L, Nk);
+    const int Nb = Nk * G;                                        // stacked queries
     int w = 0;
     for (int q0 = 0; q0 < Nb; q0 += kQBlock) w += tkv * tile_weight(min(kQBlock, Nb - q0), wide) + item_weight(min(kQBlock, Nb - q0), wide);
     return w;
@@ -304,8 +314,9 @@ __device__ __forceinline__ long long first_tile_of_block(const TcSmall* sm, cons
         if ((long long)p.H * sm->cum_w[mid] <= wt) lo = mid; else hi = mid;
     }
     const int L = min(max(p.seq_lens[lo], 0), p.L_max);
-    const int Nb = p.n_active ? min(max(p.n_active[lo], 0), p.N) : p.N;
-    const int tkv = kv_tiles_of(L, Nb);
+    const int Nk = p.n_active ? min(max(p.n_active[lo], 0), p.N) : p.N;
+    const int tkv = kv_tiles_of(L, Nk);
+    const int Nb = Nk * p.G;                                      // stacked queries
     const int wh = sm->cum_w[lo + 1] - sm->cum_w[lo], tb = sm->cum_tiles[lo + 1] - sm->cum_tiles[lo];
     const long long rem = wt - (long long)p.H * sm->cum_w[lo];
     const int h = (int)(rem / wh);
@@ -354,8 +365,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     for (int b = tid; b < p.B; b += kTcThreads) {
         const int L = min(max(p.seq_lens[b], 0), p.L_max);
         const int Nb = p.n_active ? min(max(p.n_active[b], 0), p.N) : p.N;
-        sm->cum_tiles[b + 1] = (unsigned short)tiles_of(L, Nb);
-        sm->cum_w[b + 1] = head_weight(L, Nb, NCH > 4);
+        sm->cum_tiles[b + 1] = (unsigned short)tiles_of(L, Nb, p.G);
+        sm->cum_w[b + 1] = head_weight(L, Nb, p.G, NCH > 4);
     }
     if (tid == 0) {
         for (int i = 0; i < kMaxSlots; ++i) { mbar_init(&sm->slot_full[i], 1); mbar_init(&sm->slot_empty[i], 1); }
@@ -420,11 +431,19 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 locate(sm, p, t, s);
                 const int cnt = (int)min((long long)(s.Tkv - s.lt), t_end - t);
                 const int bh = s.b * p.H + s.h;
+                const int bh_kv = s.b * p.Hkv + (s.h * p.G) / p.group;
                 ok = mbar_wait(&sm->q_empty, (seg & 1u) ^ 1u, sm, hdr, 1);
                 if (!ok) break;
                 mbar_expect_tx(&sm->q_full, (uint32_t)p.npadq * 256u);
-                tma_load_3d(smem_u32(q_buf), &tm_q, &sm->q_full, 0, s.q0, bh);
-                tma_load_3d(smem_u32(q_buf) + (uint32_t)p.npadq * 128u, &tm_q, &sm->q_full, 64, s.q0, bh);
+                if (p.G == 1) {
+                    tma_load_3d(smem_u32(q_buf), &tm_q, &sm->q_full, 0, s.q0, bh);
+                    tma_load_3d(smem_u32(q_buf) + (uint32_t)p.npadq * 128u, &tm_q, &sm->q_full, 64, s.q0, bh);
+                } else {
+                    // grouped queries: the map is (dim, head of the group, node, sequence x key/value head); a box of
+                    // all G heads by npadq / G nodes lands node-major, i.e. as stacked queries q0, q0 + 1, ...
+                    tma_load_4d(smem_u32(q_buf), &tm_q, &sm->q_full, 0, 0, s.q0 >> p.g_shift, bh);
+                    tma_load_4d(smem_u32(q_buf) + (uint32_t)p.npadq * 128u, &tm_q, &sm->q_full, 64, 0, s.q0 >> p.g_shift, bh);
+                }
                 for (int i = 0; i < cnt && ok; ++i) {
                     const int lti = s.lt + i;
                     const bool tree = lti >= s.nP;
@@ -435,8 +454,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                         const CUtensorMap* map = kv == 0 ? (tree ? &tm_kt : &tm_kc) : (tree ? &tm_vt : &tm_vc);
                         const uint32_t dst = smem_u32(ring) + slot * (uint32_t)kSlotBytes;
                         mbar_expect_tx(&sm->slot_full[slot], (uint32_t)kSlotBytes);
-                        tma_load_3d(dst, map, &sm->slot_full[slot], 0, row0, bh);
-                        tma_load_3d(dst + kSlabBytes, map, &sm->slot_full[slot], 64, row0, bh);
+                        tma_load_3d(dst, map, &sm->slot_full[slot], 0, row0, bh_kv);
+                        tma_load_3d(dst + kSlabBytes, map, &sm->slot_full[slot], 64, row0, bh_kv);
                         if (++slot == (uint32_t)NS) { slot = 0; phase ^= 1u; }
                     }
                 }
@@ -591,17 +610,18 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             // Transposition, one 32-query piece of one key's row per thread and step (consecutive threads take
             // consecutive keys, so a warp reads the same word of 32 bitsets in turn: broadcasts, no bank conflicts).
             // Rows for keys beyond the tree are never read.
-            const int n_chunks = (p.N + 31) >> 5;
+            const int NQ = p.N * p.G;                            // stacked queries: query j belongs to node j / G
+            const int n_chunks = (NQ + 31) >> 5;
             const uint32_t* anc32 = reinterpret_cast<const uint32_t*>(anc_s);
             for (int idx = tid; idx < p.N * 6; idx += 32 * 4 * kSoftmaxGroups) {
                 const int c = idx / p.N, t = idx - c * p.N;
                 uint32_t piece = 0;
                 if (c < n_chunks) {
                     const uint32_t* col = anc32 + (t >> 5);          // 32-bit half of the 64-bit word that holds bit t
-                    const int n_end = min(32, p.N - 32 * c);
+                    const int n_end = min(32, NQ - 32 * c);
 #pragma unroll 8
                     for (int i = 0; i < n_end; ++i)
-                        piece |= ((col[(size_t)(32 * c + i) * p.words * 2] >> (t & 31)) & 1u) << i;
+                        piece |= ((col[(size_t)((32 * c + i) >> p.g_shift) * p.words * 2] >> (t & 31)) & 1u) << i;
                 }
                 reinterpret_cast<uint32_t*>(&sm->dmask[t][0])[c] = piece;
             }
@@ -960,7 +980,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                                     h = __floats2bfloat162_rn(v[2], v[3]); w.y = *reinterpret_cast<uint32_t*>(&h);
                                     h = __floats2bfloat162_rn(v[4], v[5]); w.z = *reinterpret_cast<uint32_t*>(&h);
                                     h = __floats2bfloat162_rn(v[6], v[7]); w.w = *reinterpret_cast<uint32_t*>(&h);
-                                    *reinterpret_cast<uint4*>(p.out + ((size_t)bh * p.N + s.q0 + n) * 128 + 32 * wq + (lane & 24)) = w;
+                                    const int jq = s.q0 + n;          // stacked query: head jq % G of the group, node jq / G
+                                    *reinterpret_cast<uint4*>(p.out + (((size_t)bh * p.G + (jq & (p.G - 1))) * p.N + (jq >> p.g_shift)) * 128 +
+                                                              32 * wq + (lane & 24)) = w;
                                 }
                             } else {
 #pragma unroll
@@ -1049,9 +1071,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
 #pragma unroll
                                 for (int k = 0; k < 8; ++k) {
                                     const int n = col0 + 8 * (j0 + jj) + k;
-                                    if (j0 + jj < ncg && n < s.Nq)
-                                        p.out[((size_t)bh * p.N + s.q0 + n) * 128 + r] =
+                                    if (j0 + jj < ncg && n < s.Nq) {
+                                        const int jq = s.q0 + n;
+                                        p.out[(((size_t)bh * p.G + (jq & (p.G - 1))) * p.N + (jq >> p.g_shift)) * 128 + r] =
                                             __float2bfloat16_rn(lsum[jj][k] > 0.f ? o_keep[jj][k] / lsum[jj][k] : 0.f);
+                                    }
                                 }
                         }
                     }
@@ -1095,7 +1119,7 @@ static EncodeTiledFn encode_fn() {
 // buffers every step, so the encoded maps are kept in a small per-thread table (round-robin replacement).
 struct MapKey {
     const void* base;
-    int rows, bh, box_rows;
+    int rows, bh, box_rows, group;
 };
 constexpr int kMapCacheSize = 256;
 struct MapCache {
@@ -1105,25 +1129,39 @@ struct MapCache {
 };
 static thread_local MapCache g_map_cache;
 
-static bool encode_map(CUtensorMap* map, const void* base, int rows, int bh, int box_rows);
+static bool encode_map(CUtensorMap* map, const void* base, int rows, int bh, int box_rows, int group);
 
-// [BH][rows][128] bf16 tensor, boxes of box_rows x 64 columns, 128-byte swizzle, zero fill outside
-static bool make_map(CUtensorMap* map, const void* base, int rows, int bh, int box_rows) {
+// group == 1: [BH][rows][128] bf16 tensor, boxes of box_rows x 64 columns, 128-byte swizzle, zero fill outside.
+// group  > 1: the queries of a grouped-query target, [BH][group][rows][128]: dimensions (column, head of the
+//             group, row, BH) so that a box of all heads by box_rows / group rows lands row-major in shared memory.
+static bool make_map(CUtensorMap* map, const void* base, int rows, int bh, int box_rows, int group = 1) {
     MapCache& c = g_map_cache;
     for (int i = 0; i < c.used; ++i) {
         const MapKey& k = c.key[i];
-        if (k.base == base && k.rows == rows && k.bh == bh && k.box_rows == box_rows) { *map = c.map[i]; return true; }
+        if (k.base == base && k.rows == rows && k.bh == bh && k.box_rows == box_rows && k.group == group) {
+            *map = c.map[i];
+            return true;
+        }
     }
-    if (!encode_map(map, base, rows, bh, box_rows)) return false;
+    if (!encode_map(map, base, rows, bh, box_rows, group)) return false;
     const int slot = c.used < kMapCacheSize ? c.used++ : (c.next = (c.next + 1) % kMapCacheSize);
-    c.key[slot] = MapKey{base, rows, bh, box_rows};
+    c.key[slot] = MapKey{base, rows, bh, box_rows, group};
     c.map[slot] = *map;
     return true;
 }
 
-static bool encode_map(CUtensorMap* map, const void* base, int rows, int bh, int box_rows) {
+static bool encode_map(CUtensorMap* map, const void* base, int rows, int bh, int box_rows, int group) {
     EncodeTiledFn fn = encode_fn();
     if (fn == nullptr) return false;
+    if (group > 1) {
+        cuuint64_t dims[4] = {128, (cuuint64_t)group, (cuuint64_t)rows, (cuuint64_t)bh};
+        cuuint64_t strides[3] = {(cuuint64_t)rows * 256, 256, (cuuint64_t)group * rows * 256};
+        cuuint32_t box[4] = {64, (cuuint32_t)group, (cuuint32_t)(box_rows / group), 1};
+        cuuint32_t estr[4] = {1, 1, 1, 1};
+        return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    }
     cuuint64_t dims[3] = {128, (cuuint64_t)rows, (cuuint64_t)bh};
     cuuint64_t strides[2] = {256, (cuuint64_t)rows * 256};
     cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
@@ -1145,8 +1183,16 @@ static int slots_for(int nch) {
     return (int)ns;
 }
 
+// Query heads of one key/value group stacked into one work unit: the largest of 8, 4, 2, 1 that divides the group
+// and keeps the stacked queries within two query blocks.
+static int stack_for(int G, int N) {
+    for (int s = 8; s > 1; s >>= 1)
+        if (G % s == 0 && s * N <= MCSD_MAX_NODES) return s;
+    return 1;
+}
+
 bool tc_supported(const AttentionArgs& a) {
-    return a.N <= MCSD_MAX_NODES && a.B <= kMaxBatchTc && encode_fn() != nullptr;
+    return a.G >= 1 && a.H % a.G == 0 && a.N <= MCSD_MAX_NODES && a.B <= kMaxBatchTc && encode_fn() != nullptr;
 }
 
 size_t tc_workspace_bytes(int, int, int N, int, int) {
@@ -1175,19 +1221,21 @@ static int launch_tc(const CUtensorMap* maps, const TcParams& p, int grid, size_
 int tree_attention_tc(const AttentionArgs& a, WorkspaceHeader* header, void* scratch, size_t scratch_bytes,
                       cudaStream_t stream) {
     if (scratch_bytes < tc_workspace_bytes(a.B, a.H, a.N, a.D, a.L_max)) return MCSD_ERR_WORKSPACE_TOO_SMALL;
-    const int nch = chunks_for(a.N);
+    const int S = stack_for(a.G, a.N);          // query heads per work unit
+    const int nch = chunks_for(a.N * S);
     const int npadq = nch * 16;
     const int ns = slots_for(nch);
     if (ns < 4) return MCSD_ERR_BAD_SHAPE;
-    const int bh = a.B * a.H;
+    const int bh = a.B * (a.H / S);             // work units: (sequence, S query heads of one key/value group)
+    const int bh_kv = a.B * (a.H / a.G);
 
     CUtensorMap maps[5];
     const bool have_cache = a.L_max > 0;
-    bool ok = make_map(&maps[0], a.q, a.N, bh, npadq);
-    ok = ok && make_map(&maps[1], have_cache ? a.k_cache : a.k_tree, have_cache ? a.L_max : a.N, bh, kTile);
-    ok = ok && make_map(&maps[2], have_cache ? a.v_cache : a.v_tree, have_cache ? a.L_max : a.N, bh, kTile);
-    ok = ok && make_map(&maps[3], a.k_tree, a.N, bh, kTile);
-    ok = ok && make_map(&maps[4], a.v_tree, a.N, bh, kTile);
+    bool ok = make_map(&maps[0], a.q, a.N, bh, npadq, S);
+    ok = ok && make_map(&maps[1], have_cache ? a.k_cache : a.k_tree, have_cache ? a.L_max : a.N, bh_kv, kTile);
+    ok = ok && make_map(&maps[2], have_cache ? a.v_cache : a.v_tree, have_cache ? a.L_max : a.N, bh_kv, kTile);
+    ok = ok && make_map(&maps[3], a.k_tree, a.N, bh_kv, kTile);
+    ok = ok && make_map(&maps[4], a.v_tree, a.N, bh_kv, kTile);
     if (!ok) { set_last_cuda_error(cudaErrorInvalidValue); return MCSD_ERR_CUDA; }
 
     int dev = 0, sms = 0;
@@ -1206,7 +1254,11 @@ int tree_attention_tc(const AttentionArgs& a, WorkspaceHeader* header, void* scr
     p.n_active = a.n_active;
     p.anc = a.anc;
     p.words = a.words;
-    p.B = a.B; p.H = a.H; p.N = a.N; p.L_max = a.L_max;
+    p.B = a.B; p.H = a.H / S; p.N = a.N; p.L_max = a.L_max;
+    p.G = S;
+    p.g_shift = S == 8 ? 3 : S == 4 ? 2 : S == 2 ? 1 : 0;
+    p.Hkv = a.H / a.G;
+    p.group = a.G;
     p.scale_log2 = a.scale * 1.4426950408889634f;
     p.part_ml = static_cast<float*>(scratch);
     p.part_o = reinterpret_cast<float*>(static_cast<char*>(scratch) + align_up((size_t)2 * kMaxCtas * 2 * 128 * sizeof(float), 256));

@@ -77,6 +77,19 @@ def test_attention_argument_checks(m):
     assert call(N=100, words=1) == -2
 
 
+def test_attention_gqa_argument_checks(m):
+    L = m.lib
+
+    def call(Hq=8, Hkv=2, q=FAKE, wsb=1 << 30):
+        return L.mcsd_tree_attention_gqa(q, FAKE, FAKE, FAKE, FAKE, FAKE, FAKE, None, FAKE, 1, 1, Hq, Hkv, 15, 64, 128,
+                                         ctypes.c_float(0.125), 1, FAKE, wsb, None)
+    assert call(Hq=8, Hkv=3) == -2              # query heads must be a multiple of the key/value heads
+    assert call(Hkv=0) == -2
+    assert call(Hq=2, Hkv=4) == -2
+    assert call(q=None) == -1
+    assert call(wsb=16) == -5
+
+
 def test_verify_argument_checks(m):
     L = m.lib
     assert L.mcsd_verify_tree_workspace_bytes(16, 45, 32000) >= 256 + 16 * 45 * 16

@@ -201,6 +201,42 @@ def test_attention_query_split_changes_between_segments(m):
         _full_attention_case(m, w, std=1.0, rel=True, lens=lens, n_act=n_act, poison=True)
 
 
+@pytest.mark.parametrize("G,case", [(4, "stacked"), (2, "stacked"), (8, "stacked"), (3, "stacked"), (8, "stacked_small"),
+                                    (4, "too_wide"), (2, "f32")])
+def test_attention_grouped_queries(m, G, case):
+    # query heads share key/value heads; the tensor-core kernel stacks the queries of 8, 4 or 2 heads of a group into
+    # one work unit when that divides the group and fits 192 queries (G = 8, N = 45: two units of four heads; G = 3
+    # or N = 109: one head per unit, the key/value head still shared); fp32 takes the CUDA-core kernel
+    if case == "stacked":
+        w = dataclasses.replace(workload(2), B=3, H=2 * G, prefix=(40, 600))          # N = 45: 180 or 90 queries
+    elif case == "stacked_small":
+        w = dataclasses.replace(workload(1), dtype="bf16", D=128, B=2, H=G, prefix=(5, 300))   # N = 15: 120 queries
+    elif case == "too_wide":
+        w = dataclasses.replace(workload(3), B=2, H=G, prefix=(100, 300))              # N = 109: nothing to stack
+    else:
+        w = dataclasses.replace(workload(1), B=2, H=2 * G, prefix=(20, 128))           # fp32: CUDA-core kernel
+    Hkv = w.H // G
+    parent = parent_array(w.n_roots, w.branching)
+    N = len(parent)
+    inp = attention_inputs(w, 0, "cuda", std=1.0)
+    for k in ("k_cache", "v_cache", "k_tree", "v_tree"):
+        inp[k] = inp[k][:, :Hkv].contiguous()
+    rng = np.random.default_rng(60 + G)
+    lens = rng.integers(w.prefix[0], w.prefix[1] + 1, w.B).astype(np.int32)
+    n_act = np.array([N, max(1, N // 3), N - 1][: w.B], dtype=np.int32)
+    for b in range(w.B):
+        inp["k_cache"][b, :, int(lens[b]):] = float("nan")
+        inp["v_cache"][b, :, int(lens[b]):] = float("nan")
+    scale = 1.0 / np.sqrt(w.D)
+    out = _run_attention(m, w, inp, lens, n_act, parent, scale)
+    host = {k: to_np(v) for k, v in inp.items()}
+    ref = orc.tree_attention_gqa(host["q"], host["k_cache"], host["v_cache"], host["k_tree"], host["v_tree"],
+                                 lens, n_act, parent, scale)
+    rows = {(b, h): ref[b, h] for b in range(w.B) for h in range(w.H)}
+    tol = TOL_F32 if w.dtype == "f32" else TOL_BF16
+    _compare_attention(out, rows, n_act, N, tol, rel=(w.dtype != "f32"))
+
+
 def test_attention_needle_reads_out_the_mask(m):
     # tree keys share one large score and carry one-hot values, the prefix scores 0 and carries zeros:
     # out[n][j] = 1/(depth(n)+1) exactly where node n may see node j
