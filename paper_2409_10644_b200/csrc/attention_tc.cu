@@ -1019,65 +1019,79 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 group_sync_any(bar_id, false);
                 const int nparts = sm->merge_parts[wg];
                 if (nparts > 0) {
-                    // JB column groups are merged at a time: all of them when they fit in registers
-                    constexpr int JB = 1;
+                    // The other pieces sit in the workspace behind a memory system that is busy streaming keys and
+                    // values, so what counts is the number of dependent round trips: one per piece and batch of
+                    // column groups.  All O^T loads of a piece are issued first; while they are in flight the thread
+                    // that owns a query column fetches the piece's (m, l) for it, folds them into its running
+                    // reference and normaliser and leaves the two rescale factors of that column in shared memory;
+                    // after a group barrier every thread applies them to its rows.
+                    const int np1 = nparts - 1;
+                    float* const fa = &sm->wred[wg][0][0];                   // [piece parity][64]: factor for what we have
+                    float* const fw = &sm->wred[wg][2][0];                   // [piece parity][64]: factor for the new piece
+                    const bool col_owner = r < ncg * 8 && col0 + r < s.Nq;
+                    constexpr int GB = CPT < 4 ? CPT : (CPT == 7 ? 3 : 2);   // column groups per batch (what the registers allow)
 #pragma unroll
-                    for (int j0 = 0; j0 < CPT; j0 += JB) {
-                        if (j0 < ncg) {
-                            float M[JB][8], lsum[JB][8], o_keep[JB][8];
+                    for (int j0 = 0; j0 < CPT; j0 += GB) {
+                        if (j0 >= ncg) break;
+                        float acc[GB][8];
 #pragma unroll
-                            for (int jj = 0; jj < JB; ++jj) {
-                                if (j0 + jj < ncg) tc_ld8(tmem + lane_addr + kColO + col0 + 8 * (j0 + jj), o_keep[jj]);
-                            }
-                            tc_wait_ld();
+                        for (int jj = 0; jj < GB; ++jj)
+                            if (j0 + jj < CPT && j0 + jj < ncg) tc_ld8(tmem + lane_addr + kColO + col0 + 8 * (j0 + jj), acc[jj]);
+                        tc_wait_ld();
+                        float m_run = col_owner ? mref[r] : -INFINITY;       // of column r, kept by its owner
+                        float l_run2 = col_owner ? alph[r] : 0.f;
+                        for (int i = 0; i < np1; ++i) {
+                            const int slot = sm->piece_slot[which][i];
+                            float os[GB][8];
 #pragma unroll
-                            for (int jj = 0; jj < JB; ++jj)
-#pragma unroll
-                                for (int k = 0; k < 8; ++k) {
-                                    const int n = col0 + 8 * (j0 + jj) + k;
-                                    const bool on = j0 + jj < ncg && n < s.Nq;
-                                    M[jj][k] = on ? mref[n - col0] : -INFINITY;
-                                    lsum[jj][k] = on ? alph[n - col0] : 0.f;
-                                    if (!on) o_keep[jj][k] = 0.f;
-                                }
-                            for (int i = 0; i < nparts - 1; ++i) {
-                                const int slot = sm->piece_slot[which][i];
-                                float ms[JB][8], ls[JB][8], os[JB][8];
-                                // all loads of one piece are issued before any is used: one memory round trip
-#pragma unroll
-                                for (int jj = 0; jj < JB; ++jj)
-#pragma unroll
-                                    for (int k = 0; k < 8; ++k) {
-                                        const int n = col0 + 8 * (j0 + jj) + k;
-                                        const bool on = j0 + jj < ncg && n < s.Nq;
-                                        ms[jj][k] = on ? __ldcg(p.part_ml + ((size_t)slot * 2 + 0) * 128 + n) : -INFINITY;
-                                        ls[jj][k] = on ? __ldcg(p.part_ml + ((size_t)slot * 2 + 1) * 128 + n) : 0.f;
-                                        os[jj][k] = on ? __ldcg(p.part_o + ((size_t)slot * 128 + n) * 128 + r) : 0.f;
-                                    }
-#pragma unroll
-                                for (int jj = 0; jj < JB; ++jj)
-#pragma unroll
-                                    for (int k = 0; k < 8; ++k) {
-                                        const float mn = fmaxf(M[jj][k], ms[jj][k]);
-                                        if (mn == -INFINITY) continue;
-                                        const float a = exp2f(M[jj][k] - mn), w = exp2f(ms[jj][k] - mn);
-                                        lsum[jj][k] = fmaf(lsum[jj][k], a, w * ls[jj][k]);
-                                        o_keep[jj][k] = fmaf(o_keep[jj][k], a, w * os[jj][k]);
-                                        M[jj][k] = mn;
-                                    }
-                            }
-#pragma unroll
-                            for (int jj = 0; jj < JB; ++jj)
+                            for (int jj = 0; jj < GB; ++jj)
 #pragma unroll
                                 for (int k = 0; k < 8; ++k) {
                                     const int n = col0 + 8 * (j0 + jj) + k;
-                                    if (j0 + jj < ncg && n < s.Nq) {
-                                        const int jq = s.q0 + n;
-                                        p.out[(((size_t)bh * p.G + (jq & (p.G - 1))) * p.N + (jq >> p.g_shift)) * 128 + r] =
-                                            __float2bfloat16_rn(lsum[jj][k] > 0.f ? o_keep[jj][k] / lsum[jj][k] : 0.f);
-                                    }
+                                    const bool on = j0 + jj < CPT && j0 + jj < ncg && n < s.Nq;
+                                    os[jj][k] = on ? __ldcg(p.part_o + ((size_t)slot * 128 + n) * 128 + r) : 0.f;
                                 }
+                            float* const fa_i = fa + 64 * (i & 1);
+                            float* const fw_i = fw + 64 * (i & 1);
+                            if (col_owner) {
+                                const float ms = __ldcg(p.part_ml + ((size_t)slot * 2 + 0) * 128 + col0 + r);
+                                const float ls = __ldcg(p.part_ml + ((size_t)slot * 2 + 1) * 128 + col0 + r);
+                                const float mn = fmaxf(m_run, ms);
+                                const float a = (mn == -INFINITY || m_run == -INFINITY) ? 0.f : exp2f(m_run - mn);
+                                const float wgt = (mn == -INFINITY || ms == -INFINITY) ? 0.f : exp2f(ms - mn);
+                                l_run2 = l_run2 * a + ls * wgt;
+                                m_run = mn;
+                                fa_i[r] = a;
+                                fw_i[r] = wgt;
+                            }
+                            group_sync_any(bar_id, false);                   // factors of piece i are in place
+#pragma unroll
+                            for (int jj = 0; jj < GB; ++jj)
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) {
+                                    const int rel = 8 * (j0 + jj) + k;
+                                    if (j0 + jj < CPT && j0 + jj < ncg)
+                                        acc[jj][k] = fmaf(os[jj][k], fw_i[rel], acc[jj][k] * fa_i[rel]);
+                                }
+                            // piece i + 2 reuses these factor slots: by then every thread has passed the barrier of
+                            // piece i + 1, which it reaches only after the loop above
                         }
+                        // normaliser of every column, then the output rows
+                        group_sync_any(bar_id, false);                       // everybody is done with the factor slots
+                        if (col_owner) fa[r] = l_run2 > 0.f ? 1.f / l_run2 : 0.f;
+                        group_sync_any(bar_id, false);
+#pragma unroll
+                        for (int jj = 0; jj < GB; ++jj)
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const int rel = 8 * (j0 + jj) + k, n = col0 + rel;
+                                if (j0 + jj < CPT && j0 + jj < ncg && n < s.Nq) {
+                                    const int jq = s.q0 + n;
+                                    p.out[(((size_t)bh * p.G + (jq & (p.G - 1))) * p.N + (jq >> p.g_shift)) * 128 + r] =
+                                        __float2bfloat16_rn(acc[jj][k] * fa[rel]);
+                                }
+                            }
+                        group_sync_any(bar_id, false);                       // before the next batch reuses the slots
                     }
                 }
             }
@@ -1184,10 +1198,11 @@ static int slots_for(int nch) {
 }
 
 // Query heads of one key/value group stacked into one work unit: the largest of 8, 4, 2, 1 that divides the group
-// and keeps the stacked queries within two query blocks.
+// and keeps the stacked queries within one query block (a second block would stream the keys again, which is what
+// a second unit does as well, with narrower tiles).
 static int stack_for(int G, int N) {
     for (int s = 8; s > 1; s >>= 1)
-        if (G % s == 0 && s * N <= MCSD_MAX_NODES) return s;
+        if (G % s == 0 && s * N <= kQBlock) return s;
     return 1;
 }
 
