@@ -38,7 +38,7 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM traffic of the attention kernel from an `ncu --set full` capture (profiles/tree_attention_tc_b4_ncu_full.md):
 # dram__bytes_read.sum + dram__bytes_write.sum per launch on a 4-sequence case; traffic grows in proportion to the
 # batch.  The figure only holds for the kernel source it was taken on.
-_TRAFFIC_CAPTURE = {"source_sha1_12": "06dff6cd6bc9", "bytes_per_launch": 281_544_320, "batch": 4,
+_TRAFFIC_CAPTURE = {"source_sha1_12": "c1d48365f80b", "bytes_per_launch": 281_149_952, "batch": 4,
                     "workload": "long_context_b16"}
 
 
