@@ -276,6 +276,65 @@ int mcsd_commit_kv(void* const* k_cache_layers, void* const* v_cache_layers,
                    int n_levels, int B, int H, int N, int D, int L_max, int dtype, void* stream);
 
 /*
+ * mcsd_verify_tree with the vocabulary split over several GPUs (Fig. 1 steps 4-6, the procedure of
+ * mcsd_verify_tree): rank r holds columns [v0, v0 + Vs) of p and q, the way a tensor-parallel output layer leaves
+ * them, so no rank ever gathers a full row.  The four calls below are the per-rank kernels; between them the
+ * caller reduces three small buffers over the ranks (with NCCL, or any all-reduce), in this order:
+ *
+ *   mcsd_verify_shard_gather                     -> all-reduce SUM of pq_exchange
+ *   for round = 0 .. k:  mcsd_verify_shard_round -> all-reduce SUM of y_exchange   (not after round k)
+ *   mcsd_verify_shard_select                     -> all-reduce SUM of mass_exchange
+ *   mcsd_verify_shard_pick                       -> all-reduce MAX of out_tokens
+ *
+ * where k is the largest number of children of any node.  gather fetches p_u(x), q_u(x) of every candidate token
+ * from the rank that owns x.  A round takes the reduced mass of the residual pass issued in the round before,
+ * tests the next sibling of every undecided node and, on a rejection, adds up this rank's part of
+ * sum_v max(p_v - c q_v, 0) for the next residual; decisions are recomputed alike on every rank from the reduced
+ * numbers.  select follows the accepted paths (as mcsd_verify_tree) and reports this rank's share of the stop
+ * distribution's mass; pick draws the new token by inverse CDF over the ranks' column ranges in order: the rank in
+ * whose columns the running sum passes u_bonus * total writes the token, the others -1.  After the last
+ * all-reduce every rank holds the outputs of mcsd_verify_tree (next_roots is not offered).
+ *
+ *   p_shard, q_shard  [dev] float[B][N][Vs], this rank's columns
+ *   v0, V_total       first global token id of this rank's columns, size of the whole vocabulary; the ranks'
+ *                     ranges are disjoint, in rank order, and cover [0, V_total)
+ *   pq_exchange       [dev] double[B][N][2] (out of gather; read by round after the reduction)
+ *   y_exchange        [dev] double[B][N] (in: reduced sums of the previous round; out: this rank's partial sums)
+ *   mass_exchange     [dev] double[world][B][2] (out of select: row `rank` filled, others zero; read by pick)
+ *   round             0 initialises the per-node state; rounds must be issued in order
+ *   workspace         [dev] >= mcsd_verify_shard_workspace_bytes(B, N) bytes, the same one for all four calls
+ *   tokens, parent, level_start, gamma, u_accept, u_bonus, accept_len, out_tokens, out_nodes, best_root:
+ *                     as for mcsd_verify_tree, identical on every rank
+ *
+ * One launch per call on `stream`.  Errors: MCSD_ERR_NULL, MCSD_ERR_BAD_SHAPE (sizes as for mcsd_verify_tree with
+ * Vs for V; v0 < 0 or v0 + Vs > V_total; rank outside [0, world); world > 1024; round outside [0, N]),
+ * MCSD_ERR_WORKSPACE_TOO_SMALL, MCSD_ERR_CUDA.
+ */
+size_t mcsd_verify_shard_workspace_bytes(int B, int N);
+
+int mcsd_verify_shard_gather(const float* p_shard, const float* q_shard, const int32_t* tokens,
+                             const int32_t* parent, const int32_t* level_start, int n_levels,
+                             const int32_t* gamma, int B, int N, int Vs, int v0, int V_total,
+                             double* pq_exchange, void* stream);
+
+int mcsd_verify_shard_round(const float* p_shard, const float* q_shard, const int32_t* parent,
+                            const int32_t* level_start, int n_levels, const int32_t* gamma,
+                            const float* u_accept, const double* pq_exchange, double* y_exchange,
+                            int round, int B, int N, int Vs, void* workspace, size_t workspace_bytes,
+                            void* stream);
+
+int mcsd_verify_shard_select(const float* p_shard, const float* q_shard, const int32_t* tokens,
+                             int n_levels, int n_roots, int B, int N, int Vs, int v0, int V_total,
+                             int rank, int world, int32_t* accept_len, int32_t* out_tokens,
+                             int32_t* out_nodes, int32_t* best_root, double* mass_exchange,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+int mcsd_verify_shard_pick(const float* p_shard, const float* q_shard, const float* u_bonus, int n_levels,
+                           int B, int N, int Vs, int v0, int V_total, int rank, int world,
+                           const double* mass_exchange, int32_t* out_tokens, const void* workspace,
+                           size_t workspace_bytes, void* stream);
+
+/*
  * mcsd_verify_tree with built-in scratch.  (The paper has no counterpart; this is a deployment convenience.)
  *
  * Same computation, arguments and results as mcsd_verify_tree, minus the workspace: the per-node scratch

@@ -9,6 +9,7 @@ _BINDING_NAMES = (
     "mcsd_build_mask", "mcsd_tree_attention", "mcsd_tree_attention_workspace_bytes",
     "mcsd_verify_tree", "mcsd_verify_tree_logits", "mcsd_sample_roots", "mcsd_verify_tree_static", "mcsd_commit_kv", "layer_pointer_table", "mcsd_verify_tree_workspace_bytes", "mcsd_workspace_status",
     "mcsd_status_string", "mcsd_launch_count", "n_active_from_gamma", "shard_batch", "new_workspace",
+    "VocabShard", "mcsd_verify_shard_workspace_bytes",
 )
 
 

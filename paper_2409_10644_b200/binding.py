@@ -25,7 +25,8 @@ MCSD_MAX_WORDS = 3
 _EXPORTS = (
     "mcsd_status_string", "mcsd_last_cuda_error", "mcsd_launch_count", "mcsd_build_mask", "mcsd_tree_attention_workspace_bytes",
     "mcsd_tree_attention", "mcsd_tree_attention_gqa", "mcsd_workspace_status", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_logits", "mcsd_verify_tree_static", "mcsd_commit_kv", "mcsd_sample_roots",
-    "mcsd_sample_roots_logits",
+    "mcsd_sample_roots_logits", "mcsd_verify_shard_workspace_bytes", "mcsd_verify_shard_gather", "mcsd_verify_shard_round",
+    "mcsd_verify_shard_select", "mcsd_verify_shard_pick",
 )
 
 
@@ -72,6 +73,19 @@ def _load() -> ctypes.CDLL:
                                             [c_void_p] * 5 + [c_int, c_void_p])
     lib.mcsd_commit_kv.restype = c_int
     lib.mcsd_commit_kv.argtypes = [c_void_p] * 4 + [c_int] + [c_void_p] * 4 + [c_int] * 7 + [c_void_p]
+    lib.mcsd_verify_shard_workspace_bytes.restype = c_size_t
+    lib.mcsd_verify_shard_workspace_bytes.argtypes = [c_int] * 2
+    lib.mcsd_verify_shard_gather.restype = c_int
+    lib.mcsd_verify_shard_gather.argtypes = [c_void_p] * 5 + [c_int, c_void_p] + [c_int] * 5 + [c_void_p, c_void_p]
+    lib.mcsd_verify_shard_round.restype = c_int
+    lib.mcsd_verify_shard_round.argtypes = ([c_void_p] * 4 + [c_int] + [c_void_p] * 4 + [c_int] * 4 +
+                                            [c_void_p, c_size_t, c_void_p])
+    lib.mcsd_verify_shard_select.restype = c_int
+    lib.mcsd_verify_shard_select.argtypes = ([c_void_p] * 3 + [c_int] * 9 + [c_void_p] * 5 +
+                                             [c_void_p, c_size_t, c_void_p])
+    lib.mcsd_verify_shard_pick.restype = c_int
+    lib.mcsd_verify_shard_pick.argtypes = ([c_void_p] * 3 + [c_int] * 8 + [c_void_p] * 2 +
+                                           [c_void_p, c_size_t, c_void_p])
     return lib
 
 
@@ -374,6 +388,81 @@ def mcsd_commit_kv(k_cache_ptrs, v_cache_ptrs, k_tree_ptrs, v_tree_ptrs, seq_len
                                 _ptr(verify_out["best_root"]), mask.n_levels, B, H, mask.n_nodes, D, L_max, code,
                                 _stream())
     _check(st, "mcsd_commit_kv")
+
+
+def mcsd_verify_shard_workspace_bytes(B, N) -> int:
+    return int(lib.mcsd_verify_shard_workspace_bytes(B, N))
+
+
+class VocabShard:
+    """One rank's tensors and calls of the vocabulary-sharded verify step (see mcsd.h): p_shard / q_shard hold
+    columns [v0, v0 + Vs) of the two probability tensors.  The four methods launch one kernel each; the owner of
+    the object reduces `pq`, `y`, `mass` and `out["out_tokens"]` over the ranks between them."""
+
+    def __init__(self, p_shard, q_shard, v0: int, V_total: int, rank: int, world: int, tokens, mask: TreeMask,
+                 gamma, u_accept, u_bonus):
+        B, N, Vs = p_shard.shape
+        _dev_tensor(p_shard, torch.float32, "p_shard")
+        _dev_tensor(q_shard, torch.float32, "q_shard")
+        _dev_tensor(tokens, torch.int32, "tokens")
+        _dev_tensor(u_accept, torch.float32, "u_accept")
+        _dev_tensor(u_bonus, torch.float32, "u_bonus")
+        if gamma is not None:
+            _dev_tensor(gamma, torch.int32, "gamma")
+        if mask.n_nodes != N or tuple(q_shard.shape) != (B, N, Vs) or tuple(tokens.shape) != (B, N):
+            raise ValueError("shape mismatch between p_shard, q_shard, tokens and the tree")
+        dev = p_shard.device
+        self.p, self.q, self.v0, self.V_total, self.rank, self.world = p_shard, q_shard, int(v0), int(V_total), rank, world
+        self.tokens, self.mask, self.gamma, self.u_accept, self.u_bonus = tokens, mask, gamma, u_accept, u_bonus
+        self.B, self.N, self.Vs = B, N, Vs
+        nl = mask.n_levels
+        self.pq = torch.zeros((B, N, 2), dtype=torch.float64, device=dev)
+        self.y = torch.zeros((B, N), dtype=torch.float64, device=dev)
+        self.mass = torch.zeros((world, B, 2), dtype=torch.float64, device=dev)
+        self.workspace = new_workspace(mcsd_verify_shard_workspace_bytes(B, N), dev)
+        self.out = {
+            "accept_len": torch.empty(B, dtype=torch.int32, device=dev),
+            "out_tokens": torch.empty((B, nl + 1), dtype=torch.int32, device=dev),
+            "out_nodes": torch.empty((B, nl), dtype=torch.int32, device=dev),
+            "best_root": torch.empty(B, dtype=torch.int32, device=dev),
+            "next_roots": None,
+        }
+
+    def gather(self):
+        m = self.mask
+        with torch.cuda.device(self.p.device):
+            st = lib.mcsd_verify_shard_gather(_ptr(self.p), _ptr(self.q), _ptr(self.tokens), _ptr(m.parent),
+                                              _ptr(m.level_start), m.n_levels, _ptr(self.gamma), self.B, self.N,
+                                              self.Vs, self.v0, self.V_total, _ptr(self.pq), _stream())
+        _check(st, "mcsd_verify_shard_gather")
+
+    def round(self, r: int):
+        m = self.mask
+        with torch.cuda.device(self.p.device):
+            st = lib.mcsd_verify_shard_round(_ptr(self.p), _ptr(self.q), _ptr(m.parent), _ptr(m.level_start),
+                                             m.n_levels, _ptr(self.gamma), _ptr(self.u_accept), _ptr(self.pq),
+                                             _ptr(self.y), r, self.B, self.N, self.Vs, _ptr(self.workspace),
+                                             self.workspace.numel(), _stream())
+        _check(st, "mcsd_verify_shard_round")
+
+    def select(self):
+        m, o = self.mask, self.out
+        with torch.cuda.device(self.p.device):
+            st = lib.mcsd_verify_shard_select(_ptr(self.p), _ptr(self.q), _ptr(self.tokens), m.n_levels, m.n_roots,
+                                              self.B, self.N, self.Vs, self.v0, self.V_total, self.rank, self.world,
+                                              _ptr(o["accept_len"]), _ptr(o["out_tokens"]), _ptr(o["out_nodes"]),
+                                              _ptr(o["best_root"]), _ptr(self.mass), _ptr(self.workspace),
+                                              self.workspace.numel(), _stream())
+        _check(st, "mcsd_verify_shard_select")
+
+    def pick(self):
+        m = self.mask
+        with torch.cuda.device(self.p.device):
+            st = lib.mcsd_verify_shard_pick(_ptr(self.p), _ptr(self.q), _ptr(self.u_bonus), m.n_levels, self.B,
+                                            self.N, self.Vs, self.v0, self.V_total, self.rank, self.world,
+                                            _ptr(self.mass), _ptr(self.out["out_tokens"]), _ptr(self.workspace),
+                                            self.workspace.numel(), _stream())
+        _check(st, "mcsd_verify_shard_pick")
 
 
 def shard_batch(B: int, rank: int, world_size: int):

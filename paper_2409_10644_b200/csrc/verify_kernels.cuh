@@ -450,8 +450,9 @@ struct CdfScratch {
     int found;
     double total;
 };
+// pass 1: per-warp range sums and last id with mass, left in the scratch; ends with a block barrier
 template <int E, typename Load>
-__device__ int block_inverse_cdf(const Load& load, float u, int V, CdfScratch* sc, double* total_out) {
+__device__ void cdf_range_sums(const Load& load, int V, CdfScratch* sc) {
     constexpr int kStride = 32 * E;             // ids one warp covers per step
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int span = ((V + kVerifyWarps - 1) / kVerifyWarps + kStride - 1) / kStride * kStride;
@@ -474,11 +475,21 @@ __device__ int block_inverse_cdf(const Load& load, float u, int V, CdfScratch* s
         if (lane == 0) { sc->tot[warp] = (double)acc; sc->last[warp] = last; }
     }
     __syncthreads();
+}
+
+// pass 2, after cdf_range_sums: the smallest id whose running sum exceeds the target, which is t itself when
+// `absolute` and t * (total mass) otherwise; the last id with mass (V - 1 if there is none) if nothing exceeds it.
+// Every thread of the block must call it; all get the id, and *total_out the total mass.
+template <int E, typename Load>
+__device__ int cdf_locate(const Load& load, double t, bool absolute, int V, CdfScratch* sc, double* total_out) {
+    constexpr int kStride = 32 * E;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int span = ((V + kVerifyWarps - 1) / kVerifyWarps + kStride - 1) / kStride * kStride;
     if (warp == 0) {
         double total = 0.0;
         int last_pos = -1;
         for (int w = 0; w < kVerifyWarps; ++w) { total += sc->tot[w]; last_pos = max(last_pos, sc->last[w]); }
-        const double target = (double)u * total;
+        const double target = absolute ? t : t * total;
         double base = 0.0;
         int w0 = 0;
         while (w0 < kVerifyWarps && !(base + sc->tot[w0] > target)) { base += sc->tot[w0]; ++w0; }
@@ -495,8 +506,8 @@ __device__ int block_inverse_cdf(const Load& load, float u, int V, CdfScratch* s
                 float incl = ls;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
-                    const float t = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (lane >= o) incl += t;
+                    const float t2 = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += t2;
                 }
                 const bool hit = (base + (double)incl > target) && idx < hi;
                 const unsigned ballot = __ballot_sync(0xffffffffu, hit);
@@ -527,6 +538,12 @@ __device__ int block_inverse_cdf(const Load& load, float u, int V, CdfScratch* s
     __syncthreads();
     *total_out = sc->total;
     return sc->found;
+}
+
+template <int E, typename Load>
+__device__ int block_inverse_cdf(const Load& load, float u, int V, CdfScratch* sc, double* total_out) {
+    cdf_range_sums<E>(load, V, sc);
+    return cdf_locate<E>(load, (double)u, false, V, sc, total_out);
 }
 
 template <typename Rows>

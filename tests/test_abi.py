@@ -107,6 +107,45 @@ def test_verify_argument_checks(m):
     assert call(wsb=8) == -5
 
 
+def test_verify_shard_argument_checks(m):
+    L = m.lib
+    assert L.mcsd_verify_shard_workspace_bytes(16, 45) >= 256 + 16 * 45 * (16 + 24) + 16 * 8
+    assert L.mcsd_verify_shard_workspace_bytes(0, 45) == 0
+
+    def gather(p=FAKE, B=2, N=15, Vs=50, v0=0, Vt=100, nl=4):
+        return L.mcsd_verify_shard_gather(p, FAKE, FAKE, FAKE, FAKE, nl, None, B, N, Vs, v0, Vt, FAKE, None)
+    assert gather(p=None) == -1
+    assert gather(N=193) == -2
+    assert gather(Vs=0) == -2
+    assert gather(v0=60) == -2               # columns 60..110 of a 100-id vocabulary
+    assert gather(v0=-4) == -2
+    assert gather(nl=0) == -2
+
+    def rnd(y=FAKE, rd=0, B=2, N=15, Vs=50, wsb=1 << 20):
+        return L.mcsd_verify_shard_round(FAKE, FAKE, FAKE, FAKE, 4, None, FAKE, FAKE, y, rd, B, N, Vs, FAKE, wsb, None)
+    assert rnd(y=None) == -1
+    assert rnd(rd=-1) == -2
+    assert rnd(rd=16) == -2
+    assert rnd(B=0) == -2
+    assert rnd(wsb=64) == -5
+
+    def select(mass=FAKE, rank=0, world=2, nr=1, wsb=1 << 20):
+        return L.mcsd_verify_shard_select(FAKE, FAKE, FAKE, 4, nr, 2, 15, 50, 0, 100, rank, world, FAKE, FAKE, FAKE, FAKE,
+                                          mass, FAKE, wsb, None)
+    assert select(mass=None) == -1
+    assert select(rank=2) == -2
+    assert select(world=0) == -2
+    assert select(nr=0) == -2
+    assert select(wsb=64) == -5
+
+    def pick(u=FAKE, rank=1, world=2, wsb=1 << 20):
+        return L.mcsd_verify_shard_pick(FAKE, FAKE, u, 4, 2, 15, 50, 50, 100, rank, world, FAKE, FAKE, FAKE, wsb, None)
+    assert pick(u=None) == -1
+    assert pick(rank=-1) == -2
+    assert pick(world=2000) == -2
+    assert pick(wsb=64) == -5
+
+
 def test_verify_logits_argument_checks(m):
     L = m.lib
 

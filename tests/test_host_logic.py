@@ -116,3 +116,179 @@ def test_paper_shaped_workloads_and_early_stop_gammas():
         assert g.min() >= 1 and g.max() <= 5
         seen |= set(g.tolist())
     assert len(seen) >= 3
+
+
+# ----------------------------------------------------------------------------------------------
+# vocabulary-sharded verify: column ranges, and the exchange protocol over two gloo ranks
+# ----------------------------------------------------------------------------------------------
+
+def test_vocab_shard_ranges_cover_the_vocabulary():
+    from paper_2409_10644_b200.dist import max_children, vocab_shard_range
+    for V in (33, 1000, 32000, 32001, 128256):
+        for ws in (1, 2, 3, 8):
+            spans = [vocab_shard_range(V, r, ws) for r in range(ws)]
+            assert spans[0][0] == 0 and spans[-1][1] == V
+            assert all(spans[i][1] == spans[i + 1][0] for i in range(ws - 1))
+            assert all(lo % 4 == 0 and hi > lo for lo, hi in spans)
+    with pytest.raises(ValueError):
+        vocab_shard_range(13, 0, 5)          # four 4-id units cannot feed five ranks
+    with pytest.raises(ValueError):
+        vocab_shard_range(100, 2, 2)
+    assert max_children(parent_array(1, (4, 2, 2, 1))) == 4
+    assert max_children(parent_array(8, (1, 2, 2))) == 2
+    assert max_children(np.array([-1])) == 0
+
+
+class _CpuShard:
+    """Test-side stand-in for one rank's kernels (numpy, fp64) with the interface the driver expects, so that the
+    order of launches and reductions can be exercised over a CPU process group.  It restates what the four
+    per-rank steps exchange; the product has no such path."""
+
+    def __init__(self, p, q, v0, V_total, rank, world, tokens, parent, ua, ub):
+        self.p, self.q, self.v0, self.V, self.rank, self.world = p, q, v0, V_total, rank, world
+        self.tokens, self.parent, self.ua, self.ub = tokens, parent, ua, ub
+        B, N, _ = p.shape
+        self.B, self.N = B, N
+        self.kids = [[c for c in range(N) if parent[c] == u] for u in range(N)]
+        self.pq = torch.zeros((B, N, 2), dtype=torch.float64)
+        self.y = torch.zeros((B, N), dtype=torch.float64)
+        self.mass = torch.zeros((world, B, 2), dtype=torch.float64)
+        nl = int(orc.tree_levels(parent)[0].max()) + 1
+        self.nl = nl
+        self.out = {"accept_len": torch.zeros(B, dtype=torch.int32), "out_tokens": torch.full((B, nl + 1), -1, dtype=torch.int32),
+                    "out_nodes": torch.full((B, nl), -1, dtype=torch.int32), "best_root": torch.zeros(B, dtype=torch.int32)}
+
+    def gather(self):
+        self.pq.zero_()
+        for b in range(self.B):
+            for c in range(self.N):
+                u, x = self.parent[c], int(self.tokens[b, c]) - self.v0
+                if u >= 0 and 0 <= x < self.p.shape[2]:
+                    self.pq[b, c, 0], self.pq[b, c, 1] = self.p[b, u, x], self.q[b, u, x]
+
+    def round(self, r):
+        if r == 0:
+            self.stage = np.array([[0 if self.kids[u] else -1 for u in range(self.N)]] * self.B)
+            self.pend = np.zeros((self.B, self.N), dtype=bool)
+            self.c = np.zeros((self.B, self.N))
+            self.Y = np.ones((self.B, self.N))
+            self.next = -np.ones((self.B, self.N), dtype=int)
+            self.stop_c = np.zeros((self.B, self.N))
+        y_in = self.y.numpy().copy()
+        self.y.zero_()
+        for b in range(self.B):
+            for u in range(self.N):
+                if self.stage[b, u] < 0:
+                    continue
+                if self.pend[b, u]:
+                    Y = y_in[b, u]
+                    if not Y > 0:
+                        self.c[b, u], Y = 0.0, 1.0
+                    self.Y[b, u], self.pend[b, u] = Y, False
+                    self.stage[b, u] += 1
+                if self.stage[b, u] >= len(self.kids[u]):
+                    self.stop_c[b, u], self.stage[b, u] = self.c[b, u], -1
+                    continue
+                child = self.kids[u][self.stage[b, u]]
+                px, qx = float(self.pq[b, child, 0]), float(self.pq[b, child, 1])
+                num = max(px - self.c[b, u] * qx, 0.0)
+                acc = min(1.0, num / (self.Y[b, u] * qx)) if qx > 0 else (1.0 if num > 0 else 0.0)
+                if self.ua[b, child] < acc:
+                    self.next[b, u], self.stage[b, u] = child, -1
+                else:
+                    self.c[b, u] += self.Y[b, u]
+                    self.pend[b, u] = True
+                    self.y[b, u] = float(np.maximum(self.p[b, u] - self.c[b, u] * self.q[b, u], 0.0).sum())
+
+    def _dist(self, b, u):
+        return np.maximum(self.p[b, u] - self.stop_c[b, u] * self.q[b, u], 0.0)
+
+    def select(self):
+        self.mass.zero_()
+        self.stop, self.slot = [], []
+        roots = [n for n in range(self.N) if self.parent[n] < 0]
+        for b in range(self.B):
+            paths = []
+            for r in roots:
+                u, path = r, []
+                while self.next[b, u] >= 0:
+                    u = int(self.next[b, u])
+                    path.append(u)
+                paths.append(path)
+            best = max(range(len(roots)), key=lambda i: (len(paths[i]), -i))
+            toks = ([int(self.tokens[b, roots[best]])] if len(roots) > 1 else []) + [int(self.tokens[b, n]) for n in paths[best]]
+            self.out["accept_len"][b], self.out["best_root"][b] = len(paths[best]), best
+            self.out["out_tokens"][b] = -1
+            self.out["out_nodes"][b] = -1
+            self.out["out_tokens"][b, :len(toks)] = torch.tensor(toks, dtype=torch.int32)
+            self.out["out_nodes"][b, :len(paths[best])] = torch.tensor(paths[best], dtype=torch.int32)
+            u = paths[best][-1] if paths[best] else roots[best]
+            self.stop.append(u)
+            self.slot.append(len(toks))
+            d = self._dist(b, u)
+            pos = np.nonzero(d > 0)[0]
+            self.mass[self.rank, b, 0] = float(d.sum())
+            self.mass[self.rank, b, 1] = float(self.v0 + pos[-1] + 1) if pos.size else 0.0
+
+    def pick(self):
+        for b in range(self.B):
+            u = self.stop[b]
+            masses = self.mass[:, b, 0].numpy()
+            target = float(self.ub[b, u]) * float(masses.sum())
+            base, owner = 0.0, -1
+            for r in range(self.world):
+                if base + masses[r] > target:
+                    owner = r
+                    break
+                base += masses[r]
+            tok = -1
+            if owner < 0:
+                last = float(self.mass[:, b, 1].max())
+                tok = int(last) - 1 if last > 0 else self.V - 1
+            elif owner == self.rank:
+                cs = base + np.cumsum(self._dist(b, u))
+                tok = self.v0 + int(np.nonzero(cs > target)[0][0])
+            self.out["out_tokens"][b, self.slot[b]] = tok
+
+
+def _vocab_rank_main(rank, world, port, q):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2409_10644_b200.dist import _all_reduce_group, drive_vocab_shards, max_children, vocab_shard_range
+    rng = np.random.default_rng(11)
+    B, V = 6, 40
+    ok = True
+    for parent in (parent_array(1, (3, 2)), parent_array(2, (2, 1, 1))):
+        N = len(parent)
+        x = rng.random((B, N, V)) ** 4 + 1e-6
+        p = x / x.sum(-1, keepdims=True)
+        y = rng.random((B, N, V)) ** 4 + 1e-6
+        qq = y / y.sum(-1, keepdims=True)
+        tokens = rng.integers(0, V, (B, N))
+        ua, ub = rng.random((B, N)), rng.random((B, N))
+        v0, v1 = vocab_shard_range(V, rank, world)
+        shard = _CpuShard(p[:, :, v0:v1], qq[:, :, v0:v1], v0, V, rank, world, tokens, parent, ua, ub)
+        out = drive_vocab_shards([shard], _all_reduce_group(None), max_children(parent))[0]
+        full = orc.verify_tree(p, qq, tokens, parent, None, ua, ub)
+        for key in ("accept_len", "out_tokens", "out_nodes", "best_root"):     # every rank holds the whole result
+            ok &= bool(np.array_equal(out[key].numpy(), full[key]))
+    flags = [None] * world
+    dist.all_gather_object(flags, ok)
+    if rank == 0:
+        q.put(all(flags))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_vocab_sharded_verify_protocol_over_gloo(m):
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_vocab_rank_main, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    ok = q.get(timeout=120)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert ok
