@@ -391,6 +391,9 @@ def run_ours(args):
                       "tree_tokens_per_s_per_layer": float(n_act.sum()) / (attn_ms * 1e-3),
                       "mean_accept_len": float(vout["accept_len"].float().mean().item())},
     }
+    if world == 1 and args.vocab_shards > 1:
+        line["breakdown"]["vocab_sharded_verify"] = _time_vocab_sharded_verify(mcsd, w, vin, tm, gam_d, parent,
+                                                                               args.vocab_shards, vout)
     if world == 1 and not args.no_cpu_baseline:
         v, sample, threads, _ = oracle_sample(w0)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample}
@@ -398,6 +401,44 @@ def run_ours(args):
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def _time_vocab_sharded_verify(mcsd, w, vin, tm, gam_d, parent, R, vout):
+    """Kernel time of the vocabulary-sharded verify step with the R ranks' column slices all on this GPU: the ranks'
+    launches run one after the other in one stream, the all-reduces are replaced by combining the exchange buffers
+    on the device, and the whole sequence is replayed from a CUDA graph so that the host's launch path is not in the
+    number.  `ms_per_rank` = total / R still contains the stand-in reductions, so it bounds one rank's kernels from
+    above; a real job adds k + 3 small all-reduces."""
+    import torch
+    from paper_2409_10644_b200 import dist as mdist
+    k = mdist.max_children(parent)
+    shards = []
+    for r in range(R):
+        v0, v1 = mdist.vocab_shard_range(w.V, r, R)
+        shards.append(mcsd.VocabShard(vin["p"][:, :, v0:v1].contiguous(), vin["q"][:, :, v0:v1].contiguous(), v0, w.V,
+                                      r, R, vin["tokens"], tm, gam_d, vin["u_accept"], vin["u_bonus"]))
+    l0 = mcsd.mcsd_launch_count()
+    outs = mdist.drive_vocab_shards(shards, mdist.reduce_on_one_device, k)
+    launches = mcsd.mcsd_launch_count() - l0
+    torch.cuda.synchronize()
+    same = all(bool(torch.equal(o[key], vout[key])) for o in outs
+               for key in ("accept_len", "out_tokens", "out_nodes", "best_root"))
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        mdist.drive_vocab_shards(shards, mdist.reduce_on_one_device, k)
+    for _ in range(3):
+        g.replay()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 20
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(reps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    total = e0.elapsed_time(e1) / reps
+    return {"ranks_on_one_gpu": R, "rounds": k + 1, "all_reduces_per_step": k + 3, "launches_all_ranks": int(launches),
+            "ms_all_ranks": total, "ms_per_rank": total / R, "matches_single_gpu_outputs": same}
 
 
 def main():
@@ -410,6 +451,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling of a smaller case only)")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling only)")
+    ap.add_argument("--vocab-shards", type=int, default=0,
+                    help="also time the vocabulary-sharded verify step with this many ranks' column slices on one GPU")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
