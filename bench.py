@@ -173,7 +173,7 @@ def run_reference(args):
     w = workload(args.workload)
     vals = []
     for i in range(args.warmup + args.steps):
-        v, sample, threads, step_s = oracle_sample(w, budget_s=max(2.0, 60.0 / max(1, args.warmup + args.steps)))
+        v, sample, threads, step_s = oracle_sample(w, budget_s=max(2.0, 36.0 / max(1, args.warmup + args.steps)))
         if i >= args.warmup:
             vals.append((v, step_s))
     value = float(np.mean([v for v, _ in vals]))
