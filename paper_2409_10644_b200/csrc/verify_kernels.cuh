@@ -93,6 +93,24 @@ struct ProbDist {
             for (int i = 0; i < 4; ++i) r[i] = fmaxf(fmaf(-c, b[i], r[i]), 0.f);
         }
     }
+    // The same values in two steps, for row passes that issue the loads of several steps before using any of
+    // them (only for rows that allow 128-bit loads): PLAIN = the row p itself (c == 0), no draft row needed.
+    __device__ __forceinline__ bool plain() const { return c == 0.f; }
+    template <bool PLAIN> __device__ __forceinline__ void fetch(int idx, float (&a)[4], float (&b)[4]) const {
+        const float4 t = __ldg(reinterpret_cast<const float4*>(p + idx));
+        a[0] = t.x; a[1] = t.y; a[2] = t.z; a[3] = t.w;
+        if constexpr (!PLAIN) {
+            const float4 s = __ldg(reinterpret_cast<const float4*>(q + idx));
+            b[0] = s.x; b[1] = s.y; b[2] = s.z; b[3] = s.w;
+        }
+    }
+    template <bool PLAIN> __device__ __forceinline__ void finish(const float (&a)[4], const float (&b)[4], float (&r)[4]) const {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if constexpr (PLAIN) r[i] = a[i];
+            else r[i] = fmaxf(fmaf(-c, b[i], a[i]), 0.f);
+        }
+    }
 };
 
 struct ProbRows {
@@ -133,6 +151,10 @@ template <> struct LogitLoad<float> {
             for (int i = 0; i < 4; ++i) r[i] = idx + i < V ? __ldg(row + idx + i) : -INFINITY;
         }
     }
+    __device__ __forceinline__ static void load_vec(const float* __restrict__ row, int idx, float (&r)[4]) {
+        const float4 t = __ldg(reinterpret_cast<const float4*>(row + idx));
+        r[0] = t.x; r[1] = t.y; r[2] = t.z; r[3] = t.w;
+    }
     __device__ __forceinline__ static float one(const float* row, int x) { return row[x]; }
 };
 template <> struct LogitLoad<__nv_bfloat16> {
@@ -149,6 +171,15 @@ template <> struct LogitLoad<__nv_bfloat16> {
         } else {
 #pragma unroll
             for (int i = 0; i < 8; ++i) r[i] = idx + i < V ? __bfloat162float(row[idx + i]) : -INFINITY;
+        }
+    }
+    __device__ __forceinline__ static void load_vec(const __nv_bfloat16* __restrict__ row, int idx, float (&r)[8]) {
+        const uint4 t = __ldg(reinterpret_cast<const uint4*>(row + idx));
+        const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            r[2 * i] = __uint_as_float(w[i] << 16);
+            r[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
         }
     }
     __device__ __forceinline__ static float one(const __nv_bfloat16* row, int x) { return __bfloat162float(row[x]); }
@@ -192,23 +223,55 @@ template <typename T> struct LogitDist {
         }
     }
 
+    __device__ __forceinline__ bool plain() const { return cq == 0.f; }
+    template <bool PLAIN> __device__ __forceinline__ void fetch(int idx, float (&a)[E], float (&b)[E]) const {
+        LogitLoad<T>::load_vec(zt, idx, a);
+        if constexpr (!PLAIN) LogitLoad<T>::load_vec(zd, idx, b);
+    }
+    template <bool PLAIN> __device__ __forceinline__ void finish(const float (&a)[E], const float (&b)[E], float (&r)[E]) const {
+#pragma unroll
+        for (int i = 0; i < E; ++i) {
+            r[i] = ex2f((a[i] - mt) * k) * ip;
+            if constexpr (!PLAIN) r[i] = fmaxf(fmaf(-cq, ex2f((b[i] - md) * k), r[i]), 0.f);
+        }
+    }
+
     // maxima and normalisers of both rows; every thread of the block must call it
     __device__ void stats(VerifyScratch* sc) {
         float m[2] = {-INFINITY, -INFINITY}, s[2] = {0.f, 0.f};
-        for (int idx = threadIdx.x * E; idx < V; idx += kVerifyThreads * E) {
+        const float kk = k;
+        auto fold = [&m, &s, kk](int row, const float (&a)[E]) {
+            float vm = a[0];
+#pragma unroll
+            for (int i = 1; i < E; ++i) vm = fmaxf(vm, a[i]);
+            if (vm == -INFINITY) return;
+            if (vm > m[row]) { s[row] *= ex2f((m[row] - vm) * kk); m[row] = vm; }
+            float e[E];
+#pragma unroll
+            for (int i = 0; i < E; ++i) e[i] = ex2f((a[i] - m[row]) * kk);
+            s[row] += tree_sum<E>(e);
+        };
+        constexpr int kStep = kVerifyThreads * E;
+        constexpr int kBatch = 4;              // steps whose loads are issued before the first one is folded in
+        int idx = threadIdx.x * E;
+        if (vec) {
+            for (; idx + (kBatch - 1) * kStep < V; idx += kBatch * kStep) {
+                float at[kBatch][E], ad[kBatch][E];
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) {
+                    LogitLoad<T>::load_vec(zt, idx + j * kStep, at[j]);
+                    LogitLoad<T>::load_vec(zd, idx + j * kStep, ad[j]);
+                }
+#pragma unroll
+                for (int j = 0; j < kBatch; ++j) { fold(0, at[j]); fold(1, ad[j]); }
+            }
+        }
+        for (; idx < V; idx += kStep) {
 #pragma unroll
             for (int row = 0; row < 2; ++row) {
                 float a[E];
                 LogitLoad<T>::load(row == 0 ? zt : zd, idx, V, vec, a);
-                float vm = a[0];
-#pragma unroll
-                for (int i = 1; i < E; ++i) vm = fmaxf(vm, a[i]);
-                if (vm == -INFINITY) continue;
-                if (vm > m[row]) { s[row] *= ex2f((m[row] - vm) * k); m[row] = vm; }
-                float e[E];
-#pragma unroll
-                for (int i = 0; i < E; ++i) e[i] = ex2f((a[i] - m[row]) * k);
-                s[row] += tree_sum<E>(e);
+                fold(row, a);
             }
         }
 #pragma unroll
@@ -268,14 +331,49 @@ template <typename T> struct LogitRows {
 // row passes shared by both kernels
 // ------------------------------------------------------------------------------------------------------
 
+// Row passes are latency-bound for a single block (one step = one dependent trip to memory), so they run
+// kRowBatch steps at a time: all loads of the batch are issued before the first value is used.  The additions
+// keep the order of the plain loop, so the sums are the same bit for bit.
+constexpr int kRowBatch = 4;
+
+// this thread's part of sum_v dist_v: ids first, first + step, ... below end
+template <bool PLAIN, typename Dist>
+__device__ __forceinline__ float strided_sum(const Dist& d, int first, int step, int end) {
+    constexpr int E = Dist::E;
+    float acc = 0.f;
+    int idx = first;
+    for (; idx + (kRowBatch - 1) * step < end; idx += kRowBatch * step) {
+        float a[kRowBatch][E], b[kRowBatch][E];
+#pragma unroll
+        for (int j = 0; j < kRowBatch; ++j) d.template fetch<PLAIN>(idx + j * step, a[j], b[j]);
+#pragma unroll
+        for (int j = 0; j < kRowBatch; ++j) {
+            float r[E];
+            d.template finish<PLAIN>(a[j], b[j], r);
+            acc += tree_sum<E>(r);
+        }
+    }
+    for (; idx < end; idx += step) {
+        float r[E];
+        d.load(idx, r);
+        acc += tree_sum<E>(r);
+    }
+    return acc;
+}
+
 // sum_v dist_v over one row, same value in every thread of the block
 template <typename Dist> __device__ double dist_mass(const Dist& d, VerifyScratch* sc) {
     constexpr int E = Dist::E;
     float acc = 0.f;
-    for (int idx = threadIdx.x * E; idx < d.V; idx += kVerifyThreads * E) {
-        float r[E];
-        d.load(idx, r);
-        acc += tree_sum<E>(r);
+    if (d.vec) {
+        acc = d.plain() ? strided_sum<true>(d, threadIdx.x * E, kVerifyThreads * E, d.V)
+                        : strided_sum<false>(d, threadIdx.x * E, kVerifyThreads * E, d.V);
+    } else {
+        for (int idx = threadIdx.x * E; idx < d.V; idx += kVerifyThreads * E) {
+            float r[E];
+            d.load(idx, r);
+            acc += tree_sum<E>(r);
+        }
     }
     acc = warp_sum(acc);
     __syncthreads();                       // the scratch may still be read from a previous pass
@@ -477,6 +575,65 @@ __device__ void cdf_range_sums(const Load& load, int V, CdfScratch* sc) {
     __syncthreads();
 }
 
+// pass 1 for a Dist whose values `post(idx, r)` may still edit (e.g. to drop ids): batched loads when the rows
+// allow 128-bit loads (see strided_sum), the plain pass otherwise.  Same sums as cdf_range_sums bit for bit.
+template <bool PLAIN, typename Dist, typename Post>
+__device__ __forceinline__ void range_sum_batched(const Dist& d, const Post& post, int first, int step, int end,
+                                                  float& acc, int& last) {
+    constexpr int E = Dist::E;
+    int idx = first;
+    for (; idx + (kRowBatch - 1) * step < end; idx += kRowBatch * step) {
+        float a[kRowBatch][E], b[kRowBatch][E];
+#pragma unroll
+        for (int j = 0; j < kRowBatch; ++j) d.template fetch<PLAIN>(idx + j * step, a[j], b[j]);
+#pragma unroll
+        for (int j = 0; j < kRowBatch; ++j) {
+            float r[E];
+            d.template finish<PLAIN>(a[j], b[j], r);
+            post(idx + j * step, r);
+            acc += tree_sum<E>(r);
+#pragma unroll
+            for (int i = 0; i < E; ++i)
+                if (r[i] > 0.f) last = idx + j * step + i;
+        }
+    }
+    for (; idx < end; idx += step) {
+        float r[E];
+        d.load(idx, r);
+        post(idx, r);
+        acc += tree_sum<E>(r);
+#pragma unroll
+        for (int i = 0; i < E; ++i)
+            if (r[i] > 0.f) last = idx + i;
+    }
+}
+
+template <typename Dist, typename Post>
+__device__ void cdf_range_sums_dist(const Dist& d, const Post& post, int V, CdfScratch* sc) {
+    constexpr int E = Dist::E;
+    if (!d.vec) {
+        auto load = [&d, &post](int idx, float (&r)[E]) { d.load(idx, r); post(idx, r); };
+        cdf_range_sums<E>(load, V, sc);
+        return;
+    }
+    constexpr int kStride = 32 * E;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int span = ((V + kVerifyWarps - 1) / kVerifyWarps + kStride - 1) / kStride * kStride;
+    __syncthreads();                            // the scratch may still be read from a previous call
+    {
+        const int lo = warp * span, hi = min(V, lo + span);
+        float acc = 0.f;
+        int last = -1;
+        if (d.plain()) range_sum_batched<true>(d, post, lo + lane * E, kStride, hi, acc, last);
+        else range_sum_batched<false>(d, post, lo + lane * E, kStride, hi, acc, last);
+        acc = warp_sum(acc);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) last = max(last, __shfl_xor_sync(0xffffffffu, last, o));
+        if (lane == 0) { sc->tot[warp] = (double)acc; sc->last[warp] = last; }
+    }
+    __syncthreads();
+}
+
 // pass 2, after cdf_range_sums: the smallest id whose running sum exceeds the target, which is t itself when
 // `absolute` and t * (total mass) otherwise; the last id with mass (V - 1 if there is none) if nothing exceeds it.
 // Every thread of the block must call it; all get the id, and *total_out the total mass.
@@ -571,8 +728,10 @@ verify_select_kernel(Rows rows, const int32_t* __restrict__ tokens, const NodeSt
 
     // ---- new token: inverse CDF over dist_v = max(p_v - c q_v, 0) in token-id order ----
     auto load = [&d](int idx, float (&r)[E]) { d.load(idx, r); };
+    auto keep = [](int, float (&)[E]) {};
     double total;
-    const int found = block_inverse_cdf<E>(load, u_bonus[(size_t)b * N + u], V, &s_cdf, &total);
+    cdf_range_sums_dist(d, keep, V, &s_cdf);
+    const int found = cdf_locate<E>(load, (double)u_bonus[(size_t)b * N + u], false, V, &s_cdf, &total);
     if (tid == 0) out_tokens[(size_t)b * (n_levels + 1) + s_slot] = found;
 
     // ---- optional: the R most probable ids of the same distribution ----
@@ -601,8 +760,7 @@ sample_roots_kernel(Rows rows, const NodeState* __restrict__ state, const int32_
     d.set_c(state[(size_t)b * N + u].c);
     for (int i = 0; i < R; ++i) {
         const int* picks = s_pick;
-        auto load = [&d, i, picks](int idx, float (&r)[E]) {
-            d.load(idx, r);
+        auto drop = [i, picks](int idx, float (&r)[E]) {
             for (int j = 0; j < i; ++j) {                    // ids already drawn carry no mass any more
                 const int e = picks[j] - idx;
 #pragma unroll
@@ -610,8 +768,10 @@ sample_roots_kernel(Rows rows, const NodeState* __restrict__ state, const int32_
                     if (e == k) r[k] = 0.f;
             }
         };
+        auto load = [&d, &drop](int idx, float (&r)[E]) { d.load(idx, r); drop(idx, r); };
         double total;
-        int tok = block_inverse_cdf<E>(load, u_roots[(size_t)b * R + i], V, &s_cdf, &total);
+        cdf_range_sums_dist(d, drop, V, &s_cdf);
+        int tok = cdf_locate<E>(load, (double)u_roots[(size_t)b * R + i], false, V, &s_cdf, &total);
         if (!(total > 0.0)) {                                 // nothing left: the rest of the list is empty
             for (int j = i + tid; j < R; j += kVerifyThreads) next_roots[(size_t)b * R + j] = -1;
             break;

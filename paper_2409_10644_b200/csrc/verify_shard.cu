@@ -167,8 +167,8 @@ verify_shard_select_kernel(ProbRows rows, const int32_t* __restrict__ tokens, co
     const int u = s_stop;
     ProbDist d = rows.open(b, u, N, Vs, &s_scratch);
     d.set_c(st[u].c);
-    auto load = [&d](int idx, float (&r)[E]) { d.load(idx, r); };
-    cdf_range_sums<E>(load, Vs, &s_cdf);
+    auto keep = [](int, float (&)[E]) {};
+    cdf_range_sums_dist(d, keep, Vs, &s_cdf);
     if (tid == 0) {
         double total = 0.0;
         int last = -1;
@@ -214,7 +214,8 @@ verify_shard_pick_kernel(ProbRows rows, const NodeState* __restrict__ state, con
         ProbDist d = rows.open(b, u, N, Vs, &s_scratch);
         d.set_c(state[(size_t)b * N + u].c);
         auto load = [&d](int idx, float (&r)[E]) { d.load(idx, r); };
-        cdf_range_sums<E>(load, Vs, &s_cdf);
+        auto keep = [](int, float (&)[E]) {};
+        cdf_range_sums_dist(d, keep, Vs, &s_cdf);
         double local_total;
         tok = v0 + cdf_locate<E>(load, target - base, true, Vs, &s_cdf, &local_total);
     }
