@@ -411,7 +411,11 @@ verify_nodes_kernel(Rows rows, const int32_t* __restrict__ tokens, const int32_t
                     const float* __restrict__ u_accept, int N, int V, NodeState* __restrict__ state) {
     __shared__ int s_first, s_cnt, s_accept;
     __shared__ VerifyScratch s_scratch;
-    const int b = blockIdx.y, u = blockIdx.x, tid = threadIdx.x;
+    // Blocks are handed out in the order of their linear index; taking the node from its upper part starts all
+    // sequences' nodes level by level, so the nodes with the most siblings to try run first and the leaves,
+    // which have nothing to do, last.
+    const int lin = blockIdx.y * gridDim.x + blockIdx.x;
+    const int b = lin % (int)gridDim.y, u = lin / (int)gridDim.y, tid = threadIdx.x;
     const int n_act = active_nodes(gamma, level_start, n_levels, b, N);
     if (u >= n_act) return;
     int first, cnt;
