@@ -30,7 +30,21 @@ greedy_nodes_kernel(const T* __restrict__ zt, const int32_t* __restrict__ tokens
     const bool vec = (V % E == 0) && (reinterpret_cast<uintptr_t>(row) % 16 == 0);
     float bv = 0.f;
     int bi = -1;
-    for (int idx = tid * E; idx < V; idx += kVerifyThreads * E) {
+    int idx = tid * E;
+    if (vec) {                                   // several steps' loads in flight at once, compared in id order
+        constexpr int kStep = kVerifyThreads * E;
+        for (; idx + (kRowBatch - 1) * kStep < V; idx += kRowBatch * kStep) {
+            float a[kRowBatch][E];
+#pragma unroll
+            for (int j = 0; j < kRowBatch; ++j) LogitLoad<T>::load_vec(row, idx + j * kStep, a[j]);
+#pragma unroll
+            for (int j = 0; j < kRowBatch; ++j)
+#pragma unroll
+                for (int i = 0; i < E; ++i)
+                    if (bi < 0 || a[j][i] > bv) { bv = a[j][i]; bi = idx + j * kStep + i; }
+        }
+    }
+    for (; idx < V; idx += kVerifyThreads * E) {
         float a[E];
         LogitLoad<T>::load(row, idx, V, vec, a);
 #pragma unroll
