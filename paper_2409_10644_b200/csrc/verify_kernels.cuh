@@ -252,7 +252,7 @@ template <typename T> struct LogitDist {
             s[row] += tree_sum<E>(e);
         };
         constexpr int kStep = kVerifyThreads * E;
-        constexpr int kBatch = 4;              // steps whose loads are issued before the first one is folded in
+        constexpr int kBatch = E == 8 ? 2 : 4;  // steps whose loads are issued before the first one is folded in
         int idx = threadIdx.x * E;
         if (vec) {
             for (; idx + (kBatch - 1) * kStep < V; idx += kBatch * kStep) {
@@ -335,19 +335,21 @@ template <typename T> struct LogitRows {
 // kRowBatch steps at a time: all loads of the batch are issued before the first value is used.  The additions
 // keep the order of the plain loop, so the sums are the same bit for bit.
 constexpr int kRowBatch = 4;
+// two-row passes over 8-id loads keep two steps in flight: four would cost the node kernel half its resident blocks
 
 // this thread's part of sum_v dist_v: ids first, first + step, ... below end
 template <bool PLAIN, typename Dist>
 __device__ __forceinline__ float strided_sum(const Dist& d, int first, int step, int end) {
     constexpr int E = Dist::E;
+    constexpr int NB = E == 8 ? 2 : kRowBatch;
     float acc = 0.f;
     int idx = first;
-    for (; idx + (kRowBatch - 1) * step < end; idx += kRowBatch * step) {
-        float a[kRowBatch][E], b[kRowBatch][E];
+    for (; idx + (NB - 1) * step < end; idx += NB * step) {
+        float a[NB][E], b[NB][E];
 #pragma unroll
-        for (int j = 0; j < kRowBatch; ++j) d.template fetch<PLAIN>(idx + j * step, a[j], b[j]);
+        for (int j = 0; j < NB; ++j) d.template fetch<PLAIN>(idx + j * step, a[j], b[j]);
 #pragma unroll
-        for (int j = 0; j < kRowBatch; ++j) {
+        for (int j = 0; j < NB; ++j) {
             float r[E];
             d.template finish<PLAIN>(a[j], b[j], r);
             acc += tree_sum<E>(r);
@@ -585,13 +587,14 @@ template <bool PLAIN, typename Dist, typename Post>
 __device__ __forceinline__ void range_sum_batched(const Dist& d, const Post& post, int first, int step, int end,
                                                   float& acc, int& last) {
     constexpr int E = Dist::E;
+    constexpr int NB = E == 8 ? 2 : kRowBatch;
     int idx = first;
-    for (; idx + (kRowBatch - 1) * step < end; idx += kRowBatch * step) {
-        float a[kRowBatch][E], b[kRowBatch][E];
+    for (; idx + (NB - 1) * step < end; idx += NB * step) {
+        float a[NB][E], b[NB][E];
 #pragma unroll
-        for (int j = 0; j < kRowBatch; ++j) d.template fetch<PLAIN>(idx + j * step, a[j], b[j]);
+        for (int j = 0; j < NB; ++j) d.template fetch<PLAIN>(idx + j * step, a[j], b[j]);
 #pragma unroll
-        for (int j = 0; j < kRowBatch; ++j) {
+        for (int j = 0; j < NB; ++j) {
             float r[E];
             d.template finish<PLAIN>(a[j], b[j], r);
             post(idx + j * step, r);
