@@ -551,8 +551,8 @@ __device__ void top_ids(const Load& load, int V, int R, int32_t* __restrict__ ds
 struct CdfScratch {
     double tot[kVerifyWarps];
     int last[kVerifyWarps];
-    int found;
-    double total;
+    float ctot[kVerifyWarps];     // locate: totals of the chunks scanned side by side
+    int cand[kVerifyWarps];       // locate: id found in each of them, or -1
 };
 // pass 1: per-warp range sums and last id with mass, left in the scratch; ends with a block barrier
 template <int E, typename Load>
@@ -646,62 +646,72 @@ __device__ void cdf_range_sums_dist(const Dist& d, const Post& post, int V, CdfS
 // Every thread of the block must call it; all get the id, and *total_out the total mass.
 template <int E, typename Load>
 __device__ int cdf_locate(const Load& load, double t, bool absolute, int V, CdfScratch* sc, double* total_out) {
-    constexpr int kStride = 32 * E;
+    constexpr int kStride = 32 * E;             // ids of one chunk: what a warp covers in one step
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int span = ((V + kVerifyWarps - 1) / kVerifyWarps + kStride - 1) / kStride * kStride;
-    if (warp == 0) {
-        double total = 0.0;
-        int last_pos = -1;
-        for (int w = 0; w < kVerifyWarps; ++w) { total += sc->tot[w]; last_pos = max(last_pos, sc->last[w]); }
-        const double target = absolute ? t : t * total;
-        double base = 0.0;
-        int w0 = 0;
-        while (w0 < kVerifyWarps && !(base + sc->tot[w0] > target)) { base += sc->tot[w0]; ++w0; }
-        int found = -1;
-        for (int w = w0; w < kVerifyWarps && found < 0; ++w) {
-            const int lo = w * span, hi = min(V, lo + span);
-            for (int i0 = lo; i0 < hi && found < 0; i0 += kStride) {
-                const int idx = i0 + lane * E;
-                float r[E];
+    // every thread repeats the few additions over the range sums, so all agree without another barrier
+    double total = 0.0;
+    int last_pos = -1;
+    for (int w = 0; w < kVerifyWarps; ++w) { total += sc->tot[w]; last_pos = max(last_pos, sc->last[w]); }
+    const double target = absolute ? t : t * total;
+    double base = 0.0;
+    int w0 = 0;
+    while (w0 < kVerifyWarps && !(base + sc->tot[w0] > target)) { base += sc->tot[w0]; ++w0; }
+    // The running sum is carried chunk by chunk in id order, as a single warp walking the range would do, but
+    // the chunks of a range are loaded and scanned by all warps at once: warp j takes chunk j, the chunk totals
+    // are then added up in order, and the lowest chunk in which the sum passes the target gives the id.
+    int found = -1;
+    for (int w = w0; w < kVerifyWarps && found < 0; ++w) {
+        const int lo = w * span, hi = min(V, lo + span);
+        for (int c0 = lo; c0 < hi && found < 0; c0 += kVerifyWarps * kStride) {
+            const int idx = c0 + warp * kStride + lane * E;
+            float r[E];
 #pragma unroll
-                for (int i = 0; i < E; ++i) r[i] = 0.f;
-                if (idx < hi) load(idx, r);
-                const float ls = tree_sum<E>(r);
-                float incl = ls;
+            for (int i = 0; i < E; ++i) r[i] = 0.f;
+            if (idx < hi) load(idx, r);
+            const float ls = tree_sum<E>(r);
+            float incl = ls;
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const float t2 = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (lane >= o) incl += t2;
-                }
-                const bool hit = (base + (double)incl > target) && idx < hi;
-                const unsigned ballot = __ballot_sync(0xffffffffu, hit);
-                if (ballot != 0u) {
-                    const int L = __ffs(ballot) - 1;
-                    int tok = -1;
-                    if (lane == L) {
-                        const double ex = base + (double)(incl - ls);
-                        float part = 0.f;
-                        bool done = false;
-                        tok = idx + E - 1;
-#pragma unroll
-                        for (int i = 0; i < E - 1; ++i) {        // smallest i whose running sum passes the target
-                            part += r[i];
-                            if (!done && ex + (double)part > target) { tok = idx + i; done = true; }
-                        }
-                        if (tok >= V) tok = V - 1;
-                    }
-                    found = __shfl_sync(0xffffffffu, tok, L);
-                } else {
-                    base += (double)__shfl_sync(0xffffffffu, incl, 31);
-                }
+            for (int o = 1; o < 32; o <<= 1) {
+                const float t2 = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t2;
             }
+            if (lane == 31) sc->ctot[warp] = incl;
+            __syncthreads();
+            double mine = base, all = base;
+            for (int k = 0; k < kVerifyWarps; ++k) {
+                if (k == warp) mine = all;
+                all += (double)sc->ctot[k];
+            }
+            const bool hit = (mine + (double)incl > target) && idx < hi;
+            const unsigned ballot = __ballot_sync(0xffffffffu, hit);
+            int tok = -1;
+            if (ballot != 0u) {
+                const int L = __ffs(ballot) - 1;
+                if (lane == L) {
+                    const double ex = mine + (double)(incl - ls);
+                    float part = 0.f;
+                    bool done = false;
+                    tok = idx + E - 1;
+#pragma unroll
+                    for (int i = 0; i < E - 1; ++i) {        // smallest i whose running sum passes the target
+                        part += r[i];
+                        if (!done && ex + (double)part > target) { tok = idx + i; done = true; }
+                    }
+                    if (tok >= V) tok = V - 1;
+                }
+                tok = __shfl_sync(0xffffffffu, tok, L);
+            }
+            if (lane == 0) sc->cand[warp] = tok;
+            __syncthreads();
+            for (int k = 0; k < kVerifyWarps && found < 0; ++k) found = sc->cand[k];
+            base = all;
+            __syncthreads();                        // the chunk scratch is rewritten in the next step
         }
-        if (found < 0) found = last_pos >= 0 ? last_pos : V - 1;
-        if (lane == 0) { sc->found = found; sc->total = total; }
     }
-    __syncthreads();
-    *total_out = sc->total;
-    return sc->found;
+    if (found < 0) found = last_pos >= 0 ? last_pos : V - 1;
+    *total_out = total;
+    return found;
 }
 
 template <int E, typename Load>
