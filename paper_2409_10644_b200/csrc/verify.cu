@@ -29,10 +29,9 @@ extern "C" int mcsd_verify_tree(const float* p, const float* q, const int32_t* t
     mcsd::verify_nodes_kernel<mcsd::ProbRows><<<dim3(N, B), mcsd::kVerifyThreads, 0, s>>>(
         rows, tokens, parent, level_start, n_levels, gamma, u_accept, N, V, state);
     MCSD_CUDA_CHECK(cudaGetLastError());
-    mcsd::verify_select_kernel<mcsd::ProbRows><<<B, mcsd::kVerifyThreads, 0, s>>>(
-        rows, tokens, state, n_levels, n_roots, u_bonus, N, V, accept_len, out_tokens, out_nodes, best_root,
-        R > 0 ? next_roots : nullptr, R);
-    MCSD_CUDA_CHECK(cudaGetLastError());
+    MCSD_CUDA_CHECK(mcsd::launch_dependent(mcsd::verify_select_kernel<mcsd::ProbRows>, dim3(B), dim3(mcsd::kVerifyThreads), s,
+                                           rows, tokens, state, n_levels, n_roots, u_bonus, N, V, accept_len, out_tokens,
+                                           out_nodes, best_root, R > 0 ? next_roots : nullptr, R));
     mcsd::count_launches(2);
     return MCSD_OK;
 }

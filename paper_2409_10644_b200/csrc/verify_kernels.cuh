@@ -416,6 +416,9 @@ verify_nodes_kernel(Rows rows, const int32_t* __restrict__ tokens, const int32_t
     // Blocks are handed out in the order of their linear index; taking the node from its upper part starts all
     // sequences' nodes level by level, so the nodes with the most siblings to try run first and the leaves,
     // which have nothing to do, last.
+    // lets a select kernel launched as a programmatic dependent become resident while this grid still runs
+    // (it waits for this grid's completion before reading anything); no effect on an ordinary launch
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int lin = blockIdx.y * gridDim.x + blockIdx.x;
     const int b = lin % (int)gridDim.y, u = lin / (int)gridDim.y, tid = threadIdx.x;
     const int n_act = active_nodes(gamma, level_start, n_levels, b, N);
@@ -737,6 +740,9 @@ verify_select_kernel(Rows rows, const int32_t* __restrict__ tokens, const NodeSt
     __shared__ int s_bi[kVerifyWarps];
     const int b = blockIdx.x, tid = threadIdx.x;
     const NodeState* st = state + (size_t)b * N;
+    // launched as a programmatic dependent of the node kernel: wait until that grid has completed and its
+    // results are visible (returns at once on an ordinary launch)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     select_path(st, tokens, b, n_levels, n_roots, N, accept_len, out_tokens, out_nodes, best_root, s_len, &s_stop, &s_slot);
     const int u = s_stop;
@@ -796,6 +802,24 @@ sample_roots_kernel(Rows rows, const NodeState* __restrict__ state, const int32_
         if (tid == 0) { s_pick[i] = tok; next_roots[(size_t)b * R + i] = tok; }
         __syncthreads();
     }
+}
+
+// Host side: launches `kernel` as a programmatic dependent of the kernel before it in the stream.  Its blocks may
+// become resident while that kernel still runs (once all of its blocks have started) and must execute
+// griddepcontrol.wait before they read its results; this takes the launch latency off the critical path.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 }  // namespace mcsd

@@ -119,10 +119,9 @@ static int launch_logits(const void* target_logits, const void* draft_logits, fl
         verify_nodes_kernel<LogitRows<T>><<<dim3(N, B), kVerifyThreads, 0, s>>>(rows, tokens, parent, level_start, n_levels,
                                                                                gamma, u_accept, N, V, state);
         MCSD_CUDA_CHECK(cudaGetLastError());
-        verify_select_kernel<LogitRows<T>><<<B, kVerifyThreads, 0, s>>>(rows, tokens, state, n_levels, n_roots, u_bonus, N,
-                                                                       V, accept_len, out_tokens, out_nodes, best_root,
-                                                                       next_roots, R);
-        MCSD_CUDA_CHECK(cudaGetLastError());
+        MCSD_CUDA_CHECK(launch_dependent(verify_select_kernel<LogitRows<T>>, dim3(B), dim3(kVerifyThreads), s, rows, tokens,
+                                         state, n_levels, n_roots, u_bonus, N, V, accept_len, out_tokens, out_nodes,
+                                         best_root, next_roots, R));
     }
     count_launches(2);
     return MCSD_OK;
