@@ -413,6 +413,8 @@ verify_nodes_kernel(Rows rows, const int32_t* __restrict__ tokens, const int32_t
                     const float* __restrict__ u_accept, int N, int V, NodeState* __restrict__ state) {
     __shared__ int s_first, s_cnt, s_accept;
     __shared__ VerifyScratch s_scratch;
+    __shared__ double s_px[MCSD_MAX_NODES], s_qx[MCSD_MAX_NODES];
+    __shared__ float s_ua[MCSD_MAX_NODES];
     // Blocks are handed out in the order of their linear index; taking the node from its upper part starts all
     // sequences' nodes level by level, so the nodes with the most siblings to try run first and the leaves,
     // which have nothing to do, last.
@@ -431,18 +433,27 @@ verify_nodes_kernel(Rows rows, const int32_t* __restrict__ tokens, const int32_t
     // in level order a kept prefix of the tree keeps either all children of a node or none
     if (cnt > 0 && first < n_act) {
         typename Rows::Dist d = rows.open(b, u, N, V, &s_scratch);
+        // p_u(x), q_u(x) and the uniform of every sibling are fetched side by side up front, so that the sibling
+        // loop below pays for one dependent trip to memory in total instead of one per sibling
+        for (int m = tid; m < cnt; m += kVerifyThreads) {
+            const int x = tokens[(size_t)b * N + first + m];
+            const bool valid = x >= 0 && x < V;
+            s_px[m] = valid ? d.p_of(x) : -1.0;               // -1: no such token, never accepted
+            s_qx[m] = valid ? d.q_of(x) : 0.0;
+            s_ua[m] = u_accept[(size_t)b * N + first + m];
+        }
+        __syncthreads();
         double c = 0.0, Y = 1.0;
         for (int m = 0; m < cnt; ++m) {
             const int child = first + m;
             if (tid == 0) {
-                const int x = tokens[(size_t)b * N + child];
                 double a = 0.0;
-                if (x >= 0 && x < V) {
-                    const double px = d.p_of(x), qx = d.q_of(x);
+                if (s_px[m] >= 0.0) {
+                    const double px = s_px[m], qx = s_qx[m];
                     const double num = fmax(px - c * qx, 0.0);
                     a = qx > 0.0 ? fmin(1.0, num / (Y * qx)) : (num > 0.0 ? 1.0 : 0.0);
                 }
-                s_accept = ((double)u_accept[(size_t)b * N + child] < a) ? 1 : 0;
+                s_accept = ((double)s_ua[m] < a) ? 1 : 0;
             }
             __syncthreads();
             const int acc = s_accept;
