@@ -276,19 +276,58 @@ def run_ours(args):
           for _ in range(args.steps)]
     ver_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sync_all()
-    launches0 = mcsd.mcsd_launch_count()
-    t_start.record()
-    for k in range(args.steps):
-        step(ev[k])
-        ver_ev[k][1].record()
-    t_end.record()
-    sync_all()
-    launches = mcsd.mcsd_launch_count() - launches0
-    clocks = sampler.stop() if rank == 0 else None
-    ms_local = t_start.elapsed_time(t_end) / args.steps
-    attn_ms = float(np.mean([a.elapsed_time(b) for per in ev for (a, b) in per]))
-    ver_ms = float(np.mean([ev[k][-1][1].elapsed_time(ver_ev[k][1]) for k in range(args.steps)]))
+    if args.graph:
+        # The same launches replayed from two CUDA graphs (all attention layers; the verify step), so that the host's
+        # launch path (25-50 us per call from Python) is not in the numbers of workloads whose kernels are shorter.
+        def attn_layers():
+            for inp, o in zip(layers, outs):
+                mcsd.mcsd_tree_attention(inp["q"], inp["k_cache"], inp["v_cache"], inp["k_tree"], inp["v_tree"], lens_d,
+                                         nact_d, tm, out=o, softmax_scale=scale, workspace=ws_attn)
+
+        def verify_only():
+            mcsd.mcsd_verify_tree(vin["p"], vin["q"], vin["tokens"], tm, gam_d, vin["u_accept"], vin["u_bonus"],
+                                  workspace=ws_ver, out=vout)
+        l0 = mcsd.mcsd_launch_count()
+        g_attn, g_ver = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_attn):
+            attn_layers()
+        with torch.cuda.graph(g_ver):
+            verify_only()
+        per_step = mcsd.mcsd_launch_count() - l0
+        for _ in range(3):
+            g_attn.replay()
+            g_ver.replay()
+        mid = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+        beg = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+        sync_all()
+        t_start.record()
+        for k in range(args.steps):
+            beg[k].record()
+            g_attn.replay()
+            mid[k].record()
+            g_ver.replay()
+            ver_ev[k][1].record()
+        t_end.record()
+        sync_all()
+        launches = per_step * args.steps
+        clocks = sampler.stop() if rank == 0 else None
+        ms_local = t_start.elapsed_time(t_end) / args.steps
+        attn_ms = float(np.mean([beg[k].elapsed_time(mid[k]) for k in range(args.steps)])) / len(layers)
+        ver_ms = float(np.mean([mid[k].elapsed_time(ver_ev[k][1]) for k in range(args.steps)]))
+    else:
+        sync_all()
+        launches0 = mcsd.mcsd_launch_count()
+        t_start.record()
+        for k in range(args.steps):
+            step(ev[k])
+            ver_ev[k][1].record()
+        t_end.record()
+        sync_all()
+        launches = mcsd.mcsd_launch_count() - launches0
+        clocks = sampler.stop() if rank == 0 else None
+        ms_local = t_start.elapsed_time(t_end) / args.steps
+        attn_ms = float(np.mean([a.elapsed_time(b) for per in ev for (a, b) in per]))
+        ver_ms = float(np.mean([ev[k][-1][1].elapsed_time(ver_ev[k][1]) for k in range(args.steps)]))
     if mcsd.mcsd_workspace_status(ws_attn) != 0:
         raise SystemExit("a device-side wait timed out; results are invalid")
 
@@ -372,7 +411,8 @@ def run_ours(args):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic", "config": _config(w, world),
+        "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": dict(_config(w, world), launch="cuda graphs" if args.graph else "stream launches"),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                 "ms_per_step": e2e_ms,
                 "note": "per step the tree's q/k/v of every layer, p, q, tokens, uniforms, lengths and gammas are copied "
@@ -451,6 +491,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the batch (profiling of a smaller case only)")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling only)")
+    ap.add_argument("--no-graph", dest="graph", action="store_false",
+                    help="issue the step's launches one by one from Python instead of replaying them from CUDA graphs "
+                         "(the host's launch path, 25-50 us per call, then bounds workloads with shorter kernels)")
     ap.add_argument("--vocab-shards", type=int, default=0,
                     help="also time the vocabulary-sharded verify step with this many ranks' column slices on one GPU")
     args = ap.parse_args()
