@@ -182,6 +182,11 @@ int mcsd_workspace_status(const void* workspace, void* stream);
  *                 tree (Section 3.1) seeds its next step
  *   workspace     [dev] >= mcsd_verify_tree_workspace_bytes(B, N, V) bytes
  *
+ * Two launches on `stream`: one block per (sequence, node) decides the accepted child of every node, then one
+ * block per sequence follows the paths and draws the new token.  The second is a programmatic dependent launch
+ * (its blocks may become resident before the first kernel ends and wait for it on the device); to the stream's
+ * other work the pair behaves like two ordinary launches.
+ *
  * Errors: MCSD_ERR_NULL, MCSD_ERR_BAD_SHAPE (B, N, V < 1, N > MCSD_MAX_NODES, B > 65535, R < 0 or R > 32,
  * n_roots or n_levels out of range), MCSD_ERR_WORKSPACE_TOO_SMALL, MCSD_ERR_CUDA.
  */
