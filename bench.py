@@ -123,6 +123,9 @@ def _algorithmic_bytes_attention(H, D, lens, n_act, words, elt):
 # CPU oracle on a bounded sample (reported baseline; also the `--impl reference` arm)
 # ------------------------------------------------------------------------------------------------
 
+_ORACLE_POOL = {}
+
+
 def oracle_sample(w, budget_s=12.0, min_pairs=8):
     """Times the oracle, as it stands, on (sequence, head) attention problems and on verify sequences of
     workload `w`, and extrapolates to a full step.  Returns (tree-tokens/s, description, threads)."""
@@ -138,10 +141,16 @@ def oracle_sample(w, budget_s=12.0, min_pairs=8):
     # attention: one (b, h) problem at a time, drawn with the workload's seeded generator
     t_attn, pairs = 0.0, 0
     wb = dataclasses.replace(w, B=1, H=1)
+    # Generated problems are kept and taken in turn (drawing one costs more than solving it); 64 of them are a few
+    # hundred MB, more than the host's caches hold, so every solve still streams its keys and values from memory.
+    pool = _ORACLE_POOL.setdefault((w.name, w.B, w.H), {})
     while pairs < min_pairs or (t_attn < budget_s and pairs < w.B * w.H * w.n_layers):
         b = pairs % w.B
-        one = dataclasses.replace(wb, base_seed=w.seed(0, 0) + 7919 * pairs, prefix=(int(lens[b]), int(lens[b])))
-        inp = {k: v.float().numpy() for k, v in attention_inputs(one, 0, "cpu").items()}
+        slot = pairs % 64
+        if slot not in pool:
+            one = dataclasses.replace(wb, base_seed=w.seed(0, 0) + 7919 * slot, prefix=(int(lens[b]), int(lens[b])))
+            pool[slot] = {k: v.float().numpy() for k, v in attention_inputs(one, 0, "cpu").items()}
+        inp = pool[slot]
         t0 = time.perf_counter()
         orc.tree_attention(inp["q"], inp["k_cache"], inp["v_cache"], inp["k_tree"], inp["v_tree"], [int(lens[b])],
                            [int(n_act[b])], parent, scale)
@@ -160,8 +169,9 @@ def oracle_sample(w, budget_s=12.0, min_pairs=8):
         threads = max([int(i.get("num_threads", 1)) for i in threadpool_info()] or [1])
     except Exception:
         threads = os.cpu_count() or 1
-    sample = ("%d of %d (sequence, head, layer) attention problems (%.1f s) and %d of %d verify sequences (%.2f s), "
-              "extrapolated to one full step" % (pairs, w.B * w.H * w.n_layers, t_attn, nseq, w.B, t_ver))
+    sample = ("%d of %d (sequence, head, layer) attention problems (%.1f s; %d distinct seeded problems of the workload's "
+              "shapes taken in turn) and %d of %d verify sequences (%.2f s), extrapolated to one full step"
+              % (pairs, w.B * w.H * w.n_layers, t_attn, len(pool), nseq, w.B, t_ver))
     return float(n_act.sum()) / step_s, sample, threads, step_s
 
 
@@ -173,7 +183,7 @@ def run_reference(args):
     w = workload(args.workload)
     vals = []
     for i in range(args.warmup + args.steps):
-        v, sample, threads, step_s = oracle_sample(w, budget_s=max(2.0, 36.0 / max(1, args.warmup + args.steps)))
+        v, sample, threads, step_s = oracle_sample(w, budget_s=max(2.0, 60.0 / max(1, args.warmup + args.steps)))
         if i >= args.warmup:
             vals.append((v, step_s))
     value = float(np.mean([v for v, _ in vals]))
