@@ -1,12 +1,15 @@
 // Tree attention (Section 2.2 of the paper) on the fifth-generation tensor cores of sm_100a: bf16, head_dim 128.
+// This file: the kernel for up to 64 query columns per work item (trees of up to 64 nodes per head, or fewer
+// nodes with several grouped query heads stacked) and the host side of both tcgen05 kernels; the kernel for wider
+// trees is in attention_tc_wide.cu.
 //
 // One persistent thread block per SM walks a contiguous range of 128-key tiles of the flattened
 // (sequence, head, key tile) space, so the K/V stream of every (sequence, head) is read from HBM exactly once
-// and all SMs carry the same number of tiles whatever the batch and the prefix lengths are.  Where a range
+// and all SMs carry the same cost whatever the batch and the prefix lengths are.  Where a range
 // boundary cuts a (sequence, head), every side writes an unnormalised partial (running maximum, sum, weighted
 // values) and takes a ticket; the block that arrives last combines the partials: split-KV.
 //
-// The problem is set up transposed so that the small dimension (tree tokens, 16..128 per head) is the MMA N
+// The problem is set up transposed so that the small dimension (tree tokens, 16..64 per head) is the MMA N
 // and the 128 keys of a tile fill the MMA M:
 //     S^T[key][query] = K_tile[key][d] * Q[query][d]^T            (A = K tile, B = Q, both K-major, from TMA)
 //     O^T[d][query]  += V_tile[key][d]^T * P^T[key][query]        (A = V tile read MN-major, B = P^T written
@@ -26,31 +29,18 @@
 //   warp 10    bookkeeping (one thread): which other blocks share a work item with this one.
 // Every mbarrier wait is bounded; a wait that runs out raises a flag in the workspace header, all roles drain
 // and the block exits cleanly.
-#include <cuda.h>
-#include <cuda_bf16.h>
-
 #include <mutex>
-#include <type_traits>
 
-#include "attention.cuh"
+#include "attention_tc_common.cuh"
 
 namespace mcsd {
 
-constexpr int kTile = 128;                    // keys per tile
-constexpr int kQBlock = 128;                  // queries per work item
+constexpr int kQBlock = 128;                  // queries per work item (this kernel sees at most 64)
 constexpr int kSoftmaxGroups = 2;              // warpgroups that split the query columns of every tile
 constexpr int kProducerWarp = 4 * kSoftmaxGroups, kMmaWarp = kProducerWarp + 1, kHelperWarp = kMmaWarp + 1;
 constexpr int kTcThreads = 32 * (kHelperWarp + 1);
-constexpr int kSlotBytes = kTile * 128 * 2;   // one K or V tile: 128 rows x 128 bf16
-constexpr int kSlabBytes = kTile * 128;       // 64 of the 128 columns: rows of 128 bytes (the TMA swizzle span)
-constexpr int kMaxSlots = 6;
-constexpr int kMaxBatchTc = 256;
-constexpr int kTmemCols = 512;
-constexpr int kColS1 = 128, kColO = 256, kColL = 384;   // tensor-memory columns: S^T twice, O^T, row sums
-constexpr float kLazyTau = 8.0f;              // raise the reference maximum only beyond 2^8
-constexpr int kMaxParts = 64;                 // a (sequence, head) has at most 34 tiles, so at most 35 pieces
-constexpr int kMaxCtas = 160;                 // partial slots are provisioned for this many thread blocks
-constexpr long long kSpinCycles = 4000000000LL;   // about two seconds
+constexpr int kColS1 = 128, kColO = 256;      // tensor-memory columns: S^T twice, O^T
+constexpr int kNarrowNodes = 64;              // launches of this kernel have at most 64 stacked queries, so at most 64 nodes
 
 struct TcSmall {
     unsigned long long slot_full[kMaxSlots];
@@ -69,275 +59,11 @@ struct TcSmall {
     alignas(16) float m_ref[128];
     alignas(16) float alpha[128];      // rescale factors of a slow-path tile; in the epilogue: 1/l (or l) per query
     alignas(16) float wred[kSoftmaxGroups][4][64];
-    alignas(16) unsigned long long dmask[MCSD_MAX_NODES][3];
-    unsigned short cum_tiles[kMaxBatchTc + 2];   // tiles per head of the sequences before b (at most 256 * 68)
-    int cum_w[kMaxBatchTc + 1];        // the same in cost units (see tile_weight)
-    alignas(128) __nv_bfloat16 ones[256];   // 16 x 16 matrix of ones: B operand of the row-sum product (wide launches)
+    alignas(16) unsigned long long dmask[kNarrowNodes][3];   // transposed ancestor bitsets: queries that see tree key t
+    TileIndex ix;
 };
 // the small state must leave room for six 32 KB ring slots next to Q and P^T of a 48-query launch
-static_assert(sizeof(TcSmall) <= 232448 - 1024 - 6 * 32768 - 48 * 512, "TcSmall grew: the 6-slot ring no longer fits");
-
-struct TcParams {
-    __nv_bfloat16* out;
-    const int32_t* seq_lens;
-    const int32_t* n_active;
-    const uint64_t* anc;
-    int words;
-    int B, H, N, L_max;      // H: work units per sequence = query heads / G; N tree nodes (= tree keys)
-    int G, g_shift;          // query heads stacked into one work unit (1, 2, 4 or 8 = 1 << g_shift): its G * N queries
-                             // are taken node-major, query j = head j % G of the unit, node j / G
-    int Hkv, group;          // key/value heads, and query heads per key/value head (a multiple of G): unit u of a
-                             // sequence reads key/value head u * G / group
-    float scale_log2;
-    float* part_ml;      // [2 * kMaxCtas][2][128]
-    float* part_o;       // [2 * kMaxCtas][128][128]
-    int* counters;       // [B * H][query block][softmax group] arrivals per split work item; zero between launches
-    WorkspaceHeader* header;
-    int n_slots;
-    int npadq;           // rows of the Q box = 16 * (template chunk count)
-};
-
-// ------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(void* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(void* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(void* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(void* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-
-// Bounded wait.  Returns false if the wait ran out or another role already gave up; `where` names the wait.
-__device__ __noinline__ bool mbar_wait_slow(void* bar, uint32_t parity, TcSmall* sm, WorkspaceHeader* header, int where) {
-    const long long t0 = clock64();
-    for (uint32_t it = 0;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 255u) {
-            if (*(volatile int*)&sm->abort_flag) return false;
-            if (clock64() - t0 > kSpinCycles) {
-                *(volatile int*)&sm->abort_flag = 1;
-                header->detail = where;
-                header->status = MCSD_ERR_TIMEOUT;
-                __threadfence();
-                return false;
-            }
-        }
-    }
-}
-__device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, TcSmall* sm, WorkspaceHeader* header, int where) {
-    if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, sm, header, where);
-}
-
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, void* bar, int x, int y, int z) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z) : "memory");
-}
-
-__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, void* bar, int x, int y, int z, int w) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_commit(void* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
-}
-// eight consecutive fp32 columns of this thread's TMEM lane; the caller waits with tc_wait_ld()
-__device__ __forceinline__ void tc_ld8(uint32_t taddr, float* v) {
-    uint32_t r[8];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
-        : "r"(taddr) : "memory");
-#pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
-}
-__device__ __forceinline__ float tc_ld1(uint32_t taddr) {
-    float v;
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=f"(v) : "r"(taddr) : "memory");
-    return v;
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-// Calls f(j, values of 8-column group j) for the first ncg of a thread's column groups, one tensor-memory round
-// trip per group (larger batches cost registers the wide kernels do not have and measured no faster).  ncg is
-// uniform per warp.
-template <int CPT, typename F>
-__device__ __forceinline__ void sweep_groups(uint32_t taddr, int ncg, F&& f) {
-#pragma unroll
-    for (int j = 0; j < CPT; ++j) {
-        if (j < ncg) {
-            float buf[8];
-            tc_ld8(taddr + 8 * j, buf);
-            tc_wait_ld();
-            f(j, buf);
-        }
-    }
-}
-__device__ __forceinline__ void tc_st8(uint32_t taddr, const float* v) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-        ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
-          "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
-          "r"(__float_as_uint(v[7])) : "memory");
-}
-__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ float ex2_approx(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ float warp_max_f32(float v) {
-    float r;
-    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
-    return r;
-}
-// named barrier `id` over the 128 threads of one softmax warpgroup, returning the OR of `pred`
-__device__ __forceinline__ bool group_sync_any(int id, bool pred) {
-    uint32_t r;
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
-        "setp.ne.u32 p, %2, 0;\n\t"
-        "bar.red.or.pred q, %1, 128, p;\n\t"
-        "selp.u32 %0, 1, 0, q;\n\t}"
-        : "=r"(r) : "r"(id), "r"((uint32_t)pred) : "memory");
-    return r != 0;
-}
-
-// Shared-memory matrix descriptor of tcgen05.mma: start address, leading/stride byte offsets (all >> 4),
-// descriptor version 1, swizzle mode in the top bits (0 = none, 2 = 128-byte).
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
-    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
-           (1ull << 46) | ((uint64_t)layout << 61);
-}
-// Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, M = 128, N = n, operand major-ness.
-__device__ __forceinline__ uint32_t instr_desc(int n, int a_mn_major, int b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
-           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-}
-
-// ------------------------------------------------------------------ tile bookkeeping
-// Queries are processed in blocks of at most 128 (the tensor-memory budget); a tree with more nodes makes
-// each (sequence, head) two work items that read the same keys.  Tiles per work item: prefix tiles, then tree tiles.
-__device__ __forceinline__ int kv_tiles_of(int L, int Nb) {
-    return Nb > 0 ? (L + kTile - 1) / kTile + (Nb + kTile - 1) / kTile : 0;
-}
-__device__ __forceinline__ int tiles_of(int L, int Nb, int G) {
-    return kv_tiles_of(L, Nb) * ((Nb * G + kQBlock - 1) / kQBlock);
-}
-
-struct Segment {
-    int b, h, lt, Tb, L, Nb, nP;
-    int qb, q0, Nq, Tkv;      // query block, its first query, its query count, tiles per query block
-};
-
-__device__ __forceinline__ void locate(const TcSmall* sm, const TcParams& p, long long t, Segment& s) {
-    int lo = 0, hi = p.B;                      // find b with H*cum[b] <= t < H*cum[b+1]
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if ((long long)p.H * sm->cum_tiles[mid] <= t) lo = mid; else hi = mid;
-    }
-    s.b = lo;
-    s.L = min(max(p.seq_lens[lo], 0), p.L_max);
-    s.Nb = p.n_active ? min(max(p.n_active[lo], 0), p.N) : p.N;
-    s.Tb = sm->cum_tiles[lo + 1] - sm->cum_tiles[lo];
-    s.nP = (s.L + kTile - 1) / kTile;
-    const long long r = t - (long long)p.H * sm->cum_tiles[lo];
-    s.h = (int)(r / s.Tb);
-    const int rem = (int)(r % s.Tb);
-    s.Tkv = kv_tiles_of(s.L, s.Nb);
-    s.qb = rem / s.Tkv;
-    s.lt = rem % s.Tkv;
-    s.q0 = s.qb * kQBlock;
-    s.Nq = min(kQBlock, s.Nb * p.G - s.q0);
-}
-
-// Cost of one tile in units of about 100 cycles, measured on this kernel.  Launches for up to 64 query columns:
-// flat up to 32 queries (the key/value stream sets the pace), then growing with the columns the softmax threads
-// cover.  Wide launches: nearly flat, set by the 24 tensor-core instructions per tile and the shallower ring.
-// Thread blocks get equal cost, not equal tile counts, so that sequences with deep trees do not make their blocks
-// finish late.
-__device__ __forceinline__ int tile_weight(int Nq, bool wide) {
-    return wide ? 27 + Nq / 19 : 24 + (max(0, Nq - 32) * 9) / 32;
-}
-// Fixed cost of a work item (pipeline fill and drain, first-tile reference search, row sums, output of Nq columns),
-// carried by its first tile.
-__device__ __forceinline__ int item_weight(int Nq, bool wide) {
-    return (wide ? 100 : 30) + (Nq * 5) / 8;
-}
-__device__ __forceinline__ int head_weight(int L, int Nk, int G, bool wide) {  // cost of one (sequence, head): all query blocks
-    const int tkv = kv_tiles_of(L, Nk);
-    const int Nb = Nk * G;                                        // stacked queries
-    int w = 0;
-    for (int q0 = 0; q0 < Nb; q0 += kQBlock) w += tkv * tile_weight(min(kQBlock, Nb - q0), wide) + item_weight(min(kQBlock, Nb - q0), wide);
-    return w;
-}
-// cumulative cost of the tiles before the one a Segment points at
-__device__ __forceinline__ long long weight_before(const TcSmall* sm, const TcParams& p, const Segment& s) {
-    const bool wide = p.npadq > 64;
-    long long w = (long long)p.H * sm->cum_w[s.b] + (long long)s.h * (sm->cum_w[s.b + 1] - sm->cum_w[s.b]);
-    if (s.qb) w += (long long)s.Tkv * tile_weight(kQBlock, wide) + item_weight(kQBlock, wide);
-    return w + (long long)s.lt * tile_weight(s.Nq, wide) + (s.lt > 0 ? item_weight(s.Nq, wide) : 0);
-}
-// Tile t belongs to block floor(weight_before(t) * G / total_w).  First tile of block c: the first tile whose
-// cumulative cost reaches ceil(c * total_w / G).
-__device__ __forceinline__ long long first_tile_of_block(const TcSmall* sm, const TcParams& p, int c, int G, long long total_w,
-                                                         long long total_tiles) {
-    const long long wt = ((long long)c * total_w + G - 1) / G;
-    if (wt >= total_w) return total_tiles;
-    int lo = 0, hi = p.B;
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if ((long long)p.H * sm->cum_w[mid] <= wt) lo = mid; else hi = mid;
-    }
-    const int L = min(max(p.seq_lens[lo], 0), p.L_max);
-    const int Nk = p.n_active ? min(max(p.n_active[lo], 0), p.N) : p.N;
-    const int tkv = kv_tiles_of(L, Nk);
-    const int Nb = Nk * p.G;                                      // stacked queries
-    const int wh = sm->cum_w[lo + 1] - sm->cum_w[lo], tb = sm->cum_tiles[lo + 1] - sm->cum_tiles[lo];
-    const long long rem = wt - (long long)p.H * sm->cum_w[lo];
-    const int h = (int)(rem / wh);
-    int r2 = (int)(rem % wh);
-    long long t = (long long)p.H * sm->cum_tiles[lo] + (long long)h * tb;
-    // inside a work item the tiles start at cost 0, f + w, f + 2w, ... (f = fixed cost on the first tile)
-    const bool wide = p.npadq > 64;
-    const int w0 = tile_weight(min(kQBlock, Nb), wide), f0 = item_weight(min(kQBlock, Nb), wide);
-    if (r2 >= tkv * w0 + f0 && Nb > kQBlock) {         // inside the second query block
-        r2 -= tkv * w0 + f0;
-        t += tkv;
-        const int w1 = tile_weight(Nb - kQBlock, wide), f1 = item_weight(Nb - kQBlock, wide);
-        return r2 == 0 ? t : t + max(1, (r2 - f1 + w1 - 1) / w1);
-    }
-    return r2 == 0 ? t : t + max(1, (r2 - f0 + w0 - 1) / w0);
-}
-__device__ __forceinline__ int block_of_tile(const TcSmall* sm, const TcParams& p, long long t, int G, long long total_w) {
-    Segment s;
-    locate(sm, p, t, s);
-    return (int)min((long long)G - 1, weight_before(sm, p, s) * G / total_w);
-}
+static_assert(sizeof(TcSmall) <= kSmemLimit - 1024 - 6 * 32768 - 48 * 512, "TcSmall grew: the 6-slot ring no longer fits");
 
 // ------------------------------------------------------------------ the kernel
 template <int NCH>
@@ -345,6 +71,8 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kc,
                          const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kt,
                          const __grid_constant__ CUtensorMap tm_vt, const TcParams p) {
+    static_assert(NCH <= 4, "wider launches run the kernel of attention_tc_wide.cu");
+    constexpr int QB = kQBlock;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int NS = p.n_slots;
@@ -352,22 +80,12 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     unsigned char* p_buf = ring + (size_t)NS * kSlotBytes;
     unsigned char* q_buf = p_buf + (size_t)p.npadq * 256;
     TcSmall* sm = reinterpret_cast<TcSmall*>(q_buf + (size_t)p.npadq * 256);
+    const TileIndex* ix = &sm->ix;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x;
 
-    // ---- set-up: tile counts per sequence, barriers, tensor memory
-    constexpr bool WIDE = NCH > 4;              // many query columns: row sums come from the tensor cores (see below)
-    if (WIDE && tid < 256) {
-        sm->ones[tid] = __float2bfloat16_rn(1.0f);
-        fence_async_smem();                      // read by the tensor cores through the async proxy
-    }
-    for (int b = tid; b < p.B; b += kTcThreads) {
-        const int L = min(max(p.seq_lens[b], 0), p.L_max);
-        const int Nb = p.n_active ? min(max(p.n_active[b], 0), p.N) : p.N;
-        sm->cum_tiles[b + 1] = (unsigned short)tiles_of(L, Nb, p.G);
-        sm->cum_w[b + 1] = head_weight(L, Nb, p.G, NCH > 4);
-    }
+    // ---- set-up: barriers, tile counts per sequence, this block's range, tensor memory
     if (tid == 0) {
         for (int i = 0; i < kMaxSlots; ++i) { mbar_init(&sm->slot_full[i], 1); mbar_init(&sm->slot_empty[i], 1); }
         mbar_init(&sm->s_full[0], 1);
@@ -381,30 +99,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    __syncthreads();
-    if (tid == 0) {
-        int acc = 0, accw = 0;
-        sm->cum_tiles[0] = 0;
-        sm->cum_w[0] = 0;
-        for (int b = 1; b <= p.B; ++b) {
-            acc += sm->cum_tiles[b]; sm->cum_tiles[b] = (unsigned short)acc;
-            accw += sm->cum_w[b]; sm->cum_w[b] = accw;
-        }
-        // No block's share of the cost may be smaller than the heaviest tile, so that consecutive tiles never skip
-        // a block: every working block then owns at least one tile and the blocks sharing a work item are consecutive.
-        const long long tot_w = (long long)p.H * accw;
-        const int nb = (int)max(1LL, min((long long)gridDim.x, tot_w / (tile_weight(kQBlock, NCH > 4) + item_weight(kQBlock, NCH > 4))));
-        sm->n_blocks = nb;
-    }
-    __syncthreads();
-    if (tid == 0 || tid == 32) {               // the two ends of this block's range, side by side
-        const long long tot = (long long)p.H * sm->cum_tiles[p.B], tot_w = (long long)p.H * sm->cum_w[p.B];
-        const int nb = sm->n_blocks, which = tid >> 5;
-        sm->range[which] = (tot > 0 && cta < nb) ? first_tile_of_block(sm, p, cta + which, nb, tot_w, tot) : 0;
-    }
-    __syncthreads();
-    const long long total = (long long)p.H * sm->cum_tiles[p.B];
-    const long long total_w = (long long)p.H * sm->cum_w[p.B];
+    plan_ranges<QB>(&sm->ix, p, false, &sm->n_blocks, sm->range);
+    const long long total = (long long)p.H * ix->cum_tiles[p.B];
+    const long long total_w = (long long)p.H * ix->cum_w[p.B];
     const int G = sm->n_blocks;
     const long long t_begin = sm->range[0], t_end = sm->range[1];
     if (t_begin >= t_end) return;              // uniform for the whole block: nothing allocated yet
@@ -418,6 +115,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     tc_fence_after();
     const uint32_t tmem = *(volatile uint32_t*)&sm->tmem_base;
     WorkspaceHeader* hdr = p.header;
+    int* const abort_flag = &sm->abort_flag;
 
     if (warp == kProducerWarp) {
         // =========================================================== TMA producer
@@ -428,11 +126,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             bool ok = true;
             while (t < t_end && ok) {
                 Segment s;
-                locate(sm, p, t, s);
+                locate<QB>(ix, p, t, s);
                 const int cnt = (int)min((long long)(s.Tkv - s.lt), t_end - t);
                 const int bh = s.b * p.H + s.h;
                 const int bh_kv = s.b * p.Hkv + (s.h * p.G) / p.group;
-                ok = mbar_wait(&sm->q_empty, (seg & 1u) ^ 1u, sm, hdr, 1);
+                ok = mbar_wait(&sm->q_empty, (seg & 1u) ^ 1u, abort_flag, hdr, 1);
                 if (!ok) break;
                 mbar_expect_tx(&sm->q_full, (uint32_t)p.npadq * 256u);
                 if (p.G == 1) {
@@ -449,7 +147,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     const bool tree = lti >= s.nP;
                     const int row0 = (tree ? lti - s.nP : lti) * kTile;
                     for (int kv = 0; kv < 2 && ok; ++kv, ++u) {
-                        ok = mbar_wait(&sm->slot_empty[slot], phase ^ 1u, sm, hdr, 2);
+                        ok = mbar_wait(&sm->slot_empty[slot], phase ^ 1u, abort_flag, hdr, 2);
                         if (!ok) break;
                         const CUtensorMap* map = kv == 0 ? (tree ? &tm_kt : &tm_kc) : (tree ? &tm_vt : &tm_vc);
                         const uint32_t dst = smem_u32(ring) + slot * (uint32_t)kSlotBytes;
@@ -479,19 +177,19 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             // which blocks hold the other pieces of the work items this block shares with its neighbours
             for (int which = 0; which < 2; ++which) {
                 Segment sp;
-                locate(sm, p, which == 0 ? t_begin : t_end - 1, sp);
+                locate<QB>(ix, p, which == 0 ? t_begin : t_end - 1, sp);
                 const long long at = which == 0 ? t_begin : t_end - 1;
                 const long long t0 = at - sp.lt, t1 = t0 + sp.Tkv;
                 int nparts = 0;
                 const bool shared = which == 0 ? (t0 < t_begin || t1 > t_end) : (t0 > t_begin && t1 > t_end);
                 if (shared) {
-                    const int c_lo = block_of_tile(sm, p, t0, G, total_w);
-                    const int c_hi = block_of_tile(sm, p, t1 - 1, G, total_w);
+                    const int c_lo = block_of_tile<QB>(ix, p, t0, G, total_w, false);
+                    const int c_hi = block_of_tile<QB>(ix, p, t1 - 1, G, total_w, false);
                     nparts = min(c_hi - c_lo + 1, kMaxParts);
                     int others = 0;
                     for (int i = 0; i < nparts; ++i) {
                         if (c_lo + i == cta) continue;
-                        const long long start = first_tile_of_block(sm, p, c_lo + i, G, total_w, total);
+                        const long long start = first_tile_of_block<QB>(ix, p, c_lo + i, G, total_w, total, false);
                         sm->piece_slot[which][others++] = (unsigned short)(2 * (c_lo + i) + (t0 > start ? 1 : 0));
                     }
                 }
@@ -511,16 +209,16 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             const uint32_t ring_a = smem_u32(ring), q_a = smem_u32(q_buf), p_a = smem_u32(p_buf);
             while (t < t_end && ok) {
                 Segment s;
-                locate(sm, p, t, s);
+                locate<QB>(ix, p, t, s);
                 const int cnt = (int)min((long long)(s.Tkv - s.lt), t_end - t);
                 const int npad = (s.Nq + 15) & ~15;
                 const uint32_t idesc_s = instr_desc(npad, 0, 0), idesc_pv = instr_desc(npad, 1, 1);
-                ok = mbar_wait(&sm->q_full, seg & 1u, sm, hdr, 3);
+                ok = mbar_wait(&sm->q_full, seg & 1u, abort_flag, hdr, 3);
                 for (int i = 0; i <= cnt && ok; ++i) {
                     if (i < cnt) {
                         const uint32_t gi = g + (uint32_t)i, sb = gi & 1u;
                         const uint32_t slot = kslot;
-                        ok = mbar_wait(&sm->slot_full[slot], kphase, sm, hdr, 4);
+                        ok = mbar_wait(&sm->slot_full[slot], kphase, abort_flag, hdr, 4);
                         if (!ok) break;
                         kslot += 2u;
                         if (kslot >= (uint32_t)NS) { kslot -= (uint32_t)NS; kphase ^= 1u; }
@@ -540,11 +238,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     if (i >= 1) {
                         const uint32_t gj = g + (uint32_t)(i - 1);
                         const uint32_t slot = vslot;
-                        ok = mbar_wait(&sm->slot_full[slot], vphase, sm, hdr, 5);
+                        ok = mbar_wait(&sm->slot_full[slot], vphase, abort_flag, hdr, 5);
                         if (!ok) break;
                         vslot += 2u;
                         if (vslot >= (uint32_t)NS) { vslot -= (uint32_t)NS; vphase ^= 1u; }
-                        ok = mbar_wait(&sm->p_full, gj & 1u, sm, hdr, 6);
+                        ok = mbar_wait(&sm->p_full, gj & 1u, abort_flag, hdr, 6);
                         if (!ok) break;
                         tc_fence_after();
                         const uint32_t va = ring_a + slot * (uint32_t)kSlotBytes;
@@ -555,17 +253,6 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                             // P^T: 8-key groups 128 B apart (leading), 8-query groups 2 KB apart (stride), no swizzle.
                             const uint64_t db = smem_desc(p_a + k * 256, 128, 2048, 0);
                             tc_mma(tmem + kColO, da, db, idesc_pv, !(i == 1 && k == 0));
-                        }
-                        if (WIDE) {
-                            // Row sums of this tile's probabilities: L[query][.] = P[query][key] * ones[key][.], P^T read
-                            // as the A operand (queries on the accumulator's lanes), not accumulated across tiles.
-                            const uint32_t idesc_l = instr_desc(16, 1, 0);
-                            const uint64_t d1 = smem_desc(smem_u32(sm->ones), 128, 256, 0);
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                const uint64_t dp = smem_desc(p_a + k * 256, 128, 2048, 0);
-                                tc_mma(tmem + kColL, dp, d1, idesc_l, k > 0);
-                            }
                         }
                         tc_commit(&sm->slot_empty[slot]);
                         tc_commit(&sm->pv_done);
@@ -590,7 +277,6 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         // exponentiate, add to the per-thread row sums and store P^T.  Only when the vote fires (always on the
         // first tile of a segment) are exact column maxima computed and O^T rescaled.
         constexpr int CPT = NCH;                       // 8-column groups per thread (two groups share 16*NCH columns)
-        constexpr bool KEEP = CPT <= 4;                // keep the shifted scores in registers between the passes
         const int wg = warp >> 2, wq = warp & 3;
         const int r = tid & 127;
         const int bar_id = 1 + wg;
@@ -632,11 +318,10 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         long long t = t_begin;
         uint32_t u = 0, g = 0;
         bool failed = false;
-        float acc_l[KEEP ? CPT : 1][8];
-        float l_run = 0.f;                              // wide launches: row sum of query r (this thread's lane) so far
+        float acc_l[CPT][8];
         while (t < t_end) {
             Segment s;
-            locate(sm, p, t, s);
+            locate<QB>(ix, p, t, s);
             const int cnt = (int)min((long long)(s.Tkv - s.lt), t_end - t);
             const int bh = s.b * p.H + s.h;
             const int ng8 = (s.Nq + 7) >> 3;
@@ -648,11 +333,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             const unsigned long long nb_hi = s.Nq >= 128 ? ~0ull : (s.Nq > 64 ? ((1ull << (s.Nq - 64)) - 1ull) : 0ull);
             if (r < ncg * 8) mref[r] = -INFINITY;
 #pragma unroll
-            for (int j = 0; j < (KEEP ? CPT : 1); ++j)
+            for (int j = 0; j < CPT; ++j)
 #pragma unroll
                 for (int k = 0; k < 8; ++k) acc_l[j][k] = 0.f;
-            l_run = 0.f;
-            const bool own = r >= col0 && r < col0 + 8 * ncg;    // wide launches: query r is one of this group's
             if (group_sync_any(bar_id, failed)) { failed = true; break; }
 
             for (int i = 0; i < cnt; ++i) {
@@ -672,64 +355,32 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     }
                     cm = col0 >= 64 ? (c1 >> (col0 - 64)) : (col0 == 0 ? c0 : ((c0 >> col0) | (c1 << (64 - col0))));
                 }
-                if (!mbar_wait(&sm->s_full[sb], (gi >> 1) & 1u, sm, hdr, 7)) failed = true;
+                if (!mbar_wait(&sm->s_full[sb], (gi >> 1) & 1u, abort_flag, hdr, 7)) failed = true;
                 tc_fence_after();
                 const uint32_t s_addr = tmem + lane_addr + (sb ? kColS1 : 0) + col0;
-                bool l_taken = false;                   // wide launches: previous tile's row sum already added
 
                 // ---- pass A: scores minus the running reference, and the largest excess
-                float y[KEEP ? CPT : 1][8];
-                uint32_t pk[KEEP ? 1 : CPT][4];
+                float y[CPT][8];
                 float dmax = -INFINITY;
-                auto wide_pass = [&](auto masked_tag) {
-                    constexpr bool MASKED = decltype(masked_tag)::value;
-                    sweep_groups<CPT>(s_addr, ncg, [&](int j, const float* v) {
+#pragma unroll
+                for (int j = 0; j < CPT; ++j)
+                    if (j < ncg) tc_ld8(s_addr + 8 * j, y[j]);
+                tc_wait_ld();
+#pragma unroll
+                for (int j = 0; j < CPT; ++j) {
+                    if (j < ncg) {
                         const float4 m0 = *reinterpret_cast<const float4*>(&mref[8 * j]);
                         const float4 m1 = *reinterpret_cast<const float4*>(&mref[8 * j + 4]);
                         const float mr[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
                         const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
-                        float yy[8];
 #pragma unroll
                         for (int k = 0; k < 8; ++k) {
-                            yy[k] = fmaf(v[k], p.scale_log2, -mr[k]);
-                            if (MASKED && !((bits >> k) & 1u)) yy[k] = -INFINITY;
-                            dmax = fmaxf(dmax, yy[k]);
-                        }
-#pragma unroll
-                        for (int k = 0; k < 8; k += 2) {
-                            __nv_bfloat162 h2 = __floats2bfloat162_rn(ex2_approx(yy[k]), ex2_approx(yy[k + 1]));
-                            pk[KEEP ? 0 : j][k >> 1] = *reinterpret_cast<uint32_t*>(&h2);
-                        }
-                    });
-                };
-                if (KEEP) {
-#pragma unroll
-                    for (int j = 0; j < CPT; ++j)
-                        if (j < ncg) tc_ld8(s_addr + 8 * j, y[KEEP ? j : 0]);
-                    tc_wait_ld();
-                }
-                if (KEEP) {
-#pragma unroll
-                    for (int j = 0; j < CPT; ++j) {
-                        if (j < ncg) {
-                            const float4 m0 = *reinterpret_cast<const float4*>(&mref[8 * j]);
-                            const float4 m1 = *reinterpret_cast<const float4*>(&mref[8 * j + 4]);
-                            const float mr[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
-                            const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                float yy = fmaf(y[KEEP ? j : 0][k], p.scale_log2, -mr[k]);
-                                if (!full_tile && !((bits >> k) & 1u)) yy = -INFINITY;
-                                dmax = fmaxf(dmax, yy);
-                                y[KEEP ? j : 0][k] = yy;
-                            }
+                            float yy = fmaf(y[j][k], p.scale_log2, -mr[k]);
+                            if (!full_tile && !((bits >> k) & 1u)) yy = -INFINITY;
+                            dmax = fmaxf(dmax, yy);
+                            y[j][k] = yy;
                         }
                     }
-                } else {
-                    // wide launches: one sweep gives the largest excess and, optimistically, the probabilities
-                    // themselves (packed bf16, kept in registers until the P^T buffer is free); row sums come
-                    // from the tensor cores, so nothing is accumulated here that a raised reference would spoil
-                    if (full_tile) wide_pass(std::false_type{}); else wide_pass(std::true_type{});
                 }
                 if (group_sync_any(bar_id, dmax > kLazyTau || failed)) {
                     if (*(volatile int*)&sm->abort_flag) { failed = true; break; }
@@ -766,14 +417,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                         alph[r] = a;
                     }
                     const bool rescale = group_sync_any(bar_id, need);
-                    if (gi > 0 && !mbar_wait(&sm->pv_done, (gi - 1u) & 1u, sm, hdr, 8)) failed = true;
-                    if (WIDE) {
-                        // the previous tile's row sum belongs to the old reference: take it in before rescaling
-                        tc_fence_after();
-                        if (i > 0) { const float lp = tc_ld1(tmem + lane_addr + kColL); tc_wait_ld(); l_run += lp; }
-                        l_taken = true;
-                        if (own) l_run *= alph[r - col0];
-                    }
+                    if (gi > 0 && !mbar_wait(&sm->pv_done, (gi - 1u) & 1u, abort_flag, hdr, 8)) failed = true;
                     if (rescale) {
                         tc_fence_after();
 #pragma unroll
@@ -786,75 +430,56 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                                 for (int k = 0; k < 8; ++k) {
                                     const float a = alph[8 * j + k];
                                     o[k] *= a;
-                                    if (KEEP) acc_l[KEEP ? j : 0][k] *= a;
+                                    acc_l[j][k] *= a;
                                 }
                                 tc_st8(tmem + lane_addr + kColO + col0 + 8 * j, o);
                             }
                         }
                         tc_wait_st();
                     }
-                    if (KEEP) {
 #pragma unroll
-                        for (int j = 0; j < CPT; ++j) {
-                            if (j < ncg) {
-                                float v[8];
-                                tc_ld8(s_addr + 8 * j, v);
-                                tc_wait_ld();
-                                const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
+                    for (int j = 0; j < CPT; ++j) {
+                        if (j < ncg) {
+                            float v[8];
+                            tc_ld8(s_addr + 8 * j, v);
+                            tc_wait_ld();
+                            const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
 #pragma unroll
-                                for (int k = 0; k < 8; ++k) {
-                                    float yy = fmaf(v[k], p.scale_log2, -mref[8 * j + k]);
-                                    if (!full_tile && !((bits >> k) & 1u)) yy = -INFINITY;
-                                    y[KEEP ? j : 0][k] = yy;
-                                }
+                            for (int k = 0; k < 8; ++k) {
+                                float yy = fmaf(v[k], p.scale_log2, -mref[8 * j + k]);
+                                if (!full_tile && !((bits >> k) & 1u)) yy = -INFINITY;
+                                y[j][k] = yy;
                             }
                         }
-                    } else {
-                        if (full_tile) wide_pass(std::false_type{}); else wide_pass(std::true_type{});
                     }
                 }
 
                 // P buffer must no longer be read by the previous tile's MMA; this wait also keeps every thread
                 // within one phase of the p_full barrier
-                if (gi > 0 && !mbar_wait(&sm->pv_done, (gi - 1u) & 1u, sm, hdr, 8)) failed = true;
+                if (gi > 0 && !mbar_wait(&sm->pv_done, (gi - 1u) & 1u, abort_flag, hdr, 8)) failed = true;
 
                 // ---- pass B: probabilities, row sums, P^T for the second MMA
-                if (KEEP) {
 #pragma unroll
-                    for (int j = 0; j < CPT; ++j) {
-                        if (j < ncg) {
-                            uint32_t packed[4];
+                for (int j = 0; j < CPT; ++j) {
+                    if (j < ncg) {
+                        uint32_t packed[4];
 #pragma unroll
-                            for (int k = 0; k < 8; k += 2) {
-                                // 2^-inf = 0 for masked entries
-                                const float p0 = ex2_approx(y[KEEP ? j : 0][k]), p1 = ex2_approx(y[KEEP ? j : 0][k + 1]);
-                                acc_l[KEEP ? j : 0][k] += p0;
-                                acc_l[KEEP ? j : 0][k + 1] += p1;
-                                __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-                                packed[k >> 1] = *reinterpret_cast<uint32_t*>(&h2);
-                            }
-                            *reinterpret_cast<uint4*>(p_buf + (size_t)(g0 + j) * 2048 + (size_t)r * 16) =
-                                make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                        for (int k = 0; k < 8; k += 2) {
+                            // 2^-inf = 0 for masked entries
+                            const float p0 = ex2_approx(y[j][k]), p1 = ex2_approx(y[j][k + 1]);
+                            acc_l[j][k] += p0;
+                            acc_l[j][k + 1] += p1;
+                            __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
+                            packed[k >> 1] = *reinterpret_cast<uint32_t*>(&h2);
                         }
+                        *reinterpret_cast<uint4*>(p_buf + (size_t)(g0 + j) * 2048 + (size_t)r * 16) =
+                            make_uint4(packed[0], packed[1], packed[2], packed[3]);
                     }
-                } else {
-                    // the previous tile's row sum (its product has finished: pv_done) before the next one replaces it
-                    if (!l_taken && i > 0) {
-                        tc_fence_after();
-                        const float lp = tc_ld1(tmem + lane_addr + kColL);
-                        tc_wait_ld();
-                        l_run += lp;
-                    }
-#pragma unroll
-                    for (int j = 0; j < CPT; ++j)
-                        if (j < ncg)
-                            *reinterpret_cast<uint4*>(p_buf + (size_t)(g0 + j) * 2048 + (size_t)r * 16) =
-                                make_uint4(pk[KEEP ? 0 : j][0], pk[KEEP ? 0 : j][1], pk[KEEP ? 0 : j][2], pk[KEEP ? 0 : j][3]);
                 }
                 // rows of the V tile past the end of the prefix / tree may hold anything: make them zero
                 if (wg == 0 && valid < kTile) {
                     const uint32_t uv = u + 2u * (uint32_t)i + 1u, slot = uv % (uint32_t)NS;
-                    if (!mbar_wait(&sm->slot_full[slot], (uv / (uint32_t)NS) & 1u, sm, hdr, 9)) failed = true;
+                    if (!mbar_wait(&sm->slot_full[slot], (uv / (uint32_t)NS) & 1u, abort_flag, hdr, 9)) failed = true;
                     if (r >= valid && !failed) {
                         uint4* z0 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + (size_t)r * 128);
                         uint4* z1 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + kSlabBytes + (size_t)r * 128);
@@ -872,24 +497,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             const uint32_t glast = g + (uint32_t)cnt - 1u;
             const bool full = (cnt == s.Tkv);
             const int slot_id = 2 * cta + (t > t_begin ? 1 : 0);
-            if (!mbar_wait(&sm->pv_done, glast & 1u, sm, hdr, 10)) failed = true;
+            if (!mbar_wait(&sm->pv_done, glast & 1u, abort_flag, hdr, 10)) failed = true;
             tc_fence_after();
-            if (WIDE) {
-                // Row sums came from the tensor cores, query by lane: add the last tile's and hand the sum of each of
-                // this group's queries to the threads that finish its columns.
-                const float lp = tc_ld1(tmem + lane_addr + kColL);
-                tc_wait_ld();
-                const float l = l_run + lp;
-                if (own) {
-                    if (full) {
-                        alph[r - col0] = l > 0.f ? 1.f / l : 0.f;
-                    } else {
-                        alph[r - col0] = l;            // kept for the merge below
-                        p.part_ml[((size_t)slot_id * 2 + 0) * 128 + r] = mref[r - col0];
-                        p.part_ml[((size_t)slot_id * 2 + 1) * 128 + r] = l;
-                    }
-                }
-            } else {
             // Row sums: every thread holds a partial sum per query; reduce the 8 sums of a column group across the
             // warp by recursive halving (9 shuffles instead of 40): after the three exchange steps lane L holds the
             // sum of column (L >> 2) & 7 over its exchange partners, two more steps finish the reduction.
@@ -901,8 +510,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                         const bool up = lane & 16;
 #pragma unroll
                         for (int k = 0; k < 4; ++k) {
-                            const float send = up ? acc_l[KEEP ? j : 0][k] : acc_l[KEEP ? j : 0][k + 4];
-                            const float keep = up ? acc_l[KEEP ? j : 0][k + 4] : acc_l[KEEP ? j : 0][k];
+                            const float send = up ? acc_l[j][k] : acc_l[j][k + 4];
+                            const float keep = up ? acc_l[j][k + 4] : acc_l[j][k];
                             v4[k] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
                         }
                     }
@@ -934,10 +543,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     alph[r] = l > 0.f ? 1.f / l : 0.f;
                 } else {
                     alph[r] = l;                   // kept for the merge below
-                    p.part_ml[((size_t)slot_id * 2 + 0) * 128 + col0 + r] = mref[r];
-                    p.part_ml[((size_t)slot_id * 2 + 1) * 128 + col0 + r] = l;
+                    p.part_ml[((size_t)slot_id * 2 + 0) * kMaxQ + col0 + r] = mref[r];
+                    p.part_ml[((size_t)slot_id * 2 + 1) * kMaxQ + col0 + r] = l;
                 }
-            }
             }
             group_sync_any(bar_id, false);
             // O^T rows of this thread, up to four column groups per tensor-memory round trip
@@ -988,7 +596,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
 #pragma unroll
                                 for (int k = 0; k < 8; ++k) {
                                     const int n = col0 + 8 * (j0 + jj) + k;
-                                    if (n < s.Nq) p.part_o[((size_t)slot_id * 128 + n) * 128 + r] = o[jj][k];
+                                    if (n < s.Nq) p.part_o[((size_t)slot_id * kMaxQ + n) * 128 + r] = o[jj][k];
                                 }
                             }
                         }
@@ -1004,8 +612,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 group_sync_any(bar_id, false);
                 const int which = slot_id & 1;
                 if (r == 0) {
-                    if (!mbar_wait(&sm->info_ready, 0, sm, hdr, 12)) failed = true;
-                    int* counter = p.counters + ((size_t)bh * 2 + s.qb) * kSoftmaxGroups + wg;
+                    if (!mbar_wait(&sm->info_ready, 0, abort_flag, hdr, 12)) failed = true;
+                    int* counter = p.counters + ((size_t)bh * 2 + s.qb) * 4 + wg;
                     const int nparts = sm->piece_parts[which];
                     sm->merge_parts[wg] = nparts;
                     const int old = atomicAdd(counter, 1);
@@ -1029,7 +637,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     float* const fa = &sm->wred[wg][0][0];                   // [piece parity][64]: factor for what we have
                     float* const fw = &sm->wred[wg][2][0];                   // [piece parity][64]: factor for the new piece
                     const bool col_owner = r < ncg * 8 && col0 + r < s.Nq;
-                    constexpr int GB = CPT < 4 ? CPT : (CPT == 7 ? 3 : 2);   // column groups per batch (what the registers allow)
+                    constexpr int GB = CPT < 4 ? CPT : 2;                    // column groups per batch (what the registers allow)
 #pragma unroll
                     for (int j0 = 0; j0 < CPT; j0 += GB) {
                         if (j0 >= ncg) break;
@@ -1049,13 +657,13 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                                 for (int k = 0; k < 8; ++k) {
                                     const int n = col0 + 8 * (j0 + jj) + k;
                                     const bool on = j0 + jj < CPT && j0 + jj < ncg && n < s.Nq;
-                                    os[jj][k] = on ? __ldcg(p.part_o + ((size_t)slot * 128 + n) * 128 + r) : 0.f;
+                                    os[jj][k] = on ? __ldcg(p.part_o + ((size_t)slot * kMaxQ + n) * 128 + r) : 0.f;
                                 }
                             float* const fa_i = fa + 64 * (i & 1);
                             float* const fw_i = fw + 64 * (i & 1);
                             if (col_owner) {
-                                const float ms = __ldcg(p.part_ml + ((size_t)slot * 2 + 0) * 128 + col0 + r);
-                                const float ls = __ldcg(p.part_ml + ((size_t)slot * 2 + 1) * 128 + col0 + r);
+                                const float ms = __ldcg(p.part_ml + ((size_t)slot * 2 + 0) * kMaxQ + col0 + r);
+                                const float ls = __ldcg(p.part_ml + ((size_t)slot * 2 + 1) * kMaxQ + col0 + r);
                                 const float mn = fmaxf(m_run, ms);
                                 const float a = (mn == -INFINITY || m_run == -INFINITY) ? 0.f : exp2f(m_run - mn);
                                 const float wgt = (mn == -INFINITY || ms == -INFINITY) ? 0.f : exp2f(ms - mn);
@@ -1185,13 +793,15 @@ static bool encode_map(CUtensorMap* map, const void* base, int rows, int bh, int
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-static int chunks_for(int N) {
-    const int nch = ((N < kQBlock ? N : kQBlock) + 15) / 16;
-    return nch <= 3 ? 3 : nch <= 4 ? 4 : nch <= 7 ? 7 : 8;
+// Padded query columns of a launch in 16-column chunks: 3 or 4 for the kernel above, 7, 8 or 10 for the wide one
+// (10 = 160 queries in one pass; trees with more stacked queries are cut into blocks of 160).
+static int chunks_for(int nq) {
+    const int nch = ((nq < kMaxQ ? nq : kMaxQ) + 15) / 16;
+    return nch <= 3 ? 3 : nch <= 4 ? 4 : nch <= 7 ? 7 : nch <= 8 ? 8 : 10;
 }
 
 static int slots_for(int nch) {
-    const long long avail = 232448LL - 1024 - (long long)sizeof(TcSmall) - (long long)nch * 16 * 512;
+    const long long avail = (long long)kSmemLimit - 1024 - (long long)sizeof(TcSmall) - (long long)nch * 16 * 512;
     long long ns = avail / kSlotBytes;
     if (ns > kMaxSlots) ns = kMaxSlots;
     return (int)ns;
@@ -1200,24 +810,28 @@ static int slots_for(int nch) {
 // Query heads of one key/value group stacked into one work unit: the largest of 8, 4, 2, 1 that divides the group
 // and keeps the stacked queries within one query block (a second block would stream the keys again, which is what
 // a second unit does as well, with narrower tiles).
-static int stack_for(int G, int N) {
+static int tc_stack_for(int G, int N) {
     for (int s = 8; s > 1; s >>= 1)
-        if (G % s == 0 && s * N <= kQBlock) return s;
+        if (G % s == 0 && s * N <= kMaxQ) return s;
     return 1;
 }
 
+// The per-sequence prefix sums of tiles and cost units are 32-bit: bound the largest launch so that they cannot
+// wrap (a sequence of L_max keys and 192 nodes costs at most 2 * (tiles + 4) * 64 units per head).
 bool tc_supported(const AttentionArgs& a) {
-    return a.G >= 1 && a.H % a.G == 0 && a.N <= MCSD_MAX_NODES && a.B <= kMaxBatchTc && encode_fn() != nullptr;
+    if (!(a.G >= 1 && a.H % a.G == 0 && a.N <= MCSD_MAX_NODES && a.B <= kMaxBatchTc && encode_fn() != nullptr)) return false;
+    const long long tiles = (long long)a.L_max / kTile + 4;
+    return (long long)a.B * tiles * 2 * 64 < (1LL << 30);
 }
 
 size_t tc_workspace_bytes(int, int, int N, int, int) {
     if (N > MCSD_MAX_NODES) return 0;
-    return align_up((size_t)2 * kMaxCtas * 2 * 128 * sizeof(float), 256) +
-           align_up((size_t)2 * kMaxCtas * 128 * 128 * sizeof(float), 256) + (size_t)65536 * 2 * kSoftmaxGroups * sizeof(int);
+    return align_up((size_t)2 * kMaxCtas * 2 * kMaxQ * sizeof(float), 256) +
+           align_up((size_t)2 * kMaxCtas * kMaxQ * 128 * sizeof(float), 256) + (size_t)65536 * 2 * 4 * sizeof(int);
 }
 
 template <int NCH>
-static int launch_tc(const CUtensorMap* maps, const TcParams& p, int grid, size_t smem_bytes, cudaStream_t stream) {
+static int launch_tc(const TcLaunch& l, size_t smem_bytes, cudaStream_t stream) {
     // the opt-in to large dynamic shared memory is per device: done on the first launch on each device
     static std::mutex mu;
     static bool done[64] = {};
@@ -1225,10 +839,10 @@ static int launch_tc(const CUtensorMap* maps, const TcParams& p, int grid, size_
     MCSD_CUDA_CHECK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64 || !done[dev]) {
         std::lock_guard<std::mutex> lock(mu);
-        MCSD_CUDA_CHECK(cudaFuncSetAttribute(tree_attention_tc_kernel<NCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+        MCSD_CUDA_CHECK(cudaFuncSetAttribute(tree_attention_tc_kernel<NCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
         if (dev >= 0 && dev < 64) done[dev] = true;
     }
-    tree_attention_tc_kernel<NCH><<<grid, kTcThreads, smem_bytes, stream>>>(maps[0], maps[1], maps[2], maps[3], maps[4], p);
+    tree_attention_tc_kernel<NCH><<<l.grid, kTcThreads, smem_bytes, stream>>>(l.maps[0], l.maps[1], l.maps[2], l.maps[3], l.maps[4], l.p);
     MCSD_CUDA_CHECK(cudaGetLastError());
     return MCSD_OK;
 }
@@ -1236,21 +850,22 @@ static int launch_tc(const CUtensorMap* maps, const TcParams& p, int grid, size_
 int tree_attention_tc(const AttentionArgs& a, WorkspaceHeader* header, void* scratch, size_t scratch_bytes,
                       cudaStream_t stream) {
     if (scratch_bytes < tc_workspace_bytes(a.B, a.H, a.N, a.D, a.L_max)) return MCSD_ERR_WORKSPACE_TOO_SMALL;
-    const int S = stack_for(a.G, a.N);          // query heads per work unit
+    const int S = tc_stack_for(a.G, a.N);       // query heads per work unit
     const int nch = chunks_for(a.N * S);
     const int npadq = nch * 16;
-    const int ns = slots_for(nch);
+    const bool wide = nch > 4;
+    const int ns = wide ? slots_for_wide(nch) : slots_for(nch);
     if (ns < 4) return MCSD_ERR_BAD_SHAPE;
     const int bh = a.B * (a.H / S);             // work units: (sequence, S query heads of one key/value group)
     const int bh_kv = a.B * (a.H / a.G);
 
-    CUtensorMap maps[5];
+    TcLaunch l;
     const bool have_cache = a.L_max > 0;
-    bool ok = make_map(&maps[0], a.q, a.N, bh, npadq, S);
-    ok = ok && make_map(&maps[1], have_cache ? a.k_cache : a.k_tree, have_cache ? a.L_max : a.N, bh_kv, kTile);
-    ok = ok && make_map(&maps[2], have_cache ? a.v_cache : a.v_tree, have_cache ? a.L_max : a.N, bh_kv, kTile);
-    ok = ok && make_map(&maps[3], a.k_tree, a.N, bh_kv, kTile);
-    ok = ok && make_map(&maps[4], a.v_tree, a.N, bh_kv, kTile);
+    bool ok = make_map(&l.maps[0], a.q, a.N, bh, npadq, S);
+    ok = ok && make_map(&l.maps[1], have_cache ? a.k_cache : a.k_tree, have_cache ? a.L_max : a.N, bh_kv, kTile);
+    ok = ok && make_map(&l.maps[2], have_cache ? a.v_cache : a.v_tree, have_cache ? a.L_max : a.N, bh_kv, kTile);
+    ok = ok && make_map(&l.maps[3], a.k_tree, a.N, bh_kv, kTile);
+    ok = ok && make_map(&l.maps[4], a.v_tree, a.N, bh_kv, kTile);
     if (!ok) { set_last_cuda_error(cudaErrorInvalidValue); return MCSD_ERR_CUDA; }
 
     int dev = 0, sms = 0;
@@ -1261,9 +876,9 @@ int tree_attention_tc(const AttentionArgs& a, WorkspaceHeader* header, void* scr
         sms_dev = dev;
     }
     sms = sms_cached;
-    const int grid = sms < kMaxCtas ? sms : kMaxCtas;
+    l.grid = sms < kMaxCtas ? sms : kMaxCtas;
 
-    TcParams p;
+    TcParams& p = l.p;
     p.out = static_cast<__nv_bfloat16*>(a.out);
     p.seq_lens = a.seq_lens;
     p.n_active = a.n_active;
@@ -1276,19 +891,18 @@ int tree_attention_tc(const AttentionArgs& a, WorkspaceHeader* header, void* scr
     p.group = a.G;
     p.scale_log2 = a.scale * 1.4426950408889634f;
     p.part_ml = static_cast<float*>(scratch);
-    p.part_o = reinterpret_cast<float*>(static_cast<char*>(scratch) + align_up((size_t)2 * kMaxCtas * 2 * 128 * sizeof(float), 256));
-    p.counters = reinterpret_cast<int*>(reinterpret_cast<char*>(p.part_o) + align_up((size_t)2 * kMaxCtas * 128 * 128 * sizeof(float), 256));
+    p.part_o = reinterpret_cast<float*>(static_cast<char*>(scratch) + align_up((size_t)2 * kMaxCtas * 2 * kMaxQ * sizeof(float), 256));
+    p.counters = reinterpret_cast<int*>(reinterpret_cast<char*>(p.part_o) + align_up((size_t)2 * kMaxCtas * kMaxQ * 128 * sizeof(float), 256));
     p.header = header;
     p.n_slots = ns;
     p.npadq = npadq;
-    const size_t smem_bytes = 1024 + (size_t)ns * kSlotBytes + (size_t)npadq * 512 + sizeof(TcSmall);
 
     int st;
-    switch (nch) {
-        case 3: st = launch_tc<3>(maps, p, grid, smem_bytes, stream); break;
-        case 4: st = launch_tc<4>(maps, p, grid, smem_bytes, stream); break;
-        case 7: st = launch_tc<7>(maps, p, grid, smem_bytes, stream); break;
-        default: st = launch_tc<8>(maps, p, grid, smem_bytes, stream); break;
+    if (wide) {
+        st = launch_tc_wide(nch, l, stream);
+    } else {
+        const size_t smem_bytes = 1024 + (size_t)ns * kSlotBytes + (size_t)npadq * 512 + sizeof(TcSmall);
+        st = nch == 3 ? launch_tc<3>(l, smem_bytes, stream) : launch_tc<4>(l, smem_bytes, stream);
     }
     if (st != MCSD_OK) return st;
     count_launches(1);

@@ -1,0 +1,363 @@
+// Shared pieces of the two tcgen05 tree-attention kernels (Section 2.2 of the paper): launch parameters, inline-PTX
+// wrappers (mbarrier, TMA, tcgen05), and the bookkeeping that cuts the flattened (sequence, head, query block,
+// key tile) space into per-block ranges of equal cost.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "attention.cuh"
+
+namespace mcsd {
+
+constexpr int kTile = 128;                    // keys per tile
+constexpr int kSlotBytes = kTile * 128 * 2;   // one K or V tile: 128 rows x 128 bf16
+constexpr int kSlabBytes = kTile * 128;       // 64 of the 128 columns: rows of 128 bytes (the TMA swizzle span)
+constexpr int kMaxSlots = 6;
+constexpr int kMaxBatchTc = 256;
+constexpr int kTmemCols = 512;
+constexpr float kLazyTau = 8.0f;              // raise the reference maximum only beyond 2^8
+constexpr int kMaxCtas = 160;                 // partial slots are provisioned for this many thread blocks
+constexpr int kMaxParts = kMaxCtas;           // a work item is cut into at most one piece per thread block
+constexpr int kMaxQ = 160;                    // queries per work item in the widest instantiation (stride of the partials)
+constexpr long long kSpinCycles = 4000000000LL;   // about two seconds
+constexpr int kSmemLimit = 232448;            // dynamic shared memory a block may opt in to
+
+// Tiles and cost of the sequences before b, per head.
+struct TileIndex {
+    int cum_tiles[kMaxBatchTc + 1];
+    int cum_w[kMaxBatchTc + 1];
+};
+
+struct TcParams {
+    __nv_bfloat16* out;
+    const int32_t* seq_lens;
+    const int32_t* n_active;
+    const uint64_t* anc;
+    int words;
+    int B, H, N, L_max;      // H: work units per sequence = query heads / G; N tree nodes (= tree keys)
+    int G, g_shift;          // query heads stacked into one work unit (1, 2, 4 or 8 = 1 << g_shift): its G * N queries
+                             // are taken node-major, query j = head j % G of the unit, node j / G
+    int Hkv, group;          // key/value heads, and query heads per key/value head (a multiple of G): unit u of a
+                             // sequence reads key/value head u * G / group
+    float scale_log2;
+    float* part_ml;      // [2 * kMaxCtas][2][kMaxQ]
+    float* part_o;       // [2 * kMaxCtas][kMaxQ][128]
+    int* counters;       // [B * H][query block][softmax group] arrivals per split work item; zero between launches
+    WorkspaceHeader* header;
+    int n_slots;
+    int npadq;           // rows of the Q box = 16 * (template chunk count)
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(void* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(void* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(void* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(void* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  Returns false if the wait ran out or another role already gave up (abort_flag, in shared memory);
+// `where` names the wait in the workspace header.
+static __device__ __noinline__ bool mbar_wait_slow(void* bar, uint32_t parity, int* abort_flag, WorkspaceHeader* header, int where) {
+    const long long t0 = clock64();
+    for (uint32_t it = 0;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 255u) {
+            if (*(volatile int*)abort_flag) return false;
+            if (clock64() - t0 > kSpinCycles) {
+                *(volatile int*)abort_flag = 1;
+                header->detail = where;
+                header->status = MCSD_ERR_TIMEOUT;
+                __threadfence();
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, int* abort_flag, WorkspaceHeader* header, int where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, header, where);
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, void* bar, int x, int y, int z) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z) : "memory");
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, void* bar, int x, int y, int z, int w) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(void* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The same two instructions for a warp that executes them convergently: one elected lane issues.  (The lane that
+// issued the MMAs must also issue the commit that tracks them; elect.sync picks the same lane every time.)
+__device__ __forceinline__ void tc_mma_elect(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p, e;\n\t"
+        "elect.sync _|e, 0xffffffff;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "@e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_commit_elect(void* bar) {
+    asm volatile(
+        "{\n\t.reg .pred e;\n\t"
+        "elect.sync _|e, 0xffffffff;\n\t"
+        "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(smem_u32(bar)) : "memory");
+}
+// eight consecutive fp32 columns of this thread's TMEM lane; the caller waits with tc_wait_ld()
+__device__ __forceinline__ void tc_ld8(uint32_t taddr, float* v) {
+    uint32_t r[8];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+        : "r"(taddr) : "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ float tc_ld1(uint32_t taddr) {
+    float v;
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=f"(v) : "r"(taddr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void tc_st1(uint32_t taddr, float v) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x1.b32 [%0], {%1};" ::"r"(taddr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Calls f(j, values of 8-column group j) for the first ncg of a thread's column groups, one tensor-memory round
+// trip per group.  ncg is uniform per warp.
+template <int CPT, typename F>
+__device__ __forceinline__ void sweep_groups(uint32_t taddr, int ncg, F&& f) {
+#pragma unroll
+    for (int j = 0; j < CPT; ++j) {
+        if (j < ncg) {
+            float buf[8];
+            tc_ld8(taddr + 8 * j, buf);
+            tc_wait_ld();
+            f(j, buf);
+        }
+    }
+}
+__device__ __forceinline__ void tc_st8(uint32_t taddr, const float* v) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+        ::"r"(taddr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])),
+          "r"(__float_as_uint(v[3])), "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])),
+          "r"(__float_as_uint(v[7])) : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float warp_max_f32(float v) {
+    float r;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+    return r;
+}
+// named barrier `id` over the 128 threads of one softmax warpgroup, returning the OR of `pred`
+__device__ __forceinline__ bool group_sync_any(int id, bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %2, 0;\n\t"
+        "bar.red.or.pred q, %1, 128, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r) : "r"(id), "r"((uint32_t)pred) : "memory");
+    return r != 0;
+}
+
+// Shared-memory matrix descriptor of tcgen05.mma: start address, leading/stride byte offsets (all >> 4),
+// descriptor version 1, swizzle mode in the top bits (0 = none, 2 = 128-byte).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+           (1ull << 46) | ((uint64_t)layout << 61);
+}
+// Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, M = 128, N = n, operand major-ness.
+__device__ __forceinline__ uint32_t instr_desc(int n, int a_mn_major, int b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+// ------------------------------------------------------------------ tile bookkeeping
+// Queries are processed in blocks of at most QB (the tensor-memory budget: 128, or 160 in the widest kernel); a
+// tree with more stacked queries makes each (sequence, head) two work items that read the same keys.  Tiles per
+// work item: prefix tiles, then tree tiles.  Everything below is a function of (QB, wide) so that both kernels
+// and all thread blocks of a launch cut the tile space alike.
+__device__ __forceinline__ int kv_tiles_of(int L, int Nb) {
+    return Nb > 0 ? (L + kTile - 1) / kTile + (Nb + kTile - 1) / kTile : 0;
+}
+template <int QB>
+__device__ __forceinline__ int tiles_of(int L, int Nb, int G) {
+    return kv_tiles_of(L, Nb) * ((Nb * G + QB - 1) / QB);
+}
+
+struct Segment {
+    int b, h, lt, Tb, L, Nb, nP;
+    int qb, q0, Nq, Tkv;      // query block, its first query, its query count, tiles per query block
+};
+
+template <int QB>
+__device__ __forceinline__ void locate(const TileIndex* ix, const TcParams& p, long long t, Segment& s) {
+    int lo = 0, hi = p.B;                      // find b with H*cum[b] <= t < H*cum[b+1]
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if ((long long)p.H * ix->cum_tiles[mid] <= t) lo = mid; else hi = mid;
+    }
+    s.b = lo;
+    s.L = min(max(p.seq_lens[lo], 0), p.L_max);
+    s.Nb = p.n_active ? min(max(p.n_active[lo], 0), p.N) : p.N;
+    s.Tb = ix->cum_tiles[lo + 1] - ix->cum_tiles[lo];
+    s.nP = (s.L + kTile - 1) / kTile;
+    const long long r = t - (long long)p.H * ix->cum_tiles[lo];
+    s.h = (int)(r / s.Tb);
+    const int rem = (int)(r % s.Tb);
+    s.Tkv = kv_tiles_of(s.L, s.Nb);
+    s.qb = rem / s.Tkv;
+    s.lt = rem % s.Tkv;
+    s.q0 = s.qb * QB;
+    s.Nq = min(QB, s.Nb * p.G - s.q0);
+}
+
+// Cost of one tile in units of about 100 cycles, measured on these kernels.  Launches for up to 64 query columns:
+// flat up to 32 queries (the key/value stream sets the pace), then growing with the columns the softmax threads
+// cover.  Wide launches: nearly flat.  Thread blocks get equal cost, not equal tile counts, so that sequences with
+// deep trees do not make their blocks finish late.
+__device__ __forceinline__ int tile_weight(int Nq, bool wide) {
+    return wide ? 27 + Nq / 19 : 24 + (max(0, Nq - 32) * 9) / 32;
+}
+// Fixed cost of a work item (pipeline fill and drain, first-tile reference, row sums, output of Nq columns),
+// carried by its first tile.
+__device__ __forceinline__ int item_weight(int Nq, bool wide) {
+    return (wide ? 100 : 30) + (Nq * 5) / 8;
+}
+template <int QB>
+__device__ __forceinline__ int head_weight(int L, int Nk, int G, bool wide) {  // cost of one (sequence, head): all query blocks
+    const int tkv = kv_tiles_of(L, Nk);
+    const int Nb = Nk * G;                                        // stacked queries
+    int w = 0;
+    for (int q0 = 0; q0 < Nb; q0 += QB) w += tkv * tile_weight(min(QB, Nb - q0), wide) + item_weight(min(QB, Nb - q0), wide);
+    return w;
+}
+// cumulative cost of the tiles before the one a Segment points at
+template <int QB>
+__device__ __forceinline__ long long weight_before(const TileIndex* ix, const TcParams& p, const Segment& s, bool wide) {
+    long long w = (long long)p.H * ix->cum_w[s.b] + (long long)s.h * (ix->cum_w[s.b + 1] - ix->cum_w[s.b]);
+    if (s.qb) w += (long long)s.Tkv * tile_weight(QB, wide) + item_weight(QB, wide);
+    return w + (long long)s.lt * tile_weight(s.Nq, wide) + (s.lt > 0 ? item_weight(s.Nq, wide) : 0);
+}
+// Tile t belongs to block floor(weight_before(t) * G / total_w).  First tile of block c: the first tile whose
+// cumulative cost reaches ceil(c * total_w / G).
+template <int QB>
+__device__ __forceinline__ long long first_tile_of_block(const TileIndex* ix, const TcParams& p, int c, int G, long long total_w,
+                                                         long long total_tiles, bool wide) {
+    const long long wt = ((long long)c * total_w + G - 1) / G;
+    if (wt >= total_w) return total_tiles;
+    int lo = 0, hi = p.B;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if ((long long)p.H * ix->cum_w[mid] <= wt) lo = mid; else hi = mid;
+    }
+    const int L = min(max(p.seq_lens[lo], 0), p.L_max);
+    const int Nk = p.n_active ? min(max(p.n_active[lo], 0), p.N) : p.N;
+    const int tkv = kv_tiles_of(L, Nk);
+    const int Nb = Nk * p.G;                                      // stacked queries
+    const int wh = ix->cum_w[lo + 1] - ix->cum_w[lo], tb = ix->cum_tiles[lo + 1] - ix->cum_tiles[lo];
+    const long long rem = wt - (long long)p.H * ix->cum_w[lo];
+    const int h = (int)(rem / wh);
+    int r2 = (int)(rem % wh);
+    long long t = (long long)p.H * ix->cum_tiles[lo] + (long long)h * tb;
+    // inside a work item the tiles start at cost 0, f + w, f + 2w, ... (f = fixed cost on the first tile)
+    const int w0 = tile_weight(min(QB, Nb), wide), f0 = item_weight(min(QB, Nb), wide);
+    if (r2 >= tkv * w0 + f0 && Nb > QB) {              // inside the second query block
+        r2 -= tkv * w0 + f0;
+        t += tkv;
+        const int w1 = tile_weight(Nb - QB, wide), f1 = item_weight(Nb - QB, wide);
+        return r2 == 0 ? t : t + max(1, (r2 - f1 + w1 - 1) / w1);
+    }
+    return r2 == 0 ? t : t + max(1, (r2 - f0 + w0 - 1) / w0);
+}
+template <int QB>
+__device__ __forceinline__ int block_of_tile(const TileIndex* ix, const TcParams& p, long long t, int G, long long total_w, bool wide) {
+    Segment s;
+    locate<QB>(ix, p, t, s);
+    return (int)min((long long)G - 1, weight_before<QB>(ix, p, s, wide) * G / total_w);
+}
+
+// Per-block set-up shared by both kernels: tiles and cost per sequence, their prefix sums, the number of blocks
+// that get work and the two ends of this block's range.  Ends with a __syncthreads(); all threads must call it.
+template <int QB>
+__device__ __forceinline__ void plan_ranges(TileIndex* ix, const TcParams& p, bool wide, int* n_blocks, long long* range) {
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    for (int b = tid; b < p.B; b += nthr) {
+        const int L = min(max(p.seq_lens[b], 0), p.L_max);
+        const int Nb = p.n_active ? min(max(p.n_active[b], 0), p.N) : p.N;
+        ix->cum_tiles[b + 1] = tiles_of<QB>(L, Nb, p.G);
+        ix->cum_w[b + 1] = head_weight<QB>(L, Nb, p.G, wide);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int acc = 0, accw = 0;
+        ix->cum_tiles[0] = 0;
+        ix->cum_w[0] = 0;
+        for (int b = 1; b <= p.B; ++b) {
+            acc += ix->cum_tiles[b]; ix->cum_tiles[b] = acc;
+            accw += ix->cum_w[b]; ix->cum_w[b] = accw;
+        }
+        // No block's share of the cost may be smaller than the heaviest tile, so that consecutive tiles never skip
+        // a block: every working block then owns at least one tile and the blocks sharing a work item are consecutive.
+        const long long tot_w = (long long)p.H * accw;
+        *n_blocks = (int)max(1LL, min((long long)gridDim.x, tot_w / (tile_weight(QB, wide) + item_weight(QB, wide))));
+    }
+    __syncthreads();
+    if (tid == 0 || tid == 32) {               // the two ends of this block's range, side by side
+        const long long tot = (long long)p.H * ix->cum_tiles[p.B], tot_w = (long long)p.H * ix->cum_w[p.B];
+        const int nb = *n_blocks, which = tid >> 5;
+        range[which] = (tot > 0 && (int)blockIdx.x < nb) ? first_tile_of_block<QB>(ix, p, (int)blockIdx.x + which, nb, tot_w, tot, wide) : 0;
+    }
+    __syncthreads();
+}
+
+// ------------------------------------------------------------------ host side (attention_tc.cu)
+struct TcLaunch {
+    CUtensorMap maps[5];     // Q, key cache, value cache, tree keys, tree values
+    TcParams p;
+    int grid;
+};
+// widest kernel: 4 softmax warpgroups, up to 160 queries per work item (attention_tc_wide.cu)
+int launch_tc_wide(int nch, const TcLaunch& l, cudaStream_t stream);
+int slots_for_wide(int nch);
+
+}  // namespace mcsd

@@ -1,0 +1,752 @@
+// Tree attention (Section 2.2 of the paper) on tcgen05 tensor cores for wide trees: 65 to 160 query columns per
+// work item in one pass over the keys (the paper's many-candidate regime: fork width 16 and more, the target-
+// initialised forests of Section 3.1).  Same transposed formulation and the same persistent, cost-weighted
+// split-KV schedule as the kernel of attention_tc.cu:
+//     S^T[key][query] = K_tile * Q^T,   O^T[d][query] += V_tile^T * P^T,   l[query] += P * 1
+// with 128 keys on the MMA M dimension and up to 160 queries on N.  Tensor memory: S^T twice (columns 0, 160),
+// O^T (320), row sums (480 for queries 0..127, 496 for queries 128..159) = all 512 columns.
+//
+// What differs from the narrow kernel:
+//   * three softmax warpgroups (12 warps, 128 registers per thread) split the query columns of every tile; measured
+//     against two groups (168 registers) and four (96 registers, spills) on the wide workloads, three is fastest;
+//   * the probabilities of a tile are produced in one optimistic sweep (scores shifted by the running reference,
+//     checked against the lazy threshold, exponentiated, packed to bf16 in registers, tensor memory read two column
+//     groups per round trip); the sweep is redone only when the vote of a group fires;
+//   * row sums come from the tensor cores (P^T read as an MN-major A operand against a matrix of ones) and are
+//     accumulated in tensor memory across the tiles of a segment like O^T; they are touched by a thread only when
+//     the reference moves and in the epilogue;
+//   * the reference of a segment starts from the scores of the first key of its first full tile instead of an
+//     exact column maximum: any reference that no score exceeds by more than 2^8 gives the same result, and a key
+//     that does exceed it raises the vote like anywhere else.  (Segments that start on a masked tile take the
+//     exact path.)
+//
+//   * the MMA warp runs its loop convergently and one elected lane issues; descriptors are built once and advanced
+//     by constants, and there are two commits per tile (S^T done = scores ready and key slot free; products done =
+//     value slot and P^T free), because a tcgen05.mma of these shapes takes 40-60 cycles and the instructions
+//     between two of them would otherwise pace the tensor pipe;
+//   * the producer issues loads in the order in which slots come free (K0 K1 V0 K2 V1 ...), about two tiles ahead.
+//
+// Warp roles (480 threads): warps 0-11 softmax / mask / epilogue / merge, warp 12 TMA producer, warp 13 MMA issuer
+// and owner of the tensor-memory allocation, warp 14 bookkeeping.  Every mbarrier wait is bounded.
+#include <mutex>
+#include <type_traits>
+
+#include "attention_tc_common.cuh"
+
+namespace mcsd {
+
+constexpr int kWG = 3;                          // softmax warpgroups
+constexpr int kWProducerWarp = 4 * kWG, kWMmaWarp = kWProducerWarp + 1, kWHelperWarp = kWMmaWarp + 1;
+constexpr int kWideThreads = 32 * (kWHelperWarp + 1);
+constexpr int kWColS1 = 160, kWColO = 320, kWColL = 480, kWColL2 = 496;
+constexpr int kWSlots = 4;                      // ring slots that fit next to Q and P^T of 112..160 queries
+
+struct TcSmallWide {
+    unsigned long long slot_full[kWSlots];   // [0], [1]: key tile of even / odd tiles, [2], [3]: value tile
+    unsigned long long s_full[2];            // S^T of even / odd tiles finished: scores ready, key slot and (last tile) Q free
+    unsigned long long pv_done[2];           // products of even / odd tiles finished: value slot and P^T free, O^T and l current
+    unsigned long long p_full, q_full, drain, info_ready;
+    uint32_t tmem_base;
+    int abort_flag;
+    int merge_parts[kWG];              // > 0: this block finished a split work item last and merges it
+    int piece_parts[2];                // pieces of the work items at the two ends of this block's range
+    unsigned short piece_slot[2][kMaxParts];
+    long long range[2];
+    int n_blocks;
+    alignas(16) float m_ref[kWG][64];  // running reference of a group's own query columns (at most 56)
+    alignas(16) float alpha[kWG][64];  // rescale factors of a slow-path tile; in the epilogue 1/l (or l)
+    alignas(16) float wred[kWG][4][64];
+    alignas(16) unsigned long long dmask[MCSD_MAX_NODES][3];   // transposed ancestor bitsets
+    TileIndex ix;
+    alignas(128) __nv_bfloat16 ones[256];   // 16 x 16 matrix of ones: B operand of the row-sum product
+};
+static_assert(sizeof(TcSmallWide) <= kSmemLimit - 1024 - kWSlots * 32768 - 160 * 512, "TcSmallWide grew: four ring slots no longer fit");
+
+// 64 bits of a 192-bit row starting at bit `start` (bits past the row read as zero)
+__device__ __forceinline__ unsigned long long bits_from(const unsigned long long* w, int start) {
+    const int wi = start >> 6, sh = start & 63;
+    unsigned long long lo = w[wi] >> sh;
+    if (sh != 0 && wi < 2) lo |= w[wi + 1] << (64 - sh);
+    return lo;
+}
+
+template <int NCH>
+__global__ void __launch_bounds__(kWideThreads, 1)
+tree_attention_tc_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kc,
+                              const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kt,
+                              const __grid_constant__ CUtensorMap tm_vt, const TcParams p) {
+    static_assert(NCH == 7 || NCH == 8 || NCH == 10, "padded query columns: 112, 128 or 160");
+    constexpr int QB = NCH == 10 ? kMaxQ : 128;    // queries per work item
+    constexpr int CPT = (2 * NCH + kWG - 1) / kWG; // 8-column groups per thread, at most
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    unsigned char* ring = smem;                  // four 32 KB slots: keys of even / odd tiles, values of even / odd tiles
+    unsigned char* p_buf = ring + (size_t)kWSlots * kSlotBytes;
+    unsigned char* q_buf = p_buf + (size_t)p.npadq * 256;
+    TcSmallWide* sm = reinterpret_cast<TcSmallWide*>(q_buf + (size_t)p.npadq * 256);
+    const TileIndex* ix = &sm->ix;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int cta = blockIdx.x;
+
+    // ---- set-up
+    if (tid < 256) {
+        sm->ones[tid] = __float2bfloat16_rn(1.0f);
+        fence_async_smem();                      // read by the tensor cores through the async proxy
+    }
+    if (tid == 0) {
+        for (int i = 0; i < kWSlots; ++i) mbar_init(&sm->slot_full[i], 1);
+        mbar_init(&sm->s_full[0], 1);
+        mbar_init(&sm->s_full[1], 1);
+        mbar_init(&sm->pv_done[0], 1);
+        mbar_init(&sm->pv_done[1], 1);
+        mbar_init(&sm->p_full, 128 * kWG);
+        mbar_init(&sm->q_full, 1);
+        mbar_init(&sm->drain, 1);
+        mbar_init(&sm->info_ready, 1);
+        sm->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    plan_ranges<QB>(&sm->ix, p, true, &sm->n_blocks, sm->range);
+    const long long total = (long long)p.H * ix->cum_tiles[p.B];
+    const long long total_w = (long long)p.H * ix->cum_w[p.B];
+    const int G = sm->n_blocks;
+    const long long t_begin = sm->range[0], t_end = sm->range[1];
+    if (t_begin >= t_end) return;              // uniform for the whole block: nothing allocated yet
+
+    if (warp == kWMmaWarp) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sm->tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *(volatile uint32_t*)&sm->tmem_base;
+    WorkspaceHeader* hdr = p.header;
+    int* const abort_flag = &sm->abort_flag;
+
+    if (warp == kWProducerWarp) {
+        // =========================================================== TMA producer
+        // Tiles of this block are numbered n = 0, 1, ... across its segments.  Key tile n goes to slot n & 1 as soon
+        // as S^T of tile n - 2 has finished, value tile n to slot 2 + (n & 1) as soon as the products of tile n - 2
+        // have; loads are issued in the order in which their slots come free (K0 K1 V0 K2 V1 K3 ...), which keeps
+        // about two tiles in flight.  Each of these waits targets the latest completion its barrier can have
+        // reached (the next one needs the very tile being loaded), so a parity test cannot alias.
+        if (lane == 0) {
+            const uint32_t total_n = (uint32_t)(t_end - t_begin);
+            struct Cursor { long long t; Segment s; int i, cnt; };
+            auto open = [&](Cursor& c) {
+                locate<QB>(ix, p, c.t, c.s);
+                c.cnt = (int)min((long long)(c.s.Tkv - c.s.lt), t_end - c.t);
+                c.i = 0;
+            };
+            Cursor ck, cv;
+            ck.t = cv.t = t_begin;
+            open(ck);
+            cv = ck;
+            bool ok = true;
+            uint32_t nk = 0, nv = 0;                       // loads issued
+            auto load_tile = [&](const Cursor& c, bool values, uint32_t slot) {
+                const int lti = c.s.lt + c.i;
+                const bool tree = lti >= c.s.nP;
+                const int row0 = (tree ? lti - c.s.nP : lti) * kTile;
+                const int bh_kv = c.s.b * p.Hkv + (c.s.h * p.G) / p.group;
+                const CUtensorMap* map = values ? (tree ? &tm_vt : &tm_vc) : (tree ? &tm_kt : &tm_kc);
+                const uint32_t dst = smem_u32(ring) + slot * (uint32_t)kSlotBytes;
+                mbar_expect_tx(&sm->slot_full[slot], (uint32_t)kSlotBytes);
+                tma_load_3d(dst, map, &sm->slot_full[slot], 0, row0, bh_kv);
+                tma_load_3d(dst + kSlabBytes, map, &sm->slot_full[slot], 64, row0, bh_kv);
+            };
+            auto advance = [&](Cursor& c) {
+                c.t += 1;
+                if (++c.i == c.cnt && c.t < t_end) open(c);
+            };
+            for (uint32_t n = 0; n <= total_n && ok; ++n) {
+                if (n < total_n) {
+                    if (ck.i == 0) {
+                        // a new segment: its queries replace the previous segment's once that one's last S^T is done
+                        if (n > 0) ok = mbar_wait(&sm->s_full[(n - 1u) & 1u], ((n - 1u) >> 1) & 1u, abort_flag, hdr, 1);
+                        if (!ok) break;
+                        const int bh = ck.s.b * p.H + ck.s.h;
+                        mbar_expect_tx(&sm->q_full, (uint32_t)p.npadq * 256u);
+                        if (p.G == 1) {
+                            tma_load_3d(smem_u32(q_buf), &tm_q, &sm->q_full, 0, ck.s.q0, bh);
+                            tma_load_3d(smem_u32(q_buf) + (uint32_t)p.npadq * 128u, &tm_q, &sm->q_full, 64, ck.s.q0, bh);
+                        } else {
+                            // grouped queries: a box of all G heads by npadq / G nodes lands node-major, i.e. as stacked
+                            // queries q0, q0 + 1, ...
+                            tma_load_4d(smem_u32(q_buf), &tm_q, &sm->q_full, 0, 0, ck.s.q0 >> p.g_shift, bh);
+                            tma_load_4d(smem_u32(q_buf) + (uint32_t)p.npadq * 128u, &tm_q, &sm->q_full, 64, 0, ck.s.q0 >> p.g_shift, bh);
+                        }
+                    }
+                    if (n >= 2) ok = mbar_wait(&sm->s_full[n & 1u], ((n - 2u) >> 1) & 1u, abort_flag, hdr, 2);
+                    if (!ok) break;
+                    load_tile(ck, false, n & 1u);
+                    ++nk;
+                    advance(ck);
+                }
+                if (n >= 1) {
+                    const uint32_t m = n - 1u;
+                    if (m >= 2) ok = mbar_wait(&sm->pv_done[m & 1u], ((m - 2u) >> 1) & 1u, abort_flag, hdr, 2);
+                    if (!ok) break;
+                    load_tile(cv, true, 2u + (m & 1u));
+                    ++nv;
+                    advance(cv);
+                }
+            }
+            if (!ok) {
+                // gave up: let the copies already issued land before the block exits
+                for (int which = 0; which < 2; ++which) {
+                    const uint32_t cnt_issued = which ? nv : nk;
+                    for (uint32_t x = cnt_issued > 2 ? cnt_issued - 2 : 0; x < cnt_issued; ++x) {
+                        void* bar = &sm->slot_full[2 * which + (x & 1u)];
+                        const long long t0 = clock64();
+                        while (!mbar_try_wait(bar, (x >> 1) & 1u) && clock64() - t0 < kSpinCycles / 8) {}
+                    }
+                }
+            }
+        }
+    } else if (warp == kWHelperWarp) {
+        // =========================================================== bookkeeping, off everybody's critical path
+        if (lane == 0) {
+            for (int which = 0; which < 2; ++which) {
+                Segment sp;
+                locate<QB>(ix, p, which == 0 ? t_begin : t_end - 1, sp);
+                const long long at = which == 0 ? t_begin : t_end - 1;
+                const long long t0 = at - sp.lt, t1 = t0 + sp.Tkv;
+                int nparts = 0;
+                const bool shared = which == 0 ? (t0 < t_begin || t1 > t_end) : (t0 > t_begin && t1 > t_end);
+                if (shared) {
+                    const int c_lo = block_of_tile<QB>(ix, p, t0, G, total_w, true);
+                    const int c_hi = block_of_tile<QB>(ix, p, t1 - 1, G, total_w, true);
+                    nparts = min(c_hi - c_lo + 1, kMaxParts);
+                    int others = 0;
+                    for (int i = 0; i < nparts; ++i) {
+                        if (c_lo + i == cta) continue;
+                        const long long start = first_tile_of_block<QB>(ix, p, c_lo + i, G, total_w, total, true);
+                        sm->piece_slot[which][others++] = (unsigned short)(2 * (c_lo + i) + (t0 > start ? 1 : 0));
+                    }
+                }
+                sm->piece_parts[which] = nparts;
+            }
+            mbar_arrive(&sm->info_ready);
+        }
+    } else if (warp == kWMmaWarp) {
+        // =========================================================== MMA issuer
+        // The whole warp walks the loop (waits included) and one elected lane issues each tensor-core instruction
+        // and each commit; shared-memory descriptors are built once and advanced by constants, so that the few
+        // instructions between two MMAs do not pace the tensor pipe (small-N products take only 40-60 cycles).
+        {
+            long long t = t_begin;
+            uint32_t g = 0, seg = 0;
+            bool ok = true;
+            const uint32_t ring_a = smem_u32(ring), q_a = smem_u32(q_buf), p_a = smem_u32(p_buf);
+            const uint32_t idesc_l = instr_desc(16, 1, 0);
+            const uint64_t dk0 = smem_desc(ring_a, 16, 1024, 2);                       // key slot 0, first 16 head dims
+            const uint64_t dv0 = smem_desc(ring_a + 2 * kSlotBytes, kSlabBytes, 1024, 2);   // value slot 0, first 16 keys
+            const uint64_t dq0 = smem_desc(q_a, 16, 1024, 2);
+            const uint64_t dp0 = smem_desc(p_a, 128, 2048, 0);                         // P^T: B operand of O^T, A operand of l
+            const uint64_t d1 = smem_desc(smem_u32(sm->ones), 128, 256, 0);
+            const uint32_t q_slab = ((uint32_t)p.npadq * 128u) >> 4;                   // second 64 head dims of Q
+            while (t < t_end && ok) {
+                Segment s;
+                locate<QB>(ix, p, t, s);
+                const int cnt = (int)min((long long)(s.Tkv - s.lt), t_end - t);
+                const int npad = (s.Nq + 15) & ~15;
+                const uint32_t idesc_s = instr_desc(npad, 0, 0), idesc_pv = instr_desc(npad, 1, 1);
+                const bool two = NCH == 10 && s.Nq > 128;
+                ok = mbar_wait(&sm->q_full, seg & 1u, abort_flag, hdr, 3);
+                for (int i = 0; i <= cnt && ok; ++i) {
+                    if (i < cnt) {
+                        const uint32_t gi = g + (uint32_t)i, sb = gi & 1u;
+                        ok = mbar_wait(&sm->slot_full[sb], (gi >> 1) & 1u, abort_flag, hdr, 4);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint64_t da = dk0 + sb * (uint32_t)(kSlotBytes >> 4);
+                        const uint32_t d_s = tmem + (sb ? kWColS1 : 0);
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            // 16 of the 128 head dims per MMA: slab k/4, 32-byte step inside the swizzled row
+                            tc_mma_elect(d_s, da + (uint32_t)((k >> 2) * (kSlabBytes >> 4) + (k & 3) * 2),
+                                         dq0 + ((k >> 2) * q_slab + (uint32_t)(k & 3) * 2u), idesc_s, k > 0);
+                        }
+                        tc_commit_elect(&sm->s_full[sb]);
+                    }
+                    if (i >= 1) {
+                        const uint32_t gj = g + (uint32_t)(i - 1), vb = gj & 1u;
+                        ok = mbar_wait(&sm->slot_full[2u + vb], (gj >> 1) & 1u, abort_flag, hdr, 5);
+                        if (!ok) break;
+                        ok = mbar_wait(&sm->p_full, gj & 1u, abort_flag, hdr, 6);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint64_t da = dv0 + vb * (uint32_t)(kSlotBytes >> 4);
+                        const uint32_t first = (i == 1) ? 0u : 1u;      // the segment's first product overwrites
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            // 16 keys per MMA.  V^T: 8-key groups 1 KB apart; P^T: 8-key groups 128 B apart.
+                            tc_mma_elect(tmem + kWColO, da + (uint32_t)(k * (2048 >> 4)), dp0 + (uint32_t)(k * (256 >> 4)), idesc_pv,
+                                         first | (uint32_t)(k > 0));
+                        }
+                        // Row sums: l[query][.] += P[query][key] * ones[key][.], P^T read as the A operand (queries on
+                        // the accumulator's lanes); queries 128.. take a second product into their own columns.
+#pragma unroll
+                        for (int k = 0; k < 8; ++k)
+                            tc_mma_elect(tmem + kWColL, dp0 + (uint32_t)(k * (256 >> 4)), d1, idesc_l, first | (uint32_t)(k > 0));
+                        if (two) {
+#pragma unroll
+                            for (int k = 0; k < 8; ++k)
+                                tc_mma_elect(tmem + kWColL2, dp0 + (uint32_t)((16 * 2048 + k * 256) >> 4), d1, idesc_l,
+                                             first | (uint32_t)(k > 0));
+                        }
+                        tc_commit_elect(&sm->pv_done[vb]);
+                    }
+                }
+                g += (uint32_t)cnt;
+                ++seg;
+                t += cnt;
+            }
+            // all MMAs issued by this warp must have finished before tensor memory is released
+            tc_commit_elect(&sm->drain);
+            {
+                const long long t0 = clock64();
+                while (!mbar_try_wait(&sm->drain, 0) && clock64() - t0 < kSpinCycles) {}
+            }
+        }
+    } else {
+        // =========================================================== softmax / mask / epilogue
+        const int wg = warp >> 2, wq = warp & 3;
+        const int r = tid & 127;                       // key row of a tile = TMEM lane
+        const int bar_id = 1 + wg;
+        float* const mref = sm->m_ref[wg];
+        float* const alph = sm->alpha[wg];
+        // dmask[t] = set of stacked queries that may see tree key t: the ancestor bitsets transposed (staged through
+        // the P^T buffer, which is free until the first tile is finished).
+        {
+            unsigned long long* anc_s = reinterpret_cast<unsigned long long*>(p_buf);
+            const int n_words = p.N * p.words;                   // at most 192 * 3 words = 4.5 KB
+            for (int i = tid; i < n_words; i += 128 * kWG) anc_s[i] = p.anc[i];
+            asm volatile("bar.sync %0, %1;" ::"n"(kWG + 1), "n"(128 * kWG) : "memory");
+            const int NQ = p.N * p.G;                            // stacked queries: query j belongs to node j / G
+            const int n_chunks = (NQ + 31) >> 5;
+            const uint32_t* anc32 = reinterpret_cast<const uint32_t*>(anc_s);
+            for (int idx = tid; idx < p.N * 6; idx += 128 * kWG) {
+                const int c = idx / p.N, t = idx - c * p.N;
+                uint32_t piece = 0;
+                if (c < n_chunks) {
+                    const uint32_t* col = anc32 + (t >> 5);          // 32-bit half of the 64-bit word that holds bit t
+                    const int n_end = min(32, NQ - 32 * c);
+#pragma unroll 8
+                    for (int i = 0; i < n_end; ++i)
+                        piece |= ((col[(size_t)((32 * c + i) >> p.g_shift) * p.words * 2] >> (t & 31)) & 1u) << i;
+                }
+                reinterpret_cast<uint32_t*>(&sm->dmask[t][0])[c] = piece;
+            }
+            asm volatile("bar.sync %0, %1;" ::"n"(kWG + 1), "n"(128 * kWG) : "memory");
+        }
+        const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
+        long long t = t_begin;
+        uint32_t g = 0;
+        bool failed = false;
+        while (t < t_end) {
+            Segment s;
+            locate<QB>(ix, p, t, s);
+            const int cnt = (int)min((long long)(s.Tkv - s.lt), t_end - t);
+            const int bh = s.b * p.H + s.h;
+            // the groups split the segment's 8-column groups as evenly as possible
+            const int ng8 = (s.Nq + 7) >> 3;
+            const int base = ng8 / kWG, rem = ng8 % kWG;
+            const int g0 = wg * base + min(wg, rem);
+            const int ncg = base + (wg < rem ? 1 : 0);           // 8-column groups of this thread in this segment
+            const int col0 = g0 * 8;
+            // Row sums: lane q of the first set of row-sum columns holds the sum of query q, lane q - 128 of the second
+            // set that of query q >= 128; the 16 columns of a set are identical copies, and group wg only ever
+            // touches copy wg (a rescale is a read-modify-write that must not race with another group's).  A warp's
+            // 32 lanes hold queries of one set only, so the set is chosen per warp (tcgen05.ld/st are warp-wide).
+            const bool set2 = (128 + 32 * wq < col0 + 8 * ncg) && (128 + 32 * wq + 32 > col0);
+            const int oq_c = set2 ? 128 + r : r;
+            const int oq = (oq_c >= col0 && oq_c < col0 + 8 * ncg) ? oq_c : -1;   // this thread's query, if of this group
+            const uint32_t l_addr = tmem + lane_addr + (set2 ? kWColL2 : kWColL) + wg;
+            if (r < ncg * 8) mref[r] = -INFINITY;
+            if (group_sync_any(bar_id, failed)) { failed = true; break; }
+
+            for (int i = 0; i < cnt; ++i) {
+                const uint32_t gi = g + (uint32_t)i, sb = gi & 1u;
+                const int lti = s.lt + i;
+                const bool tree = lti >= s.nP;
+                const int row0 = (tree ? lti - s.nP : lti) * kTile;
+                const int valid = min(kTile, (tree ? s.Nb : s.L) - row0);
+                const bool full_tile = !tree && valid == kTile;   // every key visible to every query: no masking
+                // queries that may see this thread's key (bit n), shifted to this thread's first column
+                unsigned long long cm = 0;
+                if (!full_tile && r < valid) {
+                    const int nrem = s.Nq - col0;
+                    cm = nrem >= 64 ? ~0ull : (nrem > 0 ? ((1ull << nrem) - 1ull) : 0ull);
+                    if (tree) cm &= bits_from(sm->dmask[row0 + r], s.q0 + col0);
+                }
+                if (!mbar_wait(&sm->s_full[sb], (gi >> 1) & 1u, abort_flag, hdr, 7)) failed = true;
+                tc_fence_after();
+                const uint32_t s_addr = tmem + lane_addr + (sb ? kWColS1 : 0) + col0;
+
+                // ---- the sweep: scores of this thread's columns, shifted, checked, exponentiated, packed; tensor memory
+                // is read SB column groups per round trip (what the 128 registers of a 15-warp block allow)
+                constexpr int SB = 2;
+                uint32_t pk[CPT][4];
+                float dmax = -INFINITY;
+                auto make_probs = [&](auto masked_tag) {
+                    constexpr bool MASKED = decltype(masked_tag)::value;
+#pragma unroll
+                    for (int j0 = 0; j0 < CPT; j0 += SB) {
+                        if (j0 < ncg) {
+                            float y[SB][8];
+#pragma unroll
+                            for (int jj = 0; jj < SB; ++jj)
+                                if (j0 + jj < CPT && j0 + jj < ncg) tc_ld8(s_addr + 8 * (j0 + jj), y[jj]);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int jj = 0; jj < SB; ++jj) {
+                                const int j = j0 + jj;
+                                if (j < CPT && j < ncg) {
+                                    const float4 m0 = *reinterpret_cast<const float4*>(&mref[8 * j]);
+                                    const float4 m1 = *reinterpret_cast<const float4*>(&mref[8 * j + 4]);
+                                    const float mr[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+                                    const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
+                                    float yy[8];
+#pragma unroll
+                                    for (int k = 0; k < 8; ++k) {
+                                        yy[k] = fmaf(y[jj][k], p.scale_log2, -mr[k]);
+                                        if (MASKED && !((bits >> k) & 1u)) yy[k] = -INFINITY;
+                                    }
+                                    dmax = fmaxf(dmax, fmaxf(fmaxf(fmaxf(yy[0], yy[1]), fmaxf(yy[2], yy[3])),
+                                                             fmaxf(fmaxf(yy[4], yy[5]), fmaxf(yy[6], yy[7]))));
+#pragma unroll
+                                    for (int k = 0; k < 8; k += 2) {
+                                        __nv_bfloat162 h2 = __floats2bfloat162_rn(ex2_approx(yy[k]), ex2_approx(yy[k + 1]));
+                                        pk[j][k >> 1] = *reinterpret_cast<uint32_t*>(&h2);
+                                    }
+                                }
+                            }
+                        }
+                    }
+                };
+                if (i == 0 && full_tile) {
+                    // reference of a new segment: the scores of the tile's first key (see the file header)
+                    if (wq == 0) {
+#pragma unroll
+                        for (int j = 0; j < CPT; ++j) {
+                            if (j < ncg) {
+                                float v[8];
+                                tc_ld8(s_addr + 8 * j, v);
+                                tc_wait_ld();
+                                if (lane == 0) {
+#pragma unroll
+                                    for (int k = 0; k < 8; ++k) mref[8 * j + k] = v[k] * p.scale_log2;
+                                }
+                            }
+                        }
+                    }
+                    group_sync_any(bar_id, false);
+                }
+                if (full_tile) make_probs(std::false_type{}); else make_probs(std::true_type{});
+
+                if (group_sync_any(bar_id, dmax > kLazyTau || failed)) {
+                    if (*(volatile int*)&sm->abort_flag) { failed = true; break; }
+                    // ---- slow path: exact per-query maxima of this tile, new reference, rescale what was accumulated
+#pragma unroll
+                    for (int j = 0; j < CPT; ++j) {
+                        if (j < ncg) {
+                            float v[8];
+                            tc_ld8(s_addr + 8 * j, v);
+                            tc_wait_ld();
+                            const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
+                            float mine = -INFINITY;
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const float x = (full_tile || ((bits >> k) & 1u)) ? v[k] * p.scale_log2 : -INFINITY;
+                                const float mx = warp_max_f32(x);
+                                if (lane == k) mine = mx;
+                            }
+                            if (lane < 8) sm->wred[wg][wq][8 * j + lane] = mine;
+                        }
+                    }
+                    group_sync_any(bar_id, false);
+                    bool need = false;
+                    if (r < ncg * 8) {
+                        const float tm = fmaxf(fmaxf(sm->wred[wg][0][r], sm->wred[wg][1][r]),
+                                               fmaxf(sm->wred[wg][2][r], sm->wred[wg][3][r]));
+                        const float mo = mref[r];
+                        float a = 1.f;
+                        if (tm > mo) {
+                            a = (mo == -INFINITY) ? 0.f : exp2f(mo - tm);
+                            mref[r] = tm;
+                            need = (i > 0) && (mo != -INFINITY);
+                        }
+                        alph[r] = a;
+                    }
+                    const bool rescale = group_sync_any(bar_id, need);
+                    if (gi > 0 && !mbar_wait(&sm->pv_done[(gi - 1u) & 1u], ((gi - 1u) >> 1) & 1u, abort_flag, hdr, 8)) failed = true;
+                    if (rescale) {
+                        tc_fence_after();
+                        {                                // the row sum accumulated so far belongs to the old reference
+                            const float lp = tc_ld1(l_addr);
+                            tc_wait_ld();
+                            tc_st1(l_addr, oq >= 0 ? lp * alph[oq - col0] : lp);
+                        }
+#pragma unroll
+                        for (int j = 0; j < CPT; ++j) {
+                            if (j < ncg) {
+                                float o[8];
+                                tc_ld8(tmem + lane_addr + kWColO + col0 + 8 * j, o);
+                                tc_wait_ld();
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) o[k] *= alph[8 * j + k];
+                                tc_st8(tmem + lane_addr + kWColO + col0 + 8 * j, o);
+                            }
+                        }
+                        tc_wait_st();
+                    }
+                    dmax = -INFINITY;
+                    if (full_tile) make_probs(std::false_type{}); else make_probs(std::true_type{});
+                }
+
+                // P buffer must no longer be read by the previous tile's MMA; this wait also keeps every thread
+                // within one phase of the p_full barrier
+                if (gi > 0 && !mbar_wait(&sm->pv_done[(gi - 1u) & 1u], ((gi - 1u) >> 1) & 1u, abort_flag, hdr, 8)) failed = true;
+#pragma unroll
+                for (int j = 0; j < CPT; ++j)
+                    if (j < ncg)
+                        *reinterpret_cast<uint4*>(p_buf + (size_t)(g0 + j) * 2048 + (size_t)r * 16) =
+                            make_uint4(pk[j][0], pk[j][1], pk[j][2], pk[j][3]);
+                // rows of the V tile past the end of the prefix / tree may hold anything: make them zero
+                if (wg == 0 && valid < kTile) {
+                    const uint32_t slot = 2u + sb;
+                    if (!mbar_wait(&sm->slot_full[slot], (gi >> 1) & 1u, abort_flag, hdr, 9)) failed = true;
+                    if (r >= valid && !failed) {
+                        uint4* z0 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + (size_t)r * 128);
+                        uint4* z1 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + kSlabBytes + (size_t)r * 128);
+#pragma unroll
+                        for (int x = 0; x < 8; ++x) { z0[x] = make_uint4(0, 0, 0, 0); z1[x] = make_uint4(0, 0, 0, 0); }
+                    }
+                }
+                fence_async_smem();
+                tc_fence_before();
+                mbar_arrive(&sm->p_full);
+            }
+            if (group_sync_any(bar_id, failed)) { failed = true; break; }
+
+            // ---- epilogue of the segment: each group finishes its own query columns
+            const uint32_t glast = g + (uint32_t)cnt - 1u;
+            const bool full = (cnt == s.Tkv);
+            const int slot_id = 2 * cta + (t > t_begin ? 1 : 0);
+            if (!mbar_wait(&sm->pv_done[glast & 1u], (glast >> 1) & 1u, abort_flag, hdr, 10)) failed = true;
+            tc_fence_after();
+            const float l = tc_ld1(l_addr);
+            tc_wait_ld();
+            if (oq >= 0) {
+                // the row sum of query oq sits in this thread's lane: hand it to the threads that finish its column
+                if (full) {
+                    alph[oq - col0] = l > 0.f ? 1.f / l : 0.f;
+                } else {
+                    alph[oq - col0] = l;               // kept for the merge below
+                    p.part_ml[((size_t)slot_id * 2 + 0) * kMaxQ + oq] = mref[oq - col0];
+                    p.part_ml[((size_t)slot_id * 2 + 1) * kMaxQ + oq] = l;
+                }
+            }
+            group_sync_any(bar_id, false);
+            // O^T rows of this thread, one column group per tensor-memory round trip (registers)
+            constexpr int EB = 1;
+#pragma unroll
+            for (int j0 = 0; j0 < CPT; j0 += EB) {
+                if (j0 < ncg) {
+                    float o[EB][8];
+#pragma unroll
+                    for (int jj = 0; jj < EB; ++jj)
+                        if (j0 + jj < CPT && j0 + jj < ncg) tc_ld8(tmem + lane_addr + kWColO + col0 + 8 * (j0 + jj), o[jj]);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int jj = 0; jj < EB; ++jj) {
+                        const int j = j0 + jj;
+                        if (j < CPT && j < ncg) {
+                            if (full) {
+                                // Thread r holds head dim r of eight queries.  An 8 x 8 transpose inside every group of
+                                // eight lanes (three butterfly stages) leaves lane 8a + k with eight consecutive head
+                                // dims of query k: one 16-byte store per thread instead of eight 2-byte ones.
+                                float v[8];
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) v[k] = o[jj][k] * alph[8 * j + k];
+#pragma unroll
+                                for (int m = 4; m > 0; m >>= 1) {
+                                    const bool up = lane & m;
+#pragma unroll
+                                    for (int x = 0; x < 8; ++x) {
+                                        if (x & m) continue;
+                                        const float send = up ? v[x] : v[x | m];
+                                        const float got = __shfl_xor_sync(0xffffffffu, send, m);
+                                        if (up) v[x] = got; else v[x | m] = got;
+                                    }
+                                }
+                                const int n = col0 + 8 * j + (lane & 7);
+                                if (n < s.Nq) {
+                                    uint4 w;
+                                    __nv_bfloat162 h;
+                                    h = __floats2bfloat162_rn(v[0], v[1]); w.x = *reinterpret_cast<uint32_t*>(&h);
+                                    h = __floats2bfloat162_rn(v[2], v[3]); w.y = *reinterpret_cast<uint32_t*>(&h);
+                                    h = __floats2bfloat162_rn(v[4], v[5]); w.z = *reinterpret_cast<uint32_t*>(&h);
+                                    h = __floats2bfloat162_rn(v[6], v[7]); w.w = *reinterpret_cast<uint32_t*>(&h);
+                                    const int jq = s.q0 + n;          // stacked query: head jq % G of the group, node jq / G
+                                    *reinterpret_cast<uint4*>(p.out + (((size_t)bh * p.G + (jq & (p.G - 1))) * p.N + (jq >> p.g_shift)) * 128 +
+                                                              32 * wq + (lane & 24)) = w;
+                                }
+                            } else {
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) {
+                                    const int n = col0 + 8 * j + k;
+                                    if (n < s.Nq) p.part_o[((size_t)slot_id * kMaxQ + n) * 128 + r] = o[jj][k];
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            if (!full) {
+                // Split-KV combine: every block that finished a piece of this work item takes a ticket; the last
+                // one merges the other pieces (read back from the workspace) with its own, which is still in
+                // tensor memory.  The softmax groups own disjoint query columns and run this protocol independently.
+                __threadfence();
+                group_sync_any(bar_id, false);
+                const int which = slot_id & 1;
+                if (r == 0) {
+                    if (!mbar_wait(&sm->info_ready, 0, abort_flag, hdr, 12)) failed = true;
+                    int* counter = p.counters + ((size_t)bh * 2 + s.qb) * 4 + wg;
+                    const int nparts = sm->piece_parts[which];
+                    sm->merge_parts[wg] = nparts;
+                    const int old = atomicAdd(counter, 1);
+                    if (old == nparts - 1) {
+                        *(volatile int*)counter = 0;              // nobody else arrives in this launch: ready for the next one
+                        __threadfence();                          // acquire: the other pieces' partials are visible
+                    } else {
+                        sm->merge_parts[wg] = 0;                  // not the last: nothing more to do
+                    }
+                }
+                group_sync_any(bar_id, false);
+                const int nparts = sm->merge_parts[wg];
+                if (nparts > 0) {
+                    // One dependent round trip to the workspace per piece and batch of column groups: all O^T loads
+                    // of a piece are issued first; while they are in flight the thread that owns a query column folds
+                    // the piece's (m, l) into its running reference and normaliser and leaves the two rescale factors
+                    // of that column in shared memory; after a group barrier every thread applies them to its rows.
+                    const int np1 = nparts - 1;
+                    float* const fa = &sm->wred[wg][0][0];                   // [piece parity][64]: factor for what we have
+                    float* const fw = &sm->wred[wg][2][0];                   // [piece parity][64]: factor for the new piece
+                    const bool col_owner = r < ncg * 8 && col0 + r < s.Nq;
+                    constexpr int GB = 1;                                    // column groups per batch (what the registers allow)
+#pragma unroll
+                    for (int j0 = 0; j0 < CPT; j0 += GB) {
+                        if (j0 >= ncg) break;
+                        float acc[GB][8];
+#pragma unroll
+                        for (int jj = 0; jj < GB; ++jj)
+                            if (j0 + jj < CPT && j0 + jj < ncg) tc_ld8(tmem + lane_addr + kWColO + col0 + 8 * (j0 + jj), acc[jj]);
+                        tc_wait_ld();
+                        float m_run = col_owner ? mref[r] : -INFINITY;       // of column r, kept by its owner
+                        float l_run2 = col_owner ? alph[r] : 0.f;
+                        for (int i = 0; i < np1; ++i) {
+                            const int slot = sm->piece_slot[which][i];
+                            float os[GB][8];
+#pragma unroll
+                            for (int jj = 0; jj < GB; ++jj)
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) {
+                                    const int n = col0 + 8 * (j0 + jj) + k;
+                                    const bool on = j0 + jj < CPT && j0 + jj < ncg && n < s.Nq;
+                                    os[jj][k] = on ? __ldcg(p.part_o + ((size_t)slot * kMaxQ + n) * 128 + r) : 0.f;
+                                }
+                            float* const fa_i = fa + 64 * (i & 1);
+                            float* const fw_i = fw + 64 * (i & 1);
+                            if (col_owner) {
+                                const float ms = __ldcg(p.part_ml + ((size_t)slot * 2 + 0) * kMaxQ + col0 + r);
+                                const float ls = __ldcg(p.part_ml + ((size_t)slot * 2 + 1) * kMaxQ + col0 + r);
+                                const float mn = fmaxf(m_run, ms);
+                                const float a = (mn == -INFINITY || m_run == -INFINITY) ? 0.f : exp2f(m_run - mn);
+                                const float wgt = (mn == -INFINITY || ms == -INFINITY) ? 0.f : exp2f(ms - mn);
+                                l_run2 = l_run2 * a + ls * wgt;
+                                m_run = mn;
+                                fa_i[r] = a;
+                                fw_i[r] = wgt;
+                            }
+                            group_sync_any(bar_id, false);                   // factors of piece i are in place
+#pragma unroll
+                            for (int jj = 0; jj < GB; ++jj)
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) {
+                                    const int rel = 8 * (j0 + jj) + k;
+                                    if (j0 + jj < CPT && j0 + jj < ncg)
+                                        acc[jj][k] = fmaf(os[jj][k], fw_i[rel], acc[jj][k] * fa_i[rel]);
+                                }
+                            // piece i + 2 reuses these factor slots: by then every thread has passed the barrier of
+                            // piece i + 1, which it reaches only after the loop above
+                        }
+                        // normaliser of every column, then the output rows
+                        group_sync_any(bar_id, false);                       // everybody is done with the factor slots
+                        if (col_owner) fa[r] = l_run2 > 0.f ? 1.f / l_run2 : 0.f;
+                        group_sync_any(bar_id, false);
+#pragma unroll
+                        for (int jj = 0; jj < GB; ++jj)
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const int rel = 8 * (j0 + jj) + k, n = col0 + rel;
+                                if (j0 + jj < CPT && j0 + jj < ncg && n < s.Nq) {
+                                    const int jq = s.q0 + n;
+                                    p.out[(((size_t)bh * p.G + (jq & (p.G - 1))) * p.N + (jq >> p.g_shift)) * 128 + r] =
+                                        __float2bfloat16_rn(acc[jj][k] * fa[rel]);
+                                }
+                            }
+                        group_sync_any(bar_id, false);                       // before the next batch reuses the slots
+                    }
+                }
+            }
+            group_sync_any(bar_id, false);
+            g += (uint32_t)cnt;
+            t += cnt;
+        }
+    }
+
+    // ---- tear-down
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kWMmaWarp) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------ host side
+int slots_for_wide(int) { return kWSlots; }
+
+template <int NCH>
+static int launch_wide(const TcLaunch& l, cudaStream_t stream) {
+    // the opt-in to large dynamic shared memory is per device: done on the first launch on each device
+    static std::mutex mu;
+    static bool done[64] = {};
+    int dev = 0;
+    MCSD_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64 || !done[dev]) {
+        std::lock_guard<std::mutex> lock(mu);
+        MCSD_CUDA_CHECK(cudaFuncSetAttribute(tree_attention_tc_wide_kernel<NCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
+        if (dev >= 0 && dev < 64) done[dev] = true;
+    }
+    const size_t smem_bytes = 1024 + (size_t)kWSlots * kSlotBytes + (size_t)l.p.npadq * 512 + sizeof(TcSmallWide);
+    tree_attention_tc_wide_kernel<NCH><<<l.grid, kWideThreads, smem_bytes, stream>>>(l.maps[0], l.maps[1], l.maps[2], l.maps[3], l.maps[4], l.p);
+    MCSD_CUDA_CHECK(cudaGetLastError());
+    return MCSD_OK;
+}
+
+int launch_tc_wide(int nch, const TcLaunch& l, cudaStream_t stream) {
+    switch (nch) {
+        case 7: return launch_wide<7>(l, stream);
+        case 8: return launch_wide<8>(l, stream);
+        default: return launch_wide<10>(l, stream);
+    }
+}
+
+}  // namespace mcsd
