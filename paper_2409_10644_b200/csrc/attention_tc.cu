@@ -1,83 +1,99 @@
-// Tree attention (Section 2.2 of the paper) on the fifth-generation tensor cores of sm_100a: bf16, head_dim 128.
-// This file: the kernel for up to 64 query columns per work item (trees of up to 64 nodes per head, or fewer
-// nodes with several grouped query heads stacked) and the host side of both tcgen05 kernels; the kernel for wider
-// trees is in attention_tc_wide.cu.
+// Tree attention (Section 2.2 of the paper) on the fifth-generation tensor cores of sm_100a: bf16, head_dim 128,
+// 1 to 160 query columns per work item in one pass over the keys (narrow static trees up to the paper's
+// many-candidate regime: fork width 16 and more, the target-initialised forests of Section 3.1).
 //
 // One persistent thread block per SM walks a contiguous range of 128-key tiles of the flattened
-// (sequence, head, key tile) space, so the K/V stream of every (sequence, head) is read from HBM exactly once
-// and all SMs carry the same cost whatever the batch and the prefix lengths are.  Where a range
-// boundary cuts a (sequence, head), every side writes an unnormalised partial (running maximum, sum, weighted
-// values) and takes a ticket; the block that arrives last combines the partials: split-KV.
+// (sequence, head, query block, key tile) space, so the K/V stream of every (sequence, head) is read from HBM once
+// and all SMs carry the same cost whatever the batch and the prefix lengths are.  Where a range boundary cuts a
+// work item, every side writes an unnormalised partial (reference, sum, weighted values) and takes a ticket; the
+// block that arrives last combines the partials: split-KV with a fused combine.
 //
-// The problem is set up transposed so that the small dimension (tree tokens, 16..64 per head) is the MMA N
-// and the 128 keys of a tile fill the MMA M:
-//     S^T[key][query] = K_tile[key][d] * Q[query][d]^T            (A = K tile, B = Q, both K-major, from TMA)
-//     O^T[d][query]  += V_tile[key][d]^T * P^T[key][query]        (A = V tile read MN-major, B = P^T written
-//                                                                  by the softmax threads, MN-major)
-// Accumulators live in tensor memory: S^T double-buffered (columns 0 and 128), O^T at column 256.
+// The problem is set up transposed so that the small dimension (tree tokens) is the MMA N and the 128 keys of a
+// tile fill the MMA M:
+//     S^T[key][query] = K_tile * Q^T,   O^T[d][query] += V_tile^T * P^T,   l[query] += P * 1
+// (A = K tile and B = Q K-major from TMA; A = V tile read MN-major, B = P^T written MN-major by the softmax
+// threads).  Tensor memory: S^T twice (columns 0, 160), O^T (320), row sums (480 for queries 0..127, 496 for queries
+// 128..159) = all 512 columns.
 //
-// Warp roles (352 threads):
-//   warps 0-7  softmax, two warpgroups that split the query columns of each tile: thread r of a group owns
-//              key row r of the tile = TMEM lane r.  The running reference maximum of a query is only raised
-//              when a score exceeds it by more than 2^8 ("lazy" rescaling): the common tile costs one vote,
-//              and only then are exact column maxima reduced (redux.sync inside a warp, shared memory across
-//              warps) and O^T in tensor memory rescaled.  Row sums are kept per thread and reduced once per
-//              segment.  These threads also apply the tree mask (transposed ancestor bitsets), zero V rows
-//              past the end of a ragged tile and run the epilogue.
-//   warp 8     TMA producer: K and V tiles into a ring of 32 KB slots, Q once per segment.
-//   warp 9     MMA issuer (one thread) and owner of the tensor-memory allocation.
-//   warp 10    bookkeeping (one thread): which other blocks share a work item with this one.
-// Every mbarrier wait is bounded; a wait that runs out raises a flag in the workspace header, all roles drain
-// and the block exits cleanly.
+// How the work is organised:
+//   * three softmax warpgroups (12 warps, 128 registers per thread) split the query columns of every tile; thread r
+//     of a group owns key row r of the tile = TMEM lane r.  Measured against two groups (168 registers) and four
+//     (96 registers, spills) on the wide workloads, three is fastest;
+//   * the probabilities of a tile are produced in one optimistic sweep (scores shifted by the running reference,
+//     checked against the lazy threshold 2^8, exponentiated, packed to bf16 in registers, tensor memory read two
+//     column groups per round trip); only when the vote of a group fires are exact column maxima reduced
+//     (redux.sync inside a warp, shared memory across warps), O^T and l rescaled and the sweep redone;
+//   * row sums come from the tensor cores (P^T read as an MN-major A operand against a matrix of ones) and are
+//     accumulated in tensor memory across the tiles of a segment like O^T; they are touched by a thread only when
+//     the reference moves and in the epilogue;
+//   * the reference of a segment starts from the scores of the first key of its first full tile instead of an
+//     exact column maximum: any reference that no score exceeds by more than 2^8 gives the same result, and a key
+//     that does exceed it raises the vote like anywhere else.  (Segments that start on a masked tile take the
+//     exact path.)
+//   * the MMA warp runs its loop convergently and one elected lane issues; descriptors are built once and advanced
+//     by constants, and there are two commits per tile (S^T done = scores ready and key slot free; products done =
+//     value slot and P^T free), because a tcgen05.mma of these shapes takes 40-60 cycles and the instructions
+//     between two of them would otherwise pace the tensor pipe;
+//   * the producer issues loads in the order in which slots come free (K0 K1 V0 K2 V1 ...), about two tiles ahead.
+//
+// Warp roles (480 threads): warps 0-11 softmax / mask / epilogue / merge, warp 12 TMA producer, warp 13 MMA issuer
+// and owner of the tensor-memory allocation, warp 14 bookkeeping (which other blocks share a work item with this
+// one).  Every mbarrier wait is bounded; a wait that runs out raises a flag in the workspace header, all roles
+// drain and the block exits cleanly.
 #include <mutex>
+#include <type_traits>
 
 #include "attention_tc_common.cuh"
 
 namespace mcsd {
 
-constexpr int kQBlock = 128;                  // queries per work item (this kernel sees at most 64)
-constexpr int kSoftmaxGroups = 2;              // warpgroups that split the query columns of every tile
-constexpr int kProducerWarp = 4 * kSoftmaxGroups, kMmaWarp = kProducerWarp + 1, kHelperWarp = kMmaWarp + 1;
+constexpr int kGroups = 3;                          // softmax warpgroups
+constexpr int kProducerWarp = 4 * kGroups, kMmaWarp = kProducerWarp + 1, kHelperWarp = kMmaWarp + 1;
 constexpr int kTcThreads = 32 * (kHelperWarp + 1);
-constexpr int kColS1 = 128, kColO = 256;      // tensor-memory columns: S^T twice, O^T
-constexpr int kNarrowNodes = 64;              // launches of this kernel have at most 64 stacked queries, so at most 64 nodes
+constexpr int kColS1 = 160, kColO = 320, kColL = 480, kColL2 = 496;
+constexpr int kSlots = 4;                      // ring slots that fit next to Q and P^T of 112..160 queries
 
 struct TcSmall {
-    unsigned long long slot_full[kMaxSlots];
-    unsigned long long slot_empty[kMaxSlots];
-    unsigned long long s_full[2];
-    unsigned long long p_full, pv_done, q_full, q_empty, drain, info_ready;
+    unsigned long long slot_full[kSlots];   // [0], [1]: key tile of even / odd tiles, [2], [3]: value tile
+    unsigned long long s_full[2];            // S^T of even / odd tiles finished: scores ready, key slot and (last tile) Q free
+    unsigned long long pv_done[2];           // products of even / odd tiles finished: value slot and P^T free, O^T and l current
+    unsigned long long p_full, q_full, drain, info_ready;
     uint32_t tmem_base;
     int abort_flag;
-    int merge_parts[kSoftmaxGroups];   // > 0: this block finished a split (sequence, head) last and merges it
-    // pieces of the (at most two) work items this block shares with others: [0] the segment at the start of its
-    // range, [1] the one at the end.  Worked out once by the bookkeeping warp.
-    int piece_parts[2];
+    int merge_parts[kGroups];              // > 0: this block finished a split work item last and merges it
+    int piece_parts[2];                // pieces of the work items at the two ends of this block's range
     unsigned short piece_slot[2][kMaxParts];
-    long long range[2];                // first and one-past-last tile of this block
-    int n_blocks;                      // blocks that got tiles
-    alignas(16) float m_ref[128];
-    alignas(16) float alpha[128];      // rescale factors of a slow-path tile; in the epilogue: 1/l (or l) per query
-    alignas(16) float wred[kSoftmaxGroups][4][64];
-    alignas(16) unsigned long long dmask[kNarrowNodes][3];   // transposed ancestor bitsets: queries that see tree key t
+    long long range[2];
+    int n_blocks;
+    alignas(16) float m_ref[kGroups][64];  // running reference of a group's own query columns (at most 56)
+    alignas(16) float alpha[kGroups][64];  // rescale factors of a slow-path tile; in the epilogue 1/l (or l)
+    alignas(16) float wred[kGroups][4][64];
+    alignas(16) unsigned long long dmask[MCSD_MAX_NODES][3];   // transposed ancestor bitsets
     TileIndex ix;
+    alignas(128) __nv_bfloat16 ones[256];   // 16 x 16 matrix of ones: B operand of the row-sum product
 };
-// the small state must leave room for six 32 KB ring slots next to Q and P^T of a 48-query launch
-static_assert(sizeof(TcSmall) <= kSmemLimit - 1024 - 6 * 32768 - 48 * 512, "TcSmall grew: the 6-slot ring no longer fits");
+static_assert(sizeof(TcSmall) <= kSmemLimit - 1024 - kSlots * 32768 - 160 * 512, "TcSmall grew: four ring slots no longer fit");
 
-// ------------------------------------------------------------------ the kernel
+// 64 bits of a 192-bit row starting at bit `start` (bits past the row read as zero)
+__device__ __forceinline__ unsigned long long bits_from(const unsigned long long* w, int start) {
+    const int wi = start >> 6, sh = start & 63;
+    unsigned long long lo = w[wi] >> sh;
+    if (sh != 0 && wi < 2) lo |= w[wi + 1] << (64 - sh);
+    return lo;
+}
+
 template <int NCH>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kc,
-                         const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kt,
-                         const __grid_constant__ CUtensorMap tm_vt, const TcParams p) {
-    static_assert(NCH <= 4, "wider launches run the kernel of attention_tc_wide.cu");
-    constexpr int QB = kQBlock;
+                              const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kt,
+                              const __grid_constant__ CUtensorMap tm_vt, const TcParams p) {
+    static_assert(NCH == 3 || NCH == 4 || NCH == 7 || NCH == 8 || NCH == 10, "padded query columns: 48, 64, 112, 128 or 160");
+    constexpr int QB = NCH == 10 ? kMaxQ : 128;    // queries per work item
+    constexpr int CPT = (2 * NCH + kGroups - 1) / kGroups; // 8-column groups per thread, at most
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const int NS = p.n_slots;
-    unsigned char* ring = smem;
-    unsigned char* p_buf = ring + (size_t)NS * kSlotBytes;
+    unsigned char* ring = smem;                  // four 32 KB slots: keys of even / odd tiles, values of even / odd tiles
+    unsigned char* p_buf = ring + (size_t)kSlots * kSlotBytes;
     unsigned char* q_buf = p_buf + (size_t)p.npadq * 256;
     TcSmall* sm = reinterpret_cast<TcSmall*>(q_buf + (size_t)p.npadq * 256);
     const TileIndex* ix = &sm->ix;
@@ -85,21 +101,25 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x;
 
-    // ---- set-up: barriers, tile counts per sequence, this block's range, tensor memory
+    // ---- set-up
+    if (tid < 256) {
+        sm->ones[tid] = __float2bfloat16_rn(1.0f);
+        fence_async_smem();                      // read by the tensor cores through the async proxy
+    }
     if (tid == 0) {
-        for (int i = 0; i < kMaxSlots; ++i) { mbar_init(&sm->slot_full[i], 1); mbar_init(&sm->slot_empty[i], 1); }
+        for (int i = 0; i < kSlots; ++i) mbar_init(&sm->slot_full[i], 1);
         mbar_init(&sm->s_full[0], 1);
         mbar_init(&sm->s_full[1], 1);
-        mbar_init(&sm->p_full, 128 * kSoftmaxGroups);
-        mbar_init(&sm->pv_done, 1);
+        mbar_init(&sm->pv_done[0], 1);
+        mbar_init(&sm->pv_done[1], 1);
+        mbar_init(&sm->p_full, 128 * kGroups);
         mbar_init(&sm->q_full, 1);
-        mbar_init(&sm->q_empty, 1);
         mbar_init(&sm->drain, 1);
         mbar_init(&sm->info_ready, 1);
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    plan_ranges<QB>(&sm->ix, p, false, &sm->n_blocks, sm->range);
+    plan_ranges<QB>(&sm->ix, p, &sm->n_blocks, sm->range);
     const long long total = (long long)p.H * ix->cum_tiles[p.B];
     const long long total_w = (long long)p.H * ix->cum_w[p.B];
     const int G = sm->n_blocks;
@@ -119,62 +139,88 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
 
     if (warp == kProducerWarp) {
         // =========================================================== TMA producer
+        // Tiles of this block are numbered n = 0, 1, ... across its segments.  Key tile n goes to slot n & 1 as soon
+        // as S^T of tile n - 2 has finished, value tile n to slot 2 + (n & 1) as soon as the products of tile n - 2
+        // have; loads are issued in the order in which their slots come free (K0 K1 V0 K2 V1 K3 ...), which keeps
+        // about two tiles in flight.  Each of these waits targets the latest completion its barrier can have
+        // reached (the next one needs the very tile being loaded), so a parity test cannot alias.
         if (lane == 0) {
-            long long t = t_begin;
-            uint32_t u = 0, seg = 0;
-            uint32_t slot = 0, phase = 0;              // ring position of use u (kept incrementally: no divisions)
+            const uint32_t total_n = (uint32_t)(t_end - t_begin);
+            struct Cursor { long long t; Segment s; int i, cnt; };
+            auto open = [&](Cursor& c) {
+                locate<QB>(ix, p, c.t, c.s);
+                c.cnt = (int)min((long long)(c.s.Tkv - c.s.lt), t_end - c.t);
+                c.i = 0;
+            };
+            Cursor ck, cv;
+            ck.t = cv.t = t_begin;
+            open(ck);
+            cv = ck;
             bool ok = true;
-            while (t < t_end && ok) {
-                Segment s;
-                locate<QB>(ix, p, t, s);
-                const int cnt = (int)min((long long)(s.Tkv - s.lt), t_end - t);
-                const int bh = s.b * p.H + s.h;
-                const int bh_kv = s.b * p.Hkv + (s.h * p.G) / p.group;
-                ok = mbar_wait(&sm->q_empty, (seg & 1u) ^ 1u, abort_flag, hdr, 1);
-                if (!ok) break;
-                mbar_expect_tx(&sm->q_full, (uint32_t)p.npadq * 256u);
-                if (p.G == 1) {
-                    tma_load_3d(smem_u32(q_buf), &tm_q, &sm->q_full, 0, s.q0, bh);
-                    tma_load_3d(smem_u32(q_buf) + (uint32_t)p.npadq * 128u, &tm_q, &sm->q_full, 64, s.q0, bh);
-                } else {
-                    // grouped queries: the map is (dim, head of the group, node, sequence x key/value head); a box of
-                    // all G heads by npadq / G nodes lands node-major, i.e. as stacked queries q0, q0 + 1, ...
-                    tma_load_4d(smem_u32(q_buf), &tm_q, &sm->q_full, 0, 0, s.q0 >> p.g_shift, bh);
-                    tma_load_4d(smem_u32(q_buf) + (uint32_t)p.npadq * 128u, &tm_q, &sm->q_full, 64, 0, s.q0 >> p.g_shift, bh);
-                }
-                for (int i = 0; i < cnt && ok; ++i) {
-                    const int lti = s.lt + i;
-                    const bool tree = lti >= s.nP;
-                    const int row0 = (tree ? lti - s.nP : lti) * kTile;
-                    for (int kv = 0; kv < 2 && ok; ++kv, ++u) {
-                        ok = mbar_wait(&sm->slot_empty[slot], phase ^ 1u, abort_flag, hdr, 2);
+            uint32_t nk = 0, nv = 0;                       // loads issued
+            auto load_tile = [&](const Cursor& c, bool values, uint32_t slot) {
+                const int lti = c.s.lt + c.i;
+                const bool tree = lti >= c.s.nP;
+                const int row0 = (tree ? lti - c.s.nP : lti) * kTile;
+                const int bh_kv = c.s.b * p.Hkv + (c.s.h * p.G) / p.group;
+                const CUtensorMap* map = values ? (tree ? &tm_vt : &tm_vc) : (tree ? &tm_kt : &tm_kc);
+                const uint32_t dst = smem_u32(ring) + slot * (uint32_t)kSlotBytes;
+                mbar_expect_tx(&sm->slot_full[slot], (uint32_t)kSlotBytes);
+                tma_load_3d(dst, map, &sm->slot_full[slot], 0, row0, bh_kv);
+                tma_load_3d(dst + kSlabBytes, map, &sm->slot_full[slot], 64, row0, bh_kv);
+            };
+            auto advance = [&](Cursor& c) {
+                c.t += 1;
+                if (++c.i == c.cnt && c.t < t_end) open(c);
+            };
+            for (uint32_t n = 0; n <= total_n && ok; ++n) {
+                if (n < total_n) {
+                    if (ck.i == 0) {
+                        // a new segment: its queries replace the previous segment's once that one's last S^T is done
+                        if (n > 0) ok = mbar_wait(&sm->s_full[(n - 1u) & 1u], ((n - 1u) >> 1) & 1u, abort_flag, hdr, 1);
                         if (!ok) break;
-                        const CUtensorMap* map = kv == 0 ? (tree ? &tm_kt : &tm_kc) : (tree ? &tm_vt : &tm_vc);
-                        const uint32_t dst = smem_u32(ring) + slot * (uint32_t)kSlotBytes;
-                        mbar_expect_tx(&sm->slot_full[slot], (uint32_t)kSlotBytes);
-                        tma_load_3d(dst, map, &sm->slot_full[slot], 0, row0, bh_kv);
-                        tma_load_3d(dst + kSlabBytes, map, &sm->slot_full[slot], 64, row0, bh_kv);
-                        if (++slot == (uint32_t)NS) { slot = 0; phase ^= 1u; }
+                        const int bh = ck.s.b * p.H + ck.s.h;
+                        mbar_expect_tx(&sm->q_full, (uint32_t)p.npadq * 256u);
+                        if (p.G == 1) {
+                            tma_load_3d(smem_u32(q_buf), &tm_q, &sm->q_full, 0, ck.s.q0, bh);
+                            tma_load_3d(smem_u32(q_buf) + (uint32_t)p.npadq * 128u, &tm_q, &sm->q_full, 64, ck.s.q0, bh);
+                        } else {
+                            // grouped queries: a box of all G heads by npadq / G nodes lands node-major, i.e. as stacked
+                            // queries q0, q0 + 1, ...
+                            tma_load_4d(smem_u32(q_buf), &tm_q, &sm->q_full, 0, 0, ck.s.q0 >> p.g_shift, bh);
+                            tma_load_4d(smem_u32(q_buf) + (uint32_t)p.npadq * 128u, &tm_q, &sm->q_full, 64, 0, ck.s.q0 >> p.g_shift, bh);
+                        }
                     }
+                    if (n >= 2) ok = mbar_wait(&sm->s_full[n & 1u], ((n - 2u) >> 1) & 1u, abort_flag, hdr, 2);
+                    if (!ok) break;
+                    load_tile(ck, false, n & 1u);
+                    ++nk;
+                    advance(ck);
                 }
-                t += cnt;
-                ++seg;
+                if (n >= 1) {
+                    const uint32_t m = n - 1u;
+                    if (m >= 2) ok = mbar_wait(&sm->pv_done[m & 1u], ((m - 2u) >> 1) & 1u, abort_flag, hdr, 2);
+                    if (!ok) break;
+                    load_tile(cv, true, 2u + (m & 1u));
+                    ++nv;
+                    advance(cv);
+                }
             }
             if (!ok) {
-                // gave up: let copies already issued land before the block exits
-                const uint32_t first = u > (uint32_t)NS ? u - (uint32_t)NS : 0u;
-                for (uint32_t x = first; x < u; ++x) {
-                    void* bar = &sm->slot_full[x % (uint32_t)NS];
-                    const uint32_t par = (x / (uint32_t)NS) & 1u;
-                    const long long t0 = clock64();
-                    while (!mbar_try_wait(bar, par) && clock64() - t0 < kSpinCycles / 8) {}
+                // gave up: let the copies already issued land before the block exits
+                for (int which = 0; which < 2; ++which) {
+                    const uint32_t cnt_issued = which ? nv : nk;
+                    for (uint32_t x = cnt_issued > 2 ? cnt_issued - 2 : 0; x < cnt_issued; ++x) {
+                        void* bar = &sm->slot_full[2 * which + (x & 1u)];
+                        const long long t0 = clock64();
+                        while (!mbar_try_wait(bar, (x >> 1) & 1u) && clock64() - t0 < kSpinCycles / 8) {}
+                    }
                 }
             }
         }
     } else if (warp == kHelperWarp) {
         // =========================================================== bookkeeping, off everybody's critical path
         if (lane == 0) {
-            // which blocks hold the other pieces of the work items this block shares with its neighbours
             for (int which = 0; which < 2; ++which) {
                 Segment sp;
                 locate<QB>(ix, p, which == 0 ? t_begin : t_end - 1, sp);
@@ -183,13 +229,13 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 int nparts = 0;
                 const bool shared = which == 0 ? (t0 < t_begin || t1 > t_end) : (t0 > t_begin && t1 > t_end);
                 if (shared) {
-                    const int c_lo = block_of_tile<QB>(ix, p, t0, G, total_w, false);
-                    const int c_hi = block_of_tile<QB>(ix, p, t1 - 1, G, total_w, false);
+                    const int c_lo = block_of_tile<QB>(ix, p, t0, G, total_w);
+                    const int c_hi = block_of_tile<QB>(ix, p, t1 - 1, G, total_w);
                     nparts = min(c_hi - c_lo + 1, kMaxParts);
                     int others = 0;
                     for (int i = 0; i < nparts; ++i) {
                         if (c_lo + i == cta) continue;
-                        const long long start = first_tile_of_block<QB>(ix, p, c_lo + i, G, total_w, total, false);
+                        const long long start = first_tile_of_block<QB>(ix, p, c_lo + i, G, total_w, total);
                         sm->piece_slot[which][others++] = (unsigned short)(2 * (c_lo + i) + (t0 > start ? 1 : 0));
                     }
                 }
@@ -199,71 +245,80 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         }
     } else if (warp == kMmaWarp) {
         // =========================================================== MMA issuer
-        if (lane == 0) {
+        // The whole warp walks the loop (waits included) and one elected lane issues each tensor-core instruction
+        // and each commit; shared-memory descriptors are built once and advanced by constants, so that the few
+        // instructions between two MMAs do not pace the tensor pipe (small-N products take only 40-60 cycles).
+        {
             long long t = t_begin;
             uint32_t g = 0, seg = 0;
-            // ring positions of the next K tile (uses 0, 2, 4, ...) and the next V tile (uses 1, 3, 5, ...), kept
-            // incrementally: this thread is the pacing one, divisions by the slot count would cost it a tenth
-            uint32_t kslot = 0, kphase = 0, vslot = 1u % (uint32_t)NS, vphase = (1u / (uint32_t)NS) & 1u;
             bool ok = true;
             const uint32_t ring_a = smem_u32(ring), q_a = smem_u32(q_buf), p_a = smem_u32(p_buf);
+            const uint32_t idesc_l = instr_desc(16, 1, 0);
+            const uint64_t dk0 = smem_desc(ring_a, 16, 1024, 2);                       // key slot 0, first 16 head dims
+            const uint64_t dv0 = smem_desc(ring_a + 2 * kSlotBytes, kSlabBytes, 1024, 2);   // value slot 0, first 16 keys
+            const uint64_t dq0 = smem_desc(q_a, 16, 1024, 2);
+            const uint64_t dp0 = smem_desc(p_a, 128, 2048, 0);                         // P^T: B operand of O^T, A operand of l
+            const uint64_t d1 = smem_desc(smem_u32(sm->ones), 128, 256, 0);
+            const uint32_t q_slab = ((uint32_t)p.npadq * 128u) >> 4;                   // second 64 head dims of Q
             while (t < t_end && ok) {
                 Segment s;
                 locate<QB>(ix, p, t, s);
                 const int cnt = (int)min((long long)(s.Tkv - s.lt), t_end - t);
                 const int npad = (s.Nq + 15) & ~15;
                 const uint32_t idesc_s = instr_desc(npad, 0, 0), idesc_pv = instr_desc(npad, 1, 1);
+                const bool two = NCH == 10 && s.Nq > 128;
                 ok = mbar_wait(&sm->q_full, seg & 1u, abort_flag, hdr, 3);
                 for (int i = 0; i <= cnt && ok; ++i) {
                     if (i < cnt) {
                         const uint32_t gi = g + (uint32_t)i, sb = gi & 1u;
-                        const uint32_t slot = kslot;
-                        ok = mbar_wait(&sm->slot_full[slot], kphase, abort_flag, hdr, 4);
+                        ok = mbar_wait(&sm->slot_full[sb], (gi >> 1) & 1u, abort_flag, hdr, 4);
                         if (!ok) break;
-                        kslot += 2u;
-                        if (kslot >= (uint32_t)NS) { kslot -= (uint32_t)NS; kphase ^= 1u; }
                         tc_fence_after();
-                        const uint32_t ka = ring_a + slot * (uint32_t)kSlotBytes;
+                        const uint64_t da = dk0 + sb * (uint32_t)(kSlotBytes >> 4);
+                        const uint32_t d_s = tmem + (sb ? kColS1 : 0);
 #pragma unroll
                         for (int k = 0; k < 8; ++k) {
                             // 16 of the 128 head dims per MMA: slab k/4, 32-byte step inside the swizzled row
-                            const uint64_t da = smem_desc(ka + (k >> 2) * kSlabBytes + (k & 3) * 32, 16, 1024, 2);
-                            const uint64_t db = smem_desc(q_a + (k >> 2) * (uint32_t)p.npadq * 128u + (k & 3) * 32, 16, 1024, 2);
-                            tc_mma(tmem + (sb ? kColS1 : 0), da, db, idesc_s, k > 0);
+                            tc_mma_elect(d_s, da + (uint32_t)((k >> 2) * (kSlabBytes >> 4) + (k & 3) * 2),
+                                         dq0 + ((k >> 2) * q_slab + (uint32_t)(k & 3) * 2u), idesc_s, k > 0);
                         }
-                        tc_commit(&sm->s_full[sb]);
-                        tc_commit(&sm->slot_empty[slot]);
-                        if (i == cnt - 1) tc_commit(&sm->q_empty);
+                        tc_commit_elect(&sm->s_full[sb]);
                     }
                     if (i >= 1) {
-                        const uint32_t gj = g + (uint32_t)(i - 1);
-                        const uint32_t slot = vslot;
-                        ok = mbar_wait(&sm->slot_full[slot], vphase, abort_flag, hdr, 5);
+                        const uint32_t gj = g + (uint32_t)(i - 1), vb = gj & 1u;
+                        ok = mbar_wait(&sm->slot_full[2u + vb], (gj >> 1) & 1u, abort_flag, hdr, 5);
                         if (!ok) break;
-                        vslot += 2u;
-                        if (vslot >= (uint32_t)NS) { vslot -= (uint32_t)NS; vphase ^= 1u; }
                         ok = mbar_wait(&sm->p_full, gj & 1u, abort_flag, hdr, 6);
                         if (!ok) break;
                         tc_fence_after();
-                        const uint32_t va = ring_a + slot * (uint32_t)kSlotBytes;
+                        const uint64_t da = dv0 + vb * (uint32_t)(kSlotBytes >> 4);
+                        const uint32_t first = (i == 1) ? 0u : 1u;      // the segment's first product overwrites
 #pragma unroll
                         for (int k = 0; k < 8; ++k) {
-                            // 16 keys per MMA.  V^T: two 64-dim atoms 16 KB apart (leading), 8-key groups 1 KB apart.
-                            const uint64_t da = smem_desc(va + k * 2048, kSlabBytes, 1024, 2);
-                            // P^T: 8-key groups 128 B apart (leading), 8-query groups 2 KB apart (stride), no swizzle.
-                            const uint64_t db = smem_desc(p_a + k * 256, 128, 2048, 0);
-                            tc_mma(tmem + kColO, da, db, idesc_pv, !(i == 1 && k == 0));
+                            // 16 keys per MMA.  V^T: 8-key groups 1 KB apart; P^T: 8-key groups 128 B apart.
+                            tc_mma_elect(tmem + kColO, da + (uint32_t)(k * (2048 >> 4)), dp0 + (uint32_t)(k * (256 >> 4)), idesc_pv,
+                                         first | (uint32_t)(k > 0));
                         }
-                        tc_commit(&sm->slot_empty[slot]);
-                        tc_commit(&sm->pv_done);
+                        // Row sums: l[query][.] += P[query][key] * ones[key][.], P^T read as the A operand (queries on
+                        // the accumulator's lanes); queries 128.. take a second product into their own columns.
+#pragma unroll
+                        for (int k = 0; k < 8; ++k)
+                            tc_mma_elect(tmem + kColL, dp0 + (uint32_t)(k * (256 >> 4)), d1, idesc_l, first | (uint32_t)(k > 0));
+                        if (two) {
+#pragma unroll
+                            for (int k = 0; k < 8; ++k)
+                                tc_mma_elect(tmem + kColL2, dp0 + (uint32_t)((16 * 2048 + k * 256) >> 4), d1, idesc_l,
+                                             first | (uint32_t)(k > 0));
+                        }
+                        tc_commit_elect(&sm->pv_done[vb]);
                     }
                 }
                 g += (uint32_t)cnt;
                 ++seg;
                 t += cnt;
             }
-            // all MMAs issued by this thread must have finished before tensor memory is released
-            tc_commit(&sm->drain);
+            // all MMAs issued by this warp must have finished before tensor memory is released
+            tc_commit_elect(&sm->drain);
             {
                 const long long t0 = clock64();
                 while (!mbar_try_wait(&sm->drain, 0) && clock64() - t0 < kSpinCycles) {}
@@ -271,35 +326,22 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         }
     } else {
         // =========================================================== softmax / mask / epilogue
-        // Two warpgroups work on the same tile and split its query columns in groups of eight; thread r of
-        // either group owns key row r (TMEM lane r).  Per tile the common case is one pass: load S^T, subtract
-        // the running reference, check that nothing exceeds it by more than 2^kLazyTau (one vote per group),
-        // exponentiate, add to the per-thread row sums and store P^T.  Only when the vote fires (always on the
-        // first tile of a segment) are exact column maxima computed and O^T rescaled.
-        constexpr int CPT = NCH;                       // 8-column groups per thread (two groups share 16*NCH columns)
         const int wg = warp >> 2, wq = warp & 3;
-        const int r = tid & 127;
+        const int r = tid & 127;                       // key row of a tile = TMEM lane
         const int bar_id = 1 + wg;
-        // Reference maxima and rescale factors of this group's own query columns, indexed from the group's first
-        // column: the split of the columns between the groups changes with the segment's query count, and one group
-        // may already be in the next segment while the other still finishes this one.
-        float* const mref = sm->m_ref + 64 * wg;
-        float* const alph = sm->alpha + 64 * wg;
-        // dmask[t] = set of queries that may see tree key t: the ancestor bitsets transposed.  The bitsets are
-        // first copied to shared memory in one coalesced round trip (the P^T buffer is free until the first tile
-        // is finished), then the warps transpose them key by key.
+        float* const mref = sm->m_ref[wg];
+        float* const alph = sm->alpha[wg];
+        // dmask[t] = set of stacked queries that may see tree key t: the ancestor bitsets transposed (staged through
+        // the P^T buffer, which is free until the first tile is finished).
         {
             unsigned long long* anc_s = reinterpret_cast<unsigned long long*>(p_buf);
             const int n_words = p.N * p.words;                   // at most 192 * 3 words = 4.5 KB
-            for (int i = tid; i < n_words; i += 256) anc_s[i] = p.anc[i];
-            asm volatile("bar.sync 3, 256;" ::: "memory");
-            // Transposition, one 32-query piece of one key's row per thread and step (consecutive threads take
-            // consecutive keys, so a warp reads the same word of 32 bitsets in turn: broadcasts, no bank conflicts).
-            // Rows for keys beyond the tree are never read.
+            for (int i = tid; i < n_words; i += 128 * kGroups) anc_s[i] = p.anc[i];
+            asm volatile("bar.sync %0, %1;" ::"n"(kGroups + 1), "n"(128 * kGroups) : "memory");
             const int NQ = p.N * p.G;                            // stacked queries: query j belongs to node j / G
             const int n_chunks = (NQ + 31) >> 5;
             const uint32_t* anc32 = reinterpret_cast<const uint32_t*>(anc_s);
-            for (int idx = tid; idx < p.N * 6; idx += 32 * 4 * kSoftmaxGroups) {
+            for (int idx = tid; idx < p.N * 6; idx += 128 * kGroups) {
                 const int c = idx / p.N, t = idx - c * p.N;
                 uint32_t piece = 0;
                 if (c < n_chunks) {
@@ -311,31 +353,32 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 }
                 reinterpret_cast<uint32_t*>(&sm->dmask[t][0])[c] = piece;
             }
-            // both groups read dmask and will overwrite the staging copy: order both before any tile is processed
-            asm volatile("bar.sync 3, 256;" ::: "memory");
+            asm volatile("bar.sync %0, %1;" ::"n"(kGroups + 1), "n"(128 * kGroups) : "memory");
         }
         const uint32_t lane_addr = (uint32_t)(wq * 32) << 16;
         long long t = t_begin;
-        uint32_t u = 0, g = 0;
+        uint32_t g = 0;
         bool failed = false;
-        float acc_l[CPT][8];
         while (t < t_end) {
             Segment s;
             locate<QB>(ix, p, t, s);
             const int cnt = (int)min((long long)(s.Tkv - s.lt), t_end - t);
             const int bh = s.b * p.H + s.h;
+            // the groups split the segment's 8-column groups as evenly as possible
             const int ng8 = (s.Nq + 7) >> 3;
-            const int half = (ng8 + 1) >> 1;                     // the two groups split the columns evenly
-            const int g0 = wg * half;
-            const int ncg = wg == 0 ? half : ng8 - half;         // 8-column groups of this thread in this segment
+            const int base = ng8 / kGroups, rem = ng8 % kGroups;
+            const int g0 = wg * base + min(wg, rem);
+            const int ncg = base + (wg < rem ? 1 : 0);           // 8-column groups of this thread in this segment
             const int col0 = g0 * 8;
-            const unsigned long long nb_lo = s.Nq >= 64 ? ~0ull : ((1ull << s.Nq) - 1ull);
-            const unsigned long long nb_hi = s.Nq >= 128 ? ~0ull : (s.Nq > 64 ? ((1ull << (s.Nq - 64)) - 1ull) : 0ull);
+            // Row sums: lane q of the first set of row-sum columns holds the sum of query q, lane q - 128 of the second
+            // set that of query q >= 128; the 16 columns of a set are identical copies, and group wg only ever
+            // touches copy wg (a rescale is a read-modify-write that must not race with another group's).  A warp's
+            // 32 lanes hold queries of one set only, so the set is chosen per warp (tcgen05.ld/st are warp-wide).
+            const bool set2 = (128 + 32 * wq < col0 + 8 * ncg) && (128 + 32 * wq + 32 > col0);
+            const int oq_c = set2 ? 128 + r : r;
+            const int oq = (oq_c >= col0 && oq_c < col0 + 8 * ncg) ? oq_c : -1;   // this thread's query, if of this group
+            const uint32_t l_addr = tmem + lane_addr + (set2 ? kColL2 : kColL) + wg;
             if (r < ncg * 8) mref[r] = -INFINITY;
-#pragma unroll
-            for (int j = 0; j < CPT; ++j)
-#pragma unroll
-                for (int k = 0; k < 8; ++k) acc_l[j][k] = 0.f;
             if (group_sync_any(bar_id, failed)) { failed = true; break; }
 
             for (int i = 0; i < cnt; ++i) {
@@ -348,40 +391,75 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 // queries that may see this thread's key (bit n), shifted to this thread's first column
                 unsigned long long cm = 0;
                 if (!full_tile && r < valid) {
-                    unsigned long long c0 = nb_lo, c1 = nb_hi;
-                    if (tree) {                     // bits q0 .. q0+127 of the key's row of the transposed mask
-                        c0 &= sm->dmask[row0 + r][s.qb ? 2 : 0];
-                        c1 &= s.qb ? 0ull : sm->dmask[row0 + r][1];
-                    }
-                    cm = col0 >= 64 ? (c1 >> (col0 - 64)) : (col0 == 0 ? c0 : ((c0 >> col0) | (c1 << (64 - col0))));
+                    const int nrem = s.Nq - col0;
+                    cm = nrem >= 64 ? ~0ull : (nrem > 0 ? ((1ull << nrem) - 1ull) : 0ull);
+                    if (tree) cm &= bits_from(sm->dmask[row0 + r], s.q0 + col0);
                 }
                 if (!mbar_wait(&sm->s_full[sb], (gi >> 1) & 1u, abort_flag, hdr, 7)) failed = true;
                 tc_fence_after();
                 const uint32_t s_addr = tmem + lane_addr + (sb ? kColS1 : 0) + col0;
 
-                // ---- pass A: scores minus the running reference, and the largest excess
-                float y[CPT][8];
+                // ---- the sweep: scores of this thread's columns, shifted, checked, exponentiated, packed; tensor memory
+                // is read SB column groups per round trip (what the 128 registers of a 15-warp block allow)
+                constexpr int SB = 2;
+                uint32_t pk[CPT][4];
                 float dmax = -INFINITY;
+                auto make_probs = [&](auto masked_tag) {
+                    constexpr bool MASKED = decltype(masked_tag)::value;
 #pragma unroll
-                for (int j = 0; j < CPT; ++j)
-                    if (j < ncg) tc_ld8(s_addr + 8 * j, y[j]);
-                tc_wait_ld();
+                    for (int j0 = 0; j0 < CPT; j0 += SB) {
+                        if (j0 < ncg) {
+                            float y[SB][8];
 #pragma unroll
-                for (int j = 0; j < CPT; ++j) {
-                    if (j < ncg) {
-                        const float4 m0 = *reinterpret_cast<const float4*>(&mref[8 * j]);
-                        const float4 m1 = *reinterpret_cast<const float4*>(&mref[8 * j + 4]);
-                        const float mr[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
-                        const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
+                            for (int jj = 0; jj < SB; ++jj)
+                                if (j0 + jj < CPT && j0 + jj < ncg) tc_ld8(s_addr + 8 * (j0 + jj), y[jj]);
+                            tc_wait_ld();
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) {
-                            float yy = fmaf(y[j][k], p.scale_log2, -mr[k]);
-                            if (!full_tile && !((bits >> k) & 1u)) yy = -INFINITY;
-                            dmax = fmaxf(dmax, yy);
-                            y[j][k] = yy;
+                            for (int jj = 0; jj < SB; ++jj) {
+                                const int j = j0 + jj;
+                                if (j < CPT && j < ncg) {
+                                    const float4 m0 = *reinterpret_cast<const float4*>(&mref[8 * j]);
+                                    const float4 m1 = *reinterpret_cast<const float4*>(&mref[8 * j + 4]);
+                                    const float mr[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+                                    const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
+                                    float yy[8];
+#pragma unroll
+                                    for (int k = 0; k < 8; ++k) {
+                                        yy[k] = fmaf(y[jj][k], p.scale_log2, -mr[k]);
+                                        if (MASKED && !((bits >> k) & 1u)) yy[k] = -INFINITY;
+                                    }
+                                    dmax = fmaxf(dmax, fmaxf(fmaxf(fmaxf(yy[0], yy[1]), fmaxf(yy[2], yy[3])),
+                                                             fmaxf(fmaxf(yy[4], yy[5]), fmaxf(yy[6], yy[7]))));
+#pragma unroll
+                                    for (int k = 0; k < 8; k += 2) {
+                                        __nv_bfloat162 h2 = __floats2bfloat162_rn(ex2_approx(yy[k]), ex2_approx(yy[k + 1]));
+                                        pk[j][k >> 1] = *reinterpret_cast<uint32_t*>(&h2);
+                                    }
+                                }
+                            }
                         }
                     }
+                };
+                if (i == 0 && full_tile) {
+                    // reference of a new segment: the scores of the tile's first key (see the file header)
+                    if (wq == 0) {
+#pragma unroll
+                        for (int j = 0; j < CPT; ++j) {
+                            if (j < ncg) {
+                                float v[8];
+                                tc_ld8(s_addr + 8 * j, v);
+                                tc_wait_ld();
+                                if (lane == 0) {
+#pragma unroll
+                                    for (int k = 0; k < 8; ++k) mref[8 * j + k] = v[k] * p.scale_log2;
+                                }
+                            }
+                        }
+                    }
+                    group_sync_any(bar_id, false);
                 }
+                if (full_tile) make_probs(std::false_type{}); else make_probs(std::true_type{});
+
                 if (group_sync_any(bar_id, dmax > kLazyTau || failed)) {
                     if (*(volatile int*)&sm->abort_flag) { failed = true; break; }
                     // ---- slow path: exact per-query maxima of this tile, new reference, rescale what was accumulated
@@ -417,9 +495,14 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                         alph[r] = a;
                     }
                     const bool rescale = group_sync_any(bar_id, need);
-                    if (gi > 0 && !mbar_wait(&sm->pv_done, (gi - 1u) & 1u, abort_flag, hdr, 8)) failed = true;
+                    if (gi > 0 && !mbar_wait(&sm->pv_done[(gi - 1u) & 1u], ((gi - 1u) >> 1) & 1u, abort_flag, hdr, 8)) failed = true;
                     if (rescale) {
                         tc_fence_after();
+                        {                                // the row sum accumulated so far belongs to the old reference
+                            const float lp = tc_ld1(l_addr);
+                            tc_wait_ld();
+                            tc_st1(l_addr, oq >= 0 ? lp * alph[oq - col0] : lp);
+                        }
 #pragma unroll
                         for (int j = 0; j < CPT; ++j) {
                             if (j < ncg) {
@@ -427,59 +510,28 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                                 tc_ld8(tmem + lane_addr + kColO + col0 + 8 * j, o);
                                 tc_wait_ld();
 #pragma unroll
-                                for (int k = 0; k < 8; ++k) {
-                                    const float a = alph[8 * j + k];
-                                    o[k] *= a;
-                                    acc_l[j][k] *= a;
-                                }
+                                for (int k = 0; k < 8; ++k) o[k] *= alph[8 * j + k];
                                 tc_st8(tmem + lane_addr + kColO + col0 + 8 * j, o);
                             }
                         }
                         tc_wait_st();
                     }
-#pragma unroll
-                    for (int j = 0; j < CPT; ++j) {
-                        if (j < ncg) {
-                            float v[8];
-                            tc_ld8(s_addr + 8 * j, v);
-                            tc_wait_ld();
-                            const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                float yy = fmaf(v[k], p.scale_log2, -mref[8 * j + k]);
-                                if (!full_tile && !((bits >> k) & 1u)) yy = -INFINITY;
-                                y[j][k] = yy;
-                            }
-                        }
-                    }
+                    dmax = -INFINITY;
+                    if (full_tile) make_probs(std::false_type{}); else make_probs(std::true_type{});
                 }
 
                 // P buffer must no longer be read by the previous tile's MMA; this wait also keeps every thread
                 // within one phase of the p_full barrier
-                if (gi > 0 && !mbar_wait(&sm->pv_done, (gi - 1u) & 1u, abort_flag, hdr, 8)) failed = true;
-
-                // ---- pass B: probabilities, row sums, P^T for the second MMA
+                if (gi > 0 && !mbar_wait(&sm->pv_done[(gi - 1u) & 1u], ((gi - 1u) >> 1) & 1u, abort_flag, hdr, 8)) failed = true;
 #pragma unroll
-                for (int j = 0; j < CPT; ++j) {
-                    if (j < ncg) {
-                        uint32_t packed[4];
-#pragma unroll
-                        for (int k = 0; k < 8; k += 2) {
-                            // 2^-inf = 0 for masked entries
-                            const float p0 = ex2_approx(y[j][k]), p1 = ex2_approx(y[j][k + 1]);
-                            acc_l[j][k] += p0;
-                            acc_l[j][k + 1] += p1;
-                            __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-                            packed[k >> 1] = *reinterpret_cast<uint32_t*>(&h2);
-                        }
+                for (int j = 0; j < CPT; ++j)
+                    if (j < ncg)
                         *reinterpret_cast<uint4*>(p_buf + (size_t)(g0 + j) * 2048 + (size_t)r * 16) =
-                            make_uint4(packed[0], packed[1], packed[2], packed[3]);
-                    }
-                }
+                            make_uint4(pk[j][0], pk[j][1], pk[j][2], pk[j][3]);
                 // rows of the V tile past the end of the prefix / tree may hold anything: make them zero
                 if (wg == 0 && valid < kTile) {
-                    const uint32_t uv = u + 2u * (uint32_t)i + 1u, slot = uv % (uint32_t)NS;
-                    if (!mbar_wait(&sm->slot_full[slot], (uv / (uint32_t)NS) & 1u, abort_flag, hdr, 9)) failed = true;
+                    const uint32_t slot = 2u + sb;
+                    if (!mbar_wait(&sm->slot_full[slot], (gi >> 1) & 1u, abort_flag, hdr, 9)) failed = true;
                     if (r >= valid && !failed) {
                         uint4* z0 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + (size_t)r * 128);
                         uint4* z1 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + kSlabBytes + (size_t)r * 128);
@@ -497,59 +549,23 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             const uint32_t glast = g + (uint32_t)cnt - 1u;
             const bool full = (cnt == s.Tkv);
             const int slot_id = 2 * cta + (t > t_begin ? 1 : 0);
-            if (!mbar_wait(&sm->pv_done, glast & 1u, abort_flag, hdr, 10)) failed = true;
+            if (!mbar_wait(&sm->pv_done[glast & 1u], (glast >> 1) & 1u, abort_flag, hdr, 10)) failed = true;
             tc_fence_after();
-            // Row sums: every thread holds a partial sum per query; reduce the 8 sums of a column group across the
-            // warp by recursive halving (9 shuffles instead of 40): after the three exchange steps lane L holds the
-            // sum of column (L >> 2) & 7 over its exchange partners, two more steps finish the reduction.
-#pragma unroll
-            for (int j = 0; j < CPT; ++j) {
-                if (j < ncg) {
-                    float v4[4], v2[2], v1;
-                    {
-                        const bool up = lane & 16;
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            const float send = up ? acc_l[j][k] : acc_l[j][k + 4];
-                            const float keep = up ? acc_l[j][k + 4] : acc_l[j][k];
-                            v4[k] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
-                        }
-                    }
-                    {
-                        const bool up = lane & 8;
-#pragma unroll
-                        for (int k = 0; k < 2; ++k) {
-                            const float send = up ? v4[k] : v4[k + 2];
-                            const float keep = up ? v4[k + 2] : v4[k];
-                            v2[k] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
-                        }
-                    }
-                    {
-                        const bool up = lane & 4;
-                        const float send = up ? v2[0] : v2[1];
-                        const float keep = up ? v2[1] : v2[0];
-                        v1 = keep + __shfl_xor_sync(0xffffffffu, send, 4);
-                    }
-                    v1 += __shfl_xor_sync(0xffffffffu, v1, 2);
-                    v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
-                    // lane bits 4,3,2 select column 4*b4 + 2*b3 + b2
-                    if ((lane & 3) == 0) sm->wred[wg][wq][8 * j + ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1)] = v1;
-                }
-            }
-            if (group_sync_any(bar_id, failed)) { failed = true; break; }
-            if (r < ncg * 8) {
-                const float l = (sm->wred[wg][0][r] + sm->wred[wg][1][r]) + (sm->wred[wg][2][r] + sm->wred[wg][3][r]);
+            const float l = tc_ld1(l_addr);
+            tc_wait_ld();
+            if (oq >= 0) {
+                // the row sum of query oq sits in this thread's lane: hand it to the threads that finish its column
                 if (full) {
-                    alph[r] = l > 0.f ? 1.f / l : 0.f;
+                    alph[oq - col0] = l > 0.f ? 1.f / l : 0.f;
                 } else {
-                    alph[r] = l;                   // kept for the merge below
-                    p.part_ml[((size_t)slot_id * 2 + 0) * kMaxQ + col0 + r] = mref[r];
-                    p.part_ml[((size_t)slot_id * 2 + 1) * kMaxQ + col0 + r] = l;
+                    alph[oq - col0] = l;               // kept for the merge below
+                    p.part_ml[((size_t)slot_id * 2 + 0) * kMaxQ + oq] = mref[oq - col0];
+                    p.part_ml[((size_t)slot_id * 2 + 1) * kMaxQ + oq] = l;
                 }
             }
             group_sync_any(bar_id, false);
-            // O^T rows of this thread, up to four column groups per tensor-memory round trip
-            constexpr int EB = CPT < 4 ? CPT : 4;
+            // O^T rows of this thread, one column group per tensor-memory round trip (registers)
+            constexpr int EB = 1;
 #pragma unroll
             for (int j0 = 0; j0 < CPT; j0 += EB) {
                 if (j0 < ncg) {
@@ -560,27 +576,27 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     tc_wait_ld();
 #pragma unroll
                     for (int jj = 0; jj < EB; ++jj) {
-                        if (j0 + jj < CPT && j0 + jj < ncg) {
+                        const int j = j0 + jj;
+                        if (j < CPT && j < ncg) {
                             if (full) {
-                                // Thread r holds head dim r of eight queries.  An 8 x 8 transpose inside every group
-                                // of eight lanes (three butterfly stages) leaves lane 8a + k with eight consecutive
-                                // head dims of query k: one 16-byte store per thread instead of eight 2-byte ones.
-                                // (The same for the fp32 partials measured no faster.)
+                                // Thread r holds head dim r of eight queries.  An 8 x 8 transpose inside every group of
+                                // eight lanes (three butterfly stages) leaves lane 8a + k with eight consecutive head
+                                // dims of query k: one 16-byte store per thread instead of eight 2-byte ones.
                                 float v[8];
 #pragma unroll
-                                for (int k = 0; k < 8; ++k) v[k] = o[jj][k] * alph[8 * (j0 + jj) + k];
+                                for (int k = 0; k < 8; ++k) v[k] = o[jj][k] * alph[8 * j + k];
 #pragma unroll
                                 for (int m = 4; m > 0; m >>= 1) {
                                     const bool up = lane & m;
 #pragma unroll
-                                    for (int i = 0; i < 8; ++i) {
-                                        if (i & m) continue;
-                                        const float send = up ? v[i] : v[i | m];
+                                    for (int x = 0; x < 8; ++x) {
+                                        if (x & m) continue;
+                                        const float send = up ? v[x] : v[x | m];
                                         const float got = __shfl_xor_sync(0xffffffffu, send, m);
-                                        if (up) v[i] = got; else v[i | m] = got;
+                                        if (up) v[x] = got; else v[x | m] = got;
                                     }
                                 }
-                                const int n = col0 + 8 * (j0 + jj) + (lane & 7);
+                                const int n = col0 + 8 * j + (lane & 7);
                                 if (n < s.Nq) {
                                     uint4 w;
                                     __nv_bfloat162 h;
@@ -595,7 +611,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                             } else {
 #pragma unroll
                                 for (int k = 0; k < 8; ++k) {
-                                    const int n = col0 + 8 * (j0 + jj) + k;
+                                    const int n = col0 + 8 * j + k;
                                     if (n < s.Nq) p.part_o[((size_t)slot_id * kMaxQ + n) * 128 + r] = o[jj][k];
                                 }
                             }
@@ -607,7 +623,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             if (!full) {
                 // Split-KV combine: every block that finished a piece of this work item takes a ticket; the last
                 // one merges the other pieces (read back from the workspace) with its own, which is still in
-                // tensor memory.  The two softmax groups own disjoint query columns and run this protocol independently.
+                // tensor memory.  The softmax groups own disjoint query columns and run this protocol independently.
                 __threadfence();
                 group_sync_any(bar_id, false);
                 const int which = slot_id & 1;
@@ -627,17 +643,15 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 group_sync_any(bar_id, false);
                 const int nparts = sm->merge_parts[wg];
                 if (nparts > 0) {
-                    // The other pieces sit in the workspace behind a memory system that is busy streaming keys and
-                    // values, so what counts is the number of dependent round trips: one per piece and batch of
-                    // column groups.  All O^T loads of a piece are issued first; while they are in flight the thread
-                    // that owns a query column fetches the piece's (m, l) for it, folds them into its running
-                    // reference and normaliser and leaves the two rescale factors of that column in shared memory;
-                    // after a group barrier every thread applies them to its rows.
+                    // One dependent round trip to the workspace per piece and batch of column groups: all O^T loads
+                    // of a piece are issued first; while they are in flight the thread that owns a query column folds
+                    // the piece's (m, l) into its running reference and normaliser and leaves the two rescale factors
+                    // of that column in shared memory; after a group barrier every thread applies them to its rows.
                     const int np1 = nparts - 1;
                     float* const fa = &sm->wred[wg][0][0];                   // [piece parity][64]: factor for what we have
                     float* const fw = &sm->wred[wg][2][0];                   // [piece parity][64]: factor for the new piece
                     const bool col_owner = r < ncg * 8 && col0 + r < s.Nq;
-                    constexpr int GB = CPT < 4 ? CPT : 2;                    // column groups per batch (what the registers allow)
+                    constexpr int GB = 1;                                    // column groups per batch (what the registers allow)
 #pragma unroll
                     for (int j0 = 0; j0 < CPT; j0 += GB) {
                         if (j0 >= ncg) break;
@@ -705,7 +719,6 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             }
             group_sync_any(bar_id, false);
             g += (uint32_t)cnt;
-            u += 2u * (uint32_t)cnt;
             t += cnt;
         }
     }
@@ -793,18 +806,11 @@ static bool encode_map(CUtensorMap* map, const void* base, int rows, int bh, int
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Padded query columns of a launch in 16-column chunks: 3 or 4 for the kernel above, 7, 8 or 10 for the wide one
-// (10 = 160 queries in one pass; trees with more stacked queries are cut into blocks of 160).
+// Padded query columns of a launch in 16-column chunks: 3, 4, 7, 8 or 10 (10 = 160 queries in one pass; trees with
+// more stacked queries are cut into blocks of 160).
 static int chunks_for(int nq) {
     const int nch = ((nq < kMaxQ ? nq : kMaxQ) + 15) / 16;
     return nch <= 3 ? 3 : nch <= 4 ? 4 : nch <= 7 ? 7 : nch <= 8 ? 8 : 10;
-}
-
-static int slots_for(int nch) {
-    const long long avail = (long long)kSmemLimit - 1024 - (long long)sizeof(TcSmall) - (long long)nch * 16 * 512;
-    long long ns = avail / kSlotBytes;
-    if (ns > kMaxSlots) ns = kMaxSlots;
-    return (int)ns;
 }
 
 // Query heads of one key/value group stacked into one work unit: the largest of 8, 4, 2, 1 that divides the group
@@ -831,7 +837,7 @@ size_t tc_workspace_bytes(int, int, int N, int, int) {
 }
 
 template <int NCH>
-static int launch_tc(const TcLaunch& l, size_t smem_bytes, cudaStream_t stream) {
+static int launch_tc(const TcLaunch& l, cudaStream_t stream) {
     // the opt-in to large dynamic shared memory is per device: done on the first launch on each device
     static std::mutex mu;
     static bool done[64] = {};
@@ -842,6 +848,7 @@ static int launch_tc(const TcLaunch& l, size_t smem_bytes, cudaStream_t stream) 
         MCSD_CUDA_CHECK(cudaFuncSetAttribute(tree_attention_tc_kernel<NCH>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit));
         if (dev >= 0 && dev < 64) done[dev] = true;
     }
+    const size_t smem_bytes = 1024 + (size_t)kSlots * kSlotBytes + (size_t)l.p.npadq * 512 + sizeof(TcSmall);
     tree_attention_tc_kernel<NCH><<<l.grid, kTcThreads, smem_bytes, stream>>>(l.maps[0], l.maps[1], l.maps[2], l.maps[3], l.maps[4], l.p);
     MCSD_CUDA_CHECK(cudaGetLastError());
     return MCSD_OK;
@@ -853,9 +860,6 @@ int tree_attention_tc(const AttentionArgs& a, WorkspaceHeader* header, void* scr
     const int S = tc_stack_for(a.G, a.N);       // query heads per work unit
     const int nch = chunks_for(a.N * S);
     const int npadq = nch * 16;
-    const bool wide = nch > 4;
-    const int ns = wide ? slots_for_wide(nch) : slots_for(nch);
-    if (ns < 4) return MCSD_ERR_BAD_SHAPE;
     const int bh = a.B * (a.H / S);             // work units: (sequence, S query heads of one key/value group)
     const int bh_kv = a.B * (a.H / a.G);
 
@@ -894,15 +898,16 @@ int tree_attention_tc(const AttentionArgs& a, WorkspaceHeader* header, void* scr
     p.part_o = reinterpret_cast<float*>(static_cast<char*>(scratch) + align_up((size_t)2 * kMaxCtas * 2 * kMaxQ * sizeof(float), 256));
     p.counters = reinterpret_cast<int*>(reinterpret_cast<char*>(p.part_o) + align_up((size_t)2 * kMaxCtas * kMaxQ * 128 * sizeof(float), 256));
     p.header = header;
-    p.n_slots = ns;
+    p.n_slots = kSlots;
     p.npadq = npadq;
 
     int st;
-    if (wide) {
-        st = launch_tc_wide(nch, l, stream);
-    } else {
-        const size_t smem_bytes = 1024 + (size_t)ns * kSlotBytes + (size_t)npadq * 512 + sizeof(TcSmall);
-        st = nch == 3 ? launch_tc<3>(l, smem_bytes, stream) : launch_tc<4>(l, smem_bytes, stream);
+    switch (nch) {
+        case 3: st = launch_tc<3>(l, stream); break;
+        case 4: st = launch_tc<4>(l, stream); break;
+        case 7: st = launch_tc<7>(l, stream); break;
+        case 8: st = launch_tc<8>(l, stream); break;
+        default: st = launch_tc<10>(l, stream); break;
     }
     if (st != MCSD_OK) return st;
     count_launches(1);

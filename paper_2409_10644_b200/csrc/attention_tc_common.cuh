@@ -1,4 +1,4 @@
-// Shared pieces of the two tcgen05 tree-attention kernels (Section 2.2 of the paper): launch parameters, inline-PTX
+// Pieces of the tcgen05 tree-attention kernel (Section 2.2 of the paper) that are not its main loop: launch parameters, inline-PTX
 // wrappers (mbarrier, TMA, tcgen05), and the bookkeeping that cuts the flattened (sequence, head, query block,
 // key tile) space into per-block ranges of equal cost.
 #pragma once
@@ -109,17 +109,7 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-__device__ __forceinline__ void tc_commit(void* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
-}
-// The same two instructions for a warp that executes them convergently: one elected lane issues.  (The lane that
+// tcgen05.mma and tcgen05.commit for a warp that executes them convergently: one elected lane issues.  (The lane that
 // issued the MMAs must also issue the commit that tracks them; elect.sync picks the same lane every time.)
 __device__ __forceinline__ void tc_mma_elect(uint32_t d_tmem, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
@@ -155,20 +145,6 @@ __device__ __forceinline__ void tc_st1(uint32_t taddr, float v) {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x1.b32 [%0], {%1};" ::"r"(taddr), "f"(v) : "memory");
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-// Calls f(j, values of 8-column group j) for the first ncg of a thread's column groups, one tensor-memory round
-// trip per group.  ncg is uniform per warp.
-template <int CPT, typename F>
-__device__ __forceinline__ void sweep_groups(uint32_t taddr, int ncg, F&& f) {
-#pragma unroll
-    for (int j = 0; j < CPT; ++j) {
-        if (j < ncg) {
-            float buf[8];
-            tc_ld8(taddr + 8 * j, buf);
-            tc_wait_ld();
-            f(j, buf);
-        }
-    }
-}
 __device__ __forceinline__ void tc_st8(uint32_t taddr, const float* v) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
@@ -214,8 +190,8 @@ __device__ __forceinline__ uint32_t instr_desc(int n, int a_mn_major, int b_mn_m
 // ------------------------------------------------------------------ tile bookkeeping
 // Queries are processed in blocks of at most QB (the tensor-memory budget: 128, or 160 in the widest kernel); a
 // tree with more stacked queries makes each (sequence, head) two work items that read the same keys.  Tiles per
-// work item: prefix tiles, then tree tiles.  Everything below is a function of (QB, wide) so that both kernels
-// and all thread blocks of a launch cut the tile space alike.
+// work item: prefix tiles, then tree tiles.  Everything below is a pure function of the launch so that all thread
+// blocks cut the tile space alike.
 __device__ __forceinline__ int kv_tiles_of(int L, int Nb) {
     return Nb > 0 ? (L + kTile - 1) / kTile + (Nb + kTile - 1) / kTile : 0;
 }
@@ -251,38 +227,33 @@ __device__ __forceinline__ void locate(const TileIndex* ix, const TcParams& p, l
     s.Nq = min(QB, s.Nb * p.G - s.q0);
 }
 
-// Cost of one tile in units of about 100 cycles, measured on these kernels.  Launches for up to 64 query columns:
-// flat up to 32 queries (the key/value stream sets the pace), then growing with the columns the softmax threads
-// cover.  Wide launches: nearly flat.  Thread blocks get equal cost, not equal tile counts, so that sequences with
-// deep trees do not make their blocks finish late.
-__device__ __forceinline__ int tile_weight(int Nq, bool wide) {
-    return wide ? 27 + Nq / 19 : 24 + (max(0, Nq - 32) * 9) / 32;
-}
-// Fixed cost of a work item (pipeline fill and drain, first-tile reference, row sums, output of Nq columns),
-// carried by its first tile.
-__device__ __forceinline__ int item_weight(int Nq, bool wide) {
-    return (wide ? 100 : 30) + (Nq * 5) / 8;
-}
+// Cost of one tile and fixed cost of a work item in units of about 100 cycles, fitted to per-segment timelines of
+// the kernel.  Thread blocks get equal cost, not equal tile counts, so that sequences with deep trees do not make
+// their blocks finish late.
+__device__ __forceinline__ int tile_weight(int Nq) { return 27 + Nq / 19; }
+// Fixed cost of a work item (pipeline fill and drain, first-tile reference, output of Nq columns), carried by its
+// first tile.
+__device__ __forceinline__ int item_weight(int Nq) { return 100 + (Nq * 5) / 8; }
 template <int QB>
-__device__ __forceinline__ int head_weight(int L, int Nk, int G, bool wide) {  // cost of one (sequence, head): all query blocks
+__device__ __forceinline__ int head_weight(int L, int Nk, int G) {  // cost of one (sequence, head): all query blocks
     const int tkv = kv_tiles_of(L, Nk);
     const int Nb = Nk * G;                                        // stacked queries
     int w = 0;
-    for (int q0 = 0; q0 < Nb; q0 += QB) w += tkv * tile_weight(min(QB, Nb - q0), wide) + item_weight(min(QB, Nb - q0), wide);
+    for (int q0 = 0; q0 < Nb; q0 += QB) w += tkv * tile_weight(min(QB, Nb - q0)) + item_weight(min(QB, Nb - q0));
     return w;
 }
 // cumulative cost of the tiles before the one a Segment points at
 template <int QB>
-__device__ __forceinline__ long long weight_before(const TileIndex* ix, const TcParams& p, const Segment& s, bool wide) {
+__device__ __forceinline__ long long weight_before(const TileIndex* ix, const TcParams& p, const Segment& s) {
     long long w = (long long)p.H * ix->cum_w[s.b] + (long long)s.h * (ix->cum_w[s.b + 1] - ix->cum_w[s.b]);
-    if (s.qb) w += (long long)s.Tkv * tile_weight(QB, wide) + item_weight(QB, wide);
-    return w + (long long)s.lt * tile_weight(s.Nq, wide) + (s.lt > 0 ? item_weight(s.Nq, wide) : 0);
+    if (s.qb) w += (long long)s.Tkv * tile_weight(QB) + item_weight(QB);
+    return w + (long long)s.lt * tile_weight(s.Nq) + (s.lt > 0 ? item_weight(s.Nq) : 0);
 }
 // Tile t belongs to block floor(weight_before(t) * G / total_w).  First tile of block c: the first tile whose
 // cumulative cost reaches ceil(c * total_w / G).
 template <int QB>
 __device__ __forceinline__ long long first_tile_of_block(const TileIndex* ix, const TcParams& p, int c, int G, long long total_w,
-                                                         long long total_tiles, bool wide) {
+                                                         long long total_tiles) {
     const long long wt = ((long long)c * total_w + G - 1) / G;
     if (wt >= total_w) return total_tiles;
     int lo = 0, hi = p.B;
@@ -300,32 +271,32 @@ __device__ __forceinline__ long long first_tile_of_block(const TileIndex* ix, co
     int r2 = (int)(rem % wh);
     long long t = (long long)p.H * ix->cum_tiles[lo] + (long long)h * tb;
     // inside a work item the tiles start at cost 0, f + w, f + 2w, ... (f = fixed cost on the first tile)
-    const int w0 = tile_weight(min(QB, Nb), wide), f0 = item_weight(min(QB, Nb), wide);
+    const int w0 = tile_weight(min(QB, Nb)), f0 = item_weight(min(QB, Nb));
     if (r2 >= tkv * w0 + f0 && Nb > QB) {              // inside the second query block
         r2 -= tkv * w0 + f0;
         t += tkv;
-        const int w1 = tile_weight(Nb - QB, wide), f1 = item_weight(Nb - QB, wide);
+        const int w1 = tile_weight(Nb - QB), f1 = item_weight(Nb - QB);
         return r2 == 0 ? t : t + max(1, (r2 - f1 + w1 - 1) / w1);
     }
     return r2 == 0 ? t : t + max(1, (r2 - f0 + w0 - 1) / w0);
 }
 template <int QB>
-__device__ __forceinline__ int block_of_tile(const TileIndex* ix, const TcParams& p, long long t, int G, long long total_w, bool wide) {
+__device__ __forceinline__ int block_of_tile(const TileIndex* ix, const TcParams& p, long long t, int G, long long total_w) {
     Segment s;
     locate<QB>(ix, p, t, s);
-    return (int)min((long long)G - 1, weight_before<QB>(ix, p, s, wide) * G / total_w);
+    return (int)min((long long)G - 1, weight_before<QB>(ix, p, s) * G / total_w);
 }
 
-// Per-block set-up shared by both kernels: tiles and cost per sequence, their prefix sums, the number of blocks
-// that get work and the two ends of this block's range.  Ends with a __syncthreads(); all threads must call it.
+// Per-block set-up: tiles and cost per sequence, their prefix sums, the number of blocks that get work and the two
+// ends of this block's range.  Ends with a __syncthreads(); all threads must call it.
 template <int QB>
-__device__ __forceinline__ void plan_ranges(TileIndex* ix, const TcParams& p, bool wide, int* n_blocks, long long* range) {
+__device__ __forceinline__ void plan_ranges(TileIndex* ix, const TcParams& p, int* n_blocks, long long* range) {
     const int tid = threadIdx.x, nthr = blockDim.x;
     for (int b = tid; b < p.B; b += nthr) {
         const int L = min(max(p.seq_lens[b], 0), p.L_max);
         const int Nb = p.n_active ? min(max(p.n_active[b], 0), p.N) : p.N;
         ix->cum_tiles[b + 1] = tiles_of<QB>(L, Nb, p.G);
-        ix->cum_w[b + 1] = head_weight<QB>(L, Nb, p.G, wide);
+        ix->cum_w[b + 1] = head_weight<QB>(L, Nb, p.G);
     }
     __syncthreads();
     if (tid == 0) {
@@ -339,25 +310,21 @@ __device__ __forceinline__ void plan_ranges(TileIndex* ix, const TcParams& p, bo
         // No block's share of the cost may be smaller than the heaviest tile, so that consecutive tiles never skip
         // a block: every working block then owns at least one tile and the blocks sharing a work item are consecutive.
         const long long tot_w = (long long)p.H * accw;
-        *n_blocks = (int)max(1LL, min((long long)gridDim.x, tot_w / (tile_weight(QB, wide) + item_weight(QB, wide))));
+        *n_blocks = (int)max(1LL, min((long long)gridDim.x, tot_w / (tile_weight(QB) + item_weight(QB))));
     }
     __syncthreads();
     if (tid == 0 || tid == 32) {               // the two ends of this block's range, side by side
         const long long tot = (long long)p.H * ix->cum_tiles[p.B], tot_w = (long long)p.H * ix->cum_w[p.B];
         const int nb = *n_blocks, which = tid >> 5;
-        range[which] = (tot > 0 && (int)blockIdx.x < nb) ? first_tile_of_block<QB>(ix, p, (int)blockIdx.x + which, nb, tot_w, tot, wide) : 0;
+        range[which] = (tot > 0 && (int)blockIdx.x < nb) ? first_tile_of_block<QB>(ix, p, (int)blockIdx.x + which, nb, tot_w, tot) : 0;
     }
     __syncthreads();
 }
 
-// ------------------------------------------------------------------ host side (attention_tc.cu)
 struct TcLaunch {
     CUtensorMap maps[5];     // Q, key cache, value cache, tree keys, tree values
     TcParams p;
     int grid;
 };
-// widest kernel: 4 softmax warpgroups, up to 160 queries per work item (attention_tc_wide.cu)
-int launch_tc_wide(int nch, const TcLaunch& l, cudaStream_t stream);
-int slots_for_wide(int nch);
 
 }  // namespace mcsd
