@@ -180,12 +180,12 @@ int mcsd_workspace_status(const void* workspace, void* stream);
  *   next_roots    [dev] int32[B][R] out or NULL: the R most probable ids of the distribution the new token
  *                 was drawn from (ties to the smaller id) -- the candidates with which a target-initialised
  *                 tree (Section 3.1) seeds its next step
- *   workspace     [dev] >= mcsd_verify_tree_workspace_bytes(B, N, V) bytes
+ *   workspace     [dev] >= mcsd_verify_tree_workspace_bytes(B, N, V) bytes, zero-filled before its first use (it
+ *                 holds a per-sequence arrival counter that every call leaves at zero again)
  *
- * Two launches on `stream`: one block per (sequence, node) decides the accepted child of every node, then one
- * block per sequence follows the paths and draws the new token.  The second is a programmatic dependent launch
- * (its blocks may become resident before the first kernel ends and wait for it on the device); to the stream's
- * other work the pair behaves like two ordinary launches.
+ * One launch on `stream`: one block per (sequence, node) decides the accepted child of every node; the block
+ * that finishes a sequence's last node (an arrival counter per sequence, nothing waits) follows the paths and
+ * draws the new token.
  *
  * Errors: MCSD_ERR_NULL, MCSD_ERR_BAD_SHAPE (B, N, V < 1, N > MCSD_MAX_NODES, B > 65535, R < 0 or R > 32,
  * n_roots or n_levels out of range), MCSD_ERR_WORKSPACE_TOO_SMALL, MCSD_ERR_CUDA.
@@ -350,7 +350,7 @@ int mcsd_verify_shard_pick(const float* p_shard, const float* q_shard, const flo
  * The call itself performs no cudaMalloc/cudaFree and calls no allocating library routine.
  *
  *   limit      B * N <= MCSD_STATIC_VERIFY_MAX_STATES, otherwise MCSD_ERR_STATIC_LIMIT is returned and
- *              nothing is launched.  The array costs about 256 KB on every GPU that loads the library, for
+ *              nothing is launched.  The array costs about 320 KB on every GPU that loads the library, for
  *              the life of the process.
  *   first call The first call on each device looks up the array's device address (with that device
  *              current); make that first call outside any stream capture.

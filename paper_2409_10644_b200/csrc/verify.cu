@@ -7,7 +7,7 @@
 extern "C" size_t mcsd_verify_tree_workspace_bytes(int B, int N, int V) {
     (void)V;
     if (B < 1 || N < 1) return 0;
-    return mcsd::align_up(sizeof(mcsd::WorkspaceHeader) + sizeof(mcsd::NodeState) * (size_t)B * N, 256);
+    return mcsd::verify_tickets_offset(B, N) + mcsd::align_up(sizeof(int) * (size_t)B, 256);
 }
 
 extern "C" int mcsd_verify_tree(const float* p, const float* q, const int32_t* tokens, const int32_t* parent,
@@ -26,13 +26,12 @@ extern "C" int mcsd_verify_tree(const float* p, const float* q, const int32_t* t
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     auto* state = reinterpret_cast<mcsd::NodeState*>(static_cast<char*>(workspace) + sizeof(mcsd::WorkspaceHeader));
     const mcsd::ProbRows rows{p, q};
-    mcsd::verify_nodes_kernel<mcsd::ProbRows><<<dim3(N, B), mcsd::kVerifyThreads, 0, s>>>(
-        rows, tokens, parent, level_start, n_levels, gamma, u_accept, N, V, state);
+    int* tickets = reinterpret_cast<int*>(static_cast<char*>(workspace) + mcsd::verify_tickets_offset(B, N));
+    mcsd::verify_tree_kernel<mcsd::ProbRows><<<dim3(N, B), mcsd::kVerifyThreads, 0, s>>>(
+        rows, tokens, parent, level_start, n_levels, n_roots, gamma, u_accept, u_bonus, N, V, state, tickets, accept_len,
+        out_tokens, out_nodes, best_root, R > 0 ? next_roots : nullptr, R);
     MCSD_CUDA_CHECK(cudaGetLastError());
-    MCSD_CUDA_CHECK(mcsd::launch_dependent(mcsd::verify_select_kernel<mcsd::ProbRows>, dim3(B), dim3(mcsd::kVerifyThreads), s,
-                                           rows, tokens, state, n_levels, n_roots, u_bonus, N, V, accept_len, out_tokens,
-                                           out_nodes, best_root, R > 0 ? next_roots : nullptr, R));
-    mcsd::count_launches(2);
+    mcsd::count_launches(1);
     return MCSD_OK;
 }
 
@@ -60,8 +59,10 @@ extern "C" int mcsd_sample_roots(const float* p, const float* q, const int32_t* 
 namespace mcsd {
 
 // Scratch that lives in the library image itself: one copy per GPU that loads the library, held until the
-// process exits.  Layout: workspace header, then MCSD_STATIC_VERIFY_MAX_STATES node states.
-constexpr size_t kStaticScratchBytes = sizeof(WorkspaceHeader) + sizeof(NodeState) * (size_t)MCSD_STATIC_VERIFY_MAX_STATES;
+// process exits.  Layout as a workspace of the largest problem: header, MCSD_STATIC_VERIFY_MAX_STATES node states, one
+// ticket per sequence (at most as many sequences as states).
+constexpr size_t kStaticScratchBytes = sizeof(WorkspaceHeader) + sizeof(NodeState) * (size_t)MCSD_STATIC_VERIFY_MAX_STATES +
+                                       256 + sizeof(int) * (size_t)MCSD_STATIC_VERIFY_MAX_STATES + 256;
 static __device__ __align__(256) unsigned char g_static_verify_scratch[kStaticScratchBytes];
 
 constexpr int kMaxDevices = 64;
@@ -96,8 +97,11 @@ extern "C" int mcsd_verify_tree_static(const float* p, const float* q, const int
     void* scratch = nullptr;
     const int st = mcsd::static_scratch_for_current_device(&scratch);
     if (st != MCSD_OK) return st;
-    // the array keeps whatever the previous call left; the status line must start at zero
+    // the array keeps whatever the previous call left; the status line and this problem's tickets must start at zero
     MCSD_CUDA_CHECK(cudaMemsetAsync(scratch, 0, sizeof(mcsd::WorkspaceHeader), static_cast<cudaStream_t>(stream)));
+    if (B >= 1 && N >= 1)
+        MCSD_CUDA_CHECK(cudaMemsetAsync(static_cast<char*>(scratch) + mcsd::verify_tickets_offset(B, N), 0, sizeof(int) * (size_t)B,
+                                        static_cast<cudaStream_t>(stream)));
     return mcsd_verify_tree(p, q, tokens, parent, level_start, n_levels, n_roots, gamma, u_accept, u_bonus, B, N, V,
                             accept_len, out_tokens, out_nodes, best_root, next_roots, R, scratch,
                             mcsd::kStaticScratchBytes, stream);

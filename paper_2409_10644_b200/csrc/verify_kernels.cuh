@@ -4,16 +4,17 @@
 //
 // The walk of one root visits a node, tries its children in order and either moves to the first accepted
 // child or stops.  Uniforms are indexed by node, so what happens at a node does not depend on how the walk
-// got there.  That splits the work in two kernels:
+// got there.  That splits the work in two phases of one launch:
 //
-//   verify_nodes_kernel   one thread block per (sequence, node): decides which child, if any, is accepted
+//   node phase            one thread block per (sequence, node): decides which child, if any, is accepted
 //                         at that node.  After m rejections the target-side distribution is
 //                         max(p - c_m q, 0) / Y_m with c_0 = 0, Y_0 = 1, c_{m+1} = c_m + Y_m and
 //                         Y_m = sum_v max(p_v - c_m q_v, 0): iterating norm(max(pt - q, 0)) never needs a
 //                         vocabulary-sized write, only one reduction over the two rows per rejection.
-//   verify_select_kernel  one thread block per sequence: follows next_child from every root, keeps the
-//                         longest path (ties: lowest root), then draws the new token at its stop node by
-//                         inverse CDF in token-id order and, on request, lists the most probable ids.
+//   select phase          the block of a sequence that finishes its node last (a ticket per sequence in the
+//                         workspace; nothing waits): follows next_child from every root, keeps the longest
+//                         path (ties: lowest root), then draws the new token at its stop node by inverse CDF
+//                         in token-id order and, on request, lists the most probable ids.
 //
 // A "Rows" type hands out, for one (sequence, node), a "Dist": the pair of rows seen as the unnormalised
 // distribution  dist_v = max(p_v - c q_v, 0)  for a settable c, read E ids at a time with 128-bit loads
@@ -37,6 +38,12 @@ struct NodeState {
     int32_t top;          // greedy verification: id of the largest target logit of this node
     double c;             // stop distribution is max(p - c q, 0); c = 0 means the row p itself
 };
+
+// Workspace layout of the verify calls: header, B * N node states, then one ticket per sequence (arrivals of the
+// sequence's node blocks; zero between launches).
+inline size_t verify_tickets_offset(int B, int N) {
+    return align_up(sizeof(WorkspaceHeader) + sizeof(NodeState) * (size_t)B * N, 256);
+}
 
 // block-wide scratch of the row passes
 struct VerifyScratch {
@@ -406,69 +413,6 @@ __device__ __forceinline__ void find_children(const int32_t* __restrict__ parent
     cnt = *s_cnt;
 }
 
-template <typename Rows>
-__global__ void __launch_bounds__(kVerifyThreads)
-verify_nodes_kernel(Rows rows, const int32_t* __restrict__ tokens, const int32_t* __restrict__ parent,
-                    const int32_t* __restrict__ level_start, int n_levels, const int32_t* __restrict__ gamma,
-                    const float* __restrict__ u_accept, int N, int V, NodeState* __restrict__ state) {
-    __shared__ int s_first, s_cnt, s_accept;
-    __shared__ VerifyScratch s_scratch;
-    __shared__ double s_px[MCSD_MAX_NODES], s_qx[MCSD_MAX_NODES];
-    __shared__ float s_ua[MCSD_MAX_NODES];
-    // Blocks are handed out in the order of their linear index; taking the node from its upper part starts all
-    // sequences' nodes level by level, so the nodes with the most siblings to try run first and the leaves,
-    // which have nothing to do, last.
-    // lets a select kernel launched as a programmatic dependent become resident while this grid still runs
-    // (it waits for this grid's completion before reading anything); no effect on an ordinary launch
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const int lin = blockIdx.y * gridDim.x + blockIdx.x;
-    const int b = lin % (int)gridDim.y, u = lin / (int)gridDim.y, tid = threadIdx.x;
-    const int n_act = active_nodes(gamma, level_start, n_levels, b, N);
-    if (u >= n_act) return;
-    int first, cnt;
-    find_children(parent, u, N, &s_first, &s_cnt, first, cnt);
-
-    NodeState st;
-    st.next_child = -1; st.top = -1; st.c = 0.0;
-    // in level order a kept prefix of the tree keeps either all children of a node or none
-    if (cnt > 0 && first < n_act) {
-        typename Rows::Dist d = rows.open(b, u, N, V, &s_scratch);
-        // p_u(x), q_u(x) and the uniform of every sibling are fetched side by side up front, so that the sibling
-        // loop below pays for one dependent trip to memory in total instead of one per sibling
-        for (int m = tid; m < cnt; m += kVerifyThreads) {
-            const int x = tokens[(size_t)b * N + first + m];
-            const bool valid = x >= 0 && x < V;
-            s_px[m] = valid ? d.p_of(x) : -1.0;               // -1: no such token, never accepted
-            s_qx[m] = valid ? d.q_of(x) : 0.0;
-            s_ua[m] = u_accept[(size_t)b * N + first + m];
-        }
-        __syncthreads();
-        double c = 0.0, Y = 1.0;
-        for (int m = 0; m < cnt; ++m) {
-            const int child = first + m;
-            if (tid == 0) {
-                double a = 0.0;
-                if (s_px[m] >= 0.0) {
-                    const double px = s_px[m], qx = s_qx[m];
-                    const double num = fmax(px - c * qx, 0.0);
-                    a = qx > 0.0 ? fmin(1.0, num / (Y * qx)) : (num > 0.0 ? 1.0 : 0.0);
-                }
-                s_accept = ((double)s_ua[m] < a) ? 1 : 0;
-            }
-            __syncthreads();
-            const int acc = s_accept;
-            __syncthreads();
-            if (acc) { st.next_child = child; break; }
-            c += Y;
-            d.set_c(c);
-            Y = dist_mass(d, &s_scratch);
-            if (!(Y > 0.0)) { c = 0.0; Y = 1.0; d.set_c(0.0); }     // nothing left: back to the un-residualised row
-        }
-        if (st.next_child < 0) st.c = c;
-    }
-    if (tid == 0) state[(size_t)b * N + u] = st;
-}
-
 // (value, id) order used for the list of most probable ids: larger value first, ties to the smaller id
 __device__ __forceinline__ bool better(float va, int ia, float vb, int ib) {
     return va > vb || (va == vb && ia < ib);
@@ -485,7 +429,7 @@ __device__ __forceinline__ void select_path(const NodeState* __restrict__ st, co
     if (tid < n_roots) {
         int u = tid, len = 0;
         for (int step = 0; step < n_levels; ++step) {
-            const int nc = st[u].next_child;
+            const int nc = __ldcg(&st[u].next_child);
             if (nc < 0 || nc >= N) break;
             u = nc;
             ++len;
@@ -505,7 +449,7 @@ __device__ __forceinline__ void select_path(const NodeState* __restrict__ st, co
         if (n_roots > 1) ot[slot++] = tokens[(size_t)b * N + best];
         int u = best;
         for (int i = 0; i < s_len[best]; ++i) {
-            u = st[u].next_child;
+            u = __ldcg(&st[u].next_child);
             on[i] = u;
             ot[slot++] = tokens[(size_t)b * N + u];
         }
@@ -734,31 +678,27 @@ __device__ int block_inverse_cdf(const Load& load, float u, int V, CdfScratch* s
     return cdf_locate<E>(load, (double)u, false, V, sc, total_out);
 }
 
+// Select phase of one sequence, run by all threads of one block: the walk from every root, the longest path, the new
+// token by inverse CDF at its stop node and, on request, the R most probable ids of the same distribution.
 template <typename Rows>
-__global__ void __launch_bounds__(kVerifyThreads)
-verify_select_kernel(Rows rows, const int32_t* __restrict__ tokens, const NodeState* __restrict__ state,
-                     int n_levels, int n_roots, const float* __restrict__ u_bonus, int N, int V,
-                     int32_t* __restrict__ accept_len, int32_t* __restrict__ out_tokens,
-                     int32_t* __restrict__ out_nodes, int32_t* __restrict__ best_root,
-                     int32_t* __restrict__ next_roots, int R) {
+__device__ void select_and_draw(const Rows& rows, const int32_t* __restrict__ tokens, const NodeState* st, int b, int n_levels,
+                                int n_roots, const float* __restrict__ u_bonus, int N, int V, int32_t* __restrict__ accept_len,
+                                int32_t* __restrict__ out_tokens, int32_t* __restrict__ out_nodes,
+                                int32_t* __restrict__ best_root, int32_t* __restrict__ next_roots, int R,
+                                VerifyScratch* s_scratch) {
     using Dist = typename Rows::Dist;
     constexpr int E = Dist::E;
     __shared__ int s_len[MCSD_MAX_NODES];
     __shared__ int s_stop, s_slot;
-    __shared__ VerifyScratch s_scratch;
     __shared__ CdfScratch s_cdf;
     __shared__ float s_bv[kVerifyWarps];
     __shared__ int s_bi[kVerifyWarps];
-    const int b = blockIdx.x, tid = threadIdx.x;
-    const NodeState* st = state + (size_t)b * N;
-    // launched as a programmatic dependent of the node kernel: wait until that grid has completed and its
-    // results are visible (returns at once on an ordinary launch)
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int tid = threadIdx.x;
 
     select_path(st, tokens, b, n_levels, n_roots, N, accept_len, out_tokens, out_nodes, best_root, s_len, &s_stop, &s_slot);
     const int u = s_stop;
-    Dist d = rows.open(b, u, N, V, &s_scratch);
-    d.set_c(st[u].c);
+    Dist d = rows.open(b, u, N, V, s_scratch);
+    d.set_c(__ldcg(&st[u].c));
 
     // ---- new token: inverse CDF over dist_v = max(p_v - c q_v, 0) in token-id order ----
     auto load = [&d](int idx, float (&r)[E]) { d.load(idx, r); };
@@ -770,6 +710,82 @@ verify_select_kernel(Rows rows, const int32_t* __restrict__ tokens, const NodeSt
 
     // ---- optional: the R most probable ids of the same distribution ----
     if (next_roots != nullptr && R > 0) top_ids<E>(load, V, R, next_roots + (size_t)b * R, s_bv, s_bi);
+}
+
+template <typename Rows>
+__global__ void __launch_bounds__(kVerifyThreads)
+verify_tree_kernel(Rows rows, const int32_t* __restrict__ tokens, const int32_t* __restrict__ parent,
+                   const int32_t* __restrict__ level_start, int n_levels, int n_roots, const int32_t* __restrict__ gamma,
+                   const float* __restrict__ u_accept, const float* __restrict__ u_bonus, int N, int V,
+                   NodeState* state, int* tickets, int32_t* __restrict__ accept_len, int32_t* __restrict__ out_tokens,
+                   int32_t* __restrict__ out_nodes, int32_t* __restrict__ best_root, int32_t* __restrict__ next_roots, int R) {
+    __shared__ int s_first, s_cnt, s_accept, s_last;
+    __shared__ VerifyScratch s_scratch;
+    __shared__ double s_px[MCSD_MAX_NODES], s_qx[MCSD_MAX_NODES];
+    __shared__ float s_ua[MCSD_MAX_NODES];
+    // Blocks are handed out in the order of their linear index; taking the node from its upper part starts all
+    // sequences' nodes level by level, so the nodes with the most siblings to try run first and the leaves,
+    // which have nothing to do, last.
+    const int lin = blockIdx.y * gridDim.x + blockIdx.x;
+    const int b = lin % (int)gridDim.y, u = lin / (int)gridDim.y, tid = threadIdx.x;
+    const int n_act = active_nodes(gamma, level_start, n_levels, b, N);
+    if (u >= n_act) return;
+    int first, cnt;
+    find_children(parent, u, N, &s_first, &s_cnt, first, cnt);
+
+    NodeState st;
+    st.next_child = -1; st.top = -1; st.c = 0.0;
+    // in level order a kept prefix of the tree keeps either all children of a node or none
+    if (cnt > 0 && first < n_act) {
+        typename Rows::Dist d = rows.open(b, u, N, V, &s_scratch);
+        // p_u(x), q_u(x) and the uniform of every sibling are fetched side by side up front, so that the sibling
+        // loop below pays for one dependent trip to memory in total instead of one per sibling
+        for (int m = tid; m < cnt; m += kVerifyThreads) {
+            const int x = tokens[(size_t)b * N + first + m];
+            const bool valid = x >= 0 && x < V;
+            s_px[m] = valid ? d.p_of(x) : -1.0;               // -1: no such token, never accepted
+            s_qx[m] = valid ? d.q_of(x) : 0.0;
+            s_ua[m] = u_accept[(size_t)b * N + first + m];
+        }
+        __syncthreads();
+        double c = 0.0, Y = 1.0;
+        for (int m = 0; m < cnt; ++m) {
+            const int child = first + m;
+            if (tid == 0) {
+                double a = 0.0;
+                if (s_px[m] >= 0.0) {
+                    const double px = s_px[m], qx = s_qx[m];
+                    const double num = fmax(px - c * qx, 0.0);
+                    a = qx > 0.0 ? fmin(1.0, num / (Y * qx)) : (num > 0.0 ? 1.0 : 0.0);
+                }
+                s_accept = ((double)s_ua[m] < a) ? 1 : 0;
+            }
+            __syncthreads();
+            const int acc = s_accept;
+            __syncthreads();
+            if (acc) { st.next_child = child; break; }
+            c += Y;
+            d.set_c(c);
+            Y = dist_mass(d, &s_scratch);
+            if (!(Y > 0.0)) { c = 0.0; Y = 1.0; d.set_c(0.0); }     // nothing left: back to the un-residualised row
+        }
+        if (st.next_child < 0) st.c = c;
+    }
+    // ---- ticket: the block that finishes a sequence's last node goes on to the select phase
+    if (tid == 0) {
+        state[(size_t)b * N + u] = st;
+        __threadfence();                                   // the state is visible before the ticket is
+        const int old = atomicAdd(&tickets[b], 1);
+        s_last = (old == n_act - 1) ? 1 : 0;
+        if (s_last) {
+            *(volatile int*)&tickets[b] = 0;               // nobody else arrives in this launch: ready for the next one
+            __threadfence();                               // acquire: the other blocks' states are visible
+        }
+    }
+    __syncthreads();
+    if (!s_last) return;
+    select_and_draw(rows, tokens, state + (size_t)b * N, b, n_levels, n_roots, u_bonus, N, V, accept_len, out_tokens, out_nodes,
+                    best_root, next_roots, R, &s_scratch);
 }
 
 // Several distinct new tokens from the distribution the winning path stopped with (Section 3.1 samples more than
@@ -813,24 +829,6 @@ sample_roots_kernel(Rows rows, const NodeState* __restrict__ state, const int32_
         if (tid == 0) { s_pick[i] = tok; next_roots[(size_t)b * R + i] = tok; }
         __syncthreads();
     }
-}
-
-// Host side: launches `kernel` as a programmatic dependent of the kernel before it in the stream.  Its blocks may
-// become resident while that kernel still runs (once all of its blocks have started) and must execute
-// griddepcontrol.wait before they read its results; this takes the launch latency off the critical path.
-template <typename... KArgs, typename... Args>
-inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t stream, Args... args) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid;
-    cfg.blockDim = block;
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 }  // namespace mcsd

@@ -105,7 +105,7 @@ static int launch_logits(const void* target_logits, const void* draft_logits, fl
                          const int32_t* parent, const int32_t* level_start, int n_levels, int n_roots,
                          const int32_t* gamma, const float* u_accept, const float* u_bonus, int B, int N, int V,
                          int32_t* accept_len, int32_t* out_tokens, int32_t* out_nodes, int32_t* best_root,
-                         int32_t* next_roots, int R, NodeState* state, cudaStream_t s) {
+                         int32_t* next_roots, int R, NodeState* state, int* tickets, cudaStream_t s) {
     const T* zt = static_cast<const T*>(target_logits);
     if (temperature == 0.f) {
         greedy_nodes_kernel<T><<<dim3(N, B), kVerifyThreads, 0, s>>>(zt, tokens, parent, level_start, n_levels, gamma, N, V,
@@ -114,16 +114,15 @@ static int launch_logits(const void* target_logits, const void* draft_logits, fl
         greedy_select_kernel<T><<<B, kVerifyThreads, 0, s>>>(zt, tokens, state, n_levels, n_roots, N, V, accept_len,
                                                             out_tokens, out_nodes, best_root, next_roots, R);
         MCSD_CUDA_CHECK(cudaGetLastError());
+        count_launches(2);
     } else {
         const LogitRows<T> rows{zt, static_cast<const T*>(draft_logits), 1.4426950408889634f / temperature};
-        verify_nodes_kernel<LogitRows<T>><<<dim3(N, B), kVerifyThreads, 0, s>>>(rows, tokens, parent, level_start, n_levels,
-                                                                               gamma, u_accept, N, V, state);
+        verify_tree_kernel<LogitRows<T>><<<dim3(N, B), kVerifyThreads, 0, s>>>(
+            rows, tokens, parent, level_start, n_levels, n_roots, gamma, u_accept, u_bonus, N, V, state, tickets, accept_len,
+            out_tokens, out_nodes, best_root, next_roots, R);
         MCSD_CUDA_CHECK(cudaGetLastError());
-        MCSD_CUDA_CHECK(launch_dependent(verify_select_kernel<LogitRows<T>>, dim3(B), dim3(kVerifyThreads), s, rows, tokens,
-                                         state, n_levels, n_roots, u_bonus, N, V, accept_len, out_tokens, out_nodes,
-                                         best_root, next_roots, R));
+        count_launches(1);
     }
-    count_launches(2);
     return MCSD_OK;
 }
 
@@ -150,14 +149,15 @@ extern "C" int mcsd_verify_tree_logits(const void* target_logits, const void* dr
     if (workspace_bytes < mcsd_verify_tree_workspace_bytes(B, N, V)) return MCSD_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     auto* state = reinterpret_cast<mcsd::NodeState*>(static_cast<char*>(workspace) + sizeof(mcsd::WorkspaceHeader));
+    int* tickets = reinterpret_cast<int*>(static_cast<char*>(workspace) + mcsd::verify_tickets_offset(B, N));
     int32_t* roots = R > 0 ? next_roots : nullptr;
     if (dtype == MCSD_F32)
         return mcsd::launch_logits<float>(target_logits, draft_logits, temperature, tokens, parent, level_start, n_levels,
                                           n_roots, gamma, u_accept, u_bonus, B, N, V, accept_len, out_tokens, out_nodes,
-                                          best_root, roots, R, state, s);
+                                          best_root, roots, R, state, tickets, s);
     return mcsd::launch_logits<__nv_bfloat16>(target_logits, draft_logits, temperature, tokens, parent, level_start,
                                               n_levels, n_roots, gamma, u_accept, u_bonus, B, N, V, accept_len, out_tokens,
-                                              out_nodes, best_root, roots, R, state, s);
+                                              out_nodes, best_root, roots, R, state, tickets, s);
 }
 
 extern "C" int mcsd_sample_roots_logits(const void* target_logits, const void* draft_logits, int dtype, float temperature,
