@@ -35,23 +35,23 @@ UNIT = "tree-tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 
 
-# DRAM traffic of the attention kernel from an `ncu --set full` capture (profiles/tree_attention_tc_b4_ncu_full.md):
-# dram__bytes_read.sum + dram__bytes_write.sum per launch on a 4-sequence case; traffic grows in proportion to the
-# batch.  The figure only holds for the kernel source it was taken on.
-_TRAFFIC_CAPTURE = {"source_sha1_12": "c1d48365f80b", "bytes_per_launch": 281_149_952, "batch": 4,
-                    "workload": "long_context_b16"}
-
-
 def _traffic_for(w):
+    """DRAM bytes per launch of the attention kernel from the tracked ncu capture (profiles/attention_traffic.json:
+    dram__bytes_read.sum + dram__bytes_write.sum on a small batch; traffic grows in proportion to the batch).  The
+    figure only holds for the kernel sources it was taken on: None once they have changed."""
     import hashlib
-    src = os.path.join(ROOT, "paper_2409_10644_b200", "csrc", "attention_tc.cu")
     try:
-        sha = hashlib.sha1(open(src, "rb").read()).hexdigest()[:12]
-    except OSError:
+        with open(os.path.join(ROOT, "profiles", "attention_traffic.json")) as f:
+            cap = json.load(f)
+        h = hashlib.sha1()
+        for name in cap["sources"]:
+            with open(os.path.join(ROOT, "paper_2409_10644_b200", "csrc", name), "rb") as f:
+                h.update(f.read())
+    except (OSError, KeyError, ValueError):
         return None
-    if sha != _TRAFFIC_CAPTURE["source_sha1_12"] or w.name != _TRAFFIC_CAPTURE["workload"]:
+    if h.hexdigest()[:12] != cap.get("source_sha1_12") or w.name != cap.get("workload"):
         return None
-    return int(_TRAFFIC_CAPTURE["bytes_per_launch"] * w.B / _TRAFFIC_CAPTURE["batch"])
+    return int(cap["bytes_per_launch"] * w.B / cap["batch"])
 
 
 def _peaks():
@@ -183,7 +183,7 @@ def run_reference(args):
     w = workload(args.workload)
     vals = []
     for i in range(args.warmup + args.steps):
-        v, sample, threads, step_s = oracle_sample(w, budget_s=max(2.0, 60.0 / max(1, args.warmup + args.steps)))
+        v, sample, threads, step_s = oracle_sample(w, budget_s=max(2.0, args.oracle_seconds / max(1, args.warmup + args.steps)))
         if i >= args.warmup:
             vals.append((v, step_s))
     value = float(np.mean([v for v, _ in vals]))
@@ -199,6 +199,37 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def cpu_baseline_in_fresh_process(workload_name, seconds=24.0):
+    """The oracle leg of the GPU arm: the same program as `--impl reference` with the same untimed first pass, started
+    as a new interpreter.  (Timed cold, without that pass, the same sample reads 2.2 x slower: the first pass pays for
+    the page faults of the problem pool and the start of the BLAS threads.)"""
+    cmd = [sys.executable, os.path.abspath(__file__), "--impl", "reference", "--workload", workload_name, "--steps", "1",
+           "--warmup", "1", "--oracle-seconds", str(seconds)]
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    res = subprocess.run(cmd, stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True, env=env)
+    for ln in reversed(res.stdout.strip().splitlines()):
+        try:
+            return json.loads(ln)["cpu_baseline"]
+        except (ValueError, KeyError):
+            continue
+    return {"value": None, "unit": UNIT, "cores": None, "kind": "oracle", "sample": "oracle process failed: " + res.stderr[-300:]}
+
+
+def torchrun_command(n, argv, port, script=None):
+    """Command line that starts n ranks of this script on this node (one per GPU) the way the scaling runs do."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n), "--master-addr",
+            "127.0.0.1", "--master-port", str(port), script or os.path.abspath(__file__)] + list(argv)
+
+
+def launch_ranks(n, argv, runner=subprocess.call, script=None):
+    """`python bench.py --gpus N` outside torchrun: start the N ranks here and hand back their exit code."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    return runner(torchrun_command(n, argv, port, script))
+
+
 def _config(w, n_gpus):
     return {"workload": w.name, "batch_per_gpu": w.B, "heads": w.H, "head_dim": w.D, "prefix": list(w.prefix),
             "tree": {"n_roots": w.n_roots, "branching": list(w.branching), "nodes": w.n_nodes},
@@ -210,6 +241,93 @@ def _config(w, n_gpus):
 # ------------------------------------------------------------------------------------------------
 # GPU arm
 # ------------------------------------------------------------------------------------------------
+
+def verify_rows_read(states, parent, n_act):
+    """Probability rows (of V floats) the verify kernel reads, counted on the host from the node states it left in the
+    workspace: an internal node's pair of rows once per rejected child (the first test needs two scalars only), and
+    at the stop node of the winning path the target row, plus the draft row if a child was rejected there.  (The
+    located range of the inverse CDF is read a second time: at most a sixteenth of a row, not counted.)"""
+    parent = np.asarray(parent)
+    N = len(parent)
+    first = np.full(N, -1)
+    cnt = np.zeros(N, dtype=np.int64)
+    for c, u in enumerate(parent):
+        if u >= 0:
+            if first[u] < 0:
+                first[u] = c
+            cnt[u] += 1
+    nxt = states["next_child"].cpu().numpy()
+    cc = states["c"].cpu().numpy()
+    rows = 0
+    for b in range(nxt.shape[0]):
+        for u in range(int(n_act[b])):
+            if cnt[u] == 0 or first[u] >= n_act[b]:
+                continue
+            rej = cnt[u] if nxt[b, u] < 0 else nxt[b, u] - first[u]
+            rows += 2 * int(rej)
+    return rows, cc
+
+
+def measure_workload(mcsd, name, dev, layers, steps, flush):
+    """Attention per layer and the verify step of one workload, replayed from CUDA graphs after an L2 flush."""
+    import torch
+    from mcsd_inputs import attention_inputs, gammas, parent_array, seq_lens, verify_inputs, workload
+    w = dataclasses.replace(workload(name), n_layers=layers)
+    parent = parent_array(w.n_roots, w.branching)
+    N = len(parent)
+    elt = 4 if w.dtype == "f32" else 2
+    code = mcsd.MCSD_F32 if w.dtype == "f32" else mcsd.MCSD_BF16
+    tm = mcsd.mcsd_build_mask(parent, device=dev)
+    lens, gam = seq_lens(w), gammas(w)
+    n_act = mcsd.n_active_from_gamma(tm.level_start_host, gam)
+    lens_d, nact_d, gam_d = (torch.from_numpy(x).to(dev) for x in (lens, n_act, gam))
+    lay = [attention_inputs(w, l, dev) for l in range(layers)]
+    outs = [torch.empty_like(l["q"]) for l in lay]
+    vin = verify_inputs(w, 0, dev, parent=parent)
+    ws_a = mcsd.new_workspace(mcsd.mcsd_tree_attention_workspace_bytes(w.B, w.H, N, w.D, w.L_max, code), dev)
+    ws_v = mcsd.new_workspace(mcsd.mcsd_verify_tree_workspace_bytes(w.B, N, w.V), dev)
+    scale = 1.0 / float(np.sqrt(w.D))
+
+    def attn():
+        for inp, o in zip(lay, outs):
+            mcsd.mcsd_tree_attention(inp["q"], inp["k_cache"], inp["v_cache"], inp["k_tree"], inp["v_tree"], lens_d, nact_d, tm,
+                                     out=o, softmax_scale=scale, workspace=ws_a)
+    vout = mcsd.mcsd_verify_tree(vin["p"], vin["q"], vin["tokens"], tm, gam_d, vin["u_accept"], vin["u_bonus"], workspace=ws_v)
+
+    def ver():
+        mcsd.mcsd_verify_tree(vin["p"], vin["q"], vin["tokens"], tm, gam_d, vin["u_accept"], vin["u_bonus"], workspace=ws_v, out=vout)
+    attn()
+    torch.cuda.synchronize()
+    ga, gv = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+    with torch.cuda.graph(ga):
+        attn()
+    with torch.cuda.graph(gv):
+        ver()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    for k in range(-3, steps):
+        flush.zero_()
+        e = ev[max(k, 0)]
+        e[0].record(); ga.replay(); e[1].record(); gv.replay(); e[2].record()
+    torch.cuda.synchronize()
+    a_ms = float(np.median([e[0].elapsed_time(e[1]) for e in ev])) / layers
+    v_ms = float(np.median([e[1].elapsed_time(e[2]) for e in ev]))
+    if mcsd.mcsd_workspace_status(ws_a) != 0 or mcsd.mcsd_workspace_status(ws_v) != 0:
+        raise SystemExit("a device-side wait timed out in workload %s" % name)
+    abytes = _algorithmic_bytes_attention(w.H, w.D, lens, n_act, tm.words, elt)
+    rows, _ = verify_rows_read(mcsd.verify_node_states(ws_v, w.B, N), parent, n_act)
+    rows += 2 * w.B                                    # stop node: target row, and (upper bound) the draft row
+    peak, _ = _peaks()
+    return {"workload": w.name, "layers_timed": layers, "tree_tokens": int(n_act.sum()), "attention_ms_per_layer": a_ms,
+            "attention_GBs": abytes / (a_ms * 1e-3) / 1e9, "frac": abytes / (a_ms * 1e-3) / 1e9 / peak,
+            "attention_algorithmic_bytes": int(abytes), "verify_ms": v_ms,
+            "verify_nodes_per_s": float(n_act.sum()) / (v_ms * 1e-3),
+            "verify_lazy_bytes": int(rows) * w.V * 4, "verify_lazy_GBs": rows * w.V * 4 / (v_ms * 1e-3) / 1e9,
+            "verify_all_rows_bytes": int(n_act.sum()) * w.V * 4 * 2}
+
+
+WORKLOAD_LAYERS = {"tiny_fp32": 8, "llama7b_b1": 8, "dynamic_slice_b8": 4, "long_context_b16": 2, "target_init_b32": 2,
+                   "paper_static_2_4_3_1_1": 4, "paper_fork_w16_d5": 4}
+
 
 def run_ours(args):
     import torch
@@ -418,11 +536,13 @@ def run_ours(args):
     abytes = _algorithmic_bytes_attention(w.H, w.D, lens, n_act, tm.words, elt)
     achieved = abytes / (attn_ms * 1e-3) / 1e9
     ver_rows_bytes = int(n_act.sum()) * w.V * 4 * 2
+    lazy_rows, _ = verify_rows_read(mcsd.verify_node_states(ws_ver, w.B, N), parent, n_act)
+    lazy_bytes = int(lazy_rows + 2 * w.B) * w.V * 4
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": dict(_config(w, world), launch="cuda graphs" if args.graph else "stream launches"),
+        "config": _config(w, world), "launch": "cuda graphs" if args.graph else "stream launches",
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                 "ms_per_step": e2e_ms,
                 "note": "per step the tree's q/k/v of every layer, p, q, tokens, uniforms, lengths and gammas are copied "
@@ -438,15 +558,29 @@ def run_ours(args):
         "breakdown": {"attention_ms_per_layer": attn_ms, "verify_ms": ver_ms,
                       "verify_nodes_per_s": float(n_act.sum()) / (ver_ms * 1e-3),
                       "verify_all_rows_GBs": ver_rows_bytes / (ver_ms * 1e-3) / 1e9,
+                      "verify_lazy_bytes": lazy_bytes, "verify_lazy_GBs": lazy_bytes / (ver_ms * 1e-3) / 1e9,
+                      "verify_bytes_note": "lazy = rows the kernel reads (a node's p and q rows once per rejected child, the "
+                                           "stop node's rows), counted from the node states; all_rows = every active node's "
+                                           "two rows, an upper bound the kernel does not move",
                       "tree_tokens_per_s_per_layer": float(n_act.sum()) / (attn_ms * 1e-3),
                       "mean_accept_len": float(vout["accept_len"].float().mean().item())},
     }
+    if world == 1 and args.workloads:
+        # the other workloads on the same box and clock record: a few layers each, graph replay after an L2 flush
+        del h_layers, h_outs
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        table = []
+        for name, nl in WORKLOAD_LAYERS.items():
+            table.append(measure_workload(mcsd, name, dev, nl, 7, flush))
+            torch.cuda.empty_cache()
+        line["breakdown"]["workloads"] = table
+        line["breakdown"]["workloads_note"] = ("every workload of the input table, few layers each with their own KV caches, "
+                                               "launches replayed from CUDA graphs, L2 flushed before each replay, medians of 7")
     if world == 1 and args.vocab_shards > 1:
         line["breakdown"]["vocab_sharded_verify"] = _time_vocab_sharded_verify(mcsd, w, vin, tm, gam_d, parent,
                                                                                args.vocab_shards, vout)
     if world == 1 and not args.no_cpu_baseline:
-        v, sample, threads, _ = oracle_sample(w0)
-        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample}
+        line["cpu_baseline"] = cpu_baseline_in_fresh_process(w0.name)
     print(json.dumps(line))
     if world > 1:
         dist.barrier()
@@ -504,11 +638,17 @@ def main():
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="issue the step's launches one by one from Python instead of replaying them from CUDA graphs "
                          "(the host's launch path, 25-50 us per call, then bounds workloads with shorter kernels)")
+    ap.add_argument("--no-workloads", dest="workloads", action="store_false",
+                    help="skip the per-workload table (breakdown.workloads) of the default run")
+    ap.add_argument("--oracle-seconds", type=float, default=60.0, help="--impl reference: oracle time in total")
     ap.add_argument("--vocab-shards", type=int, default=0,
                     help="also time the vocabulary-sharded verify step with this many ranks' column slices on one GPU")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started by hand with --gpus N: become the launcher of N ranks (torchrun sets WORLD_SIZE for them)
+        sys.exit(launch_ranks(args.gpus, sys.argv[1:]))
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -24,7 +24,7 @@ MCSD_MAX_WORDS = 3
 
 _EXPORTS = (
     "mcsd_status_string", "mcsd_last_cuda_error", "mcsd_launch_count", "mcsd_build_mask", "mcsd_tree_attention_workspace_bytes",
-    "mcsd_tree_attention", "mcsd_tree_attention_gqa", "mcsd_workspace_status", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_logits", "mcsd_verify_tree_static", "mcsd_commit_kv", "mcsd_sample_roots",
+    "mcsd_tree_attention", "mcsd_tree_attention_gqa", "mcsd_workspace_status", "verify_node_states", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_logits", "mcsd_verify_tree_static", "mcsd_commit_kv", "mcsd_sample_roots",
     "mcsd_sample_roots_logits", "mcsd_verify_shard_workspace_bytes", "mcsd_verify_shard_gather", "mcsd_verify_shard_round",
     "mcsd_verify_shard_select", "mcsd_verify_shard_pick",
 )
@@ -180,6 +180,13 @@ def _dtype_code(t: torch.Tensor) -> int:
 
 def mcsd_tree_attention_workspace_bytes(B, H, N, D, L_max, dtype) -> int:
     return int(lib.mcsd_tree_attention_workspace_bytes(B, H, N, D, L_max, dtype))
+
+
+def verify_node_states(workspace: torch.Tensor, B: int, N: int):
+    """Views of what the verify call left per (sequence, node) in its workspace: `next_child` int32[B][N] (accepted
+    child or -1) and `c` float64[B][N] (the stop distribution at that node is max(p - c q, 0))."""
+    raw = workspace[256:256 + 16 * B * N]
+    return {"next_child": raw.view(torch.int32).view(B, N, 4)[..., 0], "c": raw.view(torch.float64).view(B, N, 2)[..., 1]}
 
 
 def new_workspace(nbytes: int, device) -> torch.Tensor:

@@ -292,3 +292,70 @@ def test_vocab_sharded_verify_protocol_over_gloo(m):
         p.join(timeout=60)
         assert p.exitcode == 0
     assert ok
+
+
+# ---------------------------------------------------------------------------------------------------------
+# bench.py --gpus N started by hand: it must start N ranks itself
+# ---------------------------------------------------------------------------------------------------------
+def _load_bench():
+    import importlib.util
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    spec = importlib.util.spec_from_file_location("bench_under_test", os.path.join(root, "bench.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    return mod
+
+
+def test_bench_builds_the_launcher_command_for_n_ranks():
+    bench = _load_bench()
+    seen = []
+    rc = bench.launch_ranks(4, ["--gpus", "4", "--steps", "2"], runner=lambda cmd: seen.append(cmd) or 0)
+    assert rc == 0 and len(seen) == 1
+    cmd = seen[0]
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nnodes=1" in cmd
+    assert cmd[cmd.index("--nproc-per-node") + 1] == "4"
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert 0 < int(cmd[cmd.index("--master-port") + 1]) < 65536
+    assert cmd[-4:] == ["--gpus", "4", "--steps", "2"] and cmd[-5].endswith("bench.py")
+
+
+_FAKE_RANK = """
+import os, sys
+import torch, torch.distributed as dist
+dist.init_process_group("gloo")
+t = torch.tensor([float(os.environ["RANK"]) + 1.0])
+dist.all_reduce(t)
+open(os.path.join(sys.argv[1], "rank%s" % os.environ["RANK"]), "w").write("%d %d %g" % (dist.get_world_size(), int(os.environ["LOCAL_RANK"]), t.item()))
+dist.destroy_process_group()
+"""
+
+
+def test_bench_launcher_starts_two_real_ranks(tmp_path):
+    """The launcher's command, run for real with a stand-in for the rank program: two processes that find each other
+    over 127.0.0.1, see WORLD_SIZE = 2 and distinct LOCAL_RANKs."""
+    bench = _load_bench()
+    script = tmp_path / "fake_rank.py"
+    script.write_text(_FAKE_RANK)
+    rc = bench.launch_ranks(2, [str(tmp_path)], script=str(script))
+    assert rc == 0
+    got = sorted((tmp_path / ("rank%d" % r)).read_text() for r in range(2))
+    assert got == ["2 0 3", "2 1 3"]
+
+
+def test_bench_counts_the_rows_the_verify_kernel_reads():
+    """verify_rows_read: an internal node's two rows once per rejected child, nothing for an accepted first child."""
+    import torch
+    bench = _load_bench()
+    parent = parent_array(1, (3, 1))                  # root with three children, each with one child: 7 nodes
+    N = len(parent)
+    nxt = torch.full((2, N), -1, dtype=torch.int32)
+    nxt[0, 0] = 1                                     # sequence 0: first child of the root accepted, its child rejected
+    nxt[1, 0] = 3                                     # sequence 1: two rejections at the root, third child accepted ...
+    nxt[1, 3] = 6                                     # ... and that child's only child accepted
+    states = {"next_child": nxt, "c": torch.zeros((2, N), dtype=torch.float64)}
+    rows, _ = bench.verify_rows_read(states, parent, np.array([N, N]))
+    # sequence 0: root 0 rejections; nodes 1, 2, 3 each reject their one child -> 3 rejections
+    # sequence 1: root 2 rejections; nodes 1, 2 reject their child (2), node 3 accepts (0)
+    assert rows == 2 * (3 + 2 + 2)
+    rows_cut, _ = bench.verify_rows_read(states, parent, np.array([4, 4]))     # level 2 sliced off: only the root counts
+    assert rows_cut == 2 * (0 + 2)
