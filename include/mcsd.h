@@ -104,7 +104,8 @@ int mcsd_build_mask(const int32_t* parent_host, int n_nodes,
  *   anc, words              the mask from mcsd_build_mask for the N-node tree
  *   D                       64 or 128;  N <= MCSD_MAX_NODES;  B * H <= 65535
  *   dtype                   MCSD_BF16: bf16 storage, fp32 softmax and accumulation (tensor-core products when
- *                           D == 128 and all tensors are 16-byte aligned);  MCSD_F32: fp32 throughout
+ *                           D == 128, all tensors are 16-byte aligned and the shape is one that
+ *                           mcsd_tree_attention_path() reports as MCSD_PATH_TENSOR_CORE);  MCSD_F32: fp32 throughout
  *   workspace               [dev] scratch of at least mcsd_tree_attention_workspace_bytes(...) bytes; holds
  *                           split-KV partial results and the status word.  Calls that may overlap on the
  *                           device need distinct workspaces.
@@ -124,12 +125,27 @@ int mcsd_tree_attention(const void* q, const void* k_cache, const void* v_cache,
                         int dtype, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Which kernel mcsd_tree_attention / mcsd_tree_attention_gqa runs for a shape (Section 2.2 defines the operation; the
+ * choice of kernel is this library's).  The tensor-core kernel (tcgen05, bandwidth-bound) takes bf16, D = 128,
+ * B <= 256 and B * (L_max / 128 + 4) < 2^23 (its per-sequence tables are 32-bit and live in shared memory); every
+ * other valid shape -- fp32, D = 64, larger batches, longer prefixes -- runs the CUDA-core kernel, which is
+ * arithmetic-bound and several times slower per key.  A caller with more than 256 sequences gets the fast kernel by
+ * splitting the batch over several calls.  Host only, no CUDA call.
+ *
+ * Returns MCSD_PATH_TENSOR_CORE or MCSD_PATH_CUDA_CORE, or a negative status (MCSD_ERR_BAD_SHAPE, MCSD_ERR_BAD_DTYPE)
+ * for a shape mcsd_tree_attention rejects.  (Tensors that are not 16-byte aligned also take the CUDA-core kernel.)
+ */
+#define MCSD_PATH_CUDA_CORE 0
+#define MCSD_PATH_TENSOR_CORE 1
+int mcsd_tree_attention_path(int B, int H_q, int H_kv, int N, int D, int L_max, int dtype);
+
+/*
  * mcsd_tree_attention for a target with grouped-query attention: q and out have H_q heads, the four key/value
  * tensors H_kv heads, H_q = G * H_kv, and query head h reads key/value head h / G (the paper's targets are
  * multi-head models, G = 1; Section 2.2 defines the attention itself).  Everything else as mcsd_tree_attention.
  * With bf16 and head_dim 128 the tensor-core kernel stacks the queries of S heads of a group into one work unit
- * (S the largest of 8, 4, 2 that divides G with S * N <= MCSD_MAX_NODES, else 1), so that a key/value head is
- * streamed G / S times instead of G times.
+ * (S the largest of 8, 4, 2 that divides G with S * N <= 160, the most query columns one pass over the keys takes;
+ * else 1), so that a key/value head is streamed G / S times instead of G times.
  *
  *   q, out                  [dev] dtype[B][H_q][N][D]
  *   k_cache, v_cache        [dev] dtype[B][H_kv][L_max][D]
@@ -260,7 +276,7 @@ int mcsd_sample_roots_logits(const void* target_logits, const void* draft_logits
                              const void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * KV-cache update after acceptance (Fig. 1 step 6): "update the input IDs, key-value cache".  For every layer and
+ * KV-cache update after acceptance (Fig. 1 step 6, where the accepted tokens join the sequence).  For every layer and
  * sequence b the keys/values of the winning root (node best_root[b]; with a single root that is node 0, the last
  * emitted token, which is not in the prefix cache yet) and of the accepted nodes out_nodes[b][0 .. accept_len[b]-1]
  * are copied from the tree tensors to cache rows seq_lens[b], seq_lens[b]+1, ..., then seq_lens[b] grows by

@@ -24,7 +24,7 @@ MCSD_MAX_WORDS = 3
 
 _EXPORTS = (
     "mcsd_status_string", "mcsd_last_cuda_error", "mcsd_launch_count", "mcsd_build_mask", "mcsd_tree_attention_workspace_bytes",
-    "mcsd_tree_attention", "mcsd_tree_attention_gqa", "mcsd_workspace_status", "verify_node_states", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_logits", "mcsd_verify_tree_static", "mcsd_commit_kv", "mcsd_sample_roots",
+    "mcsd_tree_attention", "mcsd_tree_attention_gqa", "mcsd_workspace_status", "verify_node_states", "mcsd_tree_attention_path", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_logits", "mcsd_verify_tree_static", "mcsd_commit_kv", "mcsd_sample_roots",
     "mcsd_sample_roots_logits", "mcsd_verify_shard_workspace_bytes", "mcsd_verify_shard_gather", "mcsd_verify_shard_round",
     "mcsd_verify_shard_select", "mcsd_verify_shard_pick",
 )
@@ -48,6 +48,8 @@ def _load() -> ctypes.CDLL:
                                     ctypes.POINTER(c_int), c_void_p]
     lib.mcsd_tree_attention_workspace_bytes.restype = c_size_t
     lib.mcsd_tree_attention_workspace_bytes.argtypes = [c_int] * 6
+    lib.mcsd_tree_attention_path.restype = c_int
+    lib.mcsd_tree_attention_path.argtypes = [c_int] * 7
     lib.mcsd_tree_attention.restype = c_int
     lib.mcsd_tree_attention.argtypes = [c_void_p] * 9 + [c_int] * 6 + [c_float, c_int, c_void_p, c_size_t, c_void_p]
     lib.mcsd_tree_attention_gqa.restype = c_int
@@ -187,6 +189,14 @@ def verify_node_states(workspace: torch.Tensor, B: int, N: int):
     child or -1) and `c` float64[B][N] (the stop distribution at that node is max(p - c q, 0))."""
     raw = workspace[256:256 + 16 * B * N]
     return {"next_child": raw.view(torch.int32).view(B, N, 4)[..., 0], "c": raw.view(torch.float64).view(B, N, 2)[..., 1]}
+
+
+def mcsd_tree_attention_path(B, H_q, H_kv, N, D, L_max, dtype_code) -> int:
+    """1 if the tensor-core kernel takes this shape, 0 if the CUDA-core kernel does (see mcsd.h); raises on bad shapes."""
+    st = int(lib.mcsd_tree_attention_path(B, H_q, H_kv, N, D, L_max, dtype_code))
+    if st < 0:
+        _check(st, "mcsd_tree_attention_path")
+    return st
 
 
 def new_workspace(nbytes: int, device) -> torch.Tensor:
@@ -364,6 +374,30 @@ def mcsd_verify_tree_static(p, q, tokens, mask: TreeMask, gamma, u_accept, u_bon
     preallocated result tensors (accept_len, out_tokens, out_nodes, best_root, next_roots), so this wrapper
     allocates nothing either.  Calls share the array: do not let two of them overlap on the GPU."""
     B, N, V = p.shape
+    # the same argument checks as mcsd_verify_tree (none of them allocates), plus the caller's result tensors
+    _dev_tensor(p, torch.float32, "p")
+    _dev_tensor(q, torch.float32, "q")
+    _dev_tensor(tokens, torch.int32, "tokens")
+    _dev_tensor(u_accept, torch.float32, "u_accept")
+    _dev_tensor(u_bonus, torch.float32, "u_bonus")
+    if gamma is not None:
+        _dev_tensor(gamma, torch.int32, "gamma")
+        if tuple(gamma.shape) != (B,):
+            raise ValueError("gamma must have one entry per sequence")
+    if (mask.n_nodes != N or tuple(q.shape) != (B, N, V) or tuple(tokens.shape) != (B, N) or
+            tuple(u_accept.shape) != (B, N) or tuple(u_bonus.shape) != (B, N)):
+        raise ValueError("shape mismatch between p, q, tokens, the uniforms and the tree")
+    nl = mask.n_levels
+    want = {"accept_len": (B,), "out_tokens": (B, nl + 1), "out_nodes": (B, nl), "best_root": (B,)}
+    if R > 0:
+        want["next_roots"] = (B, R)
+    for name, shape in want.items():
+        t = out.get(name)
+        if t is None:
+            raise ValueError("out[%r] is missing" % name)
+        _dev_tensor(t, torch.int32, "out[%r]" % name)
+        if tuple(t.shape) != shape:
+            raise ValueError("out[%r] must have shape %r" % (name, shape))
     with torch.cuda.device(p.device):
         st = lib.mcsd_verify_tree_static(_ptr(p), _ptr(q), _ptr(tokens), _ptr(mask.parent), _ptr(mask.level_start),
                                          mask.n_levels, mask.n_roots, _ptr(gamma), _ptr(u_accept), _ptr(u_bonus),

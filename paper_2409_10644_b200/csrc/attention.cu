@@ -55,6 +55,13 @@ static int run_attention(const void* q, const void* k_cache, const void* v_cache
     return mcsd::tree_attention_simt(a, scratch, s);
 }
 
+extern "C" int mcsd_tree_attention_path(int B, int H_q, int H_kv, int N, int D, int L_max, int dtype) {
+    const int st = check_shape(B, H_q, N, D, L_max, dtype);
+    if (st != MCSD_OK) return st;
+    if (H_kv < 1 || H_q < H_kv || H_q % H_kv != 0) return MCSD_ERR_BAD_SHAPE;
+    return mcsd::tc_shape_supported(B, H_q, H_q / H_kv, N, D, L_max, dtype) ? MCSD_PATH_TENSOR_CORE : MCSD_PATH_CUDA_CORE;
+}
+
 extern "C" int mcsd_tree_attention(const void* q, const void* k_cache, const void* v_cache, const void* k_tree,
                                    const void* v_tree, void* out, const int32_t* seq_lens, const int32_t* n_active,
                                    const uint64_t* anc, int words, int B, int H, int N, int D, int L_max,

@@ -27,6 +27,7 @@ size_t simt_workspace_bytes(int B, int H, int N, int D, int L_max);
 int tree_attention_simt(const AttentionArgs& a, void* scratch, cudaStream_t stream);
 
 // tcgen05 tensor-core path: bf16, D = 128
+bool tc_shape_supported(int B, int H, int G, int N, int D, int L_max, int dtype);   // shape and dtype alone
 bool tc_supported(const AttentionArgs& a);
 size_t tc_workspace_bytes(int B, int H, int N, int D, int L_max);
 int tree_attention_tc(const AttentionArgs& a, WorkspaceHeader* header, void* scratch, size_t scratch_bytes,

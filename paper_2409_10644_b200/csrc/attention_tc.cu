@@ -822,12 +822,19 @@ static int tc_stack_for(int G, int N) {
     return 1;
 }
 
-// The per-sequence prefix sums of tiles and cost units are 32-bit: bound the largest launch so that they cannot
-// wrap (a sequence of L_max keys and 192 nodes costs at most 2 * (tiles + 4) * 64 units per head).
+// Shapes the tensor-core kernel takes.  B <= 256 (per-sequence tables in shared memory); the per-sequence prefix sums
+// of tiles and cost units are 32-bit, so the largest launch is bounded so that they cannot wrap (a sequence of L_max
+// keys and 192 nodes costs at most 2 * (tiles + 4) * 64 units per head): B * (L_max / 128 + 4) < 2^23, i.e. a
+// 4-million-token prefix at B = 256 and a 500-million-token one at B = 2.
+bool tc_shape_supported(int B, int H, int G, int N, int D, int L_max, int dtype) {
+    if (dtype != MCSD_BF16 || D != 128) return false;
+    if (!(G >= 1 && H % G == 0 && N >= 1 && N <= MCSD_MAX_NODES && B >= 1 && B <= kMaxBatchTc && L_max >= 0)) return false;
+    const long long tiles = (long long)L_max / kTile + 4;
+    return (long long)B * tiles * 2 * 64 < (1LL << 30);
+}
+
 bool tc_supported(const AttentionArgs& a) {
-    if (!(a.G >= 1 && a.H % a.G == 0 && a.N <= MCSD_MAX_NODES && a.B <= kMaxBatchTc && encode_fn() != nullptr)) return false;
-    const long long tiles = (long long)a.L_max / kTile + 4;
-    return (long long)a.B * tiles * 2 * 64 < (1LL << 30);
+    return tc_shape_supported(a.B, a.H, a.G, a.N, a.D, a.L_max, a.dtype) && encode_fn() != nullptr;
 }
 
 size_t tc_workspace_bytes(int, int, int N, int, int) {

@@ -1,5 +1,5 @@
-// Multi-candidate accept/reject straight from next-token logits (Fig. 1 step 4: the target's logits "are
-// then transformed into distributions") at the two sampling settings of Section 4.1:
+// Multi-candidate accept/reject straight from next-token logits (Fig. 1 step 4, where logits become the
+// distributions that are compared) at the two sampling settings of Section 4.1:
 //
 //   temperature > 0   p = softmax(target logits / T), q = softmax(draft logits / T); the accept/reject kernels of
 //                     verify_kernels.cuh run on logit rows, so p and q are never written to memory.

@@ -199,3 +199,26 @@ def test_commit_kv_argument_checks(m):
     assert call(N=193) == -2
     assert call(nl=0) == -2
     assert call(dtype=3) == -4
+
+
+def test_attention_kernel_choice_is_a_documented_function_of_the_shape(m):
+    """mcsd_tree_attention_path: the tensor-core kernel's limits (bf16, head_dim 128, at most 256 sequences, 32-bit
+    per-sequence tile tables) are checked on the host; everything else valid runs the CUDA-core kernel."""
+    bf16, f32 = m.MCSD_BF16, m.MCSD_F32
+    path = m.mcsd_tree_attention_path
+    assert path(16, 32, 32, 45, 128, 4096, bf16) == 1
+    assert path(32, 32, 32, 160, 128, 4096, bf16) == 1
+    assert path(1, 32, 8, 45, 128, 512, bf16) == 1                 # grouped queries
+    assert path(1, 4, 4, 15, 64, 128, f32) == 0                    # fp32
+    assert path(2, 4, 4, 45, 64, 512, bf16) == 0                   # head_dim 64
+    assert path(256, 8, 8, 45, 128, 4096, bf16) == 1
+    assert path(257, 8, 8, 45, 128, 4096, bf16) == 0               # more sequences than the per-sequence tables hold
+    # the tile tables are 32-bit: B * (L_max / 128 + 4) must stay below 2^23
+    assert path(256, 1, 1, 45, 128, 4_000_000, bf16) == 1
+    assert path(256, 1, 1, 45, 128, 4_300_000, bf16) == 0
+    assert path(2, 1, 1, 192, 128, 500_000_000, bf16) == 1
+    assert path(2, 1, 1, 192, 128, 600_000_000, bf16) == 0
+    with pytest.raises(m.McsdError):
+        path(1, 4, 4, 193, 128, 128, bf16)                         # more nodes than a tree may have
+    with pytest.raises(m.McsdError):
+        path(1, 6, 4, 45, 128, 128, bf16)                          # query heads not a multiple of key/value heads

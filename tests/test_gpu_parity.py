@@ -130,9 +130,9 @@ def _all_pairs(B, H):
     return [(b, h) for b in range(B) for h in range(H)]
 
 
-def _full_attention_case(m, w, std=None, rel=False, lens=None, n_act="gamma", pairs=None, poison=False):
+def _full_attention_case(m, w, std=None, rel=False, lens=None, n_act="gamma", pairs=None, poison=False, layer=0):
     parent = parent_array(w.n_roots, w.branching)
-    inp = attention_inputs(w, 0, "cuda", std=std)
+    inp = attention_inputs(w, layer, "cuda", std=std)
     lens = seq_lens(w) if lens is None else np.asarray(lens, dtype=np.int32)
     if isinstance(n_act, str):
         _, ls = orc.tree_levels(parent)
@@ -205,10 +205,11 @@ def test_attention_query_split_changes_between_segments(m):
                                     (4, "too_wide"), (2, "f32")])
 def test_attention_grouped_queries(m, G, case):
     # query heads share key/value heads; the tensor-core kernel stacks the queries of 8, 4 or 2 heads of a group into
-    # one work unit when that divides the group and fits 192 queries (G = 8, N = 45: two units of four heads; G = 3
-    # or N = 109: one head per unit, the key/value head still shared); fp32 takes the CUDA-core kernel
+    # one work unit when that divides the group and fits the 160 query columns of one pass (N = 45: two heads per
+    # unit = 90 queries whatever G is, since four would be 180; G = 3 or N = 109: one head per unit, the key/value
+    # head still shared; N = 15, G = 8: all eight heads = 120 queries); fp32 takes the CUDA-core kernel
     if case == "stacked":
-        w = dataclasses.replace(workload(2), B=3, H=2 * G, prefix=(40, 600))          # N = 45: 180 or 90 queries
+        w = dataclasses.replace(workload(2), B=3, H=2 * G, prefix=(40, 600))          # N = 45: 90 stacked queries
     elif case == "stacked_small":
         w = dataclasses.replace(workload(1), dtype="bf16", D=128, B=2, H=G, prefix=(5, 300))   # N = 15: 120 queries
     elif case == "too_wide":
@@ -276,6 +277,38 @@ def test_attention_full_size_sampled(m, idx):
     pairs = sorted({(int(rng.integers(w.B)), int(rng.integers(w.H))) for _ in range(6)} | {(0, 0), (w.B - 1, w.H - 1)})
     _full_attention_case(m, w, pairs=pairs)
     _full_attention_case(m, w, std=1.0, rel=True, pairs=pairs)
+    if w.n_layers > 1:
+        # the long-context workload repeats the step over 32 layers with independent seeded caches: also the
+        # middle and the last layer, on their own samples of (sequence, head) pairs
+        for layer in (w.n_layers // 2 - 1, w.n_layers - 1):
+            lp = sorted({(int(rng.integers(w.B)), int(rng.integers(w.H))) for _ in range(4)})
+            _full_attention_case(m, w, pairs=lp, layer=layer)
+    torch.cuda.empty_cache()
+
+
+def test_attention_dynamic_slice_depth6_reading(m):
+    # The dynamic-slice configuration is quoted as "depth 8, 76 nodes"; its widths give 108 draft nodes and 76 is the
+    # count of the first six levels.  The other tests take the widths; this is the other reading: every sequence
+    # verified with draft length 6, i.e. 77 of the 109 rows of the mask built once for depth 8.
+    w = workload(3)
+    parent = parent_array(w.n_roots, w.branching)
+    assert orc.n_active_for_gamma(parent, 6) == 77
+    n_act = np.full(w.B, 77, dtype=np.int32)
+    rng = np.random.default_rng(36)
+    pairs = sorted({(int(rng.integers(w.B)), int(rng.integers(w.H))) for _ in range(5)} | {(0, 0)})
+    _full_attention_case(m, w, n_act=n_act, pairs=pairs)
+    _full_attention_case(m, w, std=1.0, rel=True, n_act=n_act, pairs=pairs)
+    _verify_case(m, w, gamma=np.full(w.B, 6, dtype=np.int32))
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("H,L,roots,branching", [(1, 20000, 1, (4, 2, 2, 1)), (2, 9000, 8, (1, 2, 2, 1, 1, 1))])
+def test_attention_one_work_item_cut_into_many_pieces(m, H, L, roots, branching):
+    # One or two (sequence, head) pairs with a long prefix: every thread block gets a few tiles of the same work
+    # item, so the item is merged from about as many pieces as there are blocks (the most the split allows).
+    w = dataclasses.replace(workload(2), B=1, H=H, prefix=(L, L), n_roots=roots, branching=branching)
+    _full_attention_case(m, w, std=1.0, rel=True, lens=[L - 77], n_act=None, poison=True)
+    _full_attention_case(m, w, lens=[L], n_act=None)
     torch.cuda.empty_cache()
 
 
@@ -602,12 +635,16 @@ def test_commit_kv_matches_oracle(m, idx, dtype_D):
     dev = "cuda"
     layers = [attention_inputs(w, l, dev) for l in range(w.n_layers)]
     lens = np.array([30, 41, 57, 60][: w.B], dtype=np.int32)          # the last two run out of cache rows
+    # what was accepted comes from the oracle's own verification (uniforms kept clear of its thresholds), for both
+    # sides: the library's commit gets the oracle's accept_len / out_nodes / best_root, not the library's
     vin = verify_inputs(w, 0, dev, parent=parent, V=500)
-    gam = None if w.gamma is None else torch.from_numpy(gammas(w)).to(dev)
-    vout = m.mcsd_verify_tree(vin["p"], vin["q"], vin["tokens"], tm, gam, vin["u_accept"], vin["u_bonus"])
-    torch.cuda.synchronize()
+    gam_h = None if w.gamma is None else gammas(w)
+    hvin = {k: to_np(v) for k, v in vin.items()}
+    ua, ub = condition_uniforms(hvin["p"], hvin["q"], hvin["tokens"], parent, gam_h, hvin["u_accept"], hvin["u_bonus"])
+    hv = orc.verify_tree(hvin["p"], hvin["q"], hvin["tokens"], parent, gam_h, ua, ub)
+    vout = {k: torch.from_numpy(np.ascontiguousarray(hv[k]).astype(np.int32)).to(dev)
+            for k in ("accept_len", "out_tokens", "out_nodes", "best_root")}
     host_layers = [{k: to_np(v).copy() for k, v in l.items()} for l in layers]
-    hv = {k: v.cpu().numpy() for k, v in vout.items() if v is not None}
     lens_d = torch.from_numpy(lens).to(dev)
     kc = m.layer_pointer_table([l["k_cache"] for l in layers])
     vc = m.layer_pointer_table([l["v_cache"] for l in layers])

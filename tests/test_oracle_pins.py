@@ -785,3 +785,92 @@ def test_grouped_query_attention_is_attention_with_repeated_kv_heads():
     np.testing.assert_allclose(got2[:, 1], got2[:, 0], rtol=0, atol=0)
     with pytest.raises(ValueError):
         orc.tree_attention_gqa(q[:, :5], kc, vc, kt, vt, lens, nact, parent, 0.3)
+
+
+def test_grouped_query_attention_against_library_causal_attention_on_root_paths():
+    """A pin outside the oracle: query head h of a grouped-query target, at node n, equals ordinary causal attention
+    (library routine) of that query over [prefix of key/value head h // G | the root path of n], last position."""
+    rng = np.random.default_rng(43)
+    B, Hkv, G, D = 2, 2, 3, 8
+    parent = parent_array(2, (2, 1, 2))
+    N = len(parent)
+    lens = [9, 0]
+    L = max(lens)
+    q = rng.normal(size=(B, Hkv * G, N, D))
+    kc, vc = rng.normal(size=(B, Hkv, L, D)), rng.normal(size=(B, Hkv, L, D))
+    kt, vt = rng.normal(size=(B, Hkv, N, D)), rng.normal(size=(B, Hkv, N, D))
+    scale = 0.41
+    got = orc.tree_attention_gqa(q, kc, vc, kt, vt, lens, None, parent, scale)
+    for b in range(B):
+        for h in range(Hkv * G):
+            hk = h // G
+            for n in range(N):
+                path = []
+                u = n
+                while u >= 0:
+                    path.append(u)
+                    u = int(parent[u])
+                path = path[::-1]
+                k_seq = np.concatenate([kc[b, hk, :lens[b]], kt[b, hk, path]])
+                v_seq = np.concatenate([vc[b, hk, :lens[b]], vt[b, hk, path]])
+                q_seq = np.zeros_like(k_seq)
+                q_seq[-1] = q[b, h, n]
+                ref = _sdpa_causal_last(q_seq, k_seq, v_seq, scale)[-1]
+                np.testing.assert_allclose(got[b, h, n], ref, rtol=0, atol=1e-12)
+    # a wrong head map must show: with the other key/value head the outputs differ
+    swapped = orc.tree_attention_gqa(q, kc[:, ::-1], vc[:, ::-1], kt[:, ::-1], vt[:, ::-1], lens, None, parent, scale)
+    assert np.abs(swapped - got).max() > 1e-3
+
+
+def test_decision_margins_on_hand_written_rows():
+    """Both halves of decision_margins against distances written out by hand.
+
+    Root with two children over a vocabulary of three.  Root row: p = (0.5, 0.3, 0.2), q = (0.25, 0.25, 0.5).
+    Child 1 carries token 0 (ratio p/q = 2, unclamped), child 2 carries token 2 (tested only after a rejection,
+    against the residual max(p - q, 0) = (0.25, 0.05, 0) / 0.3: ratio 0 / 0.5 = 0)."""
+    parent = parent_array(1, (2,))
+    p = np.array([[[0.5, 0.3, 0.2], [0.2, 0.2, 0.6], [0.1, 0.7, 0.2]]])
+    q = np.array([[[0.25, 0.25, 0.5], [0.3, 0.3, 0.4], [0.3, 0.3, 0.4]]])
+    tokens = np.array([[9, 0, 2]])
+    # (a) first child accepted (u = 0.75 < min(1, 2)): only its test is made; no new token at the root
+    ua = np.array([[0.5, 0.75, 0.4]])
+    ub = np.array([[0.5, 0.5, 0.95]])
+    m_acc, m_bon = orc.decision_margins(p, q, tokens, parent, None, ua, ub)
+    assert m_acc[0, 1] == pytest.approx(2.0 - 0.75, abs=1e-12)         # distance from the unclamped ratio
+    assert np.isinf(m_acc[0, 0]) and np.isinf(m_acc[0, 2])             # root never tested; sibling 2 not reached
+    assert np.isinf(m_bon[0, 0])
+    # leaves stop with their own row p: cumulative sums (0.2, 0.4, 1.0) and (0.1, 0.8, 1.0)
+    assert m_bon[0, 1] == pytest.approx(min(0.5 - 0.4, 1.0 - 0.5), abs=1e-12)      # u = 0.5 falls in token 2
+    assert m_bon[0, 2] == pytest.approx(min(0.95 - 0.8, 1.0 - 0.95), abs=1e-12)    # u = 0.95 falls in token 2
+    # (b) a uniform above 1 is not possible, so make the first test fail through the tokens: child 1 now carries
+    # token 2 (ratio 0.2 / 0.5 = 0.4), child 2 token 0, tested against the residual (0.25, 0.05, 0) / 0.3:
+    # ratio (0.25 / 0.3) / 0.25 = 10 / 3
+    tokens_b = np.array([[9, 2, 0]])
+    ua_b = np.array([[0.5, 0.9, 0.25]])
+    m_acc, m_bon = orc.decision_margins(p, q, tokens_b, parent, None, ua_b, ub)
+    assert m_acc[0, 1] == pytest.approx(0.9 - 0.4, abs=1e-12)
+    assert m_acc[0, 2] == pytest.approx(10.0 / 3.0 - 0.25, abs=1e-12)
+    assert np.isinf(m_bon[0, 0])                                       # second child accepted: no stop at the root
+    # (c) both rejected: child 2 carries token 2 again, whose residual mass is 0 -> ratio 0, rejected for any u.
+    # After it the residual is max((0.25, 0.05, 0) / 0.3 - q, 0) = (7/12, 0, 0) -> all mass on token 0: every
+    # u_bonus falls in token 0, whose cell is [0, 1]; the first token has no lower edge to cross (u * Z cannot fall
+    # below zero), so the distance is the one to the upper edge, 1 - u.
+    tokens_c = np.array([[9, 2, 2]])
+    ua_c = np.array([[0.5, 0.9, 0.3]])
+    ub_c = np.array([[0.3, 0.5, 0.5]])
+    m_acc, m_bon = orc.decision_margins(p, q, tokens_c, parent, None, ua_c, ub_c)
+    assert m_acc[0, 1] == pytest.approx(0.5, abs=1e-12)
+    assert m_acc[0, 2] == pytest.approx(0.3 - 0.0, abs=1e-12)
+    assert m_bon[0, 0] == pytest.approx(1.0 - 0.3, abs=1e-12)
+    # a stop distribution with two cells: one rejection only (gamma cuts nothing, root has a single tested child)
+    parent1 = parent_array(1, (1,))
+    m_acc, m_bon = orc.decision_margins(p[:, :2], q[:, :2], np.array([[9, 2]]), parent1, None,
+                                        np.array([[0.5, 0.9]]), np.array([[0.9, 0.5]]))
+    # residual after rejecting token 2: (0.25, 0.05, 0) / 0.3, cumulative (5/6, 1, 1); u = 0.9 falls in token 1
+    assert m_acc[0, 1] == pytest.approx(0.5, abs=1e-12)
+    assert m_bon[0, 0] == pytest.approx(min(0.9 - 5.0 / 6.0, 1.0 - 0.9), abs=1e-12)
+    # gamma = 0: the root is the stop node with its own row, cumulative (0.5, 0.8, 1.0); u = 0.9 -> token 2
+    m_acc, m_bon = orc.decision_margins(p, q, tokens, parent, np.array([0]), ua, np.array([[0.9, 0.5, 0.5]]))
+    assert np.isinf(m_acc).all()
+    assert m_bon[0, 0] == pytest.approx(min(0.9 - 0.8, 1.0 - 0.9), abs=1e-12)
+    assert np.isinf(m_bon[0, 1]) and np.isinf(m_bon[0, 2])

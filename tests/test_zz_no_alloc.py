@@ -8,6 +8,8 @@ import pytest
 import torch
 
 from mcsd_inputs import gammas, parent_array, verify_inputs, workload
+from oracle import mcsd_oracle as orc
+from tests.helpers import condition_uniforms, to_np
 
 pytestmark = pytest.mark.gpu
 
@@ -40,14 +42,22 @@ def test_static_scratch_entry_point_matches_the_workspace_one_twice_in_a_row(m):
         parent = parent_array(w.n_roots, w.branching)
         tm = m.mcsd_build_mask(parent, device=dev)
         vin = verify_inputs(w, step, dev, parent=parent, B=B, V=V)
-        gam = torch.from_numpy(gammas(dataclasses.replace(w, B=B), step)).to(dev)
-        ref = m.mcsd_verify_tree(vin["p"], vin["q"], vin["tokens"], tm, gam, vin["u_accept"], vin["u_bonus"], R=R)
+        gam_h = gammas(dataclasses.replace(w, B=B), step)
+        gam = torch.from_numpy(gam_h).to(dev)
+        # uniforms kept clear of the oracle's thresholds, so that the oracle's integers are the expected ones too
+        host = {k: to_np(v) for k, v in vin.items()}
+        ua, ub = condition_uniforms(host["p"], host["q"], host["tokens"], parent, gam_h, host["u_accept"], host["u_bonus"])
+        ua_d, ub_d = torch.from_numpy(ua).to(dev), torch.from_numpy(ub).to(dev)
+        ref = m.mcsd_verify_tree(vin["p"], vin["q"], vin["tokens"], tm, gam, ua_d, ub_d, R=R)
         out = _outputs(B, tm.n_levels, R, dev)
-        got = m.mcsd_verify_tree_static(vin["p"], vin["q"], vin["tokens"], tm, gam, vin["u_accept"], vin["u_bonus"],
-                                        out, R=R)
+        got = m.mcsd_verify_tree_static(vin["p"], vin["q"], vin["tokens"], tm, gam, ua_d, ub_d, out, R=R)
         torch.cuda.synchronize()
         for k in ("accept_len", "out_tokens", "out_nodes", "best_root", "next_roots"):
             assert torch.equal(got[k], ref[k]), k          # integer results: identical, not just close
+        # and directly against the CPU oracle, not only against the other entry point
+        exp = orc.verify_tree(host["p"], host["q"], host["tokens"], parent, gam_h, ua, ub, R=R)
+        for k in ("accept_len", "out_tokens", "out_nodes", "best_root", "next_roots"):
+            assert np.array_equal(got[k].cpu().numpy(), exp[k]), k
         assert int(ref["accept_len"].max()) >= 0
 
 
