@@ -142,3 +142,64 @@ def test_sharded_verify_equals_the_single_gpu_entry_point(m):
     torch.cuda.synchronize()
     for key in KEYS:
         assert torch.equal(outs[0][key], one[key]), key
+
+
+# ---------------------------------------------------------------------------------------------------------
+# The real driver end to end: two processes, a process group, this library's kernels in each
+# ---------------------------------------------------------------------------------------------------------
+def _two_process_rank(rank, world, port, q, widx, B, V):
+    """One rank of dist.verify_tree_vocab_sharded.  Both ranks use GPU 0 (one GPU is all there is): each launches its
+    own kernels from its own process and the reductions between them go through a gloo group, so nothing on the device
+    waits for the other rank."""
+    import os
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    import torch.distributed as dist
+    try:
+        torch.cuda.set_device(0)
+        dist.init_process_group("gloo", rank=rank, world_size=world)
+        import paper_2409_10644_b200 as m
+        from paper_2409_10644_b200 import dist as mdist
+        w = workload(widx)
+        parent = parent_array(w.n_roots, w.branching)
+        vin = verify_inputs(w, 0, "cuda", parent=parent, B=B, V=V)          # same seeds: both ranks draw the same rows
+        gamma = None if w.gamma is None else gammas(dataclasses.replace(w, B=B), 0)
+        host = {k: to_np(v) for k, v in vin.items()}
+        ua, ub = condition_uniforms(host["p"], host["q"], host["tokens"], parent, gamma, host["u_accept"], host["u_bonus"])
+        ref = orc.verify_tree(host["p"], host["q"], host["tokens"], parent, gamma, ua, ub)
+        tm = m.mcsd_build_mask(parent)
+        dev = vin["p"].device
+        g_d = None if gamma is None else torch.from_numpy(np.asarray(gamma, dtype=np.int32)).to(dev)
+        v0, v1 = mdist.vocab_shard_range(V, rank, world)
+        out = mdist.verify_tree_vocab_sharded(vin["p"][:, :, v0:v1].contiguous(), vin["q"][:, :, v0:v1].contiguous(), v0, V,
+                                              vin["tokens"], tm, g_d, torch.from_numpy(ua).to(dev), torch.from_numpy(ub).to(dev))
+        torch.cuda.synchronize()
+        bad = [k for k in KEYS if not np.array_equal(out[k].cpu().numpy(), ref[k])]
+        q.put((rank, bad, int(ref["accept_len"].sum())))
+        dist.barrier()
+        dist.destroy_process_group()
+    except Exception as e:                                       # report instead of leaving the parent waiting
+        q.put((rank, ["exception: %r" % (e,)], -1))
+        raise
+
+
+@pytest.mark.parametrize("widx,B,V", [(2, 3, 1000), (5, 4, 777)])
+def test_vocab_sharded_driver_with_two_processes_and_a_process_group(m, widx, B, V):
+    import socket
+    import torch.multiprocessing as mp
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_two_process_rank, args=(r, 2, port, q, widx, B, V)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = sorted(q.get(timeout=300) for _ in range(2))
+    for p in procs:
+        p.join(timeout=120)
+        assert p.exitcode == 0
+    assert [g[0] for g in got] == [0, 1]
+    for rank, bad, total in got:
+        assert bad == [], (rank, bad)                            # every rank ends with the oracle's integers
+    assert got[0][2] == got[1][2] and got[0][2] >= 0
