@@ -24,6 +24,28 @@ template <typename T> __device__ __forceinline__ T from_f32(float v);
 template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
+// 16 bytes of a row as floats: 4 fp32 values or 8 bf16 values (converted in registers)
+template <typename T> struct Vec16;
+template <> struct Vec16<float> {
+    static constexpr int E = 4;
+    __device__ __forceinline__ static void load(const float* p, float (&r)[4]) {
+        const float4 v = *reinterpret_cast<const float4*>(p);
+        r[0] = v.x; r[1] = v.y; r[2] = v.z; r[3] = v.w;
+    }
+};
+template <> struct Vec16<__nv_bfloat16> {
+    static constexpr int E = 8;
+    __device__ __forceinline__ static void load(const __nv_bfloat16* p, float (&r)[8]) {
+        const uint4 v = *reinterpret_cast<const uint4*>(p);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {                     // a bf16 is the upper half of the fp32 with the same value
+            r[2 * i] = __uint_as_float(w[i] << 16);
+            r[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
+};
+
 // grid: (splits, query blocks, B * H)
 template <typename T, int D>
 __global__ void __launch_bounds__(kSimtThreads)
@@ -47,16 +69,32 @@ tree_attention_simt_kernel(const T* __restrict__ q, const T* __restrict__ k_cach
     chunk = (chunk + kSimtTile - 1) / kSimtTile * kSimtTile;
     const int j_begin = split * chunk, j_end = min(total, j_begin + chunk);
 
+    constexpr int EV = Vec16<T>::E, DV = D / EV;          // elements per 16-byte load, loads per row
     const T* qb = q + (size_t)bh * N * D;
-    for (int i = tid; i < kSimtQBlock * D; i += kSimtThreads) {
-        const int r = i / D, d = i % D;
-        s_q[r][d] = (q0 + r < Nb) ? to_f32(qb[(size_t)(q0 + r) * D + d]) : 0.f;
-    }
     const size_t bkv = (size_t)b * (H / G) + (bh % H) / G;   // query head h reads key/value head h / G
     const T* kc = k_cache + bkv * L_max * D;
     const T* vc = v_cache + bkv * L_max * D;
     const T* kt = k_tree + bkv * N * D;
     const T* vt = v_tree + bkv * N * D;
+    // rows are multiples of 16 bytes long, so 128-bit loads need only 16-byte aligned tensors (uniform per launch)
+    const bool vec = ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(k_cache) | reinterpret_cast<uintptr_t>(v_cache) |
+                       reinterpret_cast<uintptr_t>(k_tree) | reinterpret_cast<uintptr_t>(v_tree)) & 15u) == 0;
+    if (vec) {
+        for (int i = tid; i < kSimtQBlock * DV; i += kSimtThreads) {
+            const int r = i / DV, d = (i % DV) * EV;
+            float v[EV];
+#pragma unroll
+            for (int e = 0; e < EV; ++e) v[e] = 0.f;
+            if (q0 + r < Nb) Vec16<T>::load(qb + (size_t)(q0 + r) * D + d, v);
+#pragma unroll
+            for (int e = 0; e < EV; ++e) s_q[r][d + e] = v[e];
+        }
+    } else {
+        for (int i = tid; i < kSimtQBlock * D; i += kSimtThreads) {
+            const int r = i / D, d = i % D;
+            s_q[r][d] = (q0 + r < Nb) ? to_f32(qb[(size_t)(q0 + r) * D + d]) : 0.f;
+        }
+    }
 
     float m[kSimtQPerWarp], l[kSimtQPerWarp], o[kSimtQPerWarp][DL];
 #pragma unroll
@@ -68,15 +106,33 @@ tree_attention_simt_kernel(const T* __restrict__ q, const T* __restrict__ k_cach
 
     for (int j0 = j_begin; j0 < j_end; j0 += kSimtTile) {
         __syncthreads();
-        for (int i = tid; i < kSimtTile * D; i += kSimtThreads) {
-            const int r = i / D, d = i % D, j = j0 + r;
-            float kv = 0.f, vv = 0.f;
-            if (j < j_end) {
-                if (j < L) { kv = to_f32(kc[(size_t)j * D + d]); vv = to_f32(vc[(size_t)j * D + d]); }
-                else { kv = to_f32(kt[(size_t)(j - L) * D + d]); vv = to_f32(vt[(size_t)(j - L) * D + d]); }
+        if (vec) {
+            // one 128-bit load of K and one of V per thread and step, converted in registers
+            for (int i = tid; i < kSimtTile * DV; i += kSimtThreads) {
+                const int r = i / DV, d = (i % DV) * EV, j = j0 + r;
+                float kv[EV], vv[EV];
+#pragma unroll
+                for (int e = 0; e < EV; ++e) { kv[e] = 0.f; vv[e] = 0.f; }
+                if (j < j_end) {
+                    const T* kr = j < L ? kc + (size_t)j * D : kt + (size_t)(j - L) * D;
+                    const T* vr = j < L ? vc + (size_t)j * D : vt + (size_t)(j - L) * D;
+                    Vec16<T>::load(kr + d, kv);
+                    Vec16<T>::load(vr + d, vv);
+                }
+#pragma unroll
+                for (int e = 0; e < EV; ++e) { s_k[r][d + e] = kv[e]; s_v[r][d + e] = vv[e]; }
             }
-            s_k[r][d] = kv;
-            s_v[r][d] = vv;
+        } else {
+            for (int i = tid; i < kSimtTile * D; i += kSimtThreads) {
+                const int r = i / D, d = i % D, j = j0 + r;
+                float kv = 0.f, vv = 0.f;
+                if (j < j_end) {
+                    if (j < L) { kv = to_f32(kc[(size_t)j * D + d]); vv = to_f32(vc[(size_t)j * D + d]); }
+                    else { kv = to_f32(kt[(size_t)(j - L) * D + d]); vv = to_f32(vt[(size_t)(j - L) * D + d]); }
+                }
+                s_k[r][d] = kv;
+                s_v[r][d] = vv;
+            }
         }
         __syncthreads();
         const int j = j0 + lane;                          // this lane's key

@@ -27,7 +27,10 @@ constexpr int kSmemLimit = 232448;            // dynamic shared memory a block m
 struct TileIndex {
     int cum_tiles[kMaxBatchTc + 1];
     int cum_w[kMaxBatchTc + 1];
+    unsigned short kv_tiles[kMaxBatchTc];   // key tiles of one work item of sequence b
+    int whole_items;                        // launch small enough to give every block whole work items (see plan_ranges)
 };
+constexpr int kWholeItemTiles = 8;          // ... which pays while a work item has at most this many key tiles
 
 struct TcParams {
     __nv_bfloat16* out;
@@ -297,26 +300,52 @@ __device__ __forceinline__ void plan_ranges(TileIndex* ix, const TcParams& p, in
         const int Nb = p.n_active ? min(max(p.n_active[b], 0), p.N) : p.N;
         ix->cum_tiles[b + 1] = tiles_of<QB>(L, Nb, p.G);
         ix->cum_w[b + 1] = head_weight<QB>(L, Nb, p.G);
+        ix->kv_tiles[b] = (unsigned short)min(kv_tiles_of(L, Nb), 65535);
     }
     __syncthreads();
     if (tid == 0) {
-        int acc = 0, accw = 0;
+        int acc = 0, accw = 0, items = 0, longest = 0;
         ix->cum_tiles[0] = 0;
         ix->cum_w[0] = 0;
         for (int b = 1; b <= p.B; ++b) {
+            const int kv = ix->kv_tiles[b - 1];
+            if (kv > 0) items += ix->cum_tiles[b] / kv;           // query blocks of the sequence
+            longest = max(longest, kv);
             acc += ix->cum_tiles[b]; ix->cum_tiles[b] = acc;
             accw += ix->cum_w[b]; ix->cum_w[b] = accw;
         }
-        // No block's share of the cost may be smaller than the heaviest tile, so that consecutive tiles never skip
-        // a block: every working block then owns at least one tile and the blocks sharing a work item are consecutive.
+        // Few short work items (one sequence with a short prefix, say): a block's fixed costs outweigh its tiles, and
+        // cutting items into pieces would add a partial and a merge to each.  Every block then takes whole items.
+        const long long n_items = (long long)p.H * items;
+        ix->whole_items = (n_items > 0 && n_items <= (long long)gridDim.x && longest <= kWholeItemTiles) ? 1 : 0;
+        // Otherwise no block's share of the cost may be smaller than the heaviest tile, so that consecutive tiles never
+        // skip a block: every working block then owns at least one tile and the blocks sharing a work item are
+        // consecutive.
         const long long tot_w = (long long)p.H * accw;
-        *n_blocks = (int)max(1LL, min((long long)gridDim.x, tot_w / (tile_weight(QB) + item_weight(QB))));
+        *n_blocks = ix->whole_items ? (int)n_items
+                                    : (int)max(1LL, min((long long)gridDim.x, tot_w / (tile_weight(QB) + item_weight(QB))));
     }
     __syncthreads();
     if (tid == 0 || tid == 32) {               // the two ends of this block's range, side by side
         const long long tot = (long long)p.H * ix->cum_tiles[p.B], tot_w = (long long)p.H * ix->cum_w[p.B];
         const int nb = *n_blocks, which = tid >> 5;
-        range[which] = (tot > 0 && (int)blockIdx.x < nb) ? first_tile_of_block<QB>(ix, p, (int)blockIdx.x + which, nb, tot_w, tot) : 0;
+        long long t = 0;
+        if (tot > 0 && (int)blockIdx.x < nb) {
+            if (ix->whole_items) {
+                // first tile of work item number c = (sequence, head, query block) in tile order
+                int c = (int)blockIdx.x + which, b = 0;
+                t = tot;
+                for (; b < p.B; ++b) {
+                    const int kv = ix->kv_tiles[b], tb = ix->cum_tiles[b + 1] - ix->cum_tiles[b];
+                    const int per_seq = kv > 0 ? p.H * (tb / kv) : 0;
+                    if (c < per_seq) { t = (long long)p.H * ix->cum_tiles[b] + (long long)c * kv; break; }
+                    c -= per_seq;
+                }
+            } else {
+                t = first_tile_of_block<QB>(ix, p, (int)blockIdx.x + which, nb, tot_w, tot);
+            }
+        }
+        range[which] = t;
     }
     __syncthreads();
 }
