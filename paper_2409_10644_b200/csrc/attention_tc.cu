@@ -5,8 +5,9 @@
 // One persistent thread block per SM walks a contiguous range of 128-key tiles of the flattened
 // (sequence, head, query block, key tile) space, so the K/V stream of every (sequence, head) is read from HBM once
 // and all SMs carry the same cost whatever the batch and the prefix lengths are.  Where a range boundary cuts a
-// work item, every side writes an unnormalised partial (reference, sum, weighted values) and takes a ticket; the
-// block that arrives last combines the partials: split-KV with a fused combine.
+// work item, the blocks that continue it write unnormalised partials (reference, sum, weighted values) as the
+// first thing they do and take a ticket; the block that started the item, whose piece is its last segment and is
+// still in tensor memory, folds them in at its end: split-KV with a fused combine.
 //
 // The problem is set up transposed so that the small dimension (tree tokens) is the MMA N and the 128 keys of a
 // tile fill the MMA M:
@@ -36,10 +37,10 @@
 //     between two of them would otherwise pace the tensor pipe;
 //   * the producer issues loads in the order in which slots come free (K0 K1 V0 K2 V1 ...), about two tiles ahead.
 //
-// Warp roles (480 threads): warps 0-11 softmax / mask / epilogue / merge, warp 12 TMA producer, warp 13 MMA issuer
-// and owner of the tensor-memory allocation, warp 14 bookkeeping (which other blocks share a work item with this
-// one).  Every mbarrier wait is bounded; a wait that runs out raises a flag in the workspace header, all roles
-// drain and the block exits cleanly.
+// Warp roles (512 threads): warps 0-11 softmax / mask / epilogue, warp 12 TMA producer, warp 13 MMA issuer and owner
+// of the tensor-memory allocation, warp 14 polls the tickets of a split last work item, warp 15 idle; at the end of
+// the block warps 12-15 together merge such an item (they reach all 128 lanes of tensor memory).  Every wait is
+// bounded; one that runs out raises a flag in the workspace header, all roles drain and the block exits cleanly.
 #include <mutex>
 #include <type_traits>
 
@@ -48,8 +49,8 @@
 namespace mcsd {
 
 constexpr int kGroups = 3;                          // softmax warpgroups
-constexpr int kProducerWarp = 4 * kGroups, kMmaWarp = kProducerWarp + 1, kHelperWarp = kMmaWarp + 1;
-constexpr int kTcThreads = 32 * (kHelperWarp + 1);
+constexpr int kProducerWarp = 4 * kGroups, kMmaWarp = kProducerWarp + 1;   // service warpgroup: warps 12..15
+constexpr int kTcThreads = 32 * (kProducerWarp + 4);
 constexpr int kColS1 = 160, kColO = 320, kColL = 480, kColL2 = 496;
 constexpr int kSlots = 4;                      // ring slots that fit next to Q and P^T of 112..160 queries
 
@@ -57,12 +58,12 @@ struct TcSmall {
     unsigned long long slot_full[kSlots];   // [0], [1]: key tile of even / odd tiles, [2], [3]: value tile
     unsigned long long s_full[2];            // S^T of even / odd tiles finished: scores ready, key slot and (last tile) Q free
     unsigned long long pv_done[2];           // products of even / odd tiles finished: value slot and P^T free, O^T and l current
-    unsigned long long p_full, q_full, drain, info_ready;
+    unsigned long long p_full, q_full, drain;
+    unsigned long long merge_bar;            // a staged copy of another block's partial has landed
+    int merge_np1;                           // pieces of later blocks to fold into this block's last segment (0: none)
+    Segment merge_item;                      // that segment's work item
     uint32_t tmem_base;
     int abort_flag;
-    int merge_parts[kGroups];              // > 0: this block finished a split work item last and merges it
-    int piece_parts[2];                // pieces of the work items at the two ends of this block's range
-    unsigned short piece_slot[2][kMaxParts];
     long long range[2];
     int n_blocks;
     alignas(16) float m_ref[kGroups][64];  // running reference of a group's own query columns (at most 56)
@@ -115,7 +116,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         mbar_init(&sm->p_full, 128 * kGroups);
         mbar_init(&sm->q_full, 1);
         mbar_init(&sm->drain, 1);
-        mbar_init(&sm->info_ready, 1);
+        mbar_init(&sm->merge_bar, 1);
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -158,6 +159,9 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             cv = ck;
             bool ok = true;
             uint32_t nk = 0, nv = 0;                       // loads issued
+            // keys and values that only one work unit reads are streamed through L2 with evict-first priority
+            const bool stream_once = p.group == p.G;
+            const uint64_t pol = l2_policy_evict_first();
             auto load_tile = [&](const Cursor& c, bool values, uint32_t slot) {
                 const int lti = c.s.lt + c.i;
                 const bool tree = lti >= c.s.nP;
@@ -166,8 +170,13 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 const CUtensorMap* map = values ? (tree ? &tm_vt : &tm_vc) : (tree ? &tm_kt : &tm_kc);
                 const uint32_t dst = smem_u32(ring) + slot * (uint32_t)kSlotBytes;
                 mbar_expect_tx(&sm->slot_full[slot], (uint32_t)kSlotBytes);
-                tma_load_3d(dst, map, &sm->slot_full[slot], 0, row0, bh_kv);
-                tma_load_3d(dst + kSlabBytes, map, &sm->slot_full[slot], 64, row0, bh_kv);
+                if (stream_once) {
+                    tma_load_3d_hint(dst, map, &sm->slot_full[slot], 0, row0, bh_kv, pol);
+                    tma_load_3d_hint(dst + kSlabBytes, map, &sm->slot_full[slot], 64, row0, bh_kv, pol);
+                } else {
+                    tma_load_3d(dst, map, &sm->slot_full[slot], 0, row0, bh_kv);
+                    tma_load_3d(dst + kSlabBytes, map, &sm->slot_full[slot], 64, row0, bh_kv);
+                }
             };
             auto advance = [&](Cursor& c) {
                 c.t += 1;
@@ -217,31 +226,6 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     }
                 }
             }
-        }
-    } else if (warp == kHelperWarp) {
-        // =========================================================== bookkeeping, off everybody's critical path
-        if (lane == 0) {
-            for (int which = 0; which < 2; ++which) {
-                Segment sp;
-                locate<QB>(ix, p, which == 0 ? t_begin : t_end - 1, sp);
-                const long long at = which == 0 ? t_begin : t_end - 1;
-                const long long t0 = at - sp.lt, t1 = t0 + sp.Tkv;
-                int nparts = 0;
-                const bool shared = which == 0 ? (t0 < t_begin || t1 > t_end) : (t0 > t_begin && t1 > t_end);
-                if (shared) {
-                    const int c_lo = block_of_tile<QB>(ix, p, t0, G, total_w);
-                    const int c_hi = block_of_tile<QB>(ix, p, t1 - 1, G, total_w);
-                    nparts = min(c_hi - c_lo + 1, kMaxParts);
-                    int others = 0;
-                    for (int i = 0; i < nparts; ++i) {
-                        if (c_lo + i == cta) continue;
-                        const long long start = first_tile_of_block<QB>(ix, p, c_lo + i, G, total_w, total);
-                        sm->piece_slot[which][others++] = (unsigned short)(2 * (c_lo + i) + (t0 > start ? 1 : 0));
-                    }
-                }
-                sm->piece_parts[which] = nparts;
-            }
-            mbar_arrive(&sm->info_ready);
         }
     } else if (warp == kMmaWarp) {
         // =========================================================== MMA issuer
@@ -324,7 +308,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 while (!mbar_try_wait(&sm->drain, 0) && clock64() - t0 < kSpinCycles) {}
             }
         }
-    } else {
+    } else if (warp < kProducerWarp) {
         // =========================================================== softmax / mask / epilogue
         const int wg = warp >> 2, wq = warp & 3;
         const int r = tid & 127;                       // key row of a tile = TMEM lane
@@ -545,9 +529,14 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             }
             if (group_sync_any(bar_id, failed)) { failed = true; break; }
 
-            // ---- epilogue of the segment: each group finishes its own query columns
+            // ---- epilogue of the segment: each group finishes its own query columns.  A segment that holds a whole work
+            // item is normalised and written out.  A piece of a split item that does not start the item is written to
+            // the workspace unnormalised and announced with a ticket.  The piece that starts a split item is always a
+            // block's last segment: it stays in tensor memory and the service warps merge the other pieces into it (see
+            // the end of the kernel), so there is nothing to do here.
             const uint32_t glast = g + (uint32_t)cnt - 1u;
             const bool full = (cnt == s.Tkv);
+            if (!full && s.lt == 0) break;
             const int slot_id = 2 * cta + (t > t_begin ? 1 : 0);
             if (!mbar_wait(&sm->pv_done[glast & 1u], (glast >> 1) & 1u, abort_flag, hdr, 10)) failed = true;
             tc_fence_after();
@@ -621,105 +610,160 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             }
             tc_fence_before();
             if (!full) {
-                // Split-KV combine: every block that finished a piece of this work item takes a ticket; the last
-                // one merges the other pieces (read back from the workspace) with its own, which is still in
-                // tensor memory.  The softmax groups own disjoint query columns and run this protocol independently.
+                // the partial is complete: make it visible, then take the ticket the merging block waits for
                 __threadfence();
                 group_sync_any(bar_id, false);
-                const int which = slot_id & 1;
-                if (r == 0) {
-                    if (!mbar_wait(&sm->info_ready, 0, abort_flag, hdr, 12)) failed = true;
-                    int* counter = p.counters + ((size_t)bh * 2 + s.qb) * 4 + wg;
-                    const int nparts = sm->piece_parts[which];
-                    sm->merge_parts[wg] = nparts;
-                    const int old = atomicAdd(counter, 1);
-                    if (old == nparts - 1) {
-                        *(volatile int*)counter = 0;              // nobody else arrives in this launch: ready for the next one
-                        __threadfence();                          // acquire: the other pieces' partials are visible
-                    } else {
-                        sm->merge_parts[wg] = 0;                  // not the last: nothing more to do
-                    }
-                }
-                group_sync_any(bar_id, false);
-                const int nparts = sm->merge_parts[wg];
-                if (nparts > 0) {
-                    // One dependent round trip to the workspace per piece and batch of column groups: all O^T loads
-                    // of a piece are issued first; while they are in flight the thread that owns a query column folds
-                    // the piece's (m, l) into its running reference and normaliser and leaves the two rescale factors
-                    // of that column in shared memory; after a group barrier every thread applies them to its rows.
-                    const int np1 = nparts - 1;
-                    float* const fa = &sm->wred[wg][0][0];                   // [piece parity][64]: factor for what we have
-                    float* const fw = &sm->wred[wg][2][0];                   // [piece parity][64]: factor for the new piece
-                    const bool col_owner = r < ncg * 8 && col0 + r < s.Nq;
-                    constexpr int GB = 1;                                    // column groups per batch (what the registers allow)
-#pragma unroll
-                    for (int j0 = 0; j0 < CPT; j0 += GB) {
-                        if (j0 >= ncg) break;
-                        float acc[GB][8];
-#pragma unroll
-                        for (int jj = 0; jj < GB; ++jj)
-                            if (j0 + jj < CPT && j0 + jj < ncg) tc_ld8(tmem + lane_addr + kColO + col0 + 8 * (j0 + jj), acc[jj]);
-                        tc_wait_ld();
-                        float m_run = col_owner ? mref[r] : -INFINITY;       // of column r, kept by its owner
-                        float l_run2 = col_owner ? alph[r] : 0.f;
-                        for (int i = 0; i < np1; ++i) {
-                            const int slot = sm->piece_slot[which][i];
-                            float os[GB][8];
-#pragma unroll
-                            for (int jj = 0; jj < GB; ++jj)
-#pragma unroll
-                                for (int k = 0; k < 8; ++k) {
-                                    const int n = col0 + 8 * (j0 + jj) + k;
-                                    const bool on = j0 + jj < CPT && j0 + jj < ncg && n < s.Nq;
-                                    os[jj][k] = on ? __ldcg(p.part_o + ((size_t)slot * kMaxQ + n) * 128 + r) : 0.f;
-                                }
-                            float* const fa_i = fa + 64 * (i & 1);
-                            float* const fw_i = fw + 64 * (i & 1);
-                            if (col_owner) {
-                                const float ms = __ldcg(p.part_ml + ((size_t)slot * 2 + 0) * kMaxQ + col0 + r);
-                                const float ls = __ldcg(p.part_ml + ((size_t)slot * 2 + 1) * kMaxQ + col0 + r);
-                                const float mn = fmaxf(m_run, ms);
-                                const float a = (mn == -INFINITY || m_run == -INFINITY) ? 0.f : exp2f(m_run - mn);
-                                const float wgt = (mn == -INFINITY || ms == -INFINITY) ? 0.f : exp2f(ms - mn);
-                                l_run2 = l_run2 * a + ls * wgt;
-                                m_run = mn;
-                                fa_i[r] = a;
-                                fw_i[r] = wgt;
-                            }
-                            group_sync_any(bar_id, false);                   // factors of piece i are in place
-#pragma unroll
-                            for (int jj = 0; jj < GB; ++jj)
-#pragma unroll
-                                for (int k = 0; k < 8; ++k) {
-                                    const int rel = 8 * (j0 + jj) + k;
-                                    if (j0 + jj < CPT && j0 + jj < ncg)
-                                        acc[jj][k] = fmaf(os[jj][k], fw_i[rel], acc[jj][k] * fa_i[rel]);
-                                }
-                            // piece i + 2 reuses these factor slots: by then every thread has passed the barrier of
-                            // piece i + 1, which it reaches only after the loop above
-                        }
-                        // normaliser of every column, then the output rows
-                        group_sync_any(bar_id, false);                       // everybody is done with the factor slots
-                        if (col_owner) fa[r] = l_run2 > 0.f ? 1.f / l_run2 : 0.f;
-                        group_sync_any(bar_id, false);
-#pragma unroll
-                        for (int jj = 0; jj < GB; ++jj)
-#pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                const int rel = 8 * (j0 + jj) + k, n = col0 + rel;
-                                if (j0 + jj < CPT && j0 + jj < ncg && n < s.Nq) {
-                                    const int jq = s.q0 + n;
-                                    p.out[(((size_t)bh * p.G + (jq & (p.G - 1))) * p.N + (jq >> p.g_shift)) * 128 + r] =
-                                        __float2bfloat16_rn(acc[jj][k] * fa[rel]);
-                                }
-                            }
-                        group_sync_any(bar_id, false);                       // before the next batch reuses the slots
-                    }
-                }
+                if (r == 0) atomicAdd(p.counters + ((size_t)bh * 2 + s.qb) * 4 + wg, 1);
             }
             group_sync_any(bar_id, false);
             g += (uint32_t)cnt;
             t += cnt;
+        }
+    }
+
+    // =========================================================== merge of a split work item (service warps)
+    // If this block's last segment starts a work item that continues in later blocks, its four service warps (done
+    // with loading and issuing by then; together they reach all 128 lanes of tensor memory) fold the other pieces,
+    // which those blocks produced as the first thing they did, into this block's own piece, still in tensor memory:
+    //     m = max(m_a, m_b),  l = l_a 2^(m_a - m) + l_b 2^(m_b - m),  O = O_a 2^(m_a - m) + O_b 2^(m_b - m),  o = O / l.
+    // Thread r holds head dim r of every query.  Under a saturated memory system a dependent trip to the workspace
+    // costs 1.5-2 us, so there is one per piece: the piece's rows and its (m, l) are brought into the (now idle)
+    // key/value ring with two bulk copies.  The tickets that say the pieces are complete are polled, at leisure, by
+    // a warp that has nothing else to do, long before they are needed.  The code lives in this branch, away from the
+    // softmax warps' tile loop, so that its registers are its own.
+    if (warp >= kProducerWarp) {
+        const int r = tid - 32 * kProducerWarp;                  // 0..127 = tensor-memory lane = head dim
+        if (warp == kMmaWarp + 1) {
+            if (lane == 0) {
+                Segment sp;
+                locate<QB>(ix, p, t_end - 1, sp);
+                const long long t0 = t_end - 1 - sp.lt, t1 = t0 + sp.Tkv;
+                int np1 = 0;
+                if (t1 > t_end && t0 >= t_begin) {
+                    np1 = min(block_of_tile<QB>(ix, p, t1 - 1, G, total_w) - cta, kMaxParts - 1);
+                    // one counter per softmax group of the writing blocks; np1 arrivals each
+                    int* counter = p.counters + ((size_t)(sp.b * p.H + sp.h) * 2 + sp.qb) * 4;
+                    const long long t_start = clock64();
+                    for (int gq = 0; gq < kGroups; ++gq) {
+                        while (*(volatile int*)(counter + gq) < np1) {
+                            __nanosleep(500);
+                            if (*(volatile int*)abort_flag || clock64() - t_start > kSpinCycles) {
+                                *(volatile int*)abort_flag = 1;
+                                hdr->detail = 14;
+                                hdr->status = MCSD_ERR_TIMEOUT;
+                                break;
+                            }
+                        }
+                        *(volatile int*)(counter + gq) = 0;       // ready for the next launch
+                    }
+                    __threadfence();                              // acquire: the pieces' partials are visible
+                }
+                sm->merge_np1 = np1;
+                sm->merge_item = sp;
+            }
+            __syncwarp();
+        }
+        // the service warps without a loop of their own park on a hardware barrier until the producer and the MMA
+        // warp are done (a spinning wait would take issue slots from the softmax warps for the whole kernel)
+        asm volatile("bar.sync %0, 128;" ::"n"(kGroups + 3) : "memory");
+        const int np1 = sm->merge_np1;
+        if (np1 > 0) {
+            const Segment sp = sm->merge_item;
+            const uint32_t lane_addr = (uint32_t)((r >> 5) * 32) << 16;
+            const int bh = sp.b * p.H + sp.h;
+            float* const l_run = &sm->wred[0][0][0];             // [160] running normaliser, at the end 1 / l
+            float* const m_run = l_run + kMaxQ;                  // [160] running reference
+            float* const w_a = m_run + kMaxQ;                    // [160] weight of what has been combined so far
+            float* const w_b = w_a + kMaxQ;                      // [160] weight of the piece being added
+            static_assert(4 * kMaxQ <= kGroups * 4 * 64, "the merge scratch must fit the per-warp reduction scratch");
+            const float* stage_o = reinterpret_cast<const float*>(ring);                     // [<= 160][128]
+            const float* stage_ml = reinterpret_cast<const float*>(ring + kMaxQ * 512);      // [2][160]
+            // column -> (softmax group, index within the group), as the softmax warps split this segment
+            const int ng8 = (sp.Nq + 7) >> 3, base = ng8 / kGroups, rem = ng8 % kGroups;
+            auto group_of = [&](int q, int& rel) {
+                const int g8 = q >> 3;
+                int gidx = 0;
+#pragma unroll
+                for (int x = 1; x < kGroups; ++x) gidx += (g8 >= x * base + min(x, rem)) ? 1 : 0;
+                rel = q - 8 * (gidx * base + min(gidx, rem));
+                return gidx;
+            };
+            // All of this block's tensor-core work must have finished: the barrier that completes exactly once, after
+            // the MMA warp's last commit (a parity wait on a barrier that is reused per tile could pass on an earlier
+            // phase).
+            bool ok = mbar_wait(&sm->drain, 0, abort_flag, hdr, 10);
+            tc_fence_after();
+            // this block's own row sums and references: lane q of the first set of row-sum columns holds query q, lane
+            // q - 128 of the second set query q; the copy kept current is number (group of q)
+            {
+                float c1[4], c2[4];
+                tc_ld4(tmem + lane_addr + kColL, c1);
+                tc_ld4(tmem + lane_addr + kColL2, c2);
+                tc_wait_ld();
+                int rel;
+                if (r < sp.Nq) { const int gq = group_of(r, rel); l_run[r] = gq == 0 ? c1[0] : gq == 1 ? c1[1] : c1[2]; m_run[r] = sm->m_ref[gq][rel]; }
+                if (128 + r < sp.Nq) { const int gq = group_of(128 + r, rel); l_run[128 + r] = gq == 0 ? c2[0] : gq == 1 ? c2[1] : c2[2]; m_run[128 + r] = sm->m_ref[gq][rel]; }
+            }
+            ok = ok && !*(volatile int*)abort_flag;
+            for (int i = 1; i <= np1 && ok; ++i) {
+                const size_t slot = (size_t)(2 * (cta + i));       // the piece is that block's first segment
+                asm volatile("bar.sync %0, 128;" ::"n"(kGroups + 2) : "memory");    // staging area and weights are free
+                if (r == 0) {
+                    const uint32_t o_bytes = (uint32_t)ng8 * 4096u, ml_bytes = 2u * kMaxQ * 4u;
+                    asm volatile("fence.proxy.async;" ::: "memory");
+                    mbar_expect_tx(&sm->merge_bar, o_bytes + ml_bytes);
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(smem_u32(stage_o)), "l"(p.part_o + slot * kMaxQ * 128), "r"(o_bytes), "r"(smem_u32(&sm->merge_bar)) : "memory");
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(smem_u32(stage_ml)), "l"(p.part_ml + slot * 2 * kMaxQ), "r"(ml_bytes), "r"(smem_u32(&sm->merge_bar)) : "memory");
+                }
+                ok = mbar_wait(&sm->merge_bar, (uint32_t)(i - 1) & 1u, abort_flag, hdr, 13);
+                const bool last = i == np1;
+                for (int q = r; q < sp.Nq; q += 128) {
+                    const float ma = m_run[q], mb = stage_ml[q], lb = stage_ml[kMaxQ + q];
+                    const float mn = fmaxf(ma, mb);
+                    const float wa = (mn == -INFINITY || ma == -INFINITY) ? 0.f : exp2f(ma - mn);
+                    const float wb = (mn == -INFINITY || mb == -INFINITY) ? 0.f : exp2f(mb - mn);
+                    const float ln = l_run[q] * wa + lb * wb;
+                    m_run[q] = mn;
+                    w_a[q] = wa;
+                    w_b[q] = wb;
+                    l_run[q] = last ? (ln > 0.f ? 1.f / ln : 0.f) : ln;
+                }
+                asm volatile("bar.sync %0, 128;" ::"n"(kGroups + 2) : "memory");
+#pragma unroll 1
+                for (int j0 = 0; j0 < ng8; j0 += 4) {                               // four column groups at a time
+                    float acc[4][8];
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj)
+                        if (j0 + jj < ng8) tc_ld8(tmem + lane_addr + kColO + 8 * (j0 + jj), acc[jj]);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj) {
+                        if (j0 + jj < ng8) {
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const int q = 8 * (j0 + jj) + k;
+                                acc[jj][k] = fmaf(stage_o[(size_t)q * 128 + r], w_b[q], acc[jj][k] * w_a[q]);
+                            }
+                            if (last) {
+#pragma unroll
+                                for (int k = 0; k < 8; ++k) {
+                                    const int q = 8 * (j0 + jj) + k;
+                                    if (q < sp.Nq) {
+                                        const int jq = sp.q0 + q;   // stacked query: head jq % G of the group, node jq / G
+                                        p.out[(((size_t)bh * p.G + (jq & (p.G - 1))) * p.N + (jq >> p.g_shift)) * 128 + r] =
+                                            __float2bfloat16_rn(acc[jj][k] * l_run[q]);
+                                    }
+                                }
+                            } else {
+                                tc_st8(tmem + lane_addr + kColO + 8 * (j0 + jj), acc[jj]);
+                            }
+                        }
+                    }
+                }
+                if (!last) tc_wait_st();
+            }
         }
     }
 
