@@ -113,7 +113,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         mbar_init(&sm->s_full[1], 1);
         mbar_init(&sm->pv_done[0], 1);
         mbar_init(&sm->pv_done[1], 1);
-        mbar_init(&sm->p_full, 128 * kGroups);
+        mbar_init(&sm->p_full, 4 * kGroups);      // one arrival per softmax warp
         mbar_init(&sm->q_full, 1);
         mbar_init(&sm->drain, 1);
         mbar_init(&sm->merge_bar, 1);
@@ -523,9 +523,12 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                         for (int x = 0; x < 8; ++x) { z0[x] = make_uint4(0, 0, 0, 0); z1[x] = make_uint4(0, 0, 0, 0); }
                     }
                 }
+                // every thread makes its own P^T stores visible to the tensor cores' proxy; then one arrival per warp (384
+                // arrivals on one shared-memory word would queue up behind one another)
                 fence_async_smem();
                 tc_fence_before();
-                mbar_arrive(&sm->p_full);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm->p_full);
             }
             if (group_sync_any(bar_id, failed)) { failed = true; break; }
 
