@@ -125,6 +125,18 @@ int mcsd_tree_attention(const void* q, const void* k_cache, const void* v_cache,
                         int dtype, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Self-test of the bounded device-side waits (the paper has no counterpart; the kernels of mcsd_tree_attention wait on
+ * hardware barriers for tiles, products and partial results, and every such wait has a limit so that a lost signal ends
+ * in a status, not in a hung GPU).  Launches one small block that waits, with the same wait routine, for a signal that
+ * never comes: after about `microseconds` (1 .. 100000) the wait gives up, the block exits normally, and the workspace
+ * header holds MCSD_ERR_TIMEOUT, which mcsd_workspace_status() then returns.  The workspace must be zero-filled again
+ * before it is used for anything else.  Nothing faults, traps or spins without limit.
+ *   workspace   [dev] >= 256 bytes, 256-byte aligned
+ * Errors: MCSD_ERR_NULL, MCSD_ERR_BAD_SHAPE, MCSD_ERR_CUDA.
+ */
+int mcsd_selftest_bounded_wait(void* workspace, size_t workspace_bytes, int microseconds, void* stream);
+
+/*
  * Which kernel mcsd_tree_attention / mcsd_tree_attention_gqa runs for a shape (Section 2.2 defines the operation; the
  * choice of kernel is this library's).  The tensor-core kernel (tcgen05, bandwidth-bound) takes bf16, D = 128,
  * B <= 256 and B * (L_max / 128 + 4) < 2^23 (its per-sequence tables are 32-bit and live in shared memory); every

@@ -24,7 +24,7 @@ MCSD_MAX_WORDS = 3
 
 _EXPORTS = (
     "mcsd_status_string", "mcsd_last_cuda_error", "mcsd_launch_count", "mcsd_build_mask", "mcsd_tree_attention_workspace_bytes",
-    "mcsd_tree_attention", "mcsd_tree_attention_gqa", "mcsd_workspace_status", "verify_node_states", "mcsd_tree_attention_path", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_logits", "mcsd_verify_tree_static", "mcsd_commit_kv", "mcsd_sample_roots",
+    "mcsd_tree_attention", "mcsd_tree_attention_gqa", "mcsd_workspace_status", "verify_node_states", "mcsd_tree_attention_path", "mcsd_selftest_bounded_wait", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_logits", "mcsd_verify_tree_static", "mcsd_commit_kv", "mcsd_sample_roots",
     "mcsd_sample_roots_logits", "mcsd_verify_shard_workspace_bytes", "mcsd_verify_shard_gather", "mcsd_verify_shard_round",
     "mcsd_verify_shard_select", "mcsd_verify_shard_pick",
 )
@@ -48,6 +48,8 @@ def _load() -> ctypes.CDLL:
                                     ctypes.POINTER(c_int), c_void_p]
     lib.mcsd_tree_attention_workspace_bytes.restype = c_size_t
     lib.mcsd_tree_attention_workspace_bytes.argtypes = [c_int] * 6
+    lib.mcsd_selftest_bounded_wait.restype = c_int
+    lib.mcsd_selftest_bounded_wait.argtypes = [c_void_p, c_size_t, c_int, c_void_p]
     lib.mcsd_tree_attention_path.restype = c_int
     lib.mcsd_tree_attention_path.argtypes = [c_int] * 7
     lib.mcsd_tree_attention.restype = c_int
@@ -189,6 +191,15 @@ def verify_node_states(workspace: torch.Tensor, B: int, N: int):
     child or -1) and `c` float64[B][N] (the stop distribution at that node is max(p - c q, 0))."""
     raw = workspace[256:256 + 16 * B * N]
     return {"next_child": raw.view(torch.int32).view(B, N, 4)[..., 0], "c": raw.view(torch.float64).view(B, N, 2)[..., 1]}
+
+
+def mcsd_selftest_bounded_wait(workspace: torch.Tensor, microseconds: int = 1000) -> None:
+    """Launches the bounded-wait self-test on `workspace` (see mcsd.h); mcsd_workspace_status(workspace) then reads
+    MCSD_ERR_TIMEOUT and the workspace has to be zero-filled again."""
+    _dev_tensor(workspace, torch.uint8, "workspace")
+    with torch.cuda.device(workspace.device):
+        st = lib.mcsd_selftest_bounded_wait(_ptr(workspace), workspace.numel(), int(microseconds), _stream())
+    _check(st, "mcsd_selftest_bounded_wait")
 
 
 def mcsd_tree_attention_path(B, H_q, H_kv, N, D, L_max, dtype_code) -> int:

@@ -55,6 +55,15 @@ static int run_attention(const void* q, const void* k_cache, const void* v_cache
     return mcsd::tree_attention_simt(a, scratch, s);
 }
 
+extern "C" int mcsd_selftest_bounded_wait(void* workspace, size_t workspace_bytes, int microseconds, void* stream) {
+    if (!workspace) return MCSD_ERR_NULL;
+    if (workspace_bytes < sizeof(mcsd::WorkspaceHeader) || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MCSD_ERR_BAD_SHAPE;
+    if (microseconds < 1 || microseconds > 100000) return MCSD_ERR_BAD_SHAPE;     // at most a tenth of a second
+    // clock64 ticks at the SM clock, at most about 2 GHz: 2000 cycles per microsecond bound the wait from above
+    return mcsd::tc_bounded_wait_selftest(static_cast<mcsd::WorkspaceHeader*>(workspace), 2000LL * microseconds, 42,
+                                          static_cast<cudaStream_t>(stream));
+}
+
 extern "C" int mcsd_tree_attention_path(int B, int H_q, int H_kv, int N, int D, int L_max, int dtype) {
     const int st = check_shape(B, H_q, N, D, L_max, dtype);
     if (st != MCSD_OK) return st;

@@ -30,6 +30,7 @@ int tree_attention_simt(const AttentionArgs& a, void* scratch, cudaStream_t stre
 bool tc_shape_supported(int B, int H, int G, int N, int D, int L_max, int dtype);   // shape and dtype alone
 bool tc_supported(const AttentionArgs& a);
 size_t tc_workspace_bytes(int B, int H, int N, int D, int L_max);
+int tc_bounded_wait_selftest(WorkspaceHeader* header, long long limit_cycles, int where, cudaStream_t stream);
 int tree_attention_tc(const AttentionArgs& a, WorkspaceHeader* header, void* scratch, size_t scratch_bytes,
                       cudaStream_t stream);
 

@@ -779,6 +779,34 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     }
 }
 
+// ------------------------------------------------------------------ self-test of the bounded waits
+// One block waits, with the kernel's own wait routine and a short limit, on a barrier that nothing ever completes:
+// the wait must give up, raise the flag the other roles watch, leave MCSD_ERR_TIMEOUT and the wait's code in the
+// workspace header, and the block must exit normally.  A second warp that starts its wait afterwards must give up
+// at once because of the flag.
+__global__ void bounded_wait_selftest_kernel(WorkspaceHeader* header, long long limit_cycles, int where) {
+    __shared__ unsigned long long bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    bool ok = true;
+    if (threadIdx.x < 32) ok = mbar_wait_slow(&bar, 0, &abort_flag, header, where, limit_cycles);
+    __syncthreads();
+    if (threadIdx.x >= 32) ok = mbar_wait_slow(&bar, 0, &abort_flag, header, where + 100, 1LL << 40);   // sees the flag: no long wait
+    if (ok) header->detail = -1;                               // must not happen
+}
+
+int tc_bounded_wait_selftest(WorkspaceHeader* header, long long limit_cycles, int where, cudaStream_t stream) {
+    bounded_wait_selftest_kernel<<<1, 64, 0, stream>>>(header, limit_cycles, where);
+    MCSD_CUDA_CHECK(cudaGetLastError());
+    count_launches(1);
+    return MCSD_OK;
+}
+
 // ------------------------------------------------------------------ host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,

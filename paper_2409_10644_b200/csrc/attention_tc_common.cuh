@@ -76,13 +76,14 @@ __device__ __forceinline__ bool mbar_try_wait(void* bar, uint32_t parity) {
 
 // Bounded wait.  Returns false if the wait ran out or another role already gave up (abort_flag, in shared memory);
 // `where` names the wait in the workspace header.
-static __device__ __noinline__ bool mbar_wait_slow(void* bar, uint32_t parity, int* abort_flag, WorkspaceHeader* header, int where) {
+static __device__ __noinline__ bool mbar_wait_slow(void* bar, uint32_t parity, int* abort_flag, WorkspaceHeader* header, int where,
+                                                   long long limit = kSpinCycles) {
     const long long t0 = clock64();
     for (uint32_t it = 0;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 255u) {
             if (*(volatile int*)abort_flag) return false;
-            if (clock64() - t0 > kSpinCycles) {
+            if (clock64() - t0 > limit) {
                 *(volatile int*)abort_flag = 1;
                 header->detail = where;
                 header->status = MCSD_ERR_TIMEOUT;

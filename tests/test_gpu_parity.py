@@ -660,3 +660,39 @@ def test_commit_kv_matches_oracle(m, idx, dtype_D):
         assert np.array_equal(to_np(l["v_cache"]), hl["v_cache"])
     assert np.array_equal(lens_d.cpu().numpy(), new_ref)
     assert (new_ref > lens).any()
+
+
+# ----------------------------------------------------------------------------------------------
+# bounded device-side waits
+# ----------------------------------------------------------------------------------------------
+
+def test_a_wait_that_runs_out_ends_in_a_status_and_a_usable_context(m):
+    """The kernels' wait routine, given a signal that never comes and a short limit: the block gives up and exits, the
+    workspace reports MCSD_ERR_TIMEOUT, and the same context and (re-zeroed) workspace then run a normal launch."""
+    w = dataclasses.replace(workload(2), B=2, H=2, prefix=(100, 300))
+    parent = parent_array(w.n_roots, w.branching)
+    N = len(parent)
+    ws = m.new_workspace(m.mcsd_tree_attention_workspace_bytes(w.B, w.H, N, w.D, w.L_max, m.MCSD_BF16), "cuda")
+    assert m.mcsd_workspace_status(ws) == 0
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    m.mcsd_selftest_bounded_wait(ws, microseconds=2000)
+    stop.record()
+    torch.cuda.synchronize()
+    assert m.mcsd_workspace_status(ws) == -7                      # MCSD_ERR_TIMEOUT
+    assert "wait" in m.mcsd_status_string(-7)
+    hdr = ws[:8].view(torch.int32).cpu().numpy()
+    assert int(hdr[1]) == 42                                      # the code of the wait that gave up, not the follower's
+    assert 0.5 <= start.elapsed_time(stop) <= 50.0                # about the 2 ms asked for, not the kernels' 2 s
+    ws.zero_()
+    inp = attention_inputs(w, 0, "cuda", std=1.0)
+    lens = np.array([100, 300], dtype=np.int32)
+    tm = m.mcsd_build_mask(parent)
+    out = torch.full_like(inp["q"], float("nan"))
+    m.mcsd_tree_attention(inp["q"], inp["k_cache"], inp["v_cache"], inp["k_tree"], inp["v_tree"],
+                          torch.from_numpy(lens).cuda(), None, tm, out=out, softmax_scale=1 / np.sqrt(w.D), workspace=ws)
+    assert m.mcsd_workspace_status(ws) == 0
+    ref = oracle_attention_rows(inp, lens, None, parent, 1 / np.sqrt(w.D), [(0, 0), (1, 1)])
+    for (b, h), rr in ref.items():
+        err = np.abs(to_np(out[b, h]).astype(np.float64) - rr).max()
+        assert err <= TOL_BF16 * np.abs(rr).max()
