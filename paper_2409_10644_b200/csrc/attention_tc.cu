@@ -76,6 +76,16 @@ struct TcSmall {
 static_assert(sizeof(TcSmall) <= kSmemLimit - 1024 - kSlots * 32768 - 160 * 512, "TcSmall grew: four ring slots no longer fit");
 
 // 64 bits of a 192-bit row starting at bit `start` (bits past the row read as zero)
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+__device__ __forceinline__ uint32_t max_u16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.u16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
 __device__ __forceinline__ unsigned long long bits_from(const unsigned long long* w, int start) {
     const int wi = start >> 6, sh = start & 63;
     unsigned long long lo = w[wi] >> sh;
@@ -272,6 +282,27 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                         const uint32_t gj = g + (uint32_t)(i - 1), vb = gj & 1u;
                         ok = mbar_wait(&sm->slot_full[2u + vb], (gj >> 1) & 1u, abort_flag, hdr, 5);
                         if (!ok) break;
+                        {
+                            // Value rows past the end of the prefix (or past the active tree nodes) may hold anything,
+                            // NaN patterns included, and 0 * NaN is NaN: they are cleared here, by the warp that waits
+                            // for the tile anyway (the softmax warps would have to wait for a tile they do not need
+                            // yet).  Rows the copy did not find in the tensor arrived as zeros.  Whole rows: the
+                            // 128-byte swizzle only permutes inside a row.
+                            const int ltv = s.lt + i - 1;
+                            const bool tree_v = ltv >= s.nP;
+                            const int row0_v = (tree_v ? ltv - s.nP : ltv) * kTile;
+                            const int valid_v = min(kTile, (tree_v ? s.Nb : s.L) - row0_v);
+                            const int have_v = min(kTile, (tree_v ? p.N : p.L_max) - row0_v);
+                            if (valid_v < have_v) {
+                                unsigned char* v0 = ring + (size_t)(2u + vb) * kSlotBytes;
+                                for (int c = valid_v * 8 + lane; c < have_v * 8; c += 32) {
+                                    *reinterpret_cast<uint4*>(v0 + (size_t)c * 16) = make_uint4(0, 0, 0, 0);
+                                    *reinterpret_cast<uint4*>(v0 + kSlabBytes + (size_t)c * 16) = make_uint4(0, 0, 0, 0);
+                                }
+                                fence_async_smem();
+                                __syncwarp();
+                            }
+                        }
                         ok = mbar_wait(&sm->p_full, gj & 1u, abort_flag, hdr, 6);
                         if (!ok) break;
                         tc_fence_after();
@@ -323,19 +354,22 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             for (int i = tid; i < n_words; i += 128 * kGroups) anc_s[i] = p.anc[i];
             asm volatile("bar.sync %0, %1;" ::"n"(kGroups + 1), "n"(128 * kGroups) : "memory");
             const int NQ = p.N * p.G;                            // stacked queries: query j belongs to node j / G
-            const int n_chunks = (NQ + 31) >> 5;
+            const int n_kb = (p.N + 31) >> 5;                    // blocks of 32 tree keys
             const uint32_t* anc32 = reinterpret_cast<const uint32_t*>(anc_s);
-            for (int idx = tid; idx < p.N * 6; idx += 128 * kGroups) {
-                const int c = idx / p.N, t = idx - c * p.N;
-                uint32_t piece = 0;
-                if (c < n_chunks) {
-                    const uint32_t* col = anc32 + (t >> 5);          // 32-bit half of the 64-bit word that holds bit t
-                    const int n_end = min(32, NQ - 32 * c);
-#pragma unroll 8
-                    for (int i = 0; i < n_end; ++i)
-                        piece |= ((col[(size_t)((32 * c + i) >> p.g_shift) * p.words * 2] >> (t & 31)) & 1u) << i;
+            // a warp transposes one 32 x 32 block of bits at a time: lane i holds the keys 32 kb .. 32 kb + 31 that
+            // stacked query 32 c + i may see; the ballot over bit j is the set of those queries that see key 32 kb + j
+            for (int pair = warp; pair < 6 * n_kb; pair += 4 * kGroups) {
+                const int c = pair / n_kb, kb = pair - c * n_kb;
+                const int qi = 32 * c + lane;
+                const uint32_t w = qi < NQ ? anc32[(size_t)(qi >> p.g_shift) * p.words * 2 + kb] : 0u;
+                uint32_t mine = 0;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const uint32_t seen_by = __ballot_sync(0xffffffffu, (w >> j) & 1u);
+                    if (lane == j) mine = seen_by;
                 }
-                reinterpret_cast<uint32_t*>(&sm->dmask[t][0])[c] = piece;
+                const int t = 32 * kb + lane;
+                if (t < p.N) reinterpret_cast<uint32_t*>(&sm->dmask[t][0])[c] = mine;
             }
             asm volatile("bar.sync %0, %1;" ::"n"(kGroups + 1), "n"(128 * kGroups) : "memory");
         }
@@ -384,12 +418,18 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 const uint32_t s_addr = tmem + lane_addr + (sb ? kColS1 : 0) + col0;
 
                 // ---- the sweep: scores of this thread's columns, shifted, checked, exponentiated, packed; tensor memory
-                // is read SB column groups per round trip (what the 128 registers of a 15-warp block allow)
+                // is read SB column groups per round trip (what the 128 registers of a 16-warp block allow).  Prefix
+                // tiles take the plain sweep: every query sees every key, and a key row past the end of a ragged last
+                // tile is this thread's own row, cleared afterwards.  Tree tiles take the masked sweep, which clears
+                // single elements: the packed probabilities are ANDed with masks grown from the visibility bits, and
+                // the largest visible probability (bf16 bit patterns of positive numbers order like the numbers)
+                // stands in for the largest shifted score.
                 constexpr int SB = 2;
                 uint32_t pk[CPT][4];
                 float dmax = -INFINITY;
                 auto make_probs = [&](auto masked_tag) {
                     constexpr bool MASKED = decltype(masked_tag)::value;
+                    uint32_t pmax = 0;
 #pragma unroll
                     for (int j0 = 0; j0 < CPT; j0 += SB) {
                         if (j0 < ncg) {
@@ -405,24 +445,34 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                                     const float4 m0 = *reinterpret_cast<const float4*>(&mref[8 * j]);
                                     const float4 m1 = *reinterpret_cast<const float4*>(&mref[8 * j + 4]);
                                     const float mr[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
-                                    const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
                                     float yy[8];
 #pragma unroll
-                                    for (int k = 0; k < 8; ++k) {
-                                        yy[k] = fmaf(y[jj][k], p.scale_log2, -mr[k]);
-                                        if (MASKED && !((bits >> k) & 1u)) yy[k] = -INFINITY;
-                                    }
-                                    dmax = fmaxf(dmax, fmaxf(fmaxf(fmaxf(yy[0], yy[1]), fmaxf(yy[2], yy[3])),
-                                                             fmaxf(fmaxf(yy[4], yy[5]), fmaxf(yy[6], yy[7]))));
+                                    for (int k = 0; k < 8; ++k) yy[k] = fmaf(y[jj][k], p.scale_log2, -mr[k]);
+                                    if (!MASKED)
+                                        dmax = fmaxf(dmax, fmaxf(fmaxf(fmaxf(yy[0], yy[1]), fmaxf(yy[2], yy[3])),
+                                                                 fmaxf(fmaxf(yy[4], yy[5]), fmaxf(yy[6], yy[7]))));
 #pragma unroll
                                     for (int k = 0; k < 8; k += 2) {
                                         __nv_bfloat162 h2 = __floats2bfloat162_rn(ex2_approx(yy[k]), ex2_approx(yy[k + 1]));
                                         pk[j][k >> 1] = *reinterpret_cast<uint32_t*>(&h2);
                                     }
+                                    if (MASKED) {
+                                        // visibility bit k -> top bit of byte k (a multiply that spreads four bits), then
+                                        // a byte permute that replicates those top bits over the halves of a word
+                                        const uint32_t bits = (uint32_t)(cm >> (8 * j)) & 0xFFu;
+                                        const uint32_t lo4 = (bits & 0xFu) * 0x10204080u, hi4 = (bits >> 4) * 0x10204080u;
+                                        pk[j][0] &= prmt(lo4, 0u, 0x9988u);
+                                        pk[j][1] &= prmt(lo4, 0u, 0xBBAAu);
+                                        pk[j][2] &= prmt(hi4, 0u, 0x9988u);
+                                        pk[j][3] &= prmt(hi4, 0u, 0xBBAAu);
+                                        pmax = max_u16x2(pmax, max_u16x2(max_u16x2(pk[j][0], pk[j][1]), max_u16x2(pk[j][2], pk[j][3])));
+                                    }
                                 }
                             }
                         }
                     }
+                    // 0x4380 is 2^kLazyTau = 256 in bf16; NaN patterns are above it too
+                    if (MASKED) dmax = max(pmax & 0xFFFFu, pmax >> 16) > 0x4380u ? INFINITY : -INFINITY;
                 };
                 if (i == 0 && full_tile) {
                     // reference of a new segment: the scores of the tile's first key (see the file header)
@@ -442,8 +492,20 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     }
                     group_sync_any(bar_id, false);
                 }
-                if (full_tile) make_probs(std::false_type{}); else make_probs(std::true_type{});
-
+                auto sweep = [&]() {
+                    if (!tree) {
+                        make_probs(std::false_type{});
+                        if (r >= valid) {                      // a key row past the end of the prefix: seen by no query
+                            dmax = -INFINITY;
+#pragma unroll
+                            for (int j = 0; j < CPT; ++j) pk[j][0] = pk[j][1] = pk[j][2] = pk[j][3] = 0u;
+                        }
+                    } else {
+                        make_probs(std::true_type{});
+                    }
+                };
+                sweep();
+                // one vote per group: does any score exceed its reference by more than the lazy threshold?
                 if (group_sync_any(bar_id, dmax > kLazyTau || failed)) {
                     if (*(volatile int*)&sm->abort_flag) { failed = true; break; }
                     // ---- slow path: exact per-query maxima of this tile, new reference, rescale what was accumulated
@@ -501,7 +563,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                         tc_wait_st();
                     }
                     dmax = -INFINITY;
-                    if (full_tile) make_probs(std::false_type{}); else make_probs(std::true_type{});
+                    sweep();
                 }
 
                 // P buffer must no longer be read by the previous tile's MMA; this wait also keeps every thread
@@ -512,17 +574,6 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     if (j < ncg)
                         *reinterpret_cast<uint4*>(p_buf + (size_t)(g0 + j) * 2048 + (size_t)r * 16) =
                             make_uint4(pk[j][0], pk[j][1], pk[j][2], pk[j][3]);
-                // rows of the V tile past the end of the prefix / tree may hold anything: make them zero
-                if (wg == 0 && valid < kTile) {
-                    const uint32_t slot = 2u + sb;
-                    if (!mbar_wait(&sm->slot_full[slot], (gi >> 1) & 1u, abort_flag, hdr, 9)) failed = true;
-                    if (r >= valid && !failed) {
-                        uint4* z0 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + (size_t)r * 128);
-                        uint4* z1 = reinterpret_cast<uint4*>(ring + (size_t)slot * kSlotBytes + kSlabBytes + (size_t)r * 128);
-#pragma unroll
-                        for (int x = 0; x < 8; ++x) { z0[x] = make_uint4(0, 0, 0, 0); z1[x] = make_uint4(0, 0, 0, 0); }
-                    }
-                }
                 // every thread makes its own P^T stores visible to the tensor cores' proxy; then one arrival per warp (384
                 // arrivals on one shared-memory word would queue up behind one another)
                 fence_async_smem();

@@ -29,6 +29,7 @@ struct TileIndex {
     int cum_w[kMaxBatchTc + 1];
     unsigned short kv_tiles[kMaxBatchTc];   // key tiles of one work item of sequence b
     int whole_items;                        // launch small enough to give every block whole work items (see plan_ranges)
+    int scan[kMaxBatchTc / 32][4];          // per-warp totals of plan_ranges' scan
 };
 constexpr int kWholeItemTiles = 8;          // ... which pays while a work item has at most this many key tiles
 
@@ -252,27 +253,31 @@ __device__ __forceinline__ void locate(const TileIndex* ix, const TcParams& p, l
     s.Nq = min(QB, s.Nb * p.G - s.q0);
 }
 
-// Cost of one tile and fixed cost of a work item in units of about 100 cycles, fitted to per-segment timelines of
-// the kernel.  Thread blocks get equal cost, not equal tile counts, so that sequences with deep trees do not make
-// their blocks finish late.
-__device__ __forceinline__ int tile_weight(int Nq) { return 27 + Nq / 19; }
-// Fixed cost of a work item (pipeline fill and drain, first-tile reference, output of Nq columns), carried by its
-// first tile.
-__device__ __forceinline__ int item_weight(int Nq) { return 100 + (Nq * 5) / 8; }
+// Cost of one tile and fixed cost of a work item in units of 30 ns: a least-squares fit of the time thread blocks
+// were busy (device clock stamps, seven workloads with several seeds each) against the tiles, work items and query
+// counts they had been given.  Thread blocks get equal cost, not equal tile counts, so that sequences with deep
+// trees do not make their blocks finish late.  At most 64 per tile and 256 per work item (the launch bound on the
+// 32-bit prefix sums counts on it).
+template <int QB>
+__device__ __forceinline__ int tile_weight(int Nq) { return QB > 128 ? 32 + (Nq * 12) / 64 : 32 + (Nq * 9) / 64; }
+// Fixed cost of a work item (the masked last tiles, the wait for the last product, output of Nq columns, locating
+// the next item), carried by its first tile.
+template <int QB>
+__device__ __forceinline__ int item_weight(int Nq) { return QB > 128 ? 161 + (Nq * 29) / 64 : 120 + (Nq * 41) / 64; }
 template <int QB>
 __device__ __forceinline__ int head_weight(int L, int Nk, int G) {  // cost of one (sequence, head): all query blocks
     const int tkv = kv_tiles_of(L, Nk);
     const int Nb = Nk * G;                                        // stacked queries
     int w = 0;
-    for (int q0 = 0; q0 < Nb; q0 += QB) w += tkv * tile_weight(min(QB, Nb - q0)) + item_weight(min(QB, Nb - q0));
+    for (int q0 = 0; q0 < Nb; q0 += QB) w += tkv * tile_weight<QB>(min(QB, Nb - q0)) + item_weight<QB>(min(QB, Nb - q0));
     return w;
 }
 // cumulative cost of the tiles before the one a Segment points at
 template <int QB>
 __device__ __forceinline__ long long weight_before(const TileIndex* ix, const TcParams& p, const Segment& s) {
     long long w = (long long)p.H * ix->cum_w[s.b] + (long long)s.h * (ix->cum_w[s.b + 1] - ix->cum_w[s.b]);
-    if (s.qb) w += (long long)s.Tkv * tile_weight(QB) + item_weight(QB);
-    return w + (long long)s.lt * tile_weight(s.Nq) + (s.lt > 0 ? item_weight(s.Nq) : 0);
+    if (s.qb) w += (long long)s.Tkv * tile_weight<QB>(QB) + item_weight<QB>(QB);
+    return w + (long long)s.lt * tile_weight<QB>(s.Nq) + (s.lt > 0 ? item_weight<QB>(s.Nq) : 0);
 }
 // Tile t belongs to block floor(weight_before(t) * G / total_w).  First tile of block c: the first tile whose
 // cumulative cost reaches ceil(c * total_w / G).
@@ -296,11 +301,11 @@ __device__ __forceinline__ long long first_tile_of_block(const TileIndex* ix, co
     int r2 = (int)(rem % wh);
     long long t = (long long)p.H * ix->cum_tiles[lo] + (long long)h * tb;
     // inside a work item the tiles start at cost 0, f + w, f + 2w, ... (f = fixed cost on the first tile)
-    const int w0 = tile_weight(min(QB, Nb)), f0 = item_weight(min(QB, Nb));
+    const int w0 = tile_weight<QB>(min(QB, Nb)), f0 = item_weight<QB>(min(QB, Nb));
     if (r2 >= tkv * w0 + f0 && Nb > QB) {              // inside the second query block
         r2 -= tkv * w0 + f0;
         t += tkv;
-        const int w1 = tile_weight(Nb - QB), f1 = item_weight(Nb - QB);
+        const int w1 = tile_weight<QB>(Nb - QB), f1 = item_weight<QB>(Nb - QB);
         return r2 == 0 ? t : t + max(1, (r2 - f1 + w1 - 1) / w1);
     }
     return r2 == 0 ? t : t + max(1, (r2 - f0 + w0 - 1) / w0);
@@ -316,36 +321,53 @@ __device__ __forceinline__ int block_of_tile(const TileIndex* ix, const TcParams
 // ends of this block's range.  Ends with a __syncthreads(); all threads must call it.
 template <int QB>
 __device__ __forceinline__ void plan_ranges(TileIndex* ix, const TcParams& p, int* n_blocks, long long* range) {
-    const int tid = threadIdx.x, nthr = blockDim.x;
-    for (int b = tid; b < p.B; b += nthr) {
-        const int L = min(max(p.seq_lens[b], 0), p.L_max);
-        const int Nb = p.n_active ? min(max(p.n_active[b], 0), p.N) : p.N;
-        ix->cum_tiles[b + 1] = tiles_of<QB>(L, Nb, p.G);
-        ix->cum_w[b + 1] = head_weight<QB>(L, Nb, p.G);
-        ix->kv_tiles[b] = (unsigned short)min(kv_tiles_of(L, Nb), 65535);
+    const int tid = threadIdx.x, lane = tid & 31, wrp = tid >> 5;
+    // thread b < B owns sequence b (B <= 256 <= blockDim.x): its tiles, cost and work items, then an inclusive scan
+    // over the sequences, by warp shuffles and one exchange of the eight warp totals
+    int v_t = 0, v_w = 0, v_i = 0, v_kv = 0;
+    if (tid < kMaxBatchTc) {
+        if (tid < p.B) {
+            const int L = min(max(p.seq_lens[tid], 0), p.L_max);
+            const int Nb = p.n_active ? min(max(p.n_active[tid], 0), p.N) : p.N;
+            v_kv = min(kv_tiles_of(L, Nb), 65535);
+            v_t = tiles_of<QB>(L, Nb, p.G);
+            v_w = head_weight<QB>(L, Nb, p.G);
+            v_i = Nb > 0 ? (Nb * p.G + QB - 1) / QB : 0;          // query blocks of the sequence
+            ix->kv_tiles[tid] = (unsigned short)v_kv;
+        }
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int a = __shfl_up_sync(0xffffffffu, v_t, o), c = __shfl_up_sync(0xffffffffu, v_w, o),
+                      d = __shfl_up_sync(0xffffffffu, v_i, o);
+            if (lane >= o) { v_t += a; v_w += c; v_i += d; }
+        }
+        v_kv = __reduce_max_sync(0xffffffffu, v_kv);
+        if (lane == 31) { ix->scan[wrp][0] = v_t; ix->scan[wrp][1] = v_w; ix->scan[wrp][2] = v_i; ix->scan[wrp][3] = v_kv; }
     }
     __syncthreads();
-    if (tid == 0) {
-        int acc = 0, accw = 0, items = 0, longest = 0;
-        ix->cum_tiles[0] = 0;
-        ix->cum_w[0] = 0;
-        for (int b = 1; b <= p.B; ++b) {
-            const int kv = ix->kv_tiles[b - 1];
-            if (kv > 0) items += ix->cum_tiles[b] / kv;           // query blocks of the sequence
-            longest = max(longest, kv);
-            acc += ix->cum_tiles[b]; ix->cum_tiles[b] = acc;
-            accw += ix->cum_w[b]; ix->cum_w[b] = accw;
+    if (tid < kMaxBatchTc) {
+        int items = 0, longest = 0;
+        for (int x = 0; x < kMaxBatchTc / 32; ++x) {
+            if (x < wrp) { v_t += ix->scan[x][0]; v_w += ix->scan[x][1]; }
+            items += ix->scan[x][2];
+            longest = max(longest, ix->scan[x][3]);
         }
-        // Few short work items (one sequence with a short prefix, say): a block's fixed costs outweigh its tiles, and
-        // cutting items into pieces would add a partial and a merge to each.  Every block then takes whole items.
-        const long long n_items = (long long)p.H * items;
-        ix->whole_items = (n_items > 0 && n_items <= (long long)gridDim.x && longest <= kWholeItemTiles) ? 1 : 0;
-        // Otherwise no block's share of the cost may be smaller than the heaviest tile, so that consecutive tiles never
-        // skip a block: every working block then owns at least one tile and the blocks sharing a work item are
-        // consecutive.
-        const long long tot_w = (long long)p.H * accw;
-        *n_blocks = ix->whole_items ? (int)n_items
-                                    : (int)max(1LL, min((long long)gridDim.x, tot_w / (tile_weight(QB) + item_weight(QB))));
+        if (tid < p.B) { ix->cum_tiles[tid + 1] = v_t; ix->cum_w[tid + 1] = v_w; }
+        if (tid == max(p.B, 1) - 1) {
+            ix->cum_tiles[0] = 0;
+            ix->cum_w[0] = 0;
+            // Few short work items (one sequence with a short prefix, say): a block's fixed costs outweigh its tiles,
+            // and cutting items into pieces would add a partial and a merge to each.  Every block then takes whole
+            // items.
+            const long long n_items = (long long)p.H * items;
+            ix->whole_items = (n_items > 0 && n_items <= (long long)gridDim.x && longest <= kWholeItemTiles) ? 1 : 0;
+            // Otherwise no block's share of the cost may be smaller than the heaviest tile, so that consecutive tiles
+            // never skip a block: every working block then owns at least one tile and the blocks sharing a work item
+            // are consecutive.
+            const long long tot_w = (long long)p.H * v_w;
+            *n_blocks = ix->whole_items ? (int)n_items
+                                        : (int)max(1LL, min((long long)gridDim.x, tot_w / (tile_weight<QB>(QB) + item_weight<QB>(QB))));
+        }
     }
     __syncthreads();
     if (tid == 0 || tid == 32) {               // the two ends of this block's range, side by side
