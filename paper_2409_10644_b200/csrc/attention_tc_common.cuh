@@ -253,17 +253,18 @@ __device__ __forceinline__ void locate(const TileIndex* ix, const TcParams& p, l
     s.Nq = min(QB, s.Nb * p.G - s.q0);
 }
 
-// Cost of one tile and fixed cost of a work item in units of 30 ns: a least-squares fit of the time thread blocks
-// were busy (device clock stamps, seven workloads with several seeds each) against the tiles, work items and query
-// counts they had been given.  Thread blocks get equal cost, not equal tile counts, so that sequences with deep
-// trees do not make their blocks finish late.  At most 64 per tile and 256 per work item (the launch bound on the
-// 32-bit prefix sums counts on it).
+// Cost of one tile and fixed cost of a work item in units of 32 ns: a least-squares fit of the time thread blocks
+// were busy (device clock stamps, the wide workloads with several seeds each) against the tiles, work items and
+// query counts they had been given.  Thread blocks get equal cost, not equal tile counts, so that sequences with
+// deep trees do not make their blocks finish late.  At most 64 per tile and 256 per work item (the launch bound on
+// the 32-bit prefix sums counts on it).
 template <int QB>
-__device__ __forceinline__ int tile_weight(int Nq) { return QB > 128 ? 32 + (Nq * 12) / 64 : 32 + (Nq * 9) / 64; }
-// Fixed cost of a work item (the masked last tiles, the wait for the last product, output of Nq columns, locating
-// the next item), carried by its first tile.
+__device__ __forceinline__ int tile_weight(int Nq) { return (QB > 128 ? 34 : 29) + (Nq * 83 + (Nq * Nq * 35) / 64) / 1024; }
+// Fixed cost of a work item (the wait for the last product, normalisation and output of Nq columns, locating the
+// next item).  The fit puts it at the item's end, so the item's last tile carries it: a block that takes only the
+// first tiles of an item does not pay it.
 template <int QB>
-__device__ __forceinline__ int item_weight(int Nq) { return QB > 128 ? 161 + (Nq * 29) / 64 : 120 + (Nq * 41) / 64; }
+__device__ __forceinline__ int item_weight(int Nq) { return QB > 128 ? 119 + (Nq * 130) / 256 : 109 + (Nq * 47) / 256; }
 template <int QB>
 __device__ __forceinline__ int head_weight(int L, int Nk, int G) {  // cost of one (sequence, head): all query blocks
     const int tkv = kv_tiles_of(L, Nk);
@@ -277,7 +278,7 @@ template <int QB>
 __device__ __forceinline__ long long weight_before(const TileIndex* ix, const TcParams& p, const Segment& s) {
     long long w = (long long)p.H * ix->cum_w[s.b] + (long long)s.h * (ix->cum_w[s.b + 1] - ix->cum_w[s.b]);
     if (s.qb) w += (long long)s.Tkv * tile_weight<QB>(QB) + item_weight<QB>(QB);
-    return w + (long long)s.lt * tile_weight<QB>(s.Nq) + (s.lt > 0 ? item_weight<QB>(s.Nq) : 0);
+    return w + (long long)s.lt * tile_weight<QB>(s.Nq);
 }
 // Tile t belongs to block floor(weight_before(t) * G / total_w).  First tile of block c: the first tile whose
 // cumulative cost reaches ceil(c * total_w / G).
@@ -300,15 +301,16 @@ __device__ __forceinline__ long long first_tile_of_block(const TileIndex* ix, co
     const int h = (int)(rem / wh);
     int r2 = (int)(rem % wh);
     long long t = (long long)p.H * ix->cum_tiles[lo] + (long long)h * tb;
-    // inside a work item the tiles start at cost 0, f + w, f + 2w, ... (f = fixed cost on the first tile)
-    const int w0 = tile_weight<QB>(min(QB, Nb)), f0 = item_weight<QB>(min(QB, Nb));
-    if (r2 >= tkv * w0 + f0 && Nb > QB) {              // inside the second query block
-        r2 -= tkv * w0 + f0;
+    // inside a work item tile k starts at cost k * w; the last tile also carries the fixed cost, so a cost beyond the
+    // start of the last tile is reached only by the first tile of what follows
+    int w = tile_weight<QB>(min(QB, Nb));
+    const int item0 = tkv * w + item_weight<QB>(min(QB, Nb));
+    if (Nb > QB && r2 >= item0) {                      // inside the second query block
+        r2 -= item0;
         t += tkv;
-        const int w1 = tile_weight<QB>(Nb - QB), f1 = item_weight<QB>(Nb - QB);
-        return r2 == 0 ? t : t + max(1, (r2 - f1 + w1 - 1) / w1);
+        w = tile_weight<QB>(Nb - QB);
     }
-    return r2 == 0 ? t : t + max(1, (r2 - f0 + w0 - 1) / w0);
+    return t + min(tkv, (r2 + w - 1) / w);
 }
 template <int QB>
 __device__ __forceinline__ int block_of_tile(const TileIndex* ix, const TcParams& p, long long t, int G, long long total_w) {
