@@ -377,11 +377,13 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         long long t = t_begin;
         uint32_t g = 0;
         bool failed = false;
+        bool ticket_owed = false;                      // the block's first segment continues another block's work item
         while (t < t_end) {
             Segment s;
             locate<QB>(ix, p, t, s);
             const int cnt = (int)min((long long)(s.Tkv - s.lt), t_end - t);
             const int bh = s.b * p.H + s.h;
+            if (t == t_begin) ticket_owed = s.lt > 0;
             // the groups split the segment's 8-column groups as evenly as possible
             const int ng8 = (s.Nq + 7) >> 3;
             const int base = ng8 / kGroups, rem = ng8 % kGroups;
@@ -664,15 +666,18 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             }
             tc_fence_before();
             if (!full) {
-                // the partial is complete: make it visible, then take the ticket the merging block waits for
-                __threadfence();
-                group_sync_any(bar_id, false);
-                if (r == 0) atomicAdd(p.counters + ((size_t)bh * 2 + s.qb) * 4 + wg, 1);
+                // The partial is complete.  Making it visible device-wide takes a microsecond or two under load, so
+                // the fence and the ticket the merging block waits for are left to the last service warp: the
+                // arrival orders this thread's stores before that warp's fence.
+                asm volatile("bar.arrive %0, %1;" ::"n"(kGroups + 4), "n"(128 * kGroups + 32) : "memory");
+                ticket_owed = false;
             }
             group_sync_any(bar_id, false);
             g += (uint32_t)cnt;
             t += cnt;
         }
+        // gave up before the partial was written: the service warp must not wait for this thread
+        if (ticket_owed) asm volatile("bar.arrive %0, %1;" ::"n"(kGroups + 4), "n"(128 * kGroups + 32) : "memory");
     }
 
     // =========================================================== merge of a split work item (service warps)
@@ -716,6 +721,18 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 sm->merge_item = sp;
             }
             __syncwarp();
+        }
+        if (warp == kMmaWarp + 2) {
+            // ticket of a partial: if this block's first segment continues a work item, the softmax warps arrive here
+            // once its partial is written; this warp makes it visible and takes one ticket per softmax group
+            Segment sf;
+            locate<QB>(ix, p, t_begin, sf);
+            if (sf.lt > 0) {
+                asm volatile("bar.sync %0, %1;" ::"n"(kGroups + 4), "n"(128 * kGroups + 32) : "memory");
+                __threadfence();
+                if (lane < kGroups && !*(volatile int*)abort_flag)
+                    atomicAdd(p.counters + ((size_t)(sf.b * p.H + sf.h) * 2 + sf.qb) * 4 + lane, 1);
+            }
         }
         // the service warps without a loop of their own park on a hardware barrier until the producer and the MMA
         // warp are done (a spinning wait would take issue slots from the softmax warps for the whole kernel)

@@ -30,6 +30,8 @@ struct TileIndex {
     unsigned short kv_tiles[kMaxBatchTc];   // key tiles of one work item of sequence b
     int whole_items;                        // launch small enough to give every block whole work items (see plan_ranges)
     int scan[kMaxBatchTc / 32][4];          // per-warp totals of plan_ranges' scan
+    int len[kMaxBatchTc];                   // clamped prefix length of sequence b
+    unsigned short nodes[kMaxBatchTc];      // clamped active tree nodes of sequence b
 };
 constexpr int kWholeItemTiles = 8;          // ... which pays while a work item has at most this many key tiles
 
@@ -239,16 +241,28 @@ __device__ __forceinline__ void locate(const TileIndex* ix, const TcParams& p, l
         if ((long long)p.H * ix->cum_tiles[mid] <= t) lo = mid; else hi = mid;
     }
     s.b = lo;
-    s.L = min(max(p.seq_lens[lo], 0), p.L_max);
-    s.Nb = p.n_active ? min(max(p.n_active[lo], 0), p.N) : p.N;
+    s.L = ix->len[lo];
+    s.Nb = ix->nodes[lo];
     s.Tb = ix->cum_tiles[lo + 1] - ix->cum_tiles[lo];
     s.nP = (s.L + kTile - 1) / kTile;
     const long long r = t - (long long)p.H * ix->cum_tiles[lo];
-    s.h = (int)(r / s.Tb);
-    const int rem = (int)(r % s.Tb);
+    int rem;
+    if ((unsigned long long)r >> 32) {                 // 64-bit division only where it is needed
+        s.h = (int)(r / s.Tb);
+        rem = (int)(r % s.Tb);
+    } else {
+        const uint32_t r32 = (uint32_t)r, h32 = r32 / (uint32_t)s.Tb;
+        s.h = (int)h32;
+        rem = (int)(r32 - h32 * (uint32_t)s.Tb);
+    }
     s.Tkv = kv_tiles_of(s.L, s.Nb);
-    s.qb = rem / s.Tkv;
-    s.lt = rem % s.Tkv;
+    if (s.Tb == s.Tkv) {                               // one query block
+        s.qb = 0;
+        s.lt = rem;
+    } else {
+        s.qb = rem / s.Tkv;
+        s.lt = rem - s.qb * s.Tkv;
+    }
     s.q0 = s.qb * QB;
     s.Nq = min(QB, s.Nb * p.G - s.q0);
 }
@@ -336,6 +350,8 @@ __device__ __forceinline__ void plan_ranges(TileIndex* ix, const TcParams& p, in
             v_w = head_weight<QB>(L, Nb, p.G);
             v_i = Nb > 0 ? (Nb * p.G + QB - 1) / QB : 0;          // query blocks of the sequence
             ix->kv_tiles[tid] = (unsigned short)v_kv;
+            ix->len[tid] = L;
+            ix->nodes[tid] = (unsigned short)Nb;
         }
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
