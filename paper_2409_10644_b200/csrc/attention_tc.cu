@@ -76,6 +76,8 @@ struct TcSmall {
 static_assert(sizeof(TcSmall) <= kSmemLimit - 1024 - kSlots * 32768 - 160 * 512, "TcSmall grew: four ring slots no longer fit");
 
 // 64 bits of a 192-bit row starting at bit `start` (bits past the row read as zero)
+// rows of a key/value tile that are fetched when `valid` of them are in use: all 128, or a box of 64
+__device__ __forceinline__ int loaded_rows(int valid) { return valid > 64 ? kTile : 64; }
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
     uint32_t d;
     asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
@@ -97,7 +99,9 @@ template <int NCH>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kc,
                               const __grid_constant__ CUtensorMap tm_vc, const __grid_constant__ CUtensorMap tm_kt,
-                              const __grid_constant__ CUtensorMap tm_vt, const TcParams p) {
+                              const __grid_constant__ CUtensorMap tm_vt, const __grid_constant__ CUtensorMap tm_kc64,
+                              const __grid_constant__ CUtensorMap tm_vc64, const __grid_constant__ CUtensorMap tm_kt64,
+                              const __grid_constant__ CUtensorMap tm_vt64, const TcParams p) {
     static_assert(NCH == 3 || NCH == 4 || NCH == 7 || NCH == 8 || NCH == 10, "padded query columns: 48, 64, 112, 128 or 160");
     constexpr int QB = NCH == 10 ? kMaxQ : 128;    // queries per work item
     constexpr int CPT = (2 * NCH + kGroups - 1) / kGroups; // 8-column groups per thread, at most
@@ -113,6 +117,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     const int cta = blockIdx.x;
 
     // ---- set-up
+    // The value slots start out finite: rows of a slot that a partial fetch leaves alone are multiplied by zero
+    // probabilities, and 0 * NaN would be NaN.
+    for (int i = tid; i < 2 * kSlotBytes / 16; i += kTcThreads)
+        reinterpret_cast<uint4*>(ring + 2 * (size_t)kSlotBytes)[i] = make_uint4(0, 0, 0, 0);
+    fence_async_smem();                          // ordered before the bulk copies that will write the slots
     if (tid < 256) {
         sm->ones[tid] = __float2bfloat16_rn(1.0f);
         fence_async_smem();                      // read by the tensor cores through the async proxy
@@ -177,9 +186,17 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 const bool tree = lti >= c.s.nP;
                 const int row0 = (tree ? lti - c.s.nP : lti) * kTile;
                 const int bh_kv = c.s.b * p.Hkv + (c.s.h * p.G) / p.group;
-                const CUtensorMap* map = values ? (tree ? &tm_vt : &tm_vc) : (tree ? &tm_kt : &tm_kc);
                 const uint32_t dst = smem_u32(ring) + slot * (uint32_t)kSlotBytes;
-                mbar_expect_tx(&sm->slot_full[slot], (uint32_t)kSlotBytes);
+                // A tile with at most 64 rows in use (the ragged end of a prefix, a small tree) is fetched as a box of
+                // 64 rows, so that fewer rows travel for nothing.  (Smaller boxes do not pay: a copy instruction has a
+                // fixed cost in the copy unit, and a tile cut into 32-row boxes streams at half the rate.)  The rows
+                // of the slot that are not fetched keep what an earlier tile left there: dead key rows are ignored,
+                // value rows are finite (see the set-up).
+                const int valid = min(kTile, (tree ? c.s.Nb : c.s.L) - row0);
+                const bool half = loaded_rows(valid) < kTile;
+                const CUtensorMap* map = half ? (values ? (tree ? &tm_vt64 : &tm_vc64) : (tree ? &tm_kt64 : &tm_kc64))
+                                              : (values ? (tree ? &tm_vt : &tm_vc) : (tree ? &tm_kt : &tm_kc));
+                mbar_expect_tx(&sm->slot_full[slot], half ? (uint32_t)kSlotBytes / 2u : (uint32_t)kSlotBytes);
                 if (stream_once) {
                     tma_load_3d_hint(dst, map, &sm->slot_full[slot], 0, row0, bh_kv, pol);
                     tma_load_3d_hint(dst + kSlabBytes, map, &sm->slot_full[slot], 64, row0, bh_kv, pol);
@@ -292,7 +309,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                             const bool tree_v = ltv >= s.nP;
                             const int row0_v = (tree_v ? ltv - s.nP : ltv) * kTile;
                             const int valid_v = min(kTile, (tree_v ? s.Nb : s.L) - row0_v);
-                            const int have_v = min(kTile, (tree_v ? p.N : p.L_max) - row0_v);
+                            // rows that were fetched and exist in the tensor
+                            const int have_v = min(loaded_rows(valid_v), (tree_v ? p.N : p.L_max) - row0_v);
                             if (valid_v < have_v) {
                                 unsigned char* v0 = ring + (size_t)(2u + vb) * kSlotBytes;
                                 for (int c = valid_v * 8 + lane; c < have_v * 8; c += 32) {
@@ -999,7 +1017,8 @@ static int launch_tc(const TcLaunch& l, cudaStream_t stream) {
         if (dev >= 0 && dev < 64) done[dev] = true;
     }
     const size_t smem_bytes = 1024 + (size_t)kSlots * kSlotBytes + (size_t)l.p.npadq * 512 + sizeof(TcSmall);
-    tree_attention_tc_kernel<NCH><<<l.grid, kTcThreads, smem_bytes, stream>>>(l.maps[0], l.maps[1], l.maps[2], l.maps[3], l.maps[4], l.p);
+    tree_attention_tc_kernel<NCH><<<l.grid, kTcThreads, smem_bytes, stream>>>(l.maps[0], l.maps[1], l.maps[2], l.maps[3], l.maps[4], l.maps[5], l.maps[6],
+                                                                              l.maps[7], l.maps[8], l.p);
     MCSD_CUDA_CHECK(cudaGetLastError());
     return MCSD_OK;
 }
@@ -1020,6 +1039,11 @@ int tree_attention_tc(const AttentionArgs& a, WorkspaceHeader* header, void* scr
     ok = ok && make_map(&l.maps[2], have_cache ? a.v_cache : a.v_tree, have_cache ? a.L_max : a.N, bh_kv, kTile);
     ok = ok && make_map(&l.maps[3], a.k_tree, a.N, bh_kv, kTile);
     ok = ok && make_map(&l.maps[4], a.v_tree, a.N, bh_kv, kTile);
+    // the same tensors in boxes of 64 rows, for tiles with few rows in use
+    ok = ok && make_map(&l.maps[5], have_cache ? a.k_cache : a.k_tree, have_cache ? a.L_max : a.N, bh_kv, kTile / 2);
+    ok = ok && make_map(&l.maps[6], have_cache ? a.v_cache : a.v_tree, have_cache ? a.L_max : a.N, bh_kv, kTile / 2);
+    ok = ok && make_map(&l.maps[7], a.k_tree, a.N, bh_kv, kTile / 2);
+    ok = ok && make_map(&l.maps[8], a.v_tree, a.N, bh_kv, kTile / 2);
     if (!ok) { set_last_cuda_error(cudaErrorInvalidValue); return MCSD_ERR_CUDA; }
 
     int dev = 0, sms = 0;

@@ -413,7 +413,7 @@ __device__ __forceinline__ void plan_ranges(TileIndex* ix, const TcParams& p, in
 }
 
 struct TcLaunch {
-    CUtensorMap maps[5];     // Q, key cache, value cache, tree keys, tree values
+    CUtensorMap maps[9];     // Q, key cache, value cache, tree keys, tree values; the last four again in boxes of 64 rows
     TcParams p;
     int grid;
 };
