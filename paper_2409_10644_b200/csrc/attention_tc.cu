@@ -117,6 +117,10 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     const int cta = blockIdx.x;
 
     // ---- set-up
+    // Programmatic dependent launch: a launch that follows this one in the stream may start its blocks as soon as
+    // this grid's blocks leave their multiprocessors, and this grid may have been started that way itself.  What
+    // comes before the wait below touches no global memory, so it overlaps the tail of the preceding kernel.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // The value slots start out finite: rows of a slot that a partial fetch leaves alone are multiplied by zero
     // probabilities, and 0 * NaN would be NaN.
     for (int i = tid; i < 2 * kSlotBytes / 16; i += kTcThreads)
@@ -139,6 +143,8 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    // everything the preceding kernel in the stream wrote is visible from here on
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     plan_ranges<QB>(&sm->ix, p, &sm->n_blocks, sm->range);
     const long long total = (long long)p.H * ix->cum_tiles[p.B];
     const long long total_w = (long long)p.H * ix->cum_w[p.B];
@@ -1017,9 +1023,18 @@ static int launch_tc(const TcLaunch& l, cudaStream_t stream) {
         if (dev >= 0 && dev < 64) done[dev] = true;
     }
     const size_t smem_bytes = 1024 + (size_t)kSlots * kSlotBytes + (size_t)l.p.npadq * 512 + sizeof(TcSmall);
-    tree_attention_tc_kernel<NCH><<<l.grid, kTcThreads, smem_bytes, stream>>>(l.maps[0], l.maps[1], l.maps[2], l.maps[3], l.maps[4], l.maps[5], l.maps[6],
-                                                                              l.maps[7], l.maps[8], l.p);
-    MCSD_CUDA_CHECK(cudaGetLastError());
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)l.grid);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see the kernel's set-up
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    MCSD_CUDA_CHECK(cudaLaunchKernelEx(&cfg, tree_attention_tc_kernel<NCH>, l.maps[0], l.maps[1], l.maps[2], l.maps[3], l.maps[4],
+                                       l.maps[5], l.maps[6], l.maps[7], l.maps[8], l.p));
     return MCSD_OK;
 }
 
