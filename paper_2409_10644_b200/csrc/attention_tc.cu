@@ -60,7 +60,9 @@ struct TcSmall {
     unsigned long long pv_done[2];           // products of even / odd tiles finished: value slot and P^T free, O^T and l current
     unsigned long long p_full, q_full, drain;
     unsigned long long merge_bar;            // a staged copy of another block's partial has landed
+    unsigned long long s_last;               // the block's last S^T has finished: key slots and Q buffer are free
     int merge_np1;                           // pieces of later blocks to fold into this block's last segment (0: none)
+    int merge_prefetched;                    // the first of those pieces is already on its way into shared memory
     Segment merge_item;                      // that segment's work item
     uint32_t tmem_base;
     int abort_flag;
@@ -140,6 +142,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         mbar_init(&sm->q_full, 1);
         mbar_init(&sm->drain, 1);
         mbar_init(&sm->merge_bar, 1);
+        mbar_init(&sm->s_last, 1);
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -300,6 +303,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                                          dq0 + ((k >> 2) * q_slab + (uint32_t)(k & 3) * 2u), idesc_s, k > 0);
                         }
                         tc_commit_elect(&sm->s_full[sb]);
+                        if (t + i + 1 == t_end) tc_commit_elect(&sm->s_last);
                     }
                     if (i >= 1) {
                         const uint32_t gj = g + (uint32_t)(i - 1), vb = gj & 1u;
@@ -704,18 +708,16 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
         if (ticket_owed) asm volatile("bar.arrive %0, %1;" ::"n"(kGroups + 4), "n"(128 * kGroups + 32) : "memory");
     }
 
-    // =========================================================== merge of a split work item (service warps)
-    // If this block's last segment starts a work item that continues in later blocks, its four service warps (done
-    // with loading and issuing by then; together they reach all 128 lanes of tensor memory) fold the other pieces,
-    // which those blocks produced as the first thing they did, into this block's own piece, still in tensor memory:
+    // =========================================================== merge of a split work item
+    // If this block's last segment starts a work item that continues in later blocks, the block folds the other
+    // pieces, which those blocks produced as the first thing they did, into its own piece, still in tensor memory:
     //     m = max(m_a, m_b),  l = l_a 2^(m_a - m) + l_b 2^(m_b - m),  O = O_a 2^(m_a - m) + O_b 2^(m_b - m),  o = O / l.
     // Thread r holds head dim r of every query.  Under a saturated memory system a dependent trip to the workspace
     // costs 1.5-2 us, so there is one per piece: the piece's rows and its (m, l) are brought into the (now idle)
     // key/value ring with two bulk copies.  The tickets that say the pieces are complete are polled, at leisure, by
-    // a warp that has nothing else to do, long before they are needed.  The code lives in this branch, away from the
-    // softmax warps' tile loop, so that its registers are its own.
+    // a warp that has nothing else to do, long before they are needed.  The code lives after the roles' branches,
+    // away from the softmax warps' tile loop, so that its registers are its own.
     if (warp >= kProducerWarp) {
-        const int r = tid - 32 * kProducerWarp;                  // 0..127 = tensor-memory lane = head dim
         if (warp == kMmaWarp + 1) {
             if (lane == 0) {
                 Segment sp;
@@ -741,6 +743,22 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     }
                     __threadfence();                              // acquire: the pieces' partials are visible
                 }
+                // The first piece is fetched as soon as there is room: once the block's last S^T has finished, the
+                // two key slots (64 KB) and the Q buffer are free, one and a half tiles before the block is done.
+                int prefetched = 0;
+                const uint32_t o_bytes = (uint32_t)((sp.Nq + 7) >> 3) * 4096u;
+                if (np1 > 0 && o_bytes <= 2u * kSlotBytes && !*(volatile int*)abort_flag &&
+                    mbar_wait(&sm->s_last, 0, abort_flag, hdr, 15)) {
+                    const size_t slot = (size_t)(2 * (cta + 1));
+                    asm volatile("fence.proxy.async;" ::: "memory");
+                    mbar_expect_tx(&sm->merge_bar, o_bytes + 2u * kMaxQ * 4u);
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(smem_u32(ring)), "l"(p.part_o + slot * kMaxQ * 128), "r"(o_bytes), "r"(smem_u32(&sm->merge_bar)) : "memory");
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(smem_u32(q_buf)), "l"(p.part_ml + slot * 2 * kMaxQ), "r"(2u * kMaxQ * 4u), "r"(smem_u32(&sm->merge_bar)) : "memory");
+                    prefetched = 1;
+                }
+                sm->merge_prefetched = prefetched;
                 sm->merge_np1 = np1;
                 sm->merge_item = sp;
             }
@@ -758,13 +776,19 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     atomicAdd(p.counters + ((size_t)(sf.b * p.H + sf.h) * 2 + sf.qb) * 4 + lane, 1);
             }
         }
-        // the service warps without a loop of their own park on a hardware barrier until the producer and the MMA
-        // warp are done (a spinning wait would take issue slots from the softmax warps for the whole kernel)
-        asm volatile("bar.sync %0, 128;" ::"n"(kGroups + 3) : "memory");
+    }
+    // Every role is done with its loop (a hardware barrier: the warps that get here early sleep instead of taking issue
+    // slots from the softmax warps).  The merge itself is shared by all sixteen warps: warp w reaches tensor-memory
+    // lanes 32 (w % 4) .., i.e. head dims, and takes every fourth 8-column group, starting with group w / 4.
+    tc_fence_before();
+    __syncthreads();
+    {
         const int np1 = sm->merge_np1;
         if (np1 > 0) {
+            const int r = 32 * (warp & 3) + lane;                // tensor-memory lane = head dim
+            const int part = warp >> 2;                          // 0..3: which column groups
             const Segment sp = sm->merge_item;
-            const uint32_t lane_addr = (uint32_t)((r >> 5) * 32) << 16;
+            const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
             const int bh = sp.b * p.H + sp.h;
             float* const l_run = &sm->wred[0][0][0];             // [160] running normaliser, at the end 1 / l
             float* const m_run = l_run + kMaxQ;                  // [160] running reference
@@ -772,7 +796,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             float* const w_b = w_a + kMaxQ;                      // [160] weight of the piece being added
             static_assert(4 * kMaxQ <= kGroups * 4 * 64, "the merge scratch must fit the per-warp reduction scratch");
             const float* stage_o = reinterpret_cast<const float*>(ring);                     // [<= 160][128]
-            const float* stage_ml = reinterpret_cast<const float*>(ring + kMaxQ * 512);      // [2][160]
+            const float* stage_ml = reinterpret_cast<const float*>(q_buf);                   // [2][160]
             // column -> (softmax group, index within the group), as the softmax warps split this segment
             const int ng8 = (sp.Nq + 7) >> 3, base = ng8 / kGroups, rem = ng8 % kGroups;
             auto group_of = [&](int q, int& rel) {
@@ -783,14 +807,12 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 rel = q - 8 * (gidx * base + min(gidx, rem));
                 return gidx;
             };
-            // All of this block's tensor-core work must have finished: the barrier that completes exactly once, after
-            // the MMA warp's last commit (a parity wait on a barrier that is reused per tile could pass on an earlier
-            // phase).
-            bool ok = mbar_wait(&sm->drain, 0, abort_flag, hdr, 10);
+            // All of this block's tensor-core work has finished (the MMA warp waited for its last commit before the
+            // barrier above).
             tc_fence_after();
             // this block's own row sums and references: lane q of the first set of row-sum columns holds query q, lane
             // q - 128 of the second set query q; the copy kept current is number (group of q)
-            {
+            if (part == 3) {
                 float c1[4], c2[4];
                 tc_ld4(tmem + lane_addr + kColL, c1);
                 tc_ld4(tmem + lane_addr + kColL2, c2);
@@ -799,11 +821,11 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                 if (r < sp.Nq) { const int gq = group_of(r, rel); l_run[r] = gq == 0 ? c1[0] : gq == 1 ? c1[1] : c1[2]; m_run[r] = sm->m_ref[gq][rel]; }
                 if (128 + r < sp.Nq) { const int gq = group_of(128 + r, rel); l_run[128 + r] = gq == 0 ? c2[0] : gq == 1 ? c2[1] : c2[2]; m_run[128 + r] = sm->m_ref[gq][rel]; }
             }
-            ok = ok && !*(volatile int*)abort_flag;
-            for (int i = 1; i <= np1 && ok; ++i) {
+            for (int i = 1; i <= np1; ++i) {
                 const size_t slot = (size_t)(2 * (cta + i));       // the piece is that block's first segment
-                asm volatile("bar.sync %0, 128;" ::"n"(kGroups + 2) : "memory");    // staging area and weights are free
-                if (r == 0) {
+                // staging area and weights are free, l_run and m_run written; all threads agree on giving up
+                if (!__syncthreads_and(!*(volatile int*)abort_flag)) break;
+                if (tid == 0 && !(i == 1 && sm->merge_prefetched)) {
                     const uint32_t o_bytes = (uint32_t)ng8 * 4096u, ml_bytes = 2u * kMaxQ * 4u;
                     asm volatile("fence.proxy.async;" ::: "memory");
                     mbar_expect_tx(&sm->merge_bar, o_bytes + ml_bytes);
@@ -812,9 +834,10 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                                  ::"r"(smem_u32(stage_ml)), "l"(p.part_ml + slot * 2 * kMaxQ), "r"(ml_bytes), "r"(smem_u32(&sm->merge_bar)) : "memory");
                 }
-                ok = mbar_wait(&sm->merge_bar, (uint32_t)(i - 1) & 1u, abort_flag, hdr, 13);
+                const bool ok = mbar_wait(&sm->merge_bar, (uint32_t)(i - 1) & 1u, abort_flag, hdr, 13);
                 const bool last = i == np1;
-                for (int q = r; q < sp.Nq; q += 128) {
+                if (tid < sp.Nq) {
+                    const int q = tid;
                     const float ma = m_run[q], mb = stage_ml[q], lb = stage_ml[kMaxQ + q];
                     const float mn = fmaxf(ma, mb);
                     const float wa = (mn == -INFINITY || ma == -INFINITY) ? 0.f : exp2f(ma - mn);
@@ -825,36 +848,29 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     w_b[q] = wb;
                     l_run[q] = last ? (ln > 0.f ? 1.f / ln : 0.f) : ln;
                 }
-                asm volatile("bar.sync %0, 128;" ::"n"(kGroups + 2) : "memory");
+                if (!__syncthreads_and(ok)) break;
 #pragma unroll 1
-                for (int j0 = 0; j0 < ng8; j0 += 4) {                               // four column groups at a time
-                    float acc[4][8];
-#pragma unroll
-                    for (int jj = 0; jj < 4; ++jj)
-                        if (j0 + jj < ng8) tc_ld8(tmem + lane_addr + kColO + 8 * (j0 + jj), acc[jj]);
+                for (int j = part; j < ng8; j += 4) {
+                    float acc[8];
+                    tc_ld8(tmem + lane_addr + kColO + 8 * j, acc);
                     tc_wait_ld();
 #pragma unroll
-                    for (int jj = 0; jj < 4; ++jj) {
-                        if (j0 + jj < ng8) {
+                    for (int k = 0; k < 8; ++k) {
+                        const int q = 8 * j + k;
+                        acc[k] = fmaf(stage_o[(size_t)q * 128 + r], w_b[q], acc[k] * w_a[q]);
+                    }
+                    if (last) {
 #pragma unroll
-                            for (int k = 0; k < 8; ++k) {
-                                const int q = 8 * (j0 + jj) + k;
-                                acc[jj][k] = fmaf(stage_o[(size_t)q * 128 + r], w_b[q], acc[jj][k] * w_a[q]);
-                            }
-                            if (last) {
-#pragma unroll
-                                for (int k = 0; k < 8; ++k) {
-                                    const int q = 8 * (j0 + jj) + k;
-                                    if (q < sp.Nq) {
-                                        const int jq = sp.q0 + q;   // stacked query: head jq % G of the group, node jq / G
-                                        p.out[(((size_t)bh * p.G + (jq & (p.G - 1))) * p.N + (jq >> p.g_shift)) * 128 + r] =
-                                            __float2bfloat16_rn(acc[jj][k] * l_run[q]);
-                                    }
-                                }
-                            } else {
-                                tc_st8(tmem + lane_addr + kColO + 8 * (j0 + jj), acc[jj]);
+                        for (int k = 0; k < 8; ++k) {
+                            const int q = 8 * j + k;
+                            if (q < sp.Nq) {
+                                const int jq = sp.q0 + q;   // stacked query: head jq % G of the group, node jq / G
+                                p.out[(((size_t)bh * p.G + (jq & (p.G - 1))) * p.N + (jq >> p.g_shift)) * 128 + r] =
+                                    __float2bfloat16_rn(acc[k] * l_run[q]);
                             }
                         }
+                    } else {
+                        tc_st8(tmem + lane_addr + kColO + 8 * j, acc);
                     }
                 }
                 if (!last) tc_wait_st();
