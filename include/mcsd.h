@@ -100,7 +100,8 @@ int mcsd_build_mask(const int32_t* parent_host, int n_nodes,
  *   k_cache, v_cache        [dev] [B][H][L_max][D]; only the first seq_lens[b] rows of sequence b are used
  *                           (later rows may hold anything, NaN bit patterns included)
  *   seq_lens                [dev] int32[B], 0 <= seq_lens[b] <= L_max
- *   n_active                [dev] int32[B], 0 <= n_active[b] <= N (a level-order prefix of the tree), or NULL = N
+ *   n_active                [dev] int32[B], 0 <= n_active[b] <= N (a level-order prefix of the tree), or NULL = N;
+ *                           rows n >= n_active[b] of k_tree and v_tree are not used and may hold anything
  *   anc, words              the mask from mcsd_build_mask for the N-node tree
  *   D                       64 or 128;  N <= MCSD_MAX_NODES;  B * H <= 65535
  *   dtype                   MCSD_BF16: bf16 storage, fp32 softmax and accumulation (tensor-core products when

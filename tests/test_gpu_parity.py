@@ -137,10 +137,13 @@ def _full_attention_case(m, w, std=None, rel=False, lens=None, n_act="gamma", pa
     if isinstance(n_act, str):
         _, ls = orc.tree_levels(parent)
         n_act = None if w.gamma is None else np.array([orc.n_active_for_gamma(parent, int(g)) for g in gammas(w)])
-    if poison:                                   # cache rows past the prefix may hold anything
+    if poison:                                   # cache rows past the prefix and tree rows past the active nodes may hold anything
         for b in range(w.B):
             inp["k_cache"][b, :, int(lens[b]):] = float("nan")
             inp["v_cache"][b, :, int(lens[b]):] = float("nan")
+            if n_act is not None:
+                inp["k_tree"][b, :, int(n_act[b]):] = float("nan")
+                inp["v_tree"][b, :, int(n_act[b]):] = float("nan")
     scale = 1.0 / np.sqrt(w.D)
     out = _run_attention(m, w, inp, lens, n_act, parent, scale)
     pairs = _all_pairs(w.B, w.H) if pairs is None else pairs
@@ -186,6 +189,18 @@ def test_attention_edge_cases(m):
     wmax = dataclasses.replace(w, n_roots=8, branching=(1, 2, 2, 1, 1, 1, 1), B=2, prefix=(150, 150))
     assert wmax.n_nodes == 192
     _full_attention_case(m, wmax, std=1.0, rel=True, n_act=None)
+
+
+def test_attention_half_filled_tiles(m):
+    # A tile with at most 64 rows in use is fetched as a 64-row box and the rest of its slot keeps older data: prefix
+    # ends and active-node counts on both sides of that limit, after full tiles and as the only tile, with NaN in
+    # every row that must not be read.  Several heads per sequence, so that slots are reused within a block.
+    w = dataclasses.replace(workload(3), B=8, H=4, prefix=(1, 400))
+    N = w.n_nodes
+    lens = [64, 65, 128 + 63, 128 + 64, 256 + 65, 1, 127, 384]
+    n_act = np.array([N, 64, 65, 1, 63, N, 32, 100], dtype=np.int32)
+    _full_attention_case(m, w, std=1.0, rel=True, lens=lens, n_act=n_act, poison=True)
+    _full_attention_case(m, w, lens=lens[::-1], n_act=n_act, poison=True)
 
 
 def test_attention_query_split_changes_between_segments(m):
