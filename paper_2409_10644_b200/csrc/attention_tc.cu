@@ -27,10 +27,10 @@
 //   * row sums come from the tensor cores (P^T read as an MN-major A operand against a matrix of ones) and are
 //     accumulated in tensor memory across the tiles of a segment like O^T; they are touched by a thread only when
 //     the reference moves and in the epilogue;
-//   * the reference of a segment starts from the scores of the first key of its first full tile instead of an
-//     exact column maximum: any reference that no score exceeds by more than 2^8 gives the same result, and a key
-//     that does exceed it raises the vote like anywhere else.  (Segments that start on a masked tile take the
-//     exact path.)
+//   * the reference of a segment starts from the scores of one key of its first full tile (key 0, 32, 64 or 96,
+//     depending on the column group) instead of an exact column maximum: any reference that no score exceeds by
+//     more than 2^8 gives the same result, and a key that does exceed it raises the vote like anywhere else.
+//     (Segments that start on a ragged or tree tile take the exact path.)
 //   * the MMA warp runs its loop convergently and one elected lane issues; descriptors are built once and advanced
 //     by constants, and there are two commits per tile (S^T done = scores ready and key slot free; products done =
 //     value slot and P^T free), because a tcgen05.mma of these shapes takes 40-60 cycles and the instructions
@@ -38,8 +38,9 @@
 //   * the producer issues loads in the order in which slots come free (K0 K1 V0 K2 V1 ...), about two tiles ahead.
 //
 // Warp roles (512 threads): warps 0-11 softmax / mask / epilogue, warp 12 TMA producer, warp 13 MMA issuer and owner
-// of the tensor-memory allocation, warp 14 polls the tickets of a split last work item, warp 15 idle; at the end of
-// the block warps 12-15 together merge such an item (they reach all 128 lanes of tensor memory).  Every wait is
+// of the tensor-memory allocation, warp 14 polls the tickets of a split last work item and fetches its first
+// partial, warp 15 publishes the partial this block writes; at the end of the block all sixteen warps together
+// merge a split item.  Every wait is
 // bounded; one that runs out raises a flag in the workspace header, all roles drain and the block exits cleanly.
 #include <mutex>
 #include <type_traits>
@@ -505,18 +506,17 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
                     if (MASKED) dmax = max(pmax & 0xFFFFu, pmax >> 16) > 0x4380u ? INFINITY : -INFINITY;
                 };
                 if (i == 0 && full_tile) {
-                    // reference of a new segment: the scores of the tile's first key (see the file header)
-                    if (wq == 0) {
+                    // reference of a new segment: the scores of one key of the tile (see the file header).  The four
+                    // warps of the group share the column groups; warp wq samples key 32 wq, the row its lane 0 holds.
 #pragma unroll
-                        for (int j = 0; j < CPT; ++j) {
-                            if (j < ncg) {
-                                float v[8];
-                                tc_ld8(s_addr + 8 * j, v);
-                                tc_wait_ld();
-                                if (lane == 0) {
+                    for (int j = 0; j < CPT; ++j) {
+                        if (j < ncg && (j & 3) == wq) {
+                            float v[8];
+                            tc_ld8(s_addr + 8 * j, v);
+                            tc_wait_ld();
+                            if (lane == 0) {
 #pragma unroll
-                                    for (int k = 0; k < 8; ++k) mref[8 * j + k] = v[k] * p.scale_log2;
-                                }
+                                for (int k = 0; k < 8; ++k) mref[8 * j + k] = v[k] * p.scale_log2;
                             }
                         }
                     }
