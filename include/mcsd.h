@@ -153,6 +153,33 @@ int mcsd_selftest_bounded_wait(void* workspace, size_t workspace_bytes, int micr
 int mcsd_tree_attention_path(int B, int H_q, int H_kv, int N, int D, int L_max, int dtype);
 
 /*
+ * How the tensor-core kernel would cut a launch among its thread blocks (the paper has no counterpart: Section 2.2
+ * defines the attention, the schedule is this library's).  The key/value tiles of a launch are numbered in the
+ * order (sequence, work unit, query block, 128-key tile; prefix tiles before tree tiles); thread block c processes
+ * tiles first_tile[c] .. first_tile[c + 1] - 1, ranges of about equal estimated cost, or whole work items when the
+ * launch is small.  The kernel evaluates the same functions on the device; this entry point evaluates them on the
+ * host, for inspection and tests.  Host only, no CUDA call; all pointers are host pointers.
+ *
+ *   seq_lens, n_active   [host] int32[B] as for mcsd_tree_attention (n_active may be NULL = N)
+ *   n_blocks             thread blocks of the launch, 1 .. 160 (the kernel uses one per multiprocessor)
+ *   first_tile           [host] int64[n_blocks + 1], written; blocks past the returned count get empty ranges
+ *   info                 [host] int64[4] or NULL, written: tiles in the launch, their total cost in the kernel's
+ *                        units, 1 if blocks take whole work items, queries per work item at most (128 or 160)
+ *   probe_tiles          [host] int64[n_probe] tile numbers to describe (n_probe may be 0)
+ *   probe_out            [host] int64[n_probe][8], written: sequence, work unit within the sequence, query block, tile
+ *                        within the work item, queries of the work item, tiles of the work item, owning block as the
+ *                        merging block computes it (-1 in whole-item mode), cost of the tiles before it;
+ *                        eight times -1 for a tile number outside the launch
+ *
+ * Returns the number of blocks that get work (0 for a launch without keys), MCSD_ERR_BAD_SHAPE for a shape the
+ * tensor-core kernel does not take (see mcsd_tree_attention_path) or a bad n_blocks, MCSD_ERR_NULL, or the status
+ * mcsd_tree_attention_path returns for an invalid shape.
+ */
+int mcsd_tree_attention_plan(int B, int H_q, int H_kv, int N, int D, int L_max, int dtype, const int32_t* seq_lens,
+                             const int32_t* n_active, int n_blocks, int64_t* first_tile, int64_t* info, int n_probe,
+                             const int64_t* probe_tiles, int64_t* probe_out);
+
+/*
  * mcsd_tree_attention for a target with grouped-query attention: q and out have H_q heads, the four key/value
  * tensors H_kv heads, H_q = G * H_kv, and query head h reads key/value head h / G (the paper's targets are
  * multi-head models, G = 1; Section 2.2 defines the attention itself).  Everything else as mcsd_tree_attention.

@@ -7,7 +7,7 @@ missing build raises -- there is no fallback path.
 _BINDING_NAMES = (
     "McsdError", "TreeMask", "lib", "MCSD_BF16", "MCSD_F32", "MCSD_MAX_NODES",
     "mcsd_build_mask", "mcsd_tree_attention", "mcsd_tree_attention_workspace_bytes",
-    "mcsd_verify_tree", "mcsd_verify_tree_logits", "mcsd_sample_roots", "mcsd_verify_tree_static", "mcsd_commit_kv", "layer_pointer_table", "mcsd_verify_tree_workspace_bytes", "mcsd_workspace_status", "verify_node_states", "mcsd_tree_attention_path", "mcsd_selftest_bounded_wait",
+    "mcsd_verify_tree", "mcsd_verify_tree_logits", "mcsd_sample_roots", "mcsd_verify_tree_static", "mcsd_commit_kv", "layer_pointer_table", "mcsd_verify_tree_workspace_bytes", "mcsd_workspace_status", "verify_node_states", "mcsd_tree_attention_path", "mcsd_tree_attention_plan", "mcsd_selftest_bounded_wait",
     "mcsd_status_string", "mcsd_launch_count", "n_active_from_gamma", "shard_batch", "new_workspace",
     "VocabShard", "mcsd_verify_shard_workspace_bytes",
 )

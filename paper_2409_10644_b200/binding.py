@@ -24,7 +24,7 @@ MCSD_MAX_WORDS = 3
 
 _EXPORTS = (
     "mcsd_status_string", "mcsd_last_cuda_error", "mcsd_launch_count", "mcsd_build_mask", "mcsd_tree_attention_workspace_bytes",
-    "mcsd_tree_attention", "mcsd_tree_attention_gqa", "mcsd_workspace_status", "verify_node_states", "mcsd_tree_attention_path", "mcsd_selftest_bounded_wait", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_logits", "mcsd_verify_tree_static", "mcsd_commit_kv", "mcsd_sample_roots",
+    "mcsd_tree_attention", "mcsd_tree_attention_gqa", "mcsd_workspace_status", "verify_node_states", "mcsd_tree_attention_path", "mcsd_tree_attention_plan", "mcsd_selftest_bounded_wait", "mcsd_verify_tree_workspace_bytes", "mcsd_verify_tree", "mcsd_verify_tree_logits", "mcsd_verify_tree_static", "mcsd_commit_kv", "mcsd_sample_roots",
     "mcsd_sample_roots_logits", "mcsd_verify_shard_workspace_bytes", "mcsd_verify_shard_gather", "mcsd_verify_shard_round",
     "mcsd_verify_shard_select", "mcsd_verify_shard_pick",
 )
@@ -52,6 +52,8 @@ def _load() -> ctypes.CDLL:
     lib.mcsd_selftest_bounded_wait.argtypes = [c_void_p, c_size_t, c_int, c_void_p]
     lib.mcsd_tree_attention_path.restype = c_int
     lib.mcsd_tree_attention_path.argtypes = [c_int] * 7
+    lib.mcsd_tree_attention_plan.restype = c_int
+    lib.mcsd_tree_attention_plan.argtypes = [c_int] * 7 + [c_void_p, c_void_p, c_int, c_void_p, c_void_p, c_int, c_void_p, c_void_p]
     lib.mcsd_tree_attention.restype = c_int
     lib.mcsd_tree_attention.argtypes = [c_void_p] * 9 + [c_int] * 6 + [c_float, c_int, c_void_p, c_size_t, c_void_p]
     lib.mcsd_tree_attention_gqa.restype = c_int
@@ -208,6 +210,34 @@ def mcsd_tree_attention_path(B, H_q, H_kv, N, D, L_max, dtype_code) -> int:
     if st < 0:
         _check(st, "mcsd_tree_attention_path")
     return st
+
+
+def mcsd_tree_attention_plan(B, H_q, H_kv, N, D, L_max, dtype_code, seq_lens, n_active=None, n_blocks=148, probe_tiles=()):
+    """How the tensor-core kernel cuts a launch among ``n_blocks`` thread blocks (host only, see mcsd.h).
+
+    ``seq_lens`` / ``n_active``: host int32 arrays.  Returns ``(blocks_used, first_tile[n_blocks + 1], info[4],
+    probe_out[len(probe_tiles)][8])`` as numpy arrays.
+    """
+    import numpy as np
+    lens = np.ascontiguousarray(seq_lens, dtype=np.int32)
+    if lens.shape != (B,):
+        raise ValueError("seq_lens must have B entries")
+    nact = None if n_active is None else np.ascontiguousarray(n_active, dtype=np.int32)
+    if nact is not None and nact.shape != (B,):
+        raise ValueError("n_active must have B entries")
+    if not 1 <= int(n_blocks) <= 160:
+        raise ValueError("n_blocks must be 1..160")
+    probes = np.ascontiguousarray(probe_tiles, dtype=np.int64).reshape(-1)
+    first = np.zeros(int(n_blocks) + 1, dtype=np.int64)
+    info = np.zeros(4, dtype=np.int64)
+    out = np.zeros((len(probes), 8), dtype=np.int64)
+    st = int(lib.mcsd_tree_attention_plan(B, H_q, H_kv, N, D, L_max, dtype_code, lens.ctypes.data,
+                                          None if nact is None else nact.ctypes.data, int(n_blocks), first.ctypes.data,
+                                          info.ctypes.data, len(probes), probes.ctypes.data if len(probes) else None,
+                                          out.ctypes.data if len(probes) else None))
+    if st < 0:
+        _check(st, "mcsd_tree_attention_plan")
+    return st, first, info, out
 
 
 def new_workspace(nbytes: int, device) -> torch.Tensor:

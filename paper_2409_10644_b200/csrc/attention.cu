@@ -71,6 +71,20 @@ extern "C" int mcsd_tree_attention_path(int B, int H_q, int H_kv, int N, int D, 
     return mcsd::tc_shape_supported(B, H_q, H_q / H_kv, N, D, L_max, dtype) ? MCSD_PATH_TENSOR_CORE : MCSD_PATH_CUDA_CORE;
 }
 
+extern "C" int mcsd_tree_attention_plan(int B, int H_q, int H_kv, int N, int D, int L_max, int dtype, const int32_t* seq_lens,
+                                        const int32_t* n_active, int n_blocks, int64_t* first_tile, int64_t* info,
+                                        int n_probe, const int64_t* probe_tiles, int64_t* probe_out) {
+    const int path = mcsd_tree_attention_path(B, H_q, H_kv, N, D, L_max, dtype);
+    if (path < 0) return path;
+    if (path != MCSD_PATH_TENSOR_CORE) return MCSD_ERR_BAD_SHAPE;
+    if (!seq_lens || !first_tile || (n_probe > 0 && (!probe_tiles || !probe_out))) return MCSD_ERR_NULL;
+    if (n_blocks < 1 || n_blocks > mcsd::kTcMaxBlocks || n_probe < 0) return MCSD_ERR_BAD_SHAPE;
+    static_assert(sizeof(long long) == sizeof(int64_t), "64-bit long long");
+    return mcsd::tc_plan_host(B, H_q, H_q / H_kv, N, L_max, seq_lens, n_active, n_blocks, reinterpret_cast<long long*>(first_tile),
+                              reinterpret_cast<long long*>(info), n_probe, reinterpret_cast<const long long*>(probe_tiles),
+                              reinterpret_cast<long long*>(probe_out));
+}
+
 extern "C" int mcsd_tree_attention(const void* q, const void* k_cache, const void* v_cache, const void* k_tree,
                                    const void* v_tree, void* out, const int32_t* seq_lens, const int32_t* n_active,
                                    const uint64_t* anc, int words, int B, int H, int N, int D, int L_max,

@@ -31,6 +31,9 @@ bool tc_shape_supported(int B, int H, int G, int N, int D, int L_max, int dtype)
 bool tc_supported(const AttentionArgs& a);
 size_t tc_workspace_bytes(int B, int H, int N, int D, int L_max);
 int tc_bounded_wait_selftest(WorkspaceHeader* header, long long limit_cycles, int where, cudaStream_t stream);
+int tc_plan_host(int B, int H, int G, int N, int L_max, const int32_t* seq_lens, const int32_t* n_active, int grid,
+                 long long* first_tile, long long* info, int n_probe, const long long* probe_tiles, long long* probe_out);
+constexpr int kTcMaxBlocks = 160;                    // thread blocks of a launch, at most (one per multiprocessor)
 int tree_attention_tc(const AttentionArgs& a, WorkspaceHeader* header, void* scratch, size_t scratch_bytes,
                       cudaStream_t stream);
 

@@ -42,6 +42,7 @@
 // partial, warp 15 publishes the partial this block writes; at the end of the block all sixteen warps together
 // merge a split item.  Every wait is
 // bounded; one that runs out raises a flag in the workspace header, all roles drain and the block exits cleanly.
+#include <algorithm>
 #include <mutex>
 #include <type_traits>
 
@@ -76,6 +77,7 @@ struct TcSmall {
     TileIndex ix;
     alignas(128) __nv_bfloat16 ones[256];   // 16 x 16 matrix of ones: B operand of the row-sum product
 };
+static_assert(kMaxCtas == kTcMaxBlocks, "the plan's public limit is the kernel's");
 static_assert(sizeof(TcSmall) <= kSmemLimit - 1024 - kSlots * 32768 - 160 * 512, "TcSmall grew: four ring slots no longer fit");
 
 // 64 bits of a 192-bit row starting at bit `start` (bits past the row read as zero)
@@ -1014,6 +1016,53 @@ bool tc_shape_supported(int B, int H, int G, int N, int D, int L_max, int dtype)
     if (!(G >= 1 && H % G == 0 && N >= 1 && N <= MCSD_MAX_NODES && B >= 1 && B <= kMaxBatchTc && L_max >= 0)) return false;
     const long long tiles = (long long)L_max / kTile + 4;
     return (long long)B * tiles * 2 * 64 < (1LL << 30);
+}
+
+// The kernel's plan evaluated on the host with the functions the kernel uses (inspection and tests): first tile of
+// every block, totals, and for each probed tile where it lies and which block owns it.
+template <int QB>
+static int plan_host(const TcParams& p, int grid, long long* first_tile, long long* info, int n_probe, const long long* probe_tiles,
+                     long long* probe_out) {
+    TileIndex ix;
+    int items = 0, longest = 0;
+    ix.cum_tiles[0] = 0;
+    ix.cum_w[0] = 0;
+    for (int b = 0; b < p.B; ++b) {
+        int t, w, i, kv;
+        plan_sequence<QB>(&ix, p, b, t, w, i, kv);
+        ix.cum_tiles[b + 1] = ix.cum_tiles[b] + t;
+        ix.cum_w[b + 1] = ix.cum_w[b] + w;
+        items += i;
+        longest = std::max(longest, kv);
+    }
+    const int nb = plan_blocks<QB>(&ix, p, grid, items, longest);
+    const long long total = (long long)p.H * ix.cum_tiles[p.B], total_w = (long long)p.H * ix.cum_w[p.B];
+    for (int c = 0; c <= grid; ++c) first_tile[c] = range_start<QB>(&ix, p, c, nb);
+    if (info) { info[0] = total; info[1] = total_w; info[2] = ix.whole_items; info[3] = QB; }
+    for (int i = 0; i < n_probe; ++i) {
+        long long* o = probe_out + 8 * (size_t)i;
+        const long long t = probe_tiles[i];
+        if (t < 0 || t >= total) { for (int k = 0; k < 8; ++k) o[k] = -1; continue; }
+        Segment sg;
+        locate<QB>(&ix, p, t, sg);
+        o[0] = sg.b; o[1] = sg.h; o[2] = sg.qb; o[3] = sg.lt; o[4] = sg.Nq; o[5] = sg.Tkv;
+        o[6] = ix.whole_items ? -1 : block_of_tile<QB>(&ix, p, t, nb, total_w);
+        o[7] = weight_before<QB>(&ix, p, sg);
+    }
+    return total > 0 ? nb : 0;
+}
+
+int tc_plan_host(int B, int H, int G, int N, int L_max, const int32_t* seq_lens, const int32_t* n_active, int grid,
+                 long long* first_tile, long long* info, int n_probe, const long long* probe_tiles, long long* probe_out) {
+    const int S = tc_stack_for(G, N);
+    TcParams p = {};
+    p.seq_lens = seq_lens;
+    p.n_active = n_active;
+    p.B = B; p.H = H / S; p.N = N; p.L_max = L_max;
+    p.G = S;
+    p.g_shift = S == 8 ? 3 : S == 4 ? 2 : S == 2 ? 1 : 0;
+    return chunks_for(N * S) == 10 ? plan_host<kMaxQ>(p, grid, first_tile, info, n_probe, probe_tiles, probe_out)
+                                   : plan_host<128>(p, grid, first_tile, info, n_probe, probe_tiles, probe_out);
 }
 
 bool tc_supported(const AttentionArgs& a) {

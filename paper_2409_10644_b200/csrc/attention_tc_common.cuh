@@ -220,11 +220,11 @@ __device__ __forceinline__ uint32_t instr_desc(int n, int a_mn_major, int b_mn_m
 // tree with more stacked queries makes each (sequence, head) two work items that read the same keys.  Tiles per
 // work item: prefix tiles, then tree tiles.  Everything below is a pure function of the launch so that all thread
 // blocks cut the tile space alike.
-__device__ __forceinline__ int kv_tiles_of(int L, int Nb) {
+__host__ __device__ __forceinline__ int kv_tiles_of(int L, int Nb) {
     return Nb > 0 ? (L + kTile - 1) / kTile + (Nb + kTile - 1) / kTile : 0;
 }
 template <int QB>
-__device__ __forceinline__ int tiles_of(int L, int Nb, int G) {
+__host__ __device__ __forceinline__ int tiles_of(int L, int Nb, int G) {
     return kv_tiles_of(L, Nb) * ((Nb * G + QB - 1) / QB);
 }
 
@@ -234,7 +234,7 @@ struct Segment {
 };
 
 template <int QB>
-__device__ __forceinline__ void locate(const TileIndex* ix, const TcParams& p, long long t, Segment& s) {
+__host__ __device__ __forceinline__ void locate(const TileIndex* ix, const TcParams& p, long long t, Segment& s) {
     int lo = 0, hi = p.B;                      // find b with H*cum[b] <= t < H*cum[b+1]
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
@@ -273,14 +273,14 @@ __device__ __forceinline__ void locate(const TileIndex* ix, const TcParams& p, l
 // deep trees do not make their blocks finish late.  At most 64 per tile and 256 per work item (the launch bound on
 // the 32-bit prefix sums counts on it).
 template <int QB>
-__device__ __forceinline__ int tile_weight(int Nq) { return (QB > 128 ? 34 : 29) + (Nq * 83 + (Nq * Nq * 35) / 64) / 1024; }
+__host__ __device__ __forceinline__ int tile_weight(int Nq) { return (QB > 128 ? 34 : 29) + (Nq * 83 + (Nq * Nq * 35) / 64) / 1024; }
 // Fixed cost of a work item (the wait for the last product, normalisation and output of Nq columns, locating the
 // next item).  The fit puts it at the item's end, so the item's last tile carries it: a block that takes only the
 // first tiles of an item does not pay it.
 template <int QB>
-__device__ __forceinline__ int item_weight(int Nq) { return QB > 128 ? 119 + (Nq * 130) / 256 : 109 + (Nq * 47) / 256; }
+__host__ __device__ __forceinline__ int item_weight(int Nq) { return QB > 128 ? 119 + (Nq * 130) / 256 : 109 + (Nq * 47) / 256; }
 template <int QB>
-__device__ __forceinline__ int head_weight(int L, int Nk, int G) {  // cost of one (sequence, head): all query blocks
+__host__ __device__ __forceinline__ int head_weight(int L, int Nk, int G) {  // cost of one (sequence, head): all query blocks
     const int tkv = kv_tiles_of(L, Nk);
     const int Nb = Nk * G;                                        // stacked queries
     int w = 0;
@@ -289,7 +289,7 @@ __device__ __forceinline__ int head_weight(int L, int Nk, int G) {  // cost of o
 }
 // cumulative cost of the tiles before the one a Segment points at
 template <int QB>
-__device__ __forceinline__ long long weight_before(const TileIndex* ix, const TcParams& p, const Segment& s) {
+__host__ __device__ __forceinline__ long long weight_before(const TileIndex* ix, const TcParams& p, const Segment& s) {
     long long w = (long long)p.H * ix->cum_w[s.b] + (long long)s.h * (ix->cum_w[s.b + 1] - ix->cum_w[s.b]);
     if (s.qb) w += (long long)s.Tkv * tile_weight<QB>(QB) + item_weight<QB>(QB);
     return w + (long long)s.lt * tile_weight<QB>(s.Nq);
@@ -297,7 +297,7 @@ __device__ __forceinline__ long long weight_before(const TileIndex* ix, const Tc
 // Tile t belongs to block floor(weight_before(t) * G / total_w).  First tile of block c: the first tile whose
 // cumulative cost reaches ceil(c * total_w / G).
 template <int QB>
-__device__ __forceinline__ long long first_tile_of_block(const TileIndex* ix, const TcParams& p, int c, int G, long long total_w,
+__host__ __device__ __forceinline__ long long first_tile_of_block(const TileIndex* ix, const TcParams& p, int c, int G, long long total_w,
                                                          long long total_tiles) {
     const long long wt = ((long long)c * total_w + G - 1) / G;
     if (wt >= total_w) return total_tiles;
@@ -327,10 +327,54 @@ __device__ __forceinline__ long long first_tile_of_block(const TileIndex* ix, co
     return t + min(tkv, (r2 + w - 1) / w);
 }
 template <int QB>
-__device__ __forceinline__ int block_of_tile(const TileIndex* ix, const TcParams& p, long long t, int G, long long total_w) {
+__host__ __device__ __forceinline__ int block_of_tile(const TileIndex* ix, const TcParams& p, long long t, int G, long long total_w) {
     Segment s;
     locate<QB>(ix, p, t, s);
     return (int)min((long long)G - 1, weight_before<QB>(ix, p, s) * G / total_w);
+}
+
+// Per-sequence entries of the tile index (the prefix sums over sequences are the caller's).
+template <int QB>
+__host__ __device__ __forceinline__ void plan_sequence(TileIndex* ix, const TcParams& p, int b, int& tiles, int& cost, int& items,
+                                                       int& kv) {
+    const int L = min(max(p.seq_lens[b], 0), p.L_max);
+    const int Nb = p.n_active ? min(max(p.n_active[b], 0), p.N) : p.N;
+    kv = min(kv_tiles_of(L, Nb), 65535);
+    tiles = tiles_of<QB>(L, Nb, p.G);
+    cost = head_weight<QB>(L, Nb, p.G);
+    items = Nb > 0 ? (Nb * p.G + QB - 1) / QB : 0;          // query blocks of the sequence
+    ix->kv_tiles[b] = (unsigned short)kv;
+    ix->len[b] = L;
+    ix->nodes[b] = (unsigned short)Nb;
+}
+// How many blocks get work, and in which mode, once the prefix sums are in place.
+template <int QB>
+__host__ __device__ __forceinline__ int plan_blocks(TileIndex* ix, const TcParams& p, int grid, int items, int longest) {
+    // Few short work items (one sequence with a short prefix, say): a block's fixed costs outweigh its tiles, and
+    // cutting items into pieces would add a partial and a merge to each.  Every block then takes whole items.
+    const long long n_items = (long long)p.H * items;
+    ix->whole_items = (n_items > 0 && n_items <= (long long)grid && longest <= kWholeItemTiles) ? 1 : 0;
+    // Otherwise no block's share of the cost may be smaller than the heaviest tile, so that consecutive tiles never
+    // skip a block: every working block then owns at least one tile and the blocks sharing a work item are
+    // consecutive.
+    const long long tot_w = (long long)p.H * ix->cum_w[p.B];
+    return ix->whole_items ? (int)n_items
+                           : (int)max(1LL, min((long long)grid, tot_w / (tile_weight<QB>(QB) + item_weight<QB>(QB))));
+}
+// First tile of block c of nb (c == nb: one past the last tile).
+template <int QB>
+__host__ __device__ __forceinline__ long long range_start(const TileIndex* ix, const TcParams& p, int c, int nb) {
+    const long long tot = (long long)p.H * ix->cum_tiles[p.B], tot_w = (long long)p.H * ix->cum_w[p.B];
+    if (tot <= 0 || c >= nb) return tot > 0 ? tot : 0;
+    if (!ix->whole_items) return first_tile_of_block<QB>(ix, p, c, nb, tot_w, tot);
+    // first tile of work item number c = (sequence, head, query block) in tile order
+    for (int b = 0; b < p.B; ++b) {
+        const int kv = ix->kv_tiles[b], tb = ix->cum_tiles[b + 1] - ix->cum_tiles[b];
+        const int per_seq = kv > 0 ? p.H * (tb / kv) : 0;
+        if (c < per_seq) return (long long)p.H * ix->cum_tiles[b] + (long long)c * kv;
+        c -= per_seq;
+    }
+    return tot;
 }
 
 // Per-block set-up: tiles and cost per sequence, their prefix sums, the number of blocks that get work and the two
@@ -342,17 +386,7 @@ __device__ __forceinline__ void plan_ranges(TileIndex* ix, const TcParams& p, in
     // over the sequences, by warp shuffles and one exchange of the eight warp totals
     int v_t = 0, v_w = 0, v_i = 0, v_kv = 0;
     if (tid < kMaxBatchTc) {
-        if (tid < p.B) {
-            const int L = min(max(p.seq_lens[tid], 0), p.L_max);
-            const int Nb = p.n_active ? min(max(p.n_active[tid], 0), p.N) : p.N;
-            v_kv = min(kv_tiles_of(L, Nb), 65535);
-            v_t = tiles_of<QB>(L, Nb, p.G);
-            v_w = head_weight<QB>(L, Nb, p.G);
-            v_i = Nb > 0 ? (Nb * p.G + QB - 1) / QB : 0;          // query blocks of the sequence
-            ix->kv_tiles[tid] = (unsigned short)v_kv;
-            ix->len[tid] = L;
-            ix->nodes[tid] = (unsigned short)Nb;
-        }
+        if (tid < p.B) plan_sequence<QB>(ix, p, tid, v_t, v_w, v_i, v_kv);
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const int a = __shfl_up_sync(0xffffffffu, v_t, o), c = __shfl_up_sync(0xffffffffu, v_w, o),
@@ -371,43 +405,14 @@ __device__ __forceinline__ void plan_ranges(TileIndex* ix, const TcParams& p, in
             longest = max(longest, ix->scan[x][3]);
         }
         if (tid < p.B) { ix->cum_tiles[tid + 1] = v_t; ix->cum_w[tid + 1] = v_w; }
-        if (tid == max(p.B, 1) - 1) {
-            ix->cum_tiles[0] = 0;
-            ix->cum_w[0] = 0;
-            // Few short work items (one sequence with a short prefix, say): a block's fixed costs outweigh its tiles,
-            // and cutting items into pieces would add a partial and a merge to each.  Every block then takes whole
-            // items.
-            const long long n_items = (long long)p.H * items;
-            ix->whole_items = (n_items > 0 && n_items <= (long long)gridDim.x && longest <= kWholeItemTiles) ? 1 : 0;
-            // Otherwise no block's share of the cost may be smaller than the heaviest tile, so that consecutive tiles
-            // never skip a block: every working block then owns at least one tile and the blocks sharing a work item
-            // are consecutive.
-            const long long tot_w = (long long)p.H * v_w;
-            *n_blocks = ix->whole_items ? (int)n_items
-                                        : (int)max(1LL, min((long long)gridDim.x, tot_w / (tile_weight<QB>(QB) + item_weight<QB>(QB))));
-        }
+        if (tid == 0) { ix->cum_tiles[0] = 0; ix->cum_w[0] = 0; }
+        // the thread that wrote the totals (plan_blocks reads only cum_w[B])
+        if (tid == max(p.B, 1) - 1) *n_blocks = plan_blocks<QB>(ix, p, (int)gridDim.x, items, longest);
     }
     __syncthreads();
     if (tid == 0 || tid == 32) {               // the two ends of this block's range, side by side
-        const long long tot = (long long)p.H * ix->cum_tiles[p.B], tot_w = (long long)p.H * ix->cum_w[p.B];
-        const int nb = *n_blocks, which = tid >> 5;
-        long long t = 0;
-        if (tot > 0 && (int)blockIdx.x < nb) {
-            if (ix->whole_items) {
-                // first tile of work item number c = (sequence, head, query block) in tile order
-                int c = (int)blockIdx.x + which, b = 0;
-                t = tot;
-                for (; b < p.B; ++b) {
-                    const int kv = ix->kv_tiles[b], tb = ix->cum_tiles[b + 1] - ix->cum_tiles[b];
-                    const int per_seq = kv > 0 ? p.H * (tb / kv) : 0;
-                    if (c < per_seq) { t = (long long)p.H * ix->cum_tiles[b] + (long long)c * kv; break; }
-                    c -= per_seq;
-                }
-            } else {
-                t = first_tile_of_block<QB>(ix, p, (int)blockIdx.x + which, nb, tot_w, tot);
-            }
-        }
-        range[which] = t;
+        const int which = tid >> 5;
+        range[which] = (int)blockIdx.x < *n_blocks ? range_start<QB>(ix, p, (int)blockIdx.x + which, *n_blocks) : 0;
     }
     __syncthreads();
 }

@@ -359,3 +359,88 @@ def test_bench_counts_the_rows_the_verify_kernel_reads():
     assert rows == 2 * (3 + 2 + 2)
     rows_cut, _ = bench.verify_rows_read(states, parent, np.array([4, 4]))     # level 2 sliced off: only the root counts
     assert rows_cut == 2 * (0 + 2)
+
+
+def _enumerate_tiles(lens, n_act, units, stack, qb):
+    """Brute force: (sequence, unit, query block, tile in item, queries, tiles in item) of every tile, in the
+    kernel's order (prefix tiles before tree tiles inside an item)."""
+    rows = []
+    for b in range(len(lens)):
+        L, Nb = int(lens[b]), int(n_act[b])
+        if Nb <= 0:
+            continue
+        tkv = -(-L // 128) + -(-Nb // 128)
+        nq = Nb * stack
+        for h in range(units):
+            for qi, q0 in enumerate(range(0, nq, qb)):
+                for lt in range(tkv):
+                    rows.append((b, h, qi, lt, min(qb, nq - q0), tkv))
+    return np.array(rows, dtype=np.int64).reshape(-1, 6)
+
+
+@pytest.mark.parametrize("seed", range(40))
+def test_attention_plan_partitions_the_tiles_of_a_launch(m, seed):
+    """mcsd_tree_attention_plan (the kernel's own work-partition functions, evaluated on the host): the blocks' ranges
+    tile the launch without gaps, every probed tile is where a brute-force enumeration puts it, the block that the
+    merging code computes for a tile is the block whose range holds it, no block's cost exceeds an even share by
+    more than one heaviest tile, and in whole-item mode every block gets exactly one work item."""
+    rng = np.random.default_rng(100 + seed)
+    B = int(rng.choice([1, 2, 5, 16, 33, 256]))
+    N = int(rng.choice([1, 15, 45, 82, 109, 128, 129, 160, 192]))
+    H_kv = int(rng.choice([1, 2, 8]))
+    G = int(rng.choice([1, 1, 2, 4, 8]))
+    H_q = H_kv * G
+    L_max = int(rng.choice([0, 100, 1000, 5000]))
+    lens = rng.integers(0, L_max + 1, B).astype(np.int32)
+    n_act = rng.integers(0, N + 1, B).astype(np.int32)
+    if seed % 3 == 0:
+        n_act[:] = N
+    if seed == 5:                                   # a small launch: whole items
+        B, lens, n_act = 1, np.array([min(L_max, 500)], dtype=np.int32), np.array([N], dtype=np.int32)
+    n_blocks = int(rng.choice([1, 7, 148, 160]))
+    assert m.mcsd_tree_attention_path(B, H_q, H_kv, N, 128, L_max, m.MCSD_BF16) == 1
+    stack = next((s for s in (8, 4, 2) if G % s == 0 and s * N <= 160), 1)
+    units = H_q // stack
+
+    used, first, info, _ = m.mcsd_tree_attention_plan(B, H_q, H_kv, N, 128, L_max, m.MCSD_BF16, lens, n_act, n_blocks)
+    total, total_cost, whole, qb = (int(x) for x in info)
+    assert qb == (160 if N * stack > 128 else 128)          # trees wider than that are cut into query blocks of 160
+    tiles = _enumerate_tiles(lens, n_act, units, stack, qb)
+    assert total == len(tiles)
+    assert first[0] == 0 and (np.diff(first) >= 0).all() and first[-1] == total
+    assert (first[used:] == total).all()
+    if total == 0:
+        assert used == 0
+        return
+    assert 1 <= used <= n_blocks and (np.diff(first[: used + 1]) > 0).all()      # every used block owns a tile
+
+    probes = np.unique(np.concatenate([first[:used], first[1: used + 1] - 1, rng.integers(0, total, 200)]))
+    _, _, _, out = m.mcsd_tree_attention_plan(B, H_q, H_kv, N, 128, L_max, m.MCSD_BF16, lens, n_act, n_blocks, probes)
+    assert (out[:, :6] == tiles[probes]).all()
+    owner = np.searchsorted(first[1: used + 1], probes, side="right")            # block whose range holds the tile
+    if whole:
+        assert (out[:, 6] == -1).all()
+        item_starts = np.flatnonzero(tiles[:, 3] == 0)
+        assert used == len(item_starts) and (first[:used] == item_starts).all()
+    else:
+        assert (out[:, 6] == owner).all()
+        # cost: block c's tiles cost (cost before its successor's first tile) - (cost before its own first tile)
+        _, _, _, edge = m.mcsd_tree_attention_plan(B, H_q, H_kv, N, 128, L_max, m.MCSD_BF16, lens, n_act, n_blocks, first[:used])
+        before = np.append(edge[:, 7], total_cost)
+        assert (np.diff(before) > 0).all()
+        heaviest = 64 + 256                                                       # a tile with an item's fixed cost on it
+        assert np.diff(before).max() <= -(-total_cost // used) + heaviest
+    # a tile number outside the launch is reported as such
+    _, _, _, bad = m.mcsd_tree_attention_plan(B, H_q, H_kv, N, 128, L_max, m.MCSD_BF16, lens, n_act, n_blocks, [total, -1])
+    assert (bad == -1).all()
+
+
+def test_attention_plan_rejects_what_the_tensor_core_kernel_does_not_take(m):
+    lens = np.array([10, 20], dtype=np.int32)
+    with pytest.raises(m.McsdError):
+        m.mcsd_tree_attention_plan(2, 4, 4, 15, 64, 128, m.MCSD_BF16, lens)                  # head_dim 64: CUDA-core kernel
+    with pytest.raises(m.McsdError):
+        m.mcsd_tree_attention_plan(2, 4, 4, 193, 128, 128, m.MCSD_BF16, lens)                # too many nodes
+    with pytest.raises(ValueError):
+        m.mcsd_tree_attention_plan(2, 4, 4, 15, 128, 128, m.MCSD_BF16, lens, n_blocks=161)
+    assert int(m.lib.mcsd_tree_attention_plan(2, 4, 4, 15, 128, 128, m.MCSD_BF16, None, None, 4, None, None, 0, None, None)) == -1
