@@ -420,16 +420,31 @@ __device__ __forceinline__ bool better(float va, int ia, float vb, int ib) {
 
 // Follows next_child from every root, keeps the longest path (ties: lowest root) and writes accept_len,
 // best_root, out_nodes and all of out_tokens but the new token.  Returns the stop node and the slot of the
-// new token through shared memory; ends with a block barrier.
+// new token through shared memory (and the stop node's residual coefficient, if asked for); ends with a block
+// barrier.  The sequence's node states and tokens are brought into shared memory with one trip to memory and the
+// walks run there: followed through global memory, every step of every walk was a dependent trip of its own.
 __device__ __forceinline__ void select_path(const NodeState* __restrict__ st, const int32_t* __restrict__ tokens, int b,
                                             int n_levels, int n_roots, int N, int32_t* __restrict__ accept_len,
                                             int32_t* __restrict__ out_tokens, int32_t* __restrict__ out_nodes,
-                                            int32_t* __restrict__ best_root, int* s_len, int* s_stop, int* s_slot) {
+                                            int32_t* __restrict__ best_root, int* s_len, int* s_stop, int* s_slot,
+                                            double* s_c_stop = nullptr, const float* __restrict__ u_bonus = nullptr,
+                                            float* s_u_stop = nullptr) {
+    __shared__ int s_next[MCSD_MAX_NODES];
+    __shared__ int s_tok[MCSD_MAX_NODES];
+    __shared__ double s_c[MCSD_MAX_NODES];
+    __shared__ float s_ub[MCSD_MAX_NODES];
     const int tid = threadIdx.x;
+    for (int i = tid; i < N; i += blockDim.x) {
+        s_next[i] = __ldcg(&st[i].next_child);
+        s_c[i] = __ldcg(&st[i].c);
+        s_tok[i] = tokens[(size_t)b * N + i];
+        if (u_bonus) s_ub[i] = u_bonus[(size_t)b * N + i];
+    }
+    __syncthreads();
     if (tid < n_roots) {
         int u = tid, len = 0;
         for (int step = 0; step < n_levels; ++step) {
-            const int nc = __ldcg(&st[u].next_child);
+            const int nc = s_next[u];
             if (nc < 0 || nc >= N) break;
             u = nc;
             ++len;
@@ -446,17 +461,19 @@ __device__ __forceinline__ void select_path(const NodeState* __restrict__ st, co
         for (int i = 0; i < n_levels + 1; ++i) ot[i] = -1;
         for (int i = 0; i < n_levels; ++i) on[i] = -1;
         int slot = 0;
-        if (n_roots > 1) ot[slot++] = tokens[(size_t)b * N + best];
+        if (n_roots > 1) ot[slot++] = s_tok[best];
         int u = best;
         for (int i = 0; i < s_len[best]; ++i) {
-            u = __ldcg(&st[u].next_child);
+            u = s_next[u];
             on[i] = u;
-            ot[slot++] = tokens[(size_t)b * N + u];
+            ot[slot++] = s_tok[u];
         }
         accept_len[b] = s_len[best];
         best_root[b] = best;
         *s_stop = u;
         *s_slot = slot;
+        if (s_c_stop) *s_c_stop = s_c[u];
+        if (s_u_stop && u_bonus) *s_u_stop = s_ub[u];
     }
     __syncthreads();
 }
@@ -690,22 +707,25 @@ __device__ void select_and_draw(const Rows& rows, const int32_t* __restrict__ to
     constexpr int E = Dist::E;
     __shared__ int s_len[MCSD_MAX_NODES];
     __shared__ int s_stop, s_slot;
+    __shared__ double s_c_stop;
+    __shared__ float s_u_stop;
     __shared__ CdfScratch s_cdf;
     __shared__ float s_bv[kVerifyWarps];
     __shared__ int s_bi[kVerifyWarps];
     const int tid = threadIdx.x;
 
-    select_path(st, tokens, b, n_levels, n_roots, N, accept_len, out_tokens, out_nodes, best_root, s_len, &s_stop, &s_slot);
+    select_path(st, tokens, b, n_levels, n_roots, N, accept_len, out_tokens, out_nodes, best_root, s_len, &s_stop, &s_slot,
+                &s_c_stop, u_bonus, &s_u_stop);
     const int u = s_stop;
     Dist d = rows.open(b, u, N, V, s_scratch);
-    d.set_c(__ldcg(&st[u].c));
+    d.set_c(s_c_stop);
 
     // ---- new token: inverse CDF over dist_v = max(p_v - c q_v, 0) in token-id order ----
     auto load = [&d](int idx, float (&r)[E]) { d.load(idx, r); };
     auto keep = [](int, float (&)[E]) {};
     double total;
     cdf_range_sums_dist(d, keep, V, &s_cdf);
-    const int found = cdf_locate<E>(load, (double)u_bonus[(size_t)b * N + u], false, V, &s_cdf, &total);
+    const int found = cdf_locate<E>(load, (double)s_u_stop, false, V, &s_cdf, &total);
     if (tid == 0) out_tokens[(size_t)b * (n_levels + 1) + s_slot] = found;
 
     // ---- optional: the R most probable ids of the same distribution ----
@@ -729,7 +749,10 @@ verify_tree_kernel(Rows rows, const int32_t* __restrict__ tokens, const int32_t*
     const int lin = blockIdx.y * gridDim.x + blockIdx.x;
     const int b = lin % (int)gridDim.y, u = lin / (int)gridDim.y, tid = threadIdx.x;
     const int n_act = active_nodes(gamma, level_start, n_levels, b, N);
-    if (u >= n_act) return;
+    if (u >= n_act) return;                    // first: a sliced forest launches many blocks that have nothing to do
+    // the sequence's tokens travel together with the parent array: one trip to memory instead of two in a row
+    __shared__ int s_tok[MCSD_MAX_NODES];
+    for (int i = tid; i < N; i += kVerifyThreads) s_tok[i] = tokens[(size_t)b * N + i];
     int first, cnt;
     find_children(parent, u, N, &s_first, &s_cnt, first, cnt);
 
@@ -741,7 +764,7 @@ verify_tree_kernel(Rows rows, const int32_t* __restrict__ tokens, const int32_t*
         // p_u(x), q_u(x) and the uniform of every sibling are fetched side by side up front, so that the sibling
         // loop below pays for one dependent trip to memory in total instead of one per sibling
         for (int m = tid; m < cnt; m += kVerifyThreads) {
-            const int x = tokens[(size_t)b * N + first + m];
+            const int x = s_tok[first + m];
             const bool valid = x >= 0 && x < V;
             s_px[m] = valid ? d.p_of(x) : -1.0;               // -1: no such token, never accepted
             s_qx[m] = valid ? d.q_of(x) : 0.0;
