@@ -797,13 +797,13 @@ verify_tree_kernel(Rows rows, const int32_t* __restrict__ tokens, const int32_t*
     // ---- ticket: the block that finishes a sequence's last node goes on to the select phase
     if (tid == 0) {
         state[(size_t)b * N + u] = st;
-        __threadfence();                                   // the state is visible before the ticket is
-        const int old = atomicAdd(&tickets[b], 1);
+        // One acquire-release ticket instead of fence, ticket, fence (three trips to memory in a row on the path of
+        // the block that finishes last): the state above is visible before the ticket is, and the block that draws
+        // the last ticket sees the states of all the others.
+        int old;
+        asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(old) : "l"(tickets + b) : "memory");
         s_last = (old == n_act - 1) ? 1 : 0;
-        if (s_last) {
-            *(volatile int*)&tickets[b] = 0;               // nobody else arrives in this launch: ready for the next one
-            __threadfence();                               // acquire: the other blocks' states are visible
-        }
+        if (s_last) *(volatile int*)&tickets[b] = 0;       // nobody else arrives in this launch: ready for the next one
     }
     __syncthreads();
     if (!s_last) return;
