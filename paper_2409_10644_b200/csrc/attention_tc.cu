@@ -35,13 +35,16 @@
 //     by constants, and there are two commits per tile (S^T done = scores ready and key slot free; products done =
 //     value slot and P^T free), because a tcgen05.mma of these shapes takes 40-60 cycles and the instructions
 //     between two of them would otherwise pace the tensor pipe;
-//   * the producer issues loads in the order in which slots come free (K0 K1 V0 K2 V1 ...), about two tiles ahead.
+//   * the producer issues loads in the order in which slots come free (K0 K1 V0 K2 V1 ...), about two tiles ahead;
+//     a tile with at most 64 rows in use is fetched as one 64-row box;
+//   * prefix tiles need no mask (a dead key row of a ragged tile is one thread's own row); tree tiles mask the packed
+//     probabilities with masks grown from the transposed ancestor bitsets by a multiply and a byte permute.
 //
 // Warp roles (512 threads): warps 0-11 softmax / mask / epilogue, warp 12 TMA producer, warp 13 MMA issuer and owner
 // of the tensor-memory allocation, warp 14 polls the tickets of a split last work item and fetches its first
 // partial, warp 15 publishes the partial this block writes; at the end of the block all sixteen warps together
-// merge a split item.  Every wait is
-// bounded; one that runs out raises a flag in the workspace header, all roles drain and the block exits cleanly.
+// merge a split item.  Every wait is bounded; one that runs out raises a flag in the workspace header, all roles
+// drain and the block exits cleanly.
 #include <algorithm>
 #include <mutex>
 #include <type_traits>
@@ -80,9 +83,9 @@ struct TcSmall {
 static_assert(kMaxCtas == kTcMaxBlocks, "the plan's public limit is the kernel's");
 static_assert(sizeof(TcSmall) <= kSmemLimit - 1024 - kSlots * 32768 - 160 * 512, "TcSmall grew: four ring slots no longer fit");
 
-// 64 bits of a 192-bit row starting at bit `start` (bits past the row read as zero)
 // rows of a key/value tile that are fetched when `valid` of them are in use: all 128, or a box of 64
 __device__ __forceinline__ int loaded_rows(int valid) { return valid > 64 ? kTile : 64; }
+// byte permute; a selector nibble with its top bit set replicates the sign bit of the selected byte
 __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
     uint32_t d;
     asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
@@ -93,6 +96,7 @@ __device__ __forceinline__ uint32_t max_u16x2(uint32_t a, uint32_t b) {
     asm("max.u16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
     return d;
 }
+// 64 bits of a 192-bit row starting at bit `start` (bits past the row read as zero)
 __device__ __forceinline__ unsigned long long bits_from(const unsigned long long* w, int start) {
     const int wi = start >> 6, sh = start & 63;
     unsigned long long lo = w[wi] >> sh;
@@ -152,7 +156,6 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
     // everything the preceding kernel in the stream wrote is visible from here on
     asm volatile("griddepcontrol.wait;" ::: "memory");
     plan_ranges<QB>(&sm->ix, p, &sm->n_blocks, sm->range);
-    const long long total = (long long)p.H * ix->cum_tiles[p.B];
     const long long total_w = (long long)p.H * ix->cum_w[p.B];
     const int G = sm->n_blocks;
     const long long t_begin = sm->range[0], t_end = sm->range[1];
@@ -618,7 +621,7 @@ tree_attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_
             // ---- epilogue of the segment: each group finishes its own query columns.  A segment that holds a whole work
             // item is normalised and written out.  A piece of a split item that does not start the item is written to
             // the workspace unnormalised and announced with a ticket.  The piece that starts a split item is always a
-            // block's last segment: it stays in tensor memory and the service warps merge the other pieces into it (see
+            // block's last segment: it stays in tensor memory and the whole block merges the other pieces into it (see
             // the end of the kernel), so there is nothing to do here.
             const uint32_t glast = g + (uint32_t)cnt - 1u;
             const bool full = (cnt == s.Tkv);
